@@ -1,0 +1,162 @@
+/*
+ * fblayout.h -- C ABI of the B200 attention-layer training step on one unified tiled layout.
+ *
+ * One transformer attention layer (pre-norm LayerNorm/RMSNorm, Q/K/V/O projections, causal or
+ * full softmax attention with optional grouped-query heads), forward and backward, where every
+ * matrix lives in a single reduction-aware tiled layout ("R-Tile", the paper's section 4.2) in
+ * both passes.  The transposes the backward needs (W^T, X^T, head split/merge) are tile-index
+ * remaps or operand-orientation flags of the tensor-core descriptors (the paper's section 4.3,
+ * Eq. 3 and Eq. 4), never copies.
+ *
+ * Conventions that hold for every call
+ *   - "dev" pointers are CUDA device pointers owned by the caller; "host" pointers are ordinary
+ *     host memory.  The library allocates no device memory, never synchronises the device and
+ *     enqueues all work on the CUDA stream handle passed as `stream` (a cudaStream_t cast to void*).
+ *   - Matrices are in the storage dtype of the plan (fp32 or bf16) in R-Tile order and have
+ *     exactly fbl_tensor_bytes() bytes; they must be 1024-byte aligned.  Vectors (gamma, beta,
+ *     biases and their gradients) are plain fp32 arrays in both dtypes.
+ *   - Padding slots of input matrices must hold zero (fbl_pack guarantees it); padding slots of
+ *     output matrices are written as zero.
+ *   - Gradients are overwritten, not accumulated.
+ *   - Return value: FBL_OK (0) or a negative fbl_status.  Nothing throws, aborts or traps.  There is
+ *     no CPU or library fallback: a shape the kernels cannot run is refused by fbl_plan_create.
+ *
+ * R-Tile, as laid out here (section 4.2: tile shape, intra-tile mapping Eq. 1, inter-tile mapping).
+ *   A matrix [R, C] with e-byte elements is cut into storage tiles of tile_h = 8 rows by
+ *   tile_w = 128/e columns (64 for bf16, 32 for fp32): one tile is 1 KiB, eight 128-byte rows,
+ *   row-major inside (the paper's "horizontal strips" case tile_w <= C_w, with C_w one 128-byte
+ *   line).  Tiles are ordered with the row-tile index fastest (the token axis is the dimension
+ *   with more tile traversals): tile (tr, tc) is tile number tc * (R_pad/8) + tr.  Hence
+ *       offset(r, c) = ((c / tile_w) * R_pad + r) * tile_w + c % tile_w          (in elements)
+ *   with R_pad = R rounded up to 8 and C a multiple of tile_w.  Token matrices [B, T, C] use row
+ *   r = b * T_pad + t with T_pad = T rounded up to 8, so every sequence starts on a tile boundary.
+ */
+#ifndef FBLAYOUT_H_
+#define FBLAYOUT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FBL_OK = 0,
+  FBL_ERR_INVALID_ARG = -1,
+  FBL_ERR_UNSUPPORTED_SHAPE = -2,
+  FBL_ERR_MISALIGNED = -3,
+  FBL_ERR_WORKSPACE_TOO_SMALL = -4,
+  FBL_ERR_CUDA = -5,
+  FBL_ERR_TIMEOUT = -6
+} fbl_status;
+
+enum { FBL_DTYPE_FP32 = 0, FBL_DTYPE_BF16 = 1 };
+enum { FBL_NORM_LAYERNORM = 0, FBL_NORM_RMSNORM = 1 };
+
+/* The fine-tuning problem's shapes and flags (the paper's motivating example: one attention
+ * block whose forward tensors are reused by the backward). */
+typedef struct {
+  int32_t batch, seq, d_model, n_q_heads, n_kv_heads, head_dim; /* GQA group = n_q_heads / n_kv_heads */
+  int32_t dtype;        /* FBL_DTYPE_*  */
+  int32_t norm;         /* FBL_NORM_*   */
+  int32_t causal;       /* 0 / 1 */
+  int32_t has_bias;     /* 0 / 1: biases on Q, K, V and O projections */
+  int32_t residual;     /* 0 / 1: Y = X + attention(norm(X)) */
+  float eps;
+  float softmax_scale;  /* <= 0 selects 1/sqrt(head_dim) */
+} fbl_layer_desc;
+
+/* Tensor ids for fbl_tensor_bytes, fbl_tile_offset, fbl_pack and fbl_unpack.  The *_HEADS ids are
+ * index-map views [B, H, T, head_dim] of the same buffers as Q, K, V and A (no data moves). */
+enum {
+  FBL_T_X = 0, FBL_T_Y, FBL_T_DY, FBL_T_DX,          /* [B, T, D]               */
+  FBL_T_WQ, FBL_T_WK, FBL_T_WV, FBL_T_WO,            /* [D,Dq] [D,Dkv] [D,Dkv] [Dq,D] (and their gradients) */
+  FBL_T_XN, FBL_T_Q, FBL_T_K, FBL_T_V, FBL_T_A,      /* [B, T, D | Dq | Dkv | Dkv | Dq] */
+  FBL_T_Q_HEADS, FBL_T_K_HEADS, FBL_T_V_HEADS, FBL_T_A_HEADS, /* [B, H, T, hd] views */
+  FBL_T_WQ_T, FBL_T_WK_T, FBL_T_WV_T, FBL_T_WO_T,    /* transposed views [C, R] of the weights */
+  FBL_T_COUNT
+};
+
+/* Tile maps f of Eq. 3 (row-major tile numbering of the source view -> of the destination view). */
+enum {
+  FBL_MAP_SPLIT_Q = 0,   /* [B*T_pad, Dq] flat view  -> [B, Hq, T_pad, hd] head view (reshape o transpose) */
+  FBL_MAP_MERGE_Q,       /* inverse                                                                   */
+  FBL_MAP_SPLIT_KV,      /* same for Dkv / Hkv                                                        */
+  FBL_MAP_MERGE_KV,
+  FBL_MAP_TRANSPOSE_WQ,  /* [D, Dq] -> [Dq, D] */
+  FBL_MAP_TRANSPOSE_WO,  /* [Dq, D] -> [D, Dq] */
+  FBL_MAP_PHYS_Q,        /* flat-view tile number -> physical tile slot in memory (inter-tile mapping) */
+  FBL_MAP_PHYS_WQ,
+  FBL_MAP_COUNT
+};
+
+typedef struct fbl_plan fbl_plan; /* opaque: padded sizes, index-map constants, kernel choices */
+
+/* Host only.  Validates the description against the tile-propagation legality checks of section 4.3
+ * (head_dim and d_model multiples of tile_w, n_q_heads a multiple of n_kv_heads) and the kernels'
+ * limits, then builds the plan.  *out is owned by the caller; release with fbl_plan_destroy. */
+int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out);
+void fbl_plan_destroy(fbl_plan* plan);
+
+/* Padded R-Tile size in bytes of a matrix (physical ids only; views return the size of their buffer). */
+int fbl_tensor_bytes(const fbl_plan* plan, int tensor_id, size_t* bytes);
+
+/* Sizes of the three caller-owned work areas: `saved` carries forward tensors into the backward
+ * (the E_reuse edges of the paper's graph, section 3.1: norm statistics, Xn, Q, K, V, A, LSE);
+ * the scratch areas hold per-call temporaries. */
+int fbl_workspace_bytes(const fbl_plan* plan, size_t* saved, size_t* scratch_fwd, size_t* scratch_bwd);
+
+/* Element map (pure host integer code): logical index -> element offset in the R-Tile buffer.
+ * idx is [b, t, c, 0] for token matrices, [r, c, 0, 0] for weights and transposed views,
+ * [b, h, t, d] for head views.  Returns < 0 if idx is out of range. */
+int64_t fbl_tile_offset(const fbl_plan* plan, int tensor_id, const int32_t idx[4]);
+
+/* Tile map f of Eq. 3, composed and strength-reduced as in Eq. 4 (host integer code). */
+int fbl_tile_map(const fbl_plan* plan, int map_id, int64_t src_tile, int64_t* dst_tile);
+
+/* Layout conversion at the graph boundary only (row-major dense <-> R-Tile), device to device.
+ * Never part of a training step. */
+int fbl_pack(const fbl_plan* plan, int tensor_id, const void* rowmajor_dev, void* tiled_dev, void* stream);
+int fbl_unpack(const fbl_plan* plan, int tensor_id, const void* tiled_dev, void* rowmajor_dev, void* stream);
+
+/* Forward: Y = [X +] softmax-attention(norm(X)) Wo [+ bo]; fills `saved`.  Biases and beta may be NULL
+ * when the plan has none. */
+int fbl_layer_fwd(const fbl_plan* plan, const void* X, const float* gamma, const float* beta,
+                  const void* Wq, const void* Wk, const void* Wv, const void* Wo,
+                  const float* bq, const float* bk, const float* bv, const float* bo,
+                  void* Y, void* saved, void* scratch, void* stream);
+
+/* Backward: every gradient of sum(Y * dY).  Matrix gradients are in the storage dtype in R-Tile
+ * order; vector gradients are fp32.  db* may be NULL when the plan has no biases, dbeta for RMSNorm. */
+int fbl_layer_bwd(const fbl_plan* plan, const void* dY, const void* X, const float* gamma,
+                  const void* Wq, const void* Wk, const void* Wv, const void* Wo, const void* saved,
+                  void* dX, void* dWq, void* dWk, void* dWv, void* dWo,
+                  float* dbq, float* dbk, float* dbv, float* dbo, float* dgamma, float* dbeta,
+                  void* scratch, void* stream);
+
+/* Token-axis column reduction used for every bias gradient (db = sum over tokens, the matmul
+ * backward's M-axis reduction of section 4.1): out[c] = sum_r M[r, c] for an R-Tile matrix of
+ * `rows` x `cols` (rows a multiple of 8, cols of tile_w) in the plan's dtype.  Two stages over tiles:
+ * per-slab partial sums into `scratch` (fbl_colsum_scratch_bytes), then a tree over slabs. */
+int fbl_colsum_scratch_bytes(const fbl_plan* plan, int64_t rows, int64_t cols, size_t* bytes);
+int fbl_colsum(const fbl_plan* plan, const void* M_dev, int64_t rows, int64_t cols,
+               float* out_dev, void* scratch_dev, void* stream);
+
+/* After the caller has synchronised the stream: reads back the device status word kept at the start
+ * of `scratch` (set when a bounded wait inside a kernel expired).  Synchronous 4-byte copy. */
+int fbl_status_poll(const fbl_plan* plan, const void* scratch, int32_t* device_status);
+
+/* Kernel family used by later calls on this plan: 0 = default (tcgen05 tensor-core kernels for bf16
+ * wherever one exists for the shape, FFMA kernels for fp32), 1 = FFMA kernels only (fp32 arithmetic on
+ * the same layout; lets a caller cross-check the tensor-core path on the device). */
+int fbl_plan_set_kernel_path(fbl_plan* plan, int path);
+
+const char* fbl_strerror(int status);
+/* Text of the last CUDA runtime error seen by this thread inside the library ("" if none). */
+const char* fbl_last_error_detail(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FBLAYOUT_H_ */

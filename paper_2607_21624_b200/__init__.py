@@ -1,0 +1,10 @@
+"""B200-native attention-layer training step on one unified tiled layout (ctypes binding).
+
+The shared library is built in-tree by ``paper_2607_21624_b200.build``; importing this
+package never falls back to another implementation: if the library is missing or a
+CUDA device is absent, calls raise.
+"""
+from .binding import (FblError, Plan, lib, load_library, LayerRunner, DTYPES, TENSOR, MAP,
+                      desc_from_config)
+
+__all__ = ["FblError", "Plan", "lib", "load_library", "LayerRunner", "DTYPES", "TENSOR", "MAP", "desc_from_config"]

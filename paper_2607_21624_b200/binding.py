@@ -1,0 +1,254 @@
+"""Thin ctypes binding over libfblayout's C ABI: argument marshalling only.
+
+``Plan`` mirrors the C entry points one to one.  ``LayerRunner`` owns the torch
+device buffers a caller needs (PyTorch is used for device memory and streams, nothing
+else) and offers pack / forward / backward / unpack in terms of them.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libfblayout.so")
+
+DTYPES = {"fp32": 0, "bf16": 1}
+NORMS = {"layernorm": 0, "rmsnorm": 1}
+TENSOR = {n: i for i, n in enumerate(
+    ["X", "Y", "DY", "DX", "WQ", "WK", "WV", "WO", "XN", "Q", "K", "V", "A",
+     "Q_HEADS", "K_HEADS", "V_HEADS", "A_HEADS", "WQ_T", "WK_T", "WV_T", "WO_T"])}
+MAP = {n: i for i, n in enumerate(
+    ["SPLIT_Q", "MERGE_Q", "SPLIT_KV", "MERGE_KV", "TRANSPOSE_WQ", "TRANSPOSE_WO", "PHYS_Q", "PHYS_WQ"])}
+
+
+class FblLayerDesc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in
+                ("batch", "seq", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "dtype", "norm", "causal",
+                 "has_bias", "residual")] + [("eps", C.c_float), ("softmax_scale", C.c_float)]
+
+
+class FblError(RuntimeError):
+    def __init__(self, code, what):
+        self.code = code
+        super().__init__(what)
+
+
+_lib = None
+
+
+def load_library():
+    """Load libfblayout.so (built in-tree).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FblError(-100, f"{LIB_PATH} is missing: run `python -m paper_2607_21624_b200.build` first")
+    L = C.CDLL(LIB_PATH)
+    vp, i64, i32, sz = C.c_void_p, C.c_int64, C.c_int32, C.c_size_t
+    L.fbl_plan_create.argtypes = [C.POINTER(FblLayerDesc), C.POINTER(vp)]
+    L.fbl_plan_destroy.argtypes = [vp]
+    L.fbl_plan_destroy.restype = None
+    L.fbl_tensor_bytes.argtypes = [vp, C.c_int, C.POINTER(sz)]
+    L.fbl_workspace_bytes.argtypes = [vp, C.POINTER(sz), C.POINTER(sz), C.POINTER(sz)]
+    L.fbl_tile_offset.argtypes = [vp, C.c_int, C.POINTER(i32)]
+    L.fbl_tile_offset.restype = i64
+    L.fbl_tile_map.argtypes = [vp, C.c_int, i64, C.POINTER(i64)]
+    L.fbl_pack.argtypes = [vp, C.c_int, vp, vp, vp]
+    L.fbl_unpack.argtypes = [vp, C.c_int, vp, vp, vp]
+    L.fbl_layer_fwd.argtypes = [vp] * 16
+    L.fbl_layer_bwd.argtypes = [vp] * 22
+    L.fbl_colsum_scratch_bytes.argtypes = [vp, i64, i64, C.POINTER(sz)]
+    L.fbl_colsum.argtypes = [vp, vp, i64, i64, vp, vp, vp]
+    L.fbl_status_poll.argtypes = [vp, vp, C.POINTER(i32)]
+    L.fbl_plan_set_kernel_path.argtypes = [vp, C.c_int]
+    L.fbl_strerror.argtypes = [C.c_int]
+    L.fbl_strerror.restype = C.c_char_p
+    L.fbl_last_error_detail.restype = C.c_char_p
+    _lib = L
+    return L
+
+
+def lib():
+    return load_library()
+
+
+def _check(code):
+    if code != 0:
+        L = lib()
+        raise FblError(code, f"{L.fbl_strerror(code).decode()} [{L.fbl_last_error_detail().decode()}]")
+
+
+def desc_from_config(cfg) -> FblLayerDesc:
+    return FblLayerDesc(cfg.batch, cfg.seq, cfg.d_model, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim,
+                        DTYPES[cfg.dtype], NORMS[cfg.norm], int(cfg.causal), int(cfg.has_bias), int(cfg.residual),
+                        cfg.eps, cfg.softmax_scale)
+
+
+class Plan:
+    """One fbl_plan.  Methods carry the C entry points' names without the ``fbl_`` prefix."""
+
+    def __init__(self, desc: FblLayerDesc):
+        self._h = C.c_void_p()
+        self.desc = desc
+        _check(lib().fbl_plan_create(C.byref(desc), C.byref(self._h)))
+
+    def close(self):
+        if self._h:
+            lib().fbl_plan_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def tensor_bytes(self, tensor_id: int) -> int:
+        out = C.c_size_t()
+        _check(lib().fbl_tensor_bytes(self._h, tensor_id, C.byref(out)))
+        return out.value
+
+    def workspace_bytes(self):
+        a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
+        _check(lib().fbl_workspace_bytes(self._h, C.byref(a), C.byref(b), C.byref(c)))
+        return a.value, b.value, c.value
+
+    def tile_offset(self, tensor_id: int, idx) -> int:
+        arr = (C.c_int32 * 4)(*(list(idx) + [0] * (4 - len(idx))))
+        return lib().fbl_tile_offset(self._h, tensor_id, arr)
+
+    def tile_map(self, map_id: int, src_tile: int) -> int:
+        out = C.c_int64()
+        _check(lib().fbl_tile_map(self._h, map_id, src_tile, C.byref(out)))
+        return out.value
+
+    def set_kernel_path(self, path: int):
+        _check(lib().fbl_plan_set_kernel_path(self._h, path))
+
+    def pack(self, tensor_id, rowmajor_ptr, tiled_ptr, stream):
+        _check(lib().fbl_pack(self._h, tensor_id, rowmajor_ptr, tiled_ptr, stream))
+
+    def unpack(self, tensor_id, tiled_ptr, rowmajor_ptr, stream):
+        _check(lib().fbl_unpack(self._h, tensor_id, tiled_ptr, rowmajor_ptr, stream))
+
+    def layer_fwd(self, X, gamma, beta, Wq, Wk, Wv, Wo, bq, bk, bv, bo, Y, saved, scratch, stream):
+        _check(lib().fbl_layer_fwd(self._h, X, gamma, beta, Wq, Wk, Wv, Wo, bq, bk, bv, bo, Y, saved, scratch, stream))
+
+    def layer_bwd(self, dY, X, gamma, Wq, Wk, Wv, Wo, saved, dX, dWq, dWk, dWv, dWo, dbq, dbk, dbv, dbo, dgamma,
+                  dbeta, scratch, stream):
+        _check(lib().fbl_layer_bwd(self._h, dY, X, gamma, Wq, Wk, Wv, Wo, saved, dX, dWq, dWk, dWv, dWo, dbq, dbk,
+                                   dbv, dbo, dgamma, dbeta, scratch, stream))
+
+    def colsum_scratch_bytes(self, rows, cols) -> int:
+        out = C.c_size_t()
+        _check(lib().fbl_colsum_scratch_bytes(self._h, rows, cols, C.byref(out)))
+        return out.value
+
+    def colsum(self, M, rows, cols, out, scratch, stream):
+        _check(lib().fbl_colsum(self._h, M, rows, cols, out, scratch, stream))
+
+    def status_poll(self, scratch) -> int:
+        out = C.c_int32()
+        code = lib().fbl_status_poll(self._h, scratch, C.byref(out))
+        if code not in (0, -6):
+            _check(code)
+        return out.value
+
+
+class LayerRunner:
+    """Device buffers for one layer plus pack/step/unpack helpers (torch for memory and streams only)."""
+
+    MATS = {"X": "X", "dY": "DY", "Wq": "WQ", "Wk": "WK", "Wv": "WV", "Wo": "WO"}
+    OUT_MATS = {"Y": "Y", "dX": "DX", "dWq": "WQ", "dWk": "WK", "dWv": "WV", "dWo": "WO"}
+
+    def __init__(self, cfg, device="cuda:0"):
+        import torch
+        if not torch.cuda.is_available():
+            raise FblError(-101, "no CUDA device: the layer has no CPU path")
+        self.torch = torch
+        self.cfg = cfg
+        self.dev = torch.device(device)
+        self.plan = Plan(desc_from_config(cfg))
+        self.tdtype = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
+        saved, sf, sb = self.plan.workspace_bytes()
+        self.sizes = dict(saved=saved, scratch_fwd=sf, scratch_bwd=sb)
+        al = lambda nbytes: torch.zeros(nbytes, dtype=torch.uint8, device=self.dev)
+        self.saved = al(saved)
+        self.scratch = al(max(sf, sb))
+        self.buf = {}
+        for name, tid in {**self.MATS, **self.OUT_MATS}.items():
+            self.buf[name] = al(self.plan.tensor_bytes(TENSOR[tid]))
+        d, dq, dkv = cfg.d_model, cfg.d_q, cfg.d_kv
+        fz = lambda n: torch.zeros(n, dtype=torch.float32, device=self.dev)
+        self.vec = {"gamma": fz(d), "beta": fz(d), "bq": fz(dq), "bk": fz(dkv), "bv": fz(dkv), "bo": fz(d),
+                    "dgamma": fz(d), "dbeta": fz(d), "dbq": fz(dq), "dbk": fz(dkv), "dbv": fz(dkv), "dbo": fz(d)}
+
+    # -- helpers ---------------------------------------------------------------------------
+    def _stream(self):
+        return self.torch.cuda.current_stream(self.dev).cuda_stream
+
+    def _shape(self, name):
+        c = self.cfg
+        return {"X": (c.batch, c.seq, c.d_model), "dY": (c.batch, c.seq, c.d_model), "Y": (c.batch, c.seq, c.d_model),
+                "dX": (c.batch, c.seq, c.d_model), "Wq": (c.d_model, c.d_q), "Wk": (c.d_model, c.d_kv),
+                "Wv": (c.d_model, c.d_kv), "Wo": (c.d_q, c.d_model), "dWq": (c.d_model, c.d_q),
+                "dWk": (c.d_model, c.d_kv), "dWv": (c.d_model, c.d_kv), "dWo": (c.d_q, c.d_model)}[name]
+
+    def to_device_rowmajor(self, arr):
+        """numpy float64/float32 array of storage-representable values -> torch tensor in the storage dtype."""
+        t = self.torch.from_numpy(arr.astype("float32"))
+        return t.to(self.dev).to(self.tdtype).contiguous()
+
+    def load_inputs(self, inp):
+        """Pack the row-major inputs of ``fbl_inputs.make_inputs`` into R-Tile device buffers."""
+        for name, tid in self.MATS.items():
+            rm = self.to_device_rowmajor(inp[name])
+            self.plan.pack(TENSOR[tid], rm.data_ptr(), self.buf[name].data_ptr(), self._stream())
+        for name in ("gamma", "beta", "bq", "bk", "bv", "bo"):
+            if inp.get(name) is not None:
+                self.vec[name].copy_(self.torch.from_numpy(inp[name].astype("float32")))
+        self.torch.cuda.synchronize(self.dev)
+
+    def forward(self):
+        c, b, v = self.cfg, self.buf, self.vec
+        ptr = lambda t: t.data_ptr()
+        bias = c.has_bias
+        self.plan.layer_fwd(ptr(b["X"]), ptr(v["gamma"]), ptr(v["beta"]) if c.norm == "layernorm" else None,
+                            ptr(b["Wq"]), ptr(b["Wk"]), ptr(b["Wv"]), ptr(b["Wo"]),
+                            ptr(v["bq"]) if bias else None, ptr(v["bk"]) if bias else None,
+                            ptr(v["bv"]) if bias else None, ptr(v["bo"]) if bias else None,
+                            ptr(b["Y"]), ptr(self.saved), ptr(self.scratch), self._stream())
+
+    def backward(self):
+        c, b, v = self.cfg, self.buf, self.vec
+        ptr = lambda t: t.data_ptr()
+        bias = c.has_bias
+        self.plan.layer_bwd(ptr(b["dY"]), ptr(b["X"]), ptr(v["gamma"]), ptr(b["Wq"]), ptr(b["Wk"]), ptr(b["Wv"]),
+                            ptr(b["Wo"]), ptr(self.saved), ptr(b["dX"]), ptr(b["dWq"]), ptr(b["dWk"]), ptr(b["dWv"]),
+                            ptr(b["dWo"]), ptr(v["dbq"]) if bias else None, ptr(v["dbk"]) if bias else None,
+                            ptr(v["dbv"]) if bias else None, ptr(v["dbo"]) if bias else None, ptr(v["dgamma"]),
+                            ptr(v["dbeta"]) if c.norm == "layernorm" else None, ptr(self.scratch), self._stream())
+
+    def step(self):
+        self.forward()
+        self.backward()
+
+    def fetch(self, name):
+        """Unpack one output matrix to a row-major float64 numpy array (or copy a vector)."""
+        torch = self.torch
+        if name in self.OUT_MATS:
+            shape = self._shape(name)
+            out = torch.empty(shape, dtype=self.tdtype, device=self.dev)
+            self.plan.unpack(TENSOR[self.OUT_MATS[name]], self.buf[name].data_ptr(), out.data_ptr(), self._stream())
+            torch.cuda.synchronize(self.dev)
+            return out.float().cpu().numpy().astype("float64")
+        torch.cuda.synchronize(self.dev)
+        return self.vec[name].cpu().numpy().astype("float64")
+
+    def saved_view(self, name):
+        """Raw R-Tile bytes of a saved matrix (Xn, Q, K, V, A) as a flat torch tensor in the storage dtype."""
+        raise NotImplementedError
+
+    def status(self) -> int:
+        self.torch.cuda.synchronize(self.dev)
+        return self.plan.status_poll(self.scratch.data_ptr())

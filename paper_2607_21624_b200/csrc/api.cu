@@ -1,0 +1,405 @@
+// C ABI: plan construction, the host-side integer index maps, and the forward/backward drivers.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "fbl_internal.h"
+
+namespace {
+
+inline int64_t up8(int64_t v) { return (v + 7) / 8 * 8; }
+
+struct MatShape { int64_t outer, rows, rows_pad; int cols; };   // rows_pad per outer slice
+
+bool mat_shape(const fbl_plan* p, int id, MatShape* s) {
+  const fbl_layer_desc& d = p->d;
+  switch (id) {
+    case FBL_T_X: case FBL_T_Y: case FBL_T_DY: case FBL_T_DX: case FBL_T_XN:
+      *s = {d.batch, d.seq, p->t_pad, d.d_model}; return true;
+    case FBL_T_Q: case FBL_T_A: case FBL_T_Q_HEADS: case FBL_T_A_HEADS:
+      *s = {d.batch, d.seq, p->t_pad, p->dq}; return true;
+    case FBL_T_K: case FBL_T_V: case FBL_T_K_HEADS: case FBL_T_V_HEADS:
+      *s = {d.batch, d.seq, p->t_pad, p->dkv}; return true;
+    case FBL_T_WQ: case FBL_T_WQ_T: *s = {1, d.d_model, up8(d.d_model), p->dq}; return true;
+    case FBL_T_WK: case FBL_T_WV: case FBL_T_WK_T: case FBL_T_WV_T:
+      *s = {1, d.d_model, up8(d.d_model), p->dkv}; return true;
+    case FBL_T_WO: case FBL_T_WO_T: *s = {1, p->dq, up8(p->dq), d.d_model}; return true;
+    default: return false;
+  }
+}
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & (FBL_ALIGN - 1)) != 0; }
+
+thread_local char g_detail[256] = "";
+
+#define FBL_CUDA(expr)                                  \
+  do {                                                  \
+    cudaError_t e__ = (expr);                           \
+    if (e__ != cudaSuccess) {                           \
+      fbl_note_cuda_error(e__, #expr);                  \
+      return FBL_ERR_CUDA;                              \
+    }                                                   \
+  } while (0)
+
+cudaError_t run_gemm(const fbl_plan* p, const GemmArgs& g, void* sk, size_t sk_bytes, int32_t* status,
+                     cudaStream_t st) {
+  if (p->use_tc && gemm_tc_supported(p, g)) return launch_gemm_tc(p, g, sk, sk_bytes, status, st);
+  return launch_gemm_simt(p->d.dtype, g, st);
+}
+
+}  // namespace
+
+void fbl_note_cuda_error(cudaError_t e, const char* where) {
+  snprintf(g_detail, sizeof(g_detail), "%s: %s", cudaGetErrorString(e), where);
+}
+
+extern "C" {
+
+const char* fbl_last_error_detail(void) { return g_detail; }
+
+int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
+  if (!desc || !out) return FBL_ERR_INVALID_ARG;
+  *out = nullptr;
+  const fbl_layer_desc& d = *desc;
+  if (d.batch <= 0 || d.seq <= 0 || d.d_model <= 0 || d.n_q_heads <= 0 || d.n_kv_heads <= 0 || d.head_dim <= 0)
+    return FBL_ERR_INVALID_ARG;
+  if (d.dtype != FBL_DTYPE_FP32 && d.dtype != FBL_DTYPE_BF16) return FBL_ERR_INVALID_ARG;
+  if (d.norm != FBL_NORM_LAYERNORM && d.norm != FBL_NORM_RMSNORM) return FBL_ERR_INVALID_ARG;
+  if (!(d.eps >= 0.f)) return FBL_ERR_INVALID_ARG;
+  const int e = d.dtype == FBL_DTYPE_FP32 ? 4 : 2;
+  const int tw = 128 / e;
+  // Tile-propagation legality (section 4.3): the GQA head map needs whole groups; the head split
+  // must fall on tile boundaries (tile_w divides head_dim) and d_model must be whole tiles.
+  if (d.n_q_heads % d.n_kv_heads != 0) return FBL_ERR_UNSUPPORTED_SHAPE;
+  if (d.head_dim % tw != 0 || d.d_model % tw != 0) return FBL_ERR_UNSUPPORTED_SHAPE;
+  if (d.dtype == FBL_DTYPE_FP32 && d.head_dim != 32 && d.head_dim != 64 && d.head_dim != 128)
+    return FBL_ERR_UNSUPPORTED_SHAPE;
+  if (d.dtype == FBL_DTYPE_BF16 && d.head_dim != 64 && d.head_dim != 128) return FBL_ERR_UNSUPPORTED_SHAPE;
+  if ((int64_t)d.batch * up8(d.seq) > (int64_t)1 << 30) return FBL_ERR_UNSUPPORTED_SHAPE;
+  if (d.d_model > 16384 || (int64_t)d.n_q_heads * d.head_dim > 16384) return FBL_ERR_UNSUPPORTED_SHAPE;
+
+  fbl_plan* p = new (std::nothrow) fbl_plan();
+  if (!p) return FBL_ERR_INVALID_ARG;
+  p->d = d;
+  p->e = e;
+  p->tw = tw;
+  p->t_pad = (int)up8(d.seq);
+  p->n_pad = (int64_t)d.batch * p->t_pad;
+  p->dq = d.n_q_heads * d.head_dim;
+  p->dkv = d.n_kv_heads * d.head_dim;
+  p->group = d.n_q_heads / d.n_kv_heads;
+  p->scale = d.softmax_scale > 0.f ? d.softmax_scale : 1.0f / sqrtf((float)d.head_dim);
+  p->sm_count = 148;
+  p->use_tc = d.dtype == FBL_DTYPE_BF16 ? 1 : 0;
+
+  const size_t n = (size_t)p->n_pad;
+  auto mat = [&](size_t cols) { return fbl_align_up(n * cols * (size_t)e, FBL_ALIGN); };
+  const size_t rows_bh = (size_t)d.batch * d.n_q_heads * p->t_pad;
+  size_t o = 0;
+  p->sv_stats = o; o += fbl_align_up(n * 2 * sizeof(float), FBL_ALIGN);
+  p->sv_xn = o;    o += mat(d.d_model);
+  p->sv_q = o;     o += mat(p->dq);
+  p->sv_k = o;     o += mat(p->dkv);
+  p->sv_v = o;     o += mat(p->dkv);
+  p->sv_a = o;     o += mat(p->dq);
+  p->sv_lse = o;   o += fbl_align_up(rows_bh * sizeof(float), FBL_ALIGN);
+  p->saved_bytes = o;
+
+  // partial-sum area: column-sum slabs or split-K slices, whichever is larger
+  size_t part = colsum_scratch_bytes(p->n_pad, d.d_model > p->dq ? d.d_model : p->dq);
+  const size_t splitk = (size_t)p->sm_count * 128 * 256 * sizeof(float) * 2;
+  if (splitk > part) part = splitk;
+  p->part_bytes = fbl_align_up(part, FBL_ALIGN);
+
+  o = FBL_ALIGN;  // status word
+  p->sf_part = o; o += p->part_bytes;
+  p->scratch_fwd_bytes = o;
+
+  o = FBL_ALIGN;
+  p->sb_da = o;    o += mat(p->dq);
+  p->sb_dvec = o;  o += fbl_align_up(rows_bh * sizeof(float), FBL_ALIGN);
+  p->sb_dqacc = o; o += fbl_align_up(n * p->dq * sizeof(float), FBL_ALIGN);
+  p->sb_dq = o;    o += mat(p->dq);
+  p->sb_dk = o;    o += mat(p->dkv);
+  p->sb_dv = o;    o += mat(p->dkv);
+  p->sb_dxn = o;   o += mat(d.d_model);
+  p->sb_part = o;  o += p->part_bytes;
+  p->scratch_bwd_bytes = o;
+  *out = p;
+  return FBL_OK;
+}
+
+void fbl_plan_destroy(fbl_plan* plan) { delete plan; }
+
+int fbl_plan_set_kernel_path(fbl_plan* plan, int path) {
+  if (!plan || (path != 0 && path != 1)) return FBL_ERR_INVALID_ARG;
+  plan->use_tc = (path == 0 && plan->d.dtype == FBL_DTYPE_BF16) ? 1 : 0;
+  return FBL_OK;
+}
+
+int fbl_tensor_bytes(const fbl_plan* plan, int tensor_id, size_t* bytes) {
+  MatShape s;
+  if (!plan || !bytes || !mat_shape(plan, tensor_id, &s)) return FBL_ERR_INVALID_ARG;
+  *bytes = (size_t)(s.outer * s.rows_pad) * s.cols * plan->e;
+  return FBL_OK;
+}
+
+int fbl_workspace_bytes(const fbl_plan* plan, size_t* saved, size_t* scratch_fwd, size_t* scratch_bwd) {
+  if (!plan) return FBL_ERR_INVALID_ARG;
+  if (saved) *saved = plan->saved_bytes;
+  if (scratch_fwd) *scratch_fwd = plan->scratch_fwd_bytes;
+  if (scratch_bwd) *scratch_bwd = plan->scratch_bwd_bytes;
+  return FBL_OK;
+}
+
+int64_t fbl_tile_offset(const fbl_plan* plan, int tensor_id, const int32_t idx[4]) {
+  MatShape s;
+  if (!plan || !idx || !mat_shape(plan, tensor_id, &s)) return -1;
+  const fbl_layer_desc& d = plan->d;
+  int64_t r, c;
+  switch (tensor_id) {
+    case FBL_T_Q_HEADS: case FBL_T_A_HEADS: case FBL_T_K_HEADS: case FBL_T_V_HEADS: {
+      const int heads = (tensor_id == FBL_T_K_HEADS || tensor_id == FBL_T_V_HEADS) ? d.n_kv_heads : d.n_q_heads;
+      if (idx[0] < 0 || idx[0] >= d.batch || idx[1] < 0 || idx[1] >= heads || idx[2] < 0 || idx[2] >= d.seq ||
+          idx[3] < 0 || idx[3] >= d.head_dim) return -1;
+      r = (int64_t)idx[0] * plan->t_pad + idx[2];
+      c = (int64_t)idx[1] * d.head_dim + idx[3];
+      break;
+    }
+    case FBL_T_WQ_T: case FBL_T_WK_T: case FBL_T_WV_T: case FBL_T_WO_T:
+      if (idx[0] < 0 || idx[0] >= s.cols || idx[1] < 0 || idx[1] >= s.rows) return -1;
+      r = idx[1]; c = idx[0];
+      break;
+    case FBL_T_WQ: case FBL_T_WK: case FBL_T_WV: case FBL_T_WO:
+      if (idx[0] < 0 || idx[0] >= s.rows || idx[1] < 0 || idx[1] >= s.cols) return -1;
+      r = idx[0]; c = idx[1];
+      break;
+    default:
+      if (idx[0] < 0 || idx[0] >= s.outer || idx[1] < 0 || idx[1] >= s.rows || idx[2] < 0 || idx[2] >= s.cols)
+        return -1;
+      r = (int64_t)idx[0] * s.rows_pad + idx[1];
+      c = idx[2];
+  }
+  return rt_off_dyn(plan->tw, s.outer * s.rows_pad, r, c);
+}
+
+int fbl_tile_map(const fbl_plan* plan, int map_id, int64_t src, int64_t* dst) {
+  if (!plan || !dst || src < 0) return FBL_ERR_INVALID_ARG;
+  const fbl_layer_desc& d = plan->d;
+  const int64_t rt = plan->n_pad / 8;            // row tiles of a token matrix
+  const int64_t st = plan->t_pad / 8;            // row tiles per sequence
+  const int64_t hw = d.head_dim / plan->tw;      // tiles across one head
+  switch (map_id) {
+    case FBL_MAP_SPLIT_Q: case FBL_MAP_SPLIT_KV: case FBL_MAP_MERGE_Q: case FBL_MAP_MERGE_KV: {
+      const int64_t heads = (map_id == FBL_MAP_SPLIT_Q || map_id == FBL_MAP_MERGE_Q) ? d.n_q_heads : d.n_kv_heads;
+      const int64_t ct = heads * hw;
+      if (src >= rt * ct) return FBL_ERR_INVALID_ARG;
+      if (map_id == FBL_MAP_SPLIT_Q || map_id == FBL_MAP_SPLIT_KV) {
+        // f = (transpose S<->H) o (reshape D -> H x HD), on tile coordinates; the inner modulo chain
+        // (src mod ct) mod hw collapses to src mod hw because hw divides ct (the paper's identity).
+        const int64_t tr = src / ct, td = src % hw, h = (src % ct) / hw;
+        const int64_t b = tr / st, ts = tr % st;
+        *dst = ((b * heads + h) * st + ts) * hw + td;
+      } else {
+        const int64_t td = src % hw, ts = (src / hw) % st, bh = src / (hw * st);
+        const int64_t b = bh / heads, h = bh % heads;
+        *dst = (b * st + ts) * ct + h * hw + td;
+      }
+      return FBL_OK;
+    }
+    case FBL_MAP_TRANSPOSE_WQ: case FBL_MAP_TRANSPOSE_WO: {
+      const int64_t rows = map_id == FBL_MAP_TRANSPOSE_WQ ? d.d_model : plan->dq;
+      const int64_t cols = map_id == FBL_MAP_TRANSPOSE_WQ ? plan->dq : d.d_model;
+      const int64_t trs = up8(rows) / 8, tcs = cols / plan->tw;
+      if (src >= trs * tcs) return FBL_ERR_INVALID_ARG;
+      *dst = (src % tcs) * trs + src / tcs;
+      return FBL_OK;
+    }
+    case FBL_MAP_PHYS_Q: {
+      const int64_t ct = d.n_q_heads * hw;
+      if (src >= rt * ct) return FBL_ERR_INVALID_ARG;
+      *dst = (src % ct) * rt + src / ct;
+      return FBL_OK;
+    }
+    case FBL_MAP_PHYS_WQ: {
+      const int64_t trs = up8(d.d_model) / 8, tcs = plan->dq / plan->tw;
+      if (src >= trs * tcs) return FBL_ERR_INVALID_ARG;
+      *dst = (src % tcs) * trs + src / tcs;
+      return FBL_OK;
+    }
+    default: return FBL_ERR_INVALID_ARG;
+  }
+}
+
+static int pack_common(const fbl_plan* plan, int tensor_id, const void* src, void* dst, void* stream, int unpack) {
+  MatShape s;
+  if (!plan || !src || !dst || !mat_shape(plan, tensor_id, &s)) return FBL_ERR_INVALID_ARG;
+  if (tensor_id >= FBL_T_Q_HEADS) return FBL_ERR_INVALID_ARG;   // views are not separate buffers
+  if (misaligned(unpack ? src : dst)) return FBL_ERR_MISALIGNED;
+  FBL_CUDA(launch_pack(plan->d.dtype, unpack, src, dst, s.outer, s.rows, s.rows_pad, s.cols, as_stream(stream)));
+  return FBL_OK;
+}
+int fbl_pack(const fbl_plan* plan, int tensor_id, const void* rowmajor_dev, void* tiled_dev, void* stream) {
+  return pack_common(plan, tensor_id, rowmajor_dev, tiled_dev, stream, 0);
+}
+int fbl_unpack(const fbl_plan* plan, int tensor_id, const void* tiled_dev, void* rowmajor_dev, void* stream) {
+  return pack_common(plan, tensor_id, tiled_dev, rowmajor_dev, stream, 1);
+}
+
+int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const float* beta, const void* Wq,
+                  const void* Wk, const void* Wv, const void* Wo, const float* bq, const float* bk, const float* bv,
+                  const float* bo, void* Y, void* saved, void* scratch, void* stream) {
+  if (!p || !X || !gamma || !Wq || !Wk || !Wv || !Wo || !Y || !saved || !scratch) return FBL_ERR_INVALID_ARG;
+  if (p->d.has_bias && (!bq || !bk || !bv || !bo)) return FBL_ERR_INVALID_ARG;
+  if (p->d.norm == FBL_NORM_LAYERNORM && !beta) return FBL_ERR_INVALID_ARG;
+  const void* ptrs[] = {X, Wq, Wk, Wv, Wo, Y, saved, scratch};
+  for (const void* q : ptrs) if (misaligned(q)) return FBL_ERR_MISALIGNED;
+  cudaStream_t st = as_stream(stream);
+  char* sv = (char*)saved;
+  char* sc = (char*)scratch;
+  int32_t* status = (int32_t*)sc;
+  float* stats = (float*)(sv + p->sv_stats);
+  void* Xn = sv + p->sv_xn; void* Q = sv + p->sv_q; void* K = sv + p->sv_k; void* V = sv + p->sv_v;
+  void* A = sv + p->sv_a; float* lse = (float*)(sv + p->sv_lse);
+  void* part = sc + p->sf_part;
+  const bool bias = p->d.has_bias;
+  const int n = (int)p->n_pad, D = p->d.d_model;
+
+  FBL_CUDA(cudaMemsetAsync(status, 0, FBL_ALIGN, st));
+  FBL_CUDA(launch_norm_fwd(p, X, gamma, beta, Xn, stats, st));
+  {
+    const void* W[3] = {Wq, Wk, Wv};
+    void* O[3] = {Q, K, V};
+    const float* B[3] = {bq, bk, bv};
+    const int cols[3] = {p->dq, p->dkv, p->dkv};
+    for (int i = 0; i < 3; ++i) {
+      GemmArgs g = {};
+      g.m = n; g.n = cols[i]; g.n_terms = 1;
+      g.t[0] = {Xn, p->n_pad, 0, W[i], D, 0, D};
+      g.c = O[i]; g.c_rpad = p->n_pad; g.bias = bias ? B[i] : nullptr;
+      g.seq = p->d.seq; g.t_pad = p->t_pad;
+      FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
+    }
+  }
+  if (p->use_tc && attn_fwd_tc_supported(p)) FBL_CUDA(launch_attn_fwd_tc(p, Q, K, V, A, lse, status, st));
+  else FBL_CUDA(launch_attn_fwd_simt(p, Q, K, V, A, lse, st));
+  {
+    GemmArgs g = {};
+    g.m = n; g.n = D; g.n_terms = 1;
+    g.t[0] = {A, p->n_pad, 0, Wo, p->dq, 0, p->dq};
+    g.c = Y; g.c_rpad = p->n_pad; g.bias = bias ? bo : nullptr;
+    g.residual = p->d.residual ? X : nullptr;
+    g.seq = p->d.seq; g.t_pad = p->t_pad;
+    FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
+  }
+  return FBL_OK;
+}
+
+int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float* gamma, const void* Wq,
+                  const void* Wk, const void* Wv, const void* Wo, const void* saved, void* dX, void* dWq, void* dWk,
+                  void* dWv, void* dWo, float* dbq, float* dbk, float* dbv, float* dbo, float* dgamma, float* dbeta,
+                  void* scratch, void* stream) {
+  if (!p || !dY || !X || !gamma || !Wq || !Wk || !Wv || !Wo || !saved || !dX || !dWq || !dWk || !dWv || !dWo ||
+      !dgamma || !scratch)
+    return FBL_ERR_INVALID_ARG;
+  if (p->d.has_bias && (!dbq || !dbk || !dbv || !dbo)) return FBL_ERR_INVALID_ARG;
+  if (p->d.norm == FBL_NORM_LAYERNORM && !dbeta) return FBL_ERR_INVALID_ARG;
+  const void* ptrs[] = {dY, X, Wq, Wk, Wv, Wo, saved, dX, dWq, dWk, dWv, dWo, scratch};
+  for (const void* q : ptrs) if (misaligned(q)) return FBL_ERR_MISALIGNED;
+  cudaStream_t st = as_stream(stream);
+  const char* sv = (const char*)saved;
+  char* sc = (char*)scratch;
+  int32_t* status = (int32_t*)sc;
+  const float* stats = (const float*)(sv + p->sv_stats);
+  const void* Xn = sv + p->sv_xn; const void* Q = sv + p->sv_q; const void* K = sv + p->sv_k;
+  const void* V = sv + p->sv_v; const void* A = sv + p->sv_a; const float* lse = (const float*)(sv + p->sv_lse);
+  void* dA = sc + p->sb_da; float* dvec = (float*)(sc + p->sb_dvec); float* dqacc = (float*)(sc + p->sb_dqacc);
+  void* dQ = sc + p->sb_dq; void* dK = sc + p->sb_dk; void* dV = sc + p->sb_dv; void* dXn = sc + p->sb_dxn;
+  void* part = sc + p->sb_part;
+  const bool bias = p->d.has_bias;
+  const int n = (int)p->n_pad, D = p->d.d_model;
+
+  FBL_CUDA(cudaMemsetAsync(status, 0, FBL_ALIGN, st));
+  {  // dA = dY Wo^T : Wo's tiles read with the roles of its two axes swapped
+    GemmArgs g = {};
+    g.m = n; g.n = p->dq; g.n_terms = 1;
+    g.t[0] = {dY, p->n_pad, 0, Wo, p->dq, 1, D};
+    g.c = dA; g.c_rpad = p->n_pad; g.seq = p->d.seq; g.t_pad = p->t_pad;
+    FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
+  }
+  {  // dWo = A^T dY : token-axis reduction
+    GemmArgs g = {};
+    g.m = p->dq; g.n = D; g.n_terms = 1;
+    g.t[0] = {A, p->n_pad, 1, dY, p->n_pad, 0, n};
+    g.c = dWo; g.c_rpad = p->dq;
+    FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
+  }
+  if (bias) FBL_CUDA(launch_colsum(p->d.dtype, dY, p->n_pad, D, dbo, (float*)part, st));
+  if (p->use_tc && attn_bwd_tc_supported(p)) FBL_CUDA(launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, status, st));
+  else FBL_CUDA(launch_attn_bwd_simt(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, st));
+  {  // dXn = dQ Wq^T + dK Wk^T + dV Wv^T : one accumulator, three reduction loops
+    GemmArgs g = {};
+    g.m = n; g.n = D; g.n_terms = 3;
+    g.t[0] = {dQ, p->n_pad, 0, Wq, D, 1, p->dq};
+    g.t[1] = {dK, p->n_pad, 0, Wk, D, 1, p->dkv};
+    g.t[2] = {dV, p->n_pad, 0, Wv, D, 1, p->dkv};
+    g.c = dXn; g.c_rpad = p->n_pad; g.seq = p->d.seq; g.t_pad = p->t_pad;
+    FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
+  }
+  {
+    const void* G[3] = {dQ, dK, dV};
+    void* DW[3] = {dWq, dWk, dWv};
+    float* DB[3] = {dbq, dbk, dbv};
+    const int cols[3] = {p->dq, p->dkv, p->dkv};
+    for (int i = 0; i < 3; ++i) {
+      GemmArgs g = {};
+      g.m = D; g.n = cols[i]; g.n_terms = 1;
+      g.t[0] = {Xn, p->n_pad, 1, G[i], p->n_pad, 0, n};
+      g.c = DW[i]; g.c_rpad = D;
+      FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
+      if (bias) FBL_CUDA(launch_colsum(p->d.dtype, G[i], p->n_pad, cols[i], DB[i], (float*)part, st));
+    }
+  }
+  FBL_CUDA(launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, st));
+  return FBL_OK;
+}
+
+int fbl_colsum_scratch_bytes(const fbl_plan* plan, int64_t rows, int64_t cols, size_t* bytes) {
+  if (!plan || !bytes || rows <= 0 || cols <= 0 || rows % 8 != 0 || cols % plan->tw != 0) return FBL_ERR_INVALID_ARG;
+  *bytes = colsum_scratch_bytes(rows, cols);
+  return FBL_OK;
+}
+
+int fbl_colsum(const fbl_plan* plan, const void* M_dev, int64_t rows, int64_t cols, float* out_dev, void* scratch_dev,
+               void* stream) {
+  if (!plan || !M_dev || !out_dev || !scratch_dev || rows <= 0 || cols <= 0 || rows % 8 != 0 || cols % plan->tw != 0)
+    return FBL_ERR_INVALID_ARG;
+  if (misaligned(M_dev)) return FBL_ERR_MISALIGNED;
+  FBL_CUDA(launch_colsum(plan->d.dtype, M_dev, rows, cols, out_dev, (float*)scratch_dev, as_stream(stream)));
+  return FBL_OK;
+}
+
+int fbl_status_poll(const fbl_plan* plan, const void* scratch, int32_t* device_status) {
+  if (!plan || !scratch || !device_status) return FBL_ERR_INVALID_ARG;
+  FBL_CUDA(cudaMemcpy(device_status, scratch, sizeof(int32_t), cudaMemcpyDeviceToHost));
+  return *device_status == 0 ? FBL_OK : FBL_ERR_TIMEOUT;
+}
+
+const char* fbl_strerror(int status) {
+  switch (status) {
+    case FBL_OK: return "ok";
+    case FBL_ERR_INVALID_ARG: return "invalid argument";
+    case FBL_ERR_UNSUPPORTED_SHAPE: return "shape not supported by the tiled layout or the kernels";
+    case FBL_ERR_MISALIGNED: return "matrix pointer is not 1024-byte aligned";
+    case FBL_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case FBL_ERR_CUDA: return "CUDA runtime error";
+    case FBL_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,96 @@
+// Internal declarations shared by the translation units of libfblayout.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fblayout.h"
+
+#define FBL_TILE_H 8
+#define FBL_ALIGN 1024
+
+// ---------------------------------------------------------------------------------------------
+// R-Tile element map (section 4.2).  Storage tile = 8 rows x 128 bytes, row-major inside; tiles
+// ordered with the row-tile index fastest.  TW = elements per 128-byte tile row.
+// ---------------------------------------------------------------------------------------------
+template <int TW>
+__host__ __device__ __forceinline__ int64_t rt_off(int64_t r_pad, int64_t r, int c) {
+  return ((int64_t)(c / TW) * r_pad + r) * TW + (c % TW);
+}
+__host__ __device__ __forceinline__ int64_t rt_off_dyn(int tw, int64_t r_pad, int64_t r, int64_t c) {
+  return ((c / tw) * r_pad + r) * tw + (c % tw);
+}
+
+template <typename T> struct tile_w_of { static constexpr int value = 128 / (int)sizeof(T); };
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+struct fbl_plan {
+  fbl_layer_desc d;
+  int e;        // bytes per element
+  int tw;       // tile_w in elements
+  int t_pad;    // seq rounded up to 8
+  int64_t n_pad;  // batch * t_pad
+  int dq, dkv, group;
+  float scale;
+  int sm_count;
+  int use_tc;   // 1: tensor-core (tcgen05) kernels where one exists for the shape; 0: FFMA kernels only
+  // byte offsets inside `saved`
+  size_t sv_stats, sv_xn, sv_q, sv_k, sv_v, sv_a, sv_lse, saved_bytes;
+  // byte offsets inside the backward scratch
+  size_t sb_da, sb_dvec, sb_dqacc, sb_dq, sb_dk, sb_dv, sb_dxn, sb_part, scratch_bwd_bytes;
+  size_t sf_part, scratch_fwd_bytes;
+  size_t part_bytes;
+};
+
+static inline size_t fbl_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---------------------------------------------------------------------------------------------
+// Kernel launchers (all asynchronous on `st`; return a cudaError_t from the launch).
+// ---------------------------------------------------------------------------------------------
+struct GemmTerm {
+  const void* a; int64_t a_rpad; int a_trans;   // logical A[m,k]; a_trans: stored as [k rows][m cols]
+  const void* b; int64_t b_rpad; int b_trans;   // logical B[k,n]; b_trans: stored as [n rows][k cols]
+  int k;
+};
+struct GemmArgs {
+  int m, n, n_terms;
+  GemmTerm t[3];
+  void* c; int64_t c_rpad;        // C[m,n] stored [m rows][n cols]
+  const float* bias;              // per output column, or nullptr
+  const void* residual;           // same layout as C, or nullptr
+  int seq, t_pad;                 // if t_pad > 0: rows with (row % t_pad) >= seq are written as zero
+};
+
+cudaError_t launch_gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);
+cudaError_t launch_gemm_tc(const fbl_plan* p, const GemmArgs& g, void* splitk_scratch, size_t splitk_bytes,
+                           int32_t* status, cudaStream_t st);
+bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g);
+bool attn_fwd_tc_supported(const fbl_plan* p);
+bool attn_bwd_tc_supported(const fbl_plan* p);
+void fbl_note_cuda_error(cudaError_t e, const char* where);
+
+cudaError_t launch_pack(int dtype, int unpack, const void* src, void* dst, int64_t outer, int64_t rows,
+                        int64_t rows_pad, int cols, cudaStream_t st);
+cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
+                            float* stats, cudaStream_t st);
+cudaError_t launch_norm_bwd(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
+                            const float* gamma, void* dX, float* dgamma, float* dbeta, cudaStream_t st);
+cudaError_t launch_colsum(int dtype, const void* M, int64_t rows, int64_t cols, float* out, float* partials,
+                          cudaStream_t st);
+size_t colsum_scratch_bytes(int64_t rows, int64_t cols);
+
+cudaError_t launch_attn_fwd_simt(const fbl_plan* p, const void* Q, const void* K, const void* V, void* A, float* lse,
+                                 cudaStream_t st);
+cudaError_t launch_attn_bwd_simt(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* A,
+                                 const void* dA, const float* lse, float* dvec, float* dqacc, void* dQ, void* dK,
+                                 void* dV, cudaStream_t st);
+cudaError_t launch_attn_fwd_tc(const fbl_plan* p, const void* Q, const void* K, const void* V, void* A, float* lse,
+                               int32_t* status, cudaStream_t st);
+cudaError_t launch_attn_bwd_tc(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* A,
+                               const void* dA, const float* lse, float* dvec, float* dqacc, void* dQ, void* dK,
+                               void* dV, int32_t* status, cudaStream_t st);

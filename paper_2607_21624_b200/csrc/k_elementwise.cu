@@ -1,0 +1,326 @@
+// HBM-bound kernels on R-Tile matrices: pack/unpack, norm forward/backward, token-axis column sums.
+// Thread mapping shared by all of them: 8 consecutive lanes cover one 128-byte tile row with one
+// 16-byte vector each, 4 rows per warp are 512 contiguous bytes, so every warp-level access is a
+// run of whole 128-byte lines.
+#include "fbl_internal.h"
+
+namespace {
+
+template <typename T> struct Vec16 { static constexpr int N = 16 / (int)sizeof(T); };
+
+template <typename T>
+__device__ __forceinline__ void load16(const T* p, float (&v)[Vec16<T>::N]) {
+  uint4 raw = *reinterpret_cast<const uint4*>(p);
+  const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+  for (int i = 0; i < Vec16<T>::N; ++i) v[i] = to_f(e[i]);
+}
+template <typename T>
+__device__ __forceinline__ void store16(T* p, const float (&v)[Vec16<T>::N]) {
+  uint4 raw;
+  T* e = reinterpret_cast<T*>(&raw);
+#pragma unroll
+  for (int i = 0; i < Vec16<T>::N; ++i) e[i] = from_f<T>(v[i]);
+  *reinterpret_cast<uint4*>(p) = raw;
+}
+
+__device__ __forceinline__ float group8_sum(float v) {
+  v += __shfl_xor_sync(0xffffffffu, v, 1);
+  v += __shfl_xor_sync(0xffffffffu, v, 2);
+  v += __shfl_xor_sync(0xffffffffu, v, 4);
+  return v;
+}
+
+// ------------------------------------------------------------------------------------------
+// pack / unpack: the only layout conversions, used at the graph boundary.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void pack_kernel(const T* __restrict__ src, T* __restrict__ dst, int64_t outer, int64_t rows,
+                            int64_t rows_pad, int cols, int64_t total) {
+  constexpr int TW = tile_w_of<T>::value;
+  const int64_t r_pad = outer * rows_pad;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    int64_t panel = i / (r_pad * TW);
+    int64_t rem = i - panel * r_pad * TW;
+    int64_t r = rem / TW;
+    int c = (int)(panel * TW + rem % TW);
+    int64_t o = r / rows_pad, row = r - o * rows_pad;
+    T v = from_f<T>(0.f);
+    if (row < rows) v = src[(o * rows + row) * cols + c];
+    dst[i] = v;
+  }
+}
+
+template <typename T>
+__global__ void unpack_kernel(const T* __restrict__ src, T* __restrict__ dst, int64_t outer, int64_t rows,
+                              int64_t rows_pad, int cols, int64_t total) {
+  constexpr int TW = tile_w_of<T>::value;
+  const int64_t r_pad = outer * rows_pad;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    int64_t orow = i / cols;
+    int c = (int)(i - orow * cols);
+    int64_t o = orow / rows, row = orow - o * rows;
+    dst[i] = src[rt_off<TW>(r_pad, o * rows_pad + row, c)];
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Pre-norm forward: row (feature-axis) reductions.  32 token rows per block.
+// stats[2r] = mean (0 for RMSNorm), stats[2r+1] = rstd.  Padding rows get zeros.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) norm_fwd_kernel(const T* __restrict__ X, const float* __restrict__ gamma,
+                                                       const float* __restrict__ beta, T* __restrict__ Xn,
+                                                       float* __restrict__ stats, int64_t n_pad, int d, int seq,
+                                                       int t_pad, int rms, float eps) {
+  constexpr int TW = tile_w_of<T>::value;
+  constexpr int V = Vec16<T>::N;
+  const int64_t r = (int64_t)blockIdx.x * 32 + threadIdx.x / 8;
+  const int l8 = threadIdx.x % 8;
+  if (r >= n_pad) return;                       // whole 8-lane groups leave together
+  const bool pad = (int)(r % t_pad) >= seq;
+  const int panels = d / TW;
+  float v[V];
+  float mean = 0.f;
+  if (!rms) {
+    float s = 0.f;
+    for (int p = 0; p < panels; ++p) {
+      load16(X + ((int64_t)p * n_pad + r) * TW + l8 * V, v);
+#pragma unroll
+      for (int i = 0; i < V; ++i) s += v[i];
+    }
+    mean = group8_sum(s) / (float)d;
+  }
+  float q = 0.f;
+  for (int p = 0; p < panels; ++p) {
+    load16(X + ((int64_t)p * n_pad + r) * TW + l8 * V, v);
+#pragma unroll
+    for (int i = 0; i < V; ++i) { float c = v[i] - mean; q += c * c; }
+  }
+  float rstd = rsqrtf(group8_sum(q) / (float)d + eps);
+  if (pad) { mean = 0.f; rstd = 0.f; }
+  if (l8 == 0) { stats[2 * r] = mean; stats[2 * r + 1] = rstd; }
+  for (int p = 0; p < panels; ++p) {
+    const int64_t off = ((int64_t)p * n_pad + r) * TW + l8 * V;
+    load16(X + off, v);
+    const int c0 = p * TW + l8 * V;
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      float y = (v[i] - mean) * rstd * gamma[c0 + i] + (beta ? beta[c0 + i] : 0.f);
+      v[i] = pad ? 0.f : y;
+    }
+    store16(Xn + off, v);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Pre-norm backward.  Row reductions mean(g), mean(g*xhat) with g = dXn*gamma give dX; the
+// token-axis reductions dgamma = sum dXn*xhat and dbeta = sum dXn are accumulated per block in
+// shared memory (a reduction over the block's 4 storage tiles) and added to the fp32 outputs.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) norm_bwd_kernel(const T* __restrict__ dXn, const T* __restrict__ X,
+                                                       const T* __restrict__ dY, const float* __restrict__ stats,
+                                                       const float* __restrict__ gamma, T* __restrict__ dX,
+                                                       float* __restrict__ dgamma, float* __restrict__ dbeta,
+                                                       int64_t n_pad, int d, int rms) {
+  constexpr int TW = tile_w_of<T>::value;
+  constexpr int V = Vec16<T>::N;
+  extern __shared__ float sh[];                 // [2][d]
+  float* s_dg = sh;
+  float* s_db = sh + d;
+  for (int i = threadIdx.x; i < 2 * d; i += blockDim.x) sh[i] = 0.f;
+  __syncthreads();
+  const int64_t r = (int64_t)blockIdx.x * 32 + threadIdx.x / 8;
+  const int l8 = threadIdx.x % 8;
+  const bool live = r < n_pad;
+  const int panels = d / TW;
+  float mean = 0.f, rstd = 0.f;
+  if (live) { mean = stats[2 * r]; rstd = stats[2 * r + 1]; }
+  float xv[V], gv[V];
+  float s1 = 0.f, s2 = 0.f;
+  for (int p = 0; p < panels; ++p) {
+    const int c0 = p * TW + l8 * V;
+    float pg[V], pb[V];
+    if (live) {
+      const int64_t off = ((int64_t)p * n_pad + r) * TW + l8 * V;
+      load16(X + off, xv);
+      load16(dXn + off, gv);
+#pragma unroll
+      for (int i = 0; i < V; ++i) {
+        float xh = (xv[i] - mean) * rstd;
+        float g = gv[i] * gamma[c0 + i];
+        s1 += g;
+        s2 += g * xh;
+        pg[i] = gv[i] * xh;
+        pb[i] = gv[i];
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < V; ++i) { pg[i] = 0.f; pb[i] = 0.f; }
+    }
+    // sum the 4 rows of this warp, then one shared-memory add per column per warp
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      pg[i] += __shfl_xor_sync(0xffffffffu, pg[i], 8);
+      pg[i] += __shfl_xor_sync(0xffffffffu, pg[i], 16);
+      pb[i] += __shfl_xor_sync(0xffffffffu, pb[i], 8);
+      pb[i] += __shfl_xor_sync(0xffffffffu, pb[i], 16);
+    }
+    if ((threadIdx.x & 31) < 8) {
+#pragma unroll
+      for (int i = 0; i < V; ++i) {
+        atomicAdd(&s_dg[c0 + i], pg[i]);
+        atomicAdd(&s_db[c0 + i], pb[i]);
+      }
+    }
+  }
+  s1 = group8_sum(s1) / (float)d;
+  s2 = group8_sum(s2) / (float)d;
+  if (rms) s1 = 0.f;
+  if (live) {
+    for (int p = 0; p < panels; ++p) {
+      const int64_t off = ((int64_t)p * n_pad + r) * TW + l8 * V;
+      const int c0 = p * TW + l8 * V;
+      load16(X + off, xv);
+      load16(dXn + off, gv);
+      float rv[V];
+      if (dY) load16(dY + off, rv);
+#pragma unroll
+      for (int i = 0; i < V; ++i) {
+        float xh = (xv[i] - mean) * rstd;
+        float o = rstd * (gv[i] * gamma[c0 + i] - s1 - xh * s2);
+        xv[i] = dY ? o + rv[i] : o;
+      }
+      store16(dX + off, xv);
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    atomicAdd(&dgamma[i], s_dg[i]);
+    if (dbeta) atomicAdd(&dbeta[i], s_db[i]);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Token-axis column sums, two stages over tiles: (1) one block per (panel, slab of 256 rows)
+// reduces its 32 storage tiles to one row of partials, (2) a tree over slabs.
+// ------------------------------------------------------------------------------------------
+constexpr int COLSUM_SLAB = 256;
+
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_stage1(const T* __restrict__ M, int64_t rows, float* __restrict__ part,
+                                                     int cols) {
+  constexpr int TW = tile_w_of<T>::value;
+  constexpr int V = Vec16<T>::N;
+  __shared__ float red[32][TW + 1];
+  const int p = blockIdx.x, slab = blockIdx.y;
+  const int rr = threadIdx.x / 8, l8 = threadIdx.x % 8;
+  float acc[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) acc[i] = 0.f;
+  const int64_t r_end = min((int64_t)(slab + 1) * COLSUM_SLAB, rows);
+  for (int64_t r = (int64_t)slab * COLSUM_SLAB + rr; r < r_end; r += 32) {
+    float v[V];
+    load16(M + ((int64_t)p * rows + r) * TW + l8 * V, v);
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] += v[i];
+  }
+#pragma unroll
+  for (int i = 0; i < V; ++i) red[rr][l8 * V + i] = acc[i];
+  __syncthreads();
+  if (threadIdx.x < TW) {
+    float s = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < 32; ++k) s += red[k][threadIdx.x];
+    part[(int64_t)slab * cols + p * TW + threadIdx.x] = s;
+  }
+}
+
+__global__ void colsum_stage2(const float* __restrict__ part, int n_slabs, int cols, float* __restrict__ out) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= cols) return;
+  float s = 0.f;
+  for (int k = 0; k < n_slabs; ++k) s += part[(int64_t)k * cols + c];
+  out[c] = s;
+}
+
+}  // namespace
+
+cudaError_t launch_pack(int dtype, int unpack, const void* src, void* dst, int64_t outer, int64_t rows,
+                        int64_t rows_pad, int cols, cudaStream_t st) {
+  const int64_t total = unpack ? outer * rows * cols : outer * rows_pad * cols;
+  if (total == 0) return cudaSuccess;
+  const int blocks = (int)min((int64_t)148 * 16, (total + 255) / 256);
+  if (dtype == FBL_DTYPE_FP32) {
+    if (unpack) unpack_kernel<float><<<blocks, 256, 0, st>>>((const float*)src, (float*)dst, outer, rows, rows_pad, cols, total);
+    else pack_kernel<float><<<blocks, 256, 0, st>>>((const float*)src, (float*)dst, outer, rows, rows_pad, cols, total);
+  } else {
+    using B = __nv_bfloat16;
+    if (unpack) unpack_kernel<B><<<blocks, 256, 0, st>>>((const B*)src, (B*)dst, outer, rows, rows_pad, cols, total);
+    else pack_kernel<B><<<blocks, 256, 0, st>>>((const B*)src, (B*)dst, outer, rows, rows_pad, cols, total);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
+                            float* stats, cudaStream_t st) {
+  const int blocks = (int)((p->n_pad + 31) / 32);
+  const int rms = p->d.norm == FBL_NORM_RMSNORM;
+  if (p->d.dtype == FBL_DTYPE_FP32)
+    norm_fwd_kernel<float><<<blocks, 256, 0, st>>>((const float*)X, gamma, rms ? nullptr : beta, (float*)Xn, stats,
+                                                   p->n_pad, p->d.d_model, p->d.seq, p->t_pad, rms, p->d.eps);
+  else
+    norm_fwd_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)X, gamma, rms ? nullptr : beta,
+                                                           (__nv_bfloat16*)Xn, stats, p->n_pad, p->d.d_model,
+                                                           p->d.seq, p->t_pad, rms, p->d.eps);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_norm_bwd(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
+                            const float* gamma, void* dX, float* dgamma, float* dbeta, cudaStream_t st) {
+  const int blocks = (int)((p->n_pad + 31) / 32);
+  const int d = p->d.d_model;
+  const int rms = p->d.norm == FBL_NORM_RMSNORM;
+  const size_t sh = 2 * (size_t)d * sizeof(float);
+  cudaError_t e = cudaMemsetAsync(dgamma, 0, d * sizeof(float), st);
+  if (e != cudaSuccess) return e;
+  if (dbeta) {
+    e = cudaMemsetAsync(dbeta, 0, d * sizeof(float), st);
+    if (e != cudaSuccess) return e;
+  }
+  if (p->d.dtype == FBL_DTYPE_FP32) {
+    auto k = norm_bwd_kernel<float>;
+    if (sh > 48 * 1024) cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
+    k<<<blocks, 256, sh, st>>>((const float*)dXn, (const float*)X, (const float*)dY, stats, gamma, (float*)dX, dgamma,
+                               rms ? nullptr : dbeta, p->n_pad, d, rms);
+  } else {
+    using B = __nv_bfloat16;
+    auto k = norm_bwd_kernel<B>;
+    if (sh > 48 * 1024) cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
+    k<<<blocks, 256, sh, st>>>((const B*)dXn, (const B*)X, (const B*)dY, stats, gamma, (B*)dX, dgamma,
+                               rms ? nullptr : dbeta, p->n_pad, d, rms);
+  }
+  return cudaGetLastError();
+}
+
+size_t colsum_scratch_bytes(int64_t rows, int64_t cols) {
+  const int64_t slabs = (rows + COLSUM_SLAB - 1) / COLSUM_SLAB;
+  return (size_t)(slabs * cols) * sizeof(float);
+}
+
+cudaError_t launch_colsum(int dtype, const void* M, int64_t rows, int64_t cols, float* out, float* partials,
+                          cudaStream_t st) {
+  const int slabs = (int)((rows + COLSUM_SLAB - 1) / COLSUM_SLAB);
+  if (dtype == FBL_DTYPE_FP32) {
+    dim3 grid((unsigned)(cols / 32), slabs);
+    colsum_stage1<float><<<grid, 256, 0, st>>>((const float*)M, rows, partials, (int)cols);
+  } else {
+    dim3 grid((unsigned)(cols / 64), slabs);
+    colsum_stage1<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)M, rows, partials, (int)cols);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  colsum_stage2<<<(unsigned)((cols + 127) / 128), 128, 0, st>>>(partials, slabs, (int)cols, out);
+  return cudaGetLastError();
+}

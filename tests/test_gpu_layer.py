@@ -1,0 +1,97 @@
+"""Parity of the CUDA path (through the C ABI) with the float64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+
+from fbl_inputs import LayerConfig, get_config, make_inputs, scaled_config
+from oracle import layer as orc
+from paper_2607_21624_b200 import LayerRunner
+
+from util import FP32_REL, bf16_ok, fp32_err, report
+
+pytestmark = pytest.mark.gpu
+
+MATS = ("Y", "dX", "dWq", "dWk", "dWv", "dWo")
+
+
+def run_and_compare(cfg, affine_noise=False, path=0):
+    inp = make_inputs(cfg, affine_noise=affine_noise)
+    Y, saved, g = orc.layer_fwd_bwd(cfg, inp)
+    ref = dict(g)
+    ref["Y"] = Y
+    run = LayerRunner(cfg)
+    run.plan.set_kernel_path(path)
+    run.load_inputs(inp)
+    run.step()
+    assert run.status() == 0
+    names = list(MATS) + ["dgamma"]
+    if cfg.norm == "layernorm":
+        names.append("dbeta")
+    if cfg.has_bias:
+        names += ["dbq", "dbk", "dbv", "dbo"]
+    bad = []
+    for n in names:
+        got = run.fetch(n)
+        assert np.isfinite(got).all(), n
+        if cfg.dtype == "fp32":
+            # dbk is identically zero in exact arithmetic; judge it against the scale of dbv
+            r = ref[n] if n != "dbk" else ref[n] + 0.0
+            err = fp32_err(got, r) if n != "dbk" else float(np.abs(got).max() / (np.abs(ref["dbv"]).max()))
+            ok = err <= FP32_REL
+            print(f"{n:7s} fp32 scale-floored rel err {err:.3e}")
+        else:
+            ok, worst = bf16_ok(n, got, ref[n])
+            print(report(n, got, ref[n]), f"worst/bound={worst:.3f}")
+        if not ok:
+            bad.append(n)
+    assert not bad, bad
+    return run
+
+
+def test_config1_fp32():
+    run_and_compare(get_config(1))
+
+
+@pytest.mark.parametrize("kw", [
+    dict(norm="layernorm", causal=True, residual=True, has_bias=True),
+    dict(norm="rmsnorm", causal=False, n_kv_heads=1),
+    dict(norm="layernorm", causal=False, seq=77, batch=3),
+    dict(norm="rmsnorm", causal=True, seq=150, head_dim=64, n_q_heads=2, n_kv_heads=1, d_model=128),
+])
+def test_fp32_variants(kw):
+    run_and_compare(scaled_config(get_config(1), **kw), affine_noise=True)
+
+
+SMALL_BF16 = [
+    # several 128-row tiles with ragged tails, biases, GQA, both norms, hd 64 and 128
+    LayerConfig("b1", 2, 200, 256, 4, 4, 64, "bf16", "layernorm", True, True, False, 1e-5, 21, 0.02),
+    LayerConfig("b2", 3, 197, 256, 4, 2, 64, "bf16", "layernorm", False, False, True, 1e-6, 22, 0.02),
+    LayerConfig("b3", 1, 333, 256, 4, 1, 64, "bf16", "rmsnorm", True, False, False, 1e-5, 23, 0.02),
+    LayerConfig("b4", 2, 130, 256, 2, 2, 128, "bf16", "rmsnorm", True, False, False, 1e-5, 24, 0.01),
+    LayerConfig("b5", 1, 8, 128, 2, 2, 64, "bf16", "layernorm", True, True, False, 1e-5, 25, 0.02),
+    LayerConfig("b6", 2, 1, 128, 2, 1, 64, "bf16", "rmsnorm", False, False, False, 1e-5, 26, 0.02),
+]
+
+
+@pytest.mark.parametrize("cfg", SMALL_BF16, ids=lambda c: c.name)
+@pytest.mark.parametrize("path", [0, 1], ids=["default", "ffma"])
+def test_bf16_small(cfg, path):
+    run_and_compare(cfg, affine_noise=True, path=path)
+
+
+@pytest.mark.parametrize("i", [2, 3])
+def test_full_configs_2_and_3(i):
+    run_and_compare(get_config(i))
+
+
+def test_padding_slots_are_zero_and_padded_equals_unpadded():
+    import torch
+    cfg = scaled_config(get_config(3), batch=2)
+    run = run_and_compare(cfg)
+    t_pad = 200
+    y = run.buf["Y"].view(torch.bfloat16).float().view(cfg.d_model // 64, cfg.batch, t_pad, 64)
+    dx = run.buf["dX"].view(torch.bfloat16).float().view(cfg.d_model // 64, cfg.batch, t_pad, 64)
+    assert float(y[:, :, cfg.seq:].abs().max()) == 0.0 and float(dx[:, :, cfg.seq:].abs().max()) == 0.0
+
+
+def test_config4_reduced_batch():
+    run_and_compare(scaled_config(get_config(4), batch=1, seq=1024))
