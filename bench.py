@@ -1,0 +1,371 @@
+#!/usr/bin/env python
+"""Benchmark of the attention-layer training step (forward + backward) on B200.
+
+One step = fbl_layer_fwd + fbl_layer_bwd over one batch of synthetic input.  The JSON
+line reports algorithmic TFLOP/s (multiply-add = 2, causal pairs counted once, no
+recompute), tokens/s, the end-to-end figure with host buffers, a roofline object for
+the dominant step and the float64 oracle timed on the host cores.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config i] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from fbl_inputs import get_config, make_inputs  # noqa: E402
+
+NOMINAL_TFLOPS, NOMINAL_GBS = 2250.0, 8000.0
+FALLBACK_TFLOPS, FALLBACK_GBS = 1590.0, 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            m = json.load(f)
+        return dict(tflops_burst=m["bf16_tflops"], tflops_sustained=m["bf16_tflops_sustained"], gbs=m["hbm_gbs"],
+                    source="measured")
+    return dict(tflops_burst=FALLBACK_TFLOPS, tflops_sustained=1400.0, gbs=FALLBACK_GBS, source="fallback")
+
+
+def workload_name(cfg):
+    return (f"{cfg.name}: B={cfg.batch} T={cfg.seq} D={cfg.d_model} Hq={cfg.n_q_heads} Hkv={cfg.n_kv_heads} "
+            f"hd={cfg.head_dim} {cfg.norm} {'causal' if cfg.causal else 'full'} {cfg.dtype}")
+
+
+def step_flops(cfg):
+    """Algorithmic flops of each named step (for the roofline of the dominant one)."""
+    n = cfg.n_tokens
+    pairs = cfg.seq * (cfg.seq + 1) / 2 if cfg.causal else float(cfg.seq) * cfg.seq
+    att = 2.0 * cfg.batch * cfg.n_q_heads * pairs * cfg.head_dim
+    pq, pk, po = 2.0 * n * cfg.d_model * cfg.d_q, 2.0 * n * cfg.d_model * cfg.d_kv, 2.0 * n * cfg.d_q * cfg.d_model
+    return {"proj_q": pq, "proj_k": pk, "proj_v": pk, "proj_qkv": pq + 2 * pk, "attn_fwd": 2 * att, "proj_o": po,
+            "dA": po, "dWo": po, "attn_bwd": 4 * att, "dXn": pq + 2 * pk, "dWq": pq, "dWk": pk, "dWv": pk,
+            "dWqkv": pq + 2 * pk}
+
+
+def step_bytes(cfg):
+    """Algorithmic HBM bytes of the bandwidth-bound steps."""
+    e = 2 if cfg.dtype == "bf16" else 4
+    nd = cfg.n_tokens * cfg.d_model * e
+    return {"norm_fwd": 2 * nd, "norm_bwd": (4 if cfg.residual else 3) * nd}
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, reasons, mx = [], set(), None
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx = float(parts[2])
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.f.name)
+        if sm:
+            sm.sort()
+            # the median over the whole window includes idle samples between steps; report the upper quartile too
+            out.update(sm_mhz=sm[len(sm) // 2], sm_mhz_p75=sm[(3 * len(sm)) // 4], sm_max_mhz=mx,
+                       reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def time_oracle(cfg, inp, repeats):
+    from oracle import layer as orc
+    t = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        orc.layer_fwd_bwd(cfg, inp)
+        t.append(time.perf_counter() - t0)
+    return t
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def run_reference(args, cfg, rank):
+    if rank != 0:
+        return
+    import numpy as np  # noqa: F401  (loads the BLAS threadpool before it is inspected)
+    # bounded sample: the workload with the batch cut down so that one oracle pass stays in the seconds range
+    from fbl_inputs import scaled_config
+    sample_batch = max(1, min(cfg.batch, int(4e10 // max(cfg.flops() / cfg.batch, 1)) or 1))
+    scfg = scaled_config(cfg, batch=sample_batch)
+    inp = make_inputs(scfg)
+    time_oracle(scfg, inp, min(args.warmup, 1))
+    t = time_oracle(scfg, inp, args.steps)
+    sec = sum(t) / len(t)
+    tfl = scfg.flops() / sec / 1e12
+    line = {"impl": "reference", "metric": "fwd+bwd layer TFLOP/s", "value": tfl, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "tokens_per_s": scfg.n_tokens / sec,
+            "config": {"workload": workload_name(cfg)},
+            "cpu_baseline": {"value": tfl, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle",
+                             "sample": f"batch {sample_batch} of {cfg.batch}, full sequence, one fwd+bwd per step"},
+            "e2e": {"value": tfl, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=2, help="1-based index into the five workloads (default: the second)")
+    ap.add_argument("--impl", default="fblayout", choices=["fblayout", "reference"])
+    ap.add_argument("--path", type=int, default=0, help="0 default kernels, 1 FFMA kernels only")
+    ap.add_argument("--no-graph", action="store_true", help="enqueue kernels directly instead of replaying a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "fblayout" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cfg = get_config(args.config)
+    if args.impl == "reference":
+        run_reference(args, cfg, rank)
+        return
+
+    import numpy as np
+    import torch
+    from paper_2607_21624_b200 import TENSOR, LayerRunner
+    from paper_2607_21624_b200.build import build
+    build()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    # replicas only: every rank runs the same workload on its own GPU, no data-path collective
+    inp = make_inputs(cfg)
+    run = LayerRunner(cfg, device=f"cuda:{local_rank}")
+    run.plan.set_kernel_path(args.path)
+    run.load_inputs(inp)
+    stream = torch.cuda.Stream()
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # 256 MiB > 126 MB L2
+
+    graph = None
+    with torch.cuda.stream(stream):
+        run.step()                      # first call sets kernel attributes; keep it outside any capture
+        stream.synchronize()
+        assert run.status() == 0
+        if not args.no_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                run.step()
+
+    def one_step():
+        if graph is not None:
+            graph.replay()
+        else:
+            run.step()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    launches0 = run.plan.launch_count()
+    with torch.cuda.stream(stream):
+        run.step()
+    launches_per_step = run.plan.launch_count() - launches0
+    torch.cuda.synchronize()
+
+    # ---- device-resident timing: L2 flushed before every step, events around each step ----------
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            flush.zero_()
+            one_step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    t_wall0 = time.perf_counter()
+    with torch.cuda.stream(stream):
+        for a, b in ev:
+            flush.zero_()
+            a.record(stream)
+            one_step()
+            b.record(stream)
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop()
+    per_step = [a.elapsed_time(b) for a, b in ev]
+    ms = sum(per_step) / len(per_step)
+    assert run.status() == 0
+
+    # ---- end to end with host buffers: H2D of X and dY, pack, step, unpack, D2H of Y and dX --------
+    tdt = run.tdtype
+    shape = (cfg.batch, cfg.seq, cfg.d_model)
+    hX = run.to_device_rowmajor(inp["X"]).cpu().pin_memory()
+    hdY = run.to_device_rowmajor(inp["dY"]).cpu().pin_memory()
+    hY = torch.empty(shape, dtype=tdt).pin_memory()
+    hdX = torch.empty(shape, dtype=tdt).pin_memory()
+    dX_rm = torch.empty(shape, dtype=tdt, device="cuda")
+    dY_rm = torch.empty(shape, dtype=tdt, device="cuda")
+    oY_rm = torch.empty(shape, dtype=tdt, device="cuda")
+    odX_rm = torch.empty(shape, dtype=tdt, device="cuda")
+
+    def e2e_step():
+        s = stream.cuda_stream
+        dX_rm.copy_(hX, non_blocking=True)
+        dY_rm.copy_(hdY, non_blocking=True)
+        run.plan.pack(TENSOR["X"], dX_rm.data_ptr(), run.buf["X"].data_ptr(), s)
+        run.plan.pack(TENSOR["DY"], dY_rm.data_ptr(), run.buf["dY"].data_ptr(), s)
+        one_step()
+        run.plan.unpack(TENSOR["Y"], run.buf["Y"].data_ptr(), oY_rm.data_ptr(), s)
+        run.plan.unpack(TENSOR["DX"], run.buf["dX"].data_ptr(), odX_rm.data_ptr(), s)
+        hY.copy_(oY_rm, non_blocking=True)
+        hdX.copy_(odX_rm, non_blocking=True)
+
+    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            flush.zero_()
+            e2e_step()
+    barrier()
+    with torch.cuda.stream(stream):
+        for a, b in ev2:
+            flush.zero_()
+            a.record(stream)
+            e2e_step()
+            b.record(stream)
+    barrier()
+    ms_e2e = sum(a.elapsed_time(b) for a, b in ev2) / len(ev2)
+    io_bytes = 2 * cfg.n_tokens * cfg.d_model * (2 if cfg.dtype == "bf16" else 4)
+
+    # ---- per-step event timing (separate pass, direct launches) for the roofline of the dominant step ----
+    run.plan.profile_enable(True)
+    acc = {}
+    reps = max(3, min(args.steps, 10))
+    with torch.cuda.stream(stream):
+        for _ in range(reps):
+            flush.zero_()
+            run.forward()
+            stream.synchronize()
+            for name, t in run.plan.profile_read():
+                acc.setdefault(name, []).append(t)
+            run.backward()
+            stream.synchronize()
+            for name, t in run.plan.profile_read():
+                acc.setdefault(name, []).append(t)
+    run.plan.profile_enable(False)
+    kernel_ms = {k: sum(v) / len(v) for k, v in acc.items()}
+
+    # max over ranks
+    if dist is not None:
+        t = torch.tensor([ms, ms_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    flops = cfg.flops()
+    tfl = world * flops / (ms * 1e-3) / 1e12
+    tfl_e2e = world * flops / (ms_e2e * 1e-3) / 1e12
+    sf, sbytes = step_flops(cfg), step_bytes(cfg)
+    dom = max(kernel_ms, key=kernel_ms.get)
+    total_k = sum(kernel_ms.values())
+    if dom in sf:
+        ach = sf[dom] / (kernel_ms[dom] * 1e-3) / 1e12
+        if cfg.dtype == "bf16" and args.path == 0:
+            roof = {"bound": "tensor", "kernel": dom, "achieved": ach, "peak": peaks["tflops_burst"], "unit": "TFLOP/s",
+                    "frac": ach / peaks["tflops_burst"], "traffic": None, "peak_source": peaks["source"] + " (burst)"}
+        else:
+            # FFMA path: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
+            alu = 148 * 128 * 2 * 1.965e9 / 1e12
+            roof = {"bound": "alu", "kernel": dom, "achieved": ach, "peak": alu, "unit": "TFLOP/s", "frac": ach / alu,
+                    "traffic": None, "peak_source": "148 SM x 128 FFMA/clk x 1.965 GHz"}
+    else:
+        ach = sbytes.get(dom, 0.0) / (kernel_ms[dom] * 1e-3) / 1e9
+        roof = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peaks["gbs"], "unit": "GB/s",
+                "frac": ach / peaks["gbs"], "traffic": None, "peak_source": peaks["source"]}
+    roof["kernel_share"] = kernel_ms[dom] / total_k
+    roof["kernel_ms"] = {k: round(v, 5) for k, v in sorted(kernel_ms.items(), key=lambda kv: -kv[1])}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        from fbl_inputs import scaled_config
+        sample_batch = max(1, min(cfg.batch, int(4e10 // max(cfg.flops() / cfg.batch, 1)) or 1))
+        scfg = scaled_config(cfg, batch=sample_batch)
+        sinp = make_inputs(scfg)
+        t = time_oracle(scfg, sinp, 2)
+        sec = min(t)
+        cpu = {"value": scfg.flops() / sec / 1e12, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle",
+               "sample": f"batch {sample_batch} of {cfg.batch}, full sequence, best of 2 fwd+bwd passes", "seconds": sec}
+
+    t_tensor = flops / (peaks["tflops_burst"] * 1e12)
+    line = {
+        "metric": "fwd+bwd layer TFLOP/s", "value": tfl, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": workload_name(cfg), "l2": "256 MiB flush write before every timed step",
+                   "launch": "cuda graph replay" if graph is not None else "direct launches",
+                   "kernel_path": "default" if args.path == 0 else "ffma", "parallelism": "replicas only"},
+        "tokens_per_s": world * cfg.n_tokens / (ms * 1e-3),
+        "layer_roofline": {"t_tensor_us_at_measured_burst": t_tensor * 1e6, "frac_of_measured_burst": t_tensor / (ms * 1e-3),
+                           "frac_of_nominal_2250": flops / (NOMINAL_TFLOPS * 1e12) / (ms * 1e-3)},
+        "activation_bytes": {"saved": run.sizes["saved"], "scratch": max(run.sizes["scratch_fwd"], run.sizes["scratch_bwd"])},
+        "e2e": {"value": tfl_e2e, "unit": "TFLOP/s", "ms_per_step": ms_e2e, "h2d_bytes_per_step": io_bytes,
+                "d2h_bytes_per_step": io_bytes},
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks, "roofline": roof, "cpu_baseline": cpu, "wall_s_timed_region": t_wall,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

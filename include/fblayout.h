@@ -152,6 +152,15 @@ int fbl_status_poll(const fbl_plan* plan, const void* scratch, int32_t* device_s
  * the same layout; lets a caller cross-check the tensor-core path on the device). */
 int fbl_plan_set_kernel_path(fbl_plan* plan, int path);
 
+/* Optional per-step device timing.  fbl_profile_enable(plan, 1) creates CUDA events (host objects); while
+ * enabled, fbl_layer_fwd / fbl_layer_bwd record one event after each of their steps.  After the caller has
+ * synchronised, fbl_profile_read returns the number of steps of the most recent call and fills their names
+ * (static strings) and durations in milliseconds.  fbl_launch_count is the number of kernels this plan
+ * has enqueued since it was created. */
+int fbl_profile_enable(fbl_plan* plan, int enable);
+int fbl_profile_read(const fbl_plan* plan, int max_steps, const char** names, float* ms);
+int64_t fbl_launch_count(const fbl_plan* plan);
+
 const char* fbl_strerror(int status);
 /* Text of the last CUDA runtime error seen by this thread inside the library ("" if none). */
 const char* fbl_last_error_detail(void);

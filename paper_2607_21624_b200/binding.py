@@ -61,6 +61,10 @@ def load_library():
     L.fbl_colsum.argtypes = [vp, vp, i64, i64, vp, vp, vp]
     L.fbl_status_poll.argtypes = [vp, vp, C.POINTER(i32)]
     L.fbl_plan_set_kernel_path.argtypes = [vp, C.c_int]
+    L.fbl_profile_enable.argtypes = [vp, C.c_int]
+    L.fbl_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_char_p), C.POINTER(C.c_float)]
+    L.fbl_launch_count.argtypes = [vp]
+    L.fbl_launch_count.restype = i64
     L.fbl_strerror.argtypes = [C.c_int]
     L.fbl_strerror.restype = C.c_char_p
     L.fbl_last_error_detail.restype = C.c_char_p
@@ -146,6 +150,20 @@ class Plan:
 
     def colsum(self, M, rows, cols, out, scratch, stream):
         _check(lib().fbl_colsum(self._h, M, rows, cols, out, scratch, stream))
+
+    def profile_enable(self, on: bool):
+        _check(lib().fbl_profile_enable(self._h, int(on)))
+
+    def profile_read(self):
+        names = (C.c_char_p * 32)()
+        ms = (C.c_float * 32)()
+        n = lib().fbl_profile_read(self._h, 32, names, ms)
+        if n < 0:
+            _check(n)
+        return [(names[i].decode(), float(ms[i])) for i in range(n)]
+
+    def launch_count(self) -> int:
+        return lib().fbl_launch_count(self._h)
 
     def status_poll(self, scratch) -> int:
         out = C.c_int32()

@@ -45,6 +45,26 @@ thread_local char g_detail[256] = "";
     }                                                   \
   } while (0)
 
+// One named step of a driver: launch, count the kernels it enqueued, and (when profiling is on) record an
+// event after it so the per-step device time can be read back later.
+#define FBL_STEP(name, kernels, expr)                              \
+  do {                                                             \
+    FBL_CUDA(expr);                                                \
+    fbl_plan* mp__ = const_cast<fbl_plan*>(p);                     \
+    mp__->launches += (kernels);                                   \
+    if (mp__->prof_on && mp__->prof_n < FBL_PROF_MAX) {            \
+      mp__->prof_name[mp__->prof_n] = (name);                      \
+      FBL_CUDA(cudaEventRecord(mp__->prof_ev[1 + mp__->prof_n], st)); \
+      mp__->prof_n++;                                              \
+    }                                                              \
+  } while (0)
+
+#define FBL_PROF_BEGIN()                                           \
+  do {                                                             \
+    fbl_plan* mp__ = const_cast<fbl_plan*>(p);                     \
+    if (mp__->prof_on) { mp__->prof_n = 0; FBL_CUDA(cudaEventRecord(mp__->prof_ev[0], st)); } \
+  } while (0)
+
 cudaError_t run_gemm(const fbl_plan* p, const GemmArgs& g, void* sk, size_t sk_bytes, int32_t* status,
                      cudaStream_t st) {
   if (p->use_tc && gemm_tc_supported(p, g)) return launch_gemm_tc(p, g, sk, sk_bytes, status, st);
@@ -133,7 +153,37 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   return FBL_OK;
 }
 
-void fbl_plan_destroy(fbl_plan* plan) { delete plan; }
+void fbl_plan_destroy(fbl_plan* plan) {
+  if (!plan) return;
+  if (plan->prof_on)
+    for (int i = 0; i <= FBL_PROF_MAX; ++i) cudaEventDestroy(plan->prof_ev[i]);
+  delete plan;
+}
+
+int fbl_profile_enable(fbl_plan* plan, int enable) {
+  if (!plan) return FBL_ERR_INVALID_ARG;
+  if (enable && !plan->prof_on) {
+    for (int i = 0; i <= FBL_PROF_MAX; ++i) FBL_CUDA(cudaEventCreate(&plan->prof_ev[i]));
+    plan->prof_on = 1;
+  } else if (!enable && plan->prof_on) {
+    for (int i = 0; i <= FBL_PROF_MAX; ++i) cudaEventDestroy(plan->prof_ev[i]);
+    plan->prof_on = 0;
+  }
+  plan->prof_n = 0;
+  return FBL_OK;
+}
+
+int fbl_profile_read(const fbl_plan* plan, int max_steps, const char** names, float* ms) {
+  if (!plan || !names || !ms || !plan->prof_on) return FBL_ERR_INVALID_ARG;
+  int n = plan->prof_n < max_steps ? plan->prof_n : max_steps;
+  for (int i = 0; i < n; ++i) {
+    names[i] = plan->prof_name[i];
+    FBL_CUDA(cudaEventElapsedTime(&ms[i], plan->prof_ev[i], plan->prof_ev[i + 1]));
+  }
+  return n;
+}
+
+int64_t fbl_launch_count(const fbl_plan* plan) { return plan ? plan->launches : -1; }
 
 int fbl_plan_set_kernel_path(fbl_plan* plan, int path) {
   if (!plan || (path != 0 && path != 1)) return FBL_ERR_INVALID_ARG;
@@ -270,7 +320,8 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
   const int n = (int)p->n_pad, D = p->d.d_model;
 
   FBL_CUDA(cudaMemsetAsync(status, 0, FBL_ALIGN, st));
-  FBL_CUDA(launch_norm_fwd(p, X, gamma, beta, Xn, stats, st));
+  FBL_PROF_BEGIN();
+  FBL_STEP("norm_fwd", 1, launch_norm_fwd(p, X, gamma, beta, Xn, stats, st));
   {
     const void* W[3] = {Wq, Wk, Wv};
     void* O[3] = {Q, K, V};
@@ -282,11 +333,11 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
       g.t[0] = {Xn, p->n_pad, 0, W[i], D, 0, D};
       g.c = O[i]; g.c_rpad = p->n_pad; g.bias = bias ? B[i] : nullptr;
       g.seq = p->d.seq; g.t_pad = p->t_pad;
-      FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
+      FBL_STEP(i == 0 ? "proj_q" : i == 1 ? "proj_k" : "proj_v", 1, run_gemm(p, g, part, p->part_bytes, status, st));
     }
   }
-  if (p->use_tc && attn_fwd_tc_supported(p)) FBL_CUDA(launch_attn_fwd_tc(p, Q, K, V, A, lse, status, st));
-  else FBL_CUDA(launch_attn_fwd_simt(p, Q, K, V, A, lse, st));
+  if (p->use_tc && attn_fwd_tc_supported(p)) FBL_STEP("attn_fwd", 1, launch_attn_fwd_tc(p, Q, K, V, A, lse, status, st));
+  else FBL_STEP("attn_fwd", 1, launch_attn_fwd_simt(p, Q, K, V, A, lse, st));
   {
     GemmArgs g = {};
     g.m = n; g.n = D; g.n_terms = 1;
@@ -294,7 +345,7 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
     g.c = Y; g.c_rpad = p->n_pad; g.bias = bias ? bo : nullptr;
     g.residual = p->d.residual ? X : nullptr;
     g.seq = p->d.seq; g.t_pad = p->t_pad;
-    FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
+    FBL_STEP("proj_o", 1, run_gemm(p, g, part, p->part_bytes, status, st));
   }
   return FBL_OK;
 }
@@ -324,23 +375,24 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
   const int n = (int)p->n_pad, D = p->d.d_model;
 
   FBL_CUDA(cudaMemsetAsync(status, 0, FBL_ALIGN, st));
+  FBL_PROF_BEGIN();
   {  // dA = dY Wo^T : Wo's tiles read with the roles of its two axes swapped
     GemmArgs g = {};
     g.m = n; g.n = p->dq; g.n_terms = 1;
     g.t[0] = {dY, p->n_pad, 0, Wo, p->dq, 1, D};
     g.c = dA; g.c_rpad = p->n_pad; g.seq = p->d.seq; g.t_pad = p->t_pad;
-    FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
+    FBL_STEP("dA", 1, run_gemm(p, g, part, p->part_bytes, status, st));
   }
   {  // dWo = A^T dY : token-axis reduction
     GemmArgs g = {};
     g.m = p->dq; g.n = D; g.n_terms = 1;
     g.t[0] = {A, p->n_pad, 1, dY, p->n_pad, 0, n};
     g.c = dWo; g.c_rpad = p->dq;
-    FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
+    FBL_STEP("dWo", 1, run_gemm(p, g, part, p->part_bytes, status, st));
   }
-  if (bias) FBL_CUDA(launch_colsum(p->d.dtype, dY, p->n_pad, D, dbo, (float*)part, st));
-  if (p->use_tc && attn_bwd_tc_supported(p)) FBL_CUDA(launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, status, st));
-  else FBL_CUDA(launch_attn_bwd_simt(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, st));
+  if (bias) FBL_STEP("dbo", 2, launch_colsum(p->d.dtype, dY, p->n_pad, D, dbo, (float*)part, st));
+  if (p->use_tc && attn_bwd_tc_supported(p)) FBL_STEP("attn_bwd", 3, launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, status, st));
+  else FBL_STEP("attn_bwd", 3, launch_attn_bwd_simt(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, st));
   {  // dXn = dQ Wq^T + dK Wk^T + dV Wv^T : one accumulator, three reduction loops
     GemmArgs g = {};
     g.m = n; g.n = D; g.n_terms = 3;
@@ -348,7 +400,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
     g.t[1] = {dK, p->n_pad, 0, Wk, D, 1, p->dkv};
     g.t[2] = {dV, p->n_pad, 0, Wv, D, 1, p->dkv};
     g.c = dXn; g.c_rpad = p->n_pad; g.seq = p->d.seq; g.t_pad = p->t_pad;
-    FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
+    FBL_STEP("dXn", 1, run_gemm(p, g, part, p->part_bytes, status, st));
   }
   {
     const void* G[3] = {dQ, dK, dV};
@@ -360,11 +412,11 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
       g.m = D; g.n = cols[i]; g.n_terms = 1;
       g.t[0] = {Xn, p->n_pad, 1, G[i], p->n_pad, 0, n};
       g.c = DW[i]; g.c_rpad = D;
-      FBL_CUDA(run_gemm(p, g, part, p->part_bytes, status, st));
-      if (bias) FBL_CUDA(launch_colsum(p->d.dtype, G[i], p->n_pad, cols[i], DB[i], (float*)part, st));
+      FBL_STEP(i == 0 ? "dWq" : i == 1 ? "dWk" : "dWv", 1, run_gemm(p, g, part, p->part_bytes, status, st));
+      if (bias) FBL_STEP(i == 0 ? "dbq" : i == 1 ? "dbk" : "dbv", 2, launch_colsum(p->d.dtype, G[i], p->n_pad, cols[i], DB[i], (float*)part, st));
     }
   }
-  FBL_CUDA(launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, st));
+  FBL_STEP("norm_bwd", 1, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, st));
   return FBL_OK;
 }
 

@@ -8,6 +8,7 @@
 
 #define FBL_TILE_H 8
 #define FBL_ALIGN 1024
+#define FBL_PROF_MAX 32
 
 // ---------------------------------------------------------------------------------------------
 // R-Tile element map (section 4.2).  Storage tile = 8 rows x 128 bytes, row-major inside; tiles
@@ -45,6 +46,11 @@ struct fbl_plan {
   size_t sb_da, sb_dvec, sb_dqacc, sb_dq, sb_dk, sb_dv, sb_dxn, sb_part, scratch_bwd_bytes;
   size_t sf_part, scratch_fwd_bytes;
   size_t part_bytes;
+  // bookkeeping: kernels enqueued so far, optional per-step event timing
+  int64_t launches;
+  int prof_on, prof_n;
+  cudaEvent_t prof_ev[FBL_PROF_MAX + 1];
+  const char* prof_name[FBL_PROF_MAX];
 };
 
 static inline size_t fbl_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
