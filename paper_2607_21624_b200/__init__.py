@@ -5,6 +5,6 @@ package never falls back to another implementation: if the library is missing or
 CUDA device is absent, calls raise.
 """
 from .binding import (FblError, Plan, lib, load_library, LayerRunner, DTYPES, TENSOR, MAP,
-                      desc_from_config)
+                      desc_from_config, aligned_bytes)
 
-__all__ = ["FblError", "Plan", "lib", "load_library", "LayerRunner", "DTYPES", "TENSOR", "MAP", "desc_from_config"]
+__all__ = ["FblError", "Plan", "lib", "load_library", "LayerRunner", "DTYPES", "TENSOR", "MAP", "desc_from_config", "aligned_bytes"]

@@ -59,6 +59,7 @@ def load_library():
     L.fbl_layer_bwd.argtypes = [vp] * 22
     L.fbl_colsum_scratch_bytes.argtypes = [vp, i64, i64, C.POINTER(sz)]
     L.fbl_colsum.argtypes = [vp, vp, i64, i64, vp, vp, vp]
+    L.fbl_colsum_noalloc.argtypes = [vp, vp, i64, i64, vp, vp]
     L.fbl_status_poll.argtypes = [vp, vp, C.POINTER(i32)]
     L.fbl_plan_set_kernel_path.argtypes = [vp, C.c_int]
     L.fbl_profile_enable.argtypes = [vp, C.c_int]
@@ -151,6 +152,10 @@ class Plan:
     def colsum(self, M, rows, cols, out, scratch, stream):
         _check(lib().fbl_colsum(self._h, M, rows, cols, out, scratch, stream))
 
+    def colsum_noalloc(self, M, rows, cols, out, stream):
+        """fbl_colsum with the partial sums kept in the library's own fixed array (allocates nothing)."""
+        _check(lib().fbl_colsum_noalloc(self._h, M, rows, cols, out, stream))
+
     def profile_enable(self, on: bool):
         _check(lib().fbl_profile_enable(self._h, int(on)))
 
@@ -173,6 +178,14 @@ class Plan:
         return out.value
 
 
+def aligned_bytes(torch, nbytes, device, align=1024, zero=True):
+    """A uint8 device tensor of ``nbytes`` whose data pointer is ``align``-byte aligned (torch only
+    promises 512)."""
+    raw = (torch.zeros if zero else torch.empty)(nbytes + align, dtype=torch.uint8, device=device)
+    off = (-raw.data_ptr()) % align
+    return raw[off:off + nbytes]
+
+
 class LayerRunner:
     """Device buffers for one layer plus pack/step/unpack helpers (torch for memory and streams only)."""
 
@@ -190,7 +203,7 @@ class LayerRunner:
         self.tdtype = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
         saved, sf, sb = self.plan.workspace_bytes()
         self.sizes = dict(saved=saved, scratch_fwd=sf, scratch_bwd=sb)
-        al = lambda nbytes: torch.zeros(nbytes, dtype=torch.uint8, device=self.dev)
+        al = lambda nbytes: aligned_bytes(torch, nbytes, self.dev)
         self.saved = al(saved)
         self.scratch = al(max(sf, sb))
         self.buf = {}
