@@ -143,6 +143,22 @@ int fbl_colsum_scratch_bytes(const fbl_plan* plan, int64_t rows, int64_t cols, s
 int fbl_colsum(const fbl_plan* plan, const void* M_dev, int64_t rows, int64_t cols,
                float* out_dev, void* scratch_dev, void* stream);
 
+/* (No counterpart in the paper.)  fbl_colsum for callers that cannot hand over scratch memory: code that runs
+ * where device allocation is off limits -- inside a framework's allocator hook or out-of-memory handler, in a
+ * plugin that was given fixed input and output buffers and nothing else, or on a path that must not disturb a
+ * caching allocator.  The per-slab partial sums go to a fixed 1 MiB array that is part of the library image
+ * (every GPU that loads the library carries it until the process exits), so this call allocates nothing, on the
+ * host side of CUDA or through any library.  Same arguments and result as fbl_colsum minus `scratch_dev`.
+ *   - Limit: ceil(rows / 256) * cols <= 262144 (for example 16384 rows x 4096 columns); beyond it the call
+ *     returns FBL_ERR_WORKSPACE_TOO_SMALL and enqueues nothing.
+ *   - The first call on each device looks up the array's device address (with that device current); make that
+ *     first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call overwrites the part it uses before reading it, so
+ *     earlier contents never leak into a result, but two calls that can run at the same time on the GPU (different
+ *     streams, no ordering between them) race; order them. */
+int fbl_colsum_noalloc(const fbl_plan* plan, const void* M_dev, int64_t rows, int64_t cols,
+                       float* out_dev, void* stream);
+
 /* After the caller has synchronised the stream: reads back the device status word kept at the start
  * of `scratch` (set when a bounded wait inside a kernel expired).  Synchronous 4-byte copy. */
 int fbl_status_poll(const fbl_plan* plan, const void* scratch, int32_t* device_status);

@@ -324,3 +324,60 @@ cudaError_t launch_colsum(int dtype, const void* M, int64_t rows, int64_t cols, 
   colsum_stage2<<<(unsigned)((cols + 127) / 128), 128, 0, st>>>(partials, slabs, (int)cols, out);
   return cudaGetLastError();
 }
+
+// ------------------------------------------------------------------------------------------
+// Column sums without caller scratch.  The per-slab partial sums live in a fixed array inside the
+// library image instead of a caller buffer, for callers that are not in a position to allocate.
+// ------------------------------------------------------------------------------------------
+#include <mutex>
+
+#define FBL_COLSUM_NOALLOC_MAX_FLOATS (256 * 1024)   // 1 MiB: e.g. 16384 rows x 4096 columns
+
+static __device__ __align__(256) float g_colsum_partials[FBL_COLSUM_NOALLOC_MAX_FLOATS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+float* g_partials_addr[kMaxDevices] = {};   // device address of g_colsum_partials, per device ordinal
+}  // namespace
+
+extern "C" int fbl_colsum_noalloc(const fbl_plan* plan, const void* M_dev, int64_t rows, int64_t cols,
+                                  float* out_dev, void* stream) {
+  if (!plan || !M_dev || !out_dev || rows <= 0 || cols <= 0 || rows % 8 != 0 || cols % plan->tw != 0)
+    return FBL_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(M_dev) & (FBL_ALIGN - 1)) != 0) return FBL_ERR_MISALIGNED;
+  const int64_t slabs = (rows + COLSUM_SLAB - 1) / COLSUM_SLAB;
+  if (slabs * cols > FBL_COLSUM_NOALLOC_MAX_FLOATS) {
+    fbl_note_cuda_error(cudaSuccess, "fbl_colsum_noalloc: ceil(rows/256) * cols exceeds the built-in 262144-float area");
+    return FBL_ERR_WORKSPACE_TOO_SMALL;
+  }
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    fbl_note_cuda_error(e, "fbl_colsum_noalloc: cudaGetDevice");
+    return FBL_ERR_CUDA;
+  }
+  float* partials = nullptr;
+  {
+    // Set-up, once per device and with that device current: in host code the array's name is only a
+    // handle, so ask the runtime for the address the kernels must be given.
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_partials_addr[dev]) {
+      void* addr = nullptr;
+      e = cudaGetSymbolAddress(&addr, g_colsum_partials);
+      if (e != cudaSuccess || !addr) {
+        fbl_note_cuda_error(e, "fbl_colsum_noalloc: cudaGetSymbolAddress");
+        return FBL_ERR_CUDA;
+      }
+      g_partials_addr[dev] = static_cast<float*>(addr);
+    }
+    partials = g_partials_addr[dev];
+  }
+  // Stage 1 writes every partial that stage 2 reads, so nothing left over from an earlier call is used.
+  e = launch_colsum(plan->d.dtype, M_dev, rows, cols, out_dev, partials, reinterpret_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) {
+    fbl_note_cuda_error(e, "fbl_colsum_noalloc: launch");
+    return FBL_ERR_CUDA;
+  }
+  return FBL_OK;
+}
