@@ -327,13 +327,22 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
     void* O[3] = {Q, K, V};
     const float* B[3] = {bq, bk, bv};
     const int cols[3] = {p->dq, p->dkv, p->dkv};
+    GemmArgs gs[3];
+    bool tc = p->use_tc != 0;
     for (int i = 0; i < 3; ++i) {
-      GemmArgs g = {};
+      GemmArgs& g = gs[i];
+      g = GemmArgs{};
       g.m = n; g.n = cols[i]; g.n_terms = 1;
       g.t[0] = {Xn, p->n_pad, 0, W[i], D, 0, D};
       g.c = O[i]; g.c_rpad = p->n_pad; g.bias = bias ? B[i] : nullptr;
       g.seq = p->d.seq; g.t_pad = p->t_pad;
-      FBL_STEP(i == 0 ? "proj_q" : i == 1 ? "proj_k" : "proj_v", 1, run_gemm(p, g, part, p->part_bytes, status, st));
+      tc = tc && gemm_tc_supported(p, g);
+    }
+    if (tc) {
+      FBL_STEP("proj_qkv", 1, launch_gemm_tc_group(p, gs, 3, status, st));   // one launch, blockIdx.z picks Q, K or V
+    } else {
+      for (int i = 0; i < 3; ++i)
+        FBL_STEP(i == 0 ? "proj_q" : i == 1 ? "proj_k" : "proj_v", 1, launch_gemm_simt(p->d.dtype, gs[i], st));
     }
   }
   if (p->use_tc && attn_fwd_tc_supported(p)) FBL_STEP("attn_fwd", 1, launch_attn_fwd_tc(p, Q, K, V, A, lse, status, st));
@@ -407,14 +416,26 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
     void* DW[3] = {dWq, dWk, dWv};
     float* DB[3] = {dbq, dbk, dbv};
     const int cols[3] = {p->dq, p->dkv, p->dkv};
+    GemmArgs gs[3];
+    bool tc = p->use_tc != 0;
     for (int i = 0; i < 3; ++i) {
-      GemmArgs g = {};
+      GemmArgs& g = gs[i];
+      g = GemmArgs{};
       g.m = D; g.n = cols[i]; g.n_terms = 1;
       g.t[0] = {Xn, p->n_pad, 1, G[i], p->n_pad, 0, n};
       g.c = DW[i]; g.c_rpad = D;
-      FBL_STEP(i == 0 ? "dWq" : i == 1 ? "dWk" : "dWv", 1, run_gemm(p, g, part, p->part_bytes, status, st));
-      if (bias) FBL_STEP(i == 0 ? "dbq" : i == 1 ? "dbk" : "dbv", 2, launch_colsum(p->d.dtype, G[i], p->n_pad, cols[i], DB[i], (float*)part, st));
+      tc = tc && gemm_tc_supported(p, g);
     }
+    if (tc) {
+      FBL_STEP("dWqkv", 1, launch_gemm_tc_group(p, gs, 3, status, st));
+    } else {
+      for (int i = 0; i < 3; ++i)
+        FBL_STEP(i == 0 ? "dWq" : i == 1 ? "dWk" : "dWv", 1, launch_gemm_simt(p->d.dtype, gs[i], st));
+    }
+    if (bias)
+      for (int i = 0; i < 3; ++i)
+        FBL_STEP(i == 0 ? "dbq" : i == 1 ? "dbk" : "dbv", 2,
+                 launch_colsum(p->d.dtype, G[i], p->n_pad, cols[i], DB[i], (float*)part, st));
   }
   FBL_STEP("norm_bwd", 1, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, st));
   return FBL_OK;

@@ -76,6 +76,7 @@ cudaError_t launch_gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);
 cudaError_t launch_gemm_tc(const fbl_plan* p, const GemmArgs& g, void* splitk_scratch, size_t splitk_bytes,
                            int32_t* status, cudaStream_t st);
 bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g);
+cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st);
 bool attn_fwd_tc_supported(const fbl_plan* p);
 bool attn_bwd_tc_supported(const fbl_plan* p);
 void fbl_note_cuda_error(cudaError_t e, const char* where);

@@ -1,3 +1,254 @@
+// Projection GEMMs on tcgen05 tensor cores (bf16 in, fp32 accumulate in TMEM, bf16 out), operands in
+// R-Tile order fetched by TMA.  One kernel serves all six projection steps and their transposed forms:
+// each operand is declared K-major or MN-major in the descriptors, so W / W^T and X / X^T are the same
+// tiles in HBM and in shared memory.  Up to three reduction loops feed one accumulator (dXn), and up
+// to three problems that share a launch are selected by blockIdx.z (Q/K/V projections, dWq/dWk/dWv).
+#include <string.h>
+
+#include <mutex>
+
 #include "fbl_internal.h"
-bool gemm_tc_supported(const fbl_plan*, const GemmArgs&) { return false; }
-cudaError_t launch_gemm_tc(const fbl_plan*, const GemmArgs&, void*, size_t, int32_t*, cudaStream_t) { return cudaErrorNotSupported; }
+#include "tc_common.cuh"
+
+namespace {
+
+constexpr int BM = 128, BK = 64;
+constexpr int MAX_TERMS = 3, MAX_PROBLEMS = 3;
+
+struct alignas(64) TcProblem {
+  CUtensorMap ta[MAX_TERMS], tb[MAX_TERMS];
+  int n_terms;
+  int kblocks[MAX_TERMS];
+  int a_mn[MAX_TERMS], b_mn[MAX_TERMS];   // 1: operand is MN-major in shared memory (its rows are K indices)
+  int m, n;
+  __nv_bfloat16* c;
+  long long c_rpad;
+  const float* bias;
+  const __nv_bfloat16* residual;
+  int seq, t_pad;
+};
+struct alignas(64) TcGroup {
+  TcProblem p[MAX_PROBLEMS];
+  int count;
+  int32_t* status;
+};
+
+template <int BN, int STAGES>
+struct SmemPlan {
+  static constexpr uint32_t A_BYTES = BM * 128;
+  static constexpr uint32_t B_BYTES = BN * 128;
+  static constexpr uint32_t STAGE = A_BYTES + B_BYTES;
+  static constexpr uint32_t BAR_OFF = STAGES * STAGE;
+  static constexpr uint32_t TOTAL = BAR_OFF + 8 * (2 * STAGES + 2) + 1024;   // + alignment slack
+};
+
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__ TcGroup G) {
+  using SP = SmemPlan<BN, STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  const TcProblem& P = G.p[blockIdx.z];
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  if (m0 >= P.m || n0 >= P.n) return;          // uniform per block: problems of a group differ in size
+  const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = base + SP::BAR_OFF;
+  const uint32_t bar_acc = bars + 16 * STAGES;
+  const uint32_t slot = bar_acc + 8;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  int32_t* status = G.status;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      tc::mbar_init(bars + 8 * s, 1);                 // full[s]: one producer arrival + transaction bytes
+      tc::mbar_init(bars + 8 * (STAGES + s), 1);      // empty[s]: one tcgen05.commit arrival
+    }
+    tc::mbar_init(bar_acc, 1);
+    tc::fence_barrier_init();
+  }
+  if (warp == 1) {
+    tc::tmem_alloc(slot, BN);                         // BN fp32 columns x 128 lanes
+    tc::tmem_relinquish();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  uint32_t tmem_base;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
+
+  if (warp == 0 && lane == 0) {
+    // ---- TMA producer ----------------------------------------------------------------------
+    int it = 0;
+    bool ok = true;
+    for (int t = 0; t < P.n_terms && ok; ++t) {
+      tc::tma_prefetch_desc(&P.ta[t]);
+      tc::tma_prefetch_desc(&P.tb[t]);
+      for (int kb = 0; kb < P.kblocks[t]; ++kb, ++it) {
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1;
+        if (!tc::mbar_wait(bars + 8 * (STAGES + s), ph ^ 1, status, 101)) { ok = false; break; }
+        const uint32_t full = bars + 8 * s;
+        const uint32_t sa = base + s * SP::STAGE, sb = sa + SP::A_BYTES;
+        tc::mbar_expect_tx(full, SP::STAGE);
+        if (P.a_mn[t]) tc::tma_load_3d(sa, &P.ta[t], full, 0, kb * BK, m0 / 64);
+        else tc::tma_load_3d(sa, &P.ta[t], full, 0, m0, kb);
+        if (P.b_mn[t]) tc::tma_load_3d(sb, &P.tb[t], full, 0, kb * BK, n0 / 64);
+        else tc::tma_load_3d(sb, &P.tb[t], full, 0, n0, kb);
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---- MMA issuer ------------------------------------------------------------------------
+    int it = 0;
+    bool ok = true;
+    for (int t = 0; t < P.n_terms && ok; ++t) {
+      const uint32_t idesc = tc::idesc_bf16(BM, BN, P.a_mn[t], P.b_mn[t]);
+      // K-major: 8-row groups 1024 B apart, 16 K elements = 32 B along the row.
+      // MN-major: 64-wide M/N blocks 8 KiB apart (64 K rows x 128 B), 16 K rows = 2 KiB.
+      const uint32_t a_lbo = P.a_mn[t] ? 8192u : 16u, a_step = P.a_mn[t] ? 2048u : 32u;
+      const uint32_t b_lbo = P.b_mn[t] ? 8192u : 16u, b_step = P.b_mn[t] ? 2048u : 32u;
+      for (int kb = 0; kb < P.kblocks[t]; ++kb, ++it) {
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1;
+        if (!tc::mbar_wait(bars + 8 * s, ph, status, 102)) { ok = false; break; }
+        tc::tc_fence_after();
+        const uint32_t sa = base + s * SP::STAGE, sb = sa + SP::A_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < BK / 16; ++kk) {
+          const uint64_t da = tc::smem_desc_sw128(sa + kk * a_step, a_lbo, 1024);
+          const uint64_t db = tc::smem_desc_sw128(sb + kk * b_step, b_lbo, 1024);
+          tc::mma_bf16_ss(tmem_base, da, db, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+        }
+        tc::mma_commit(bars + 8 * (STAGES + s));      // frees the stage once these MMAs have read it
+      }
+    }
+    if (ok) tc::mma_commit(bar_acc);
+  } else if (warp >= 2) {
+    // ---- epilogue: TMEM -> registers -> R-Tile rows (each thread owns one output row) -----------
+    const int q = warp % 4;                           // the TMEM lane quarter this warp may access
+    const bool ok = tc::mbar_wait(bar_acc, 0, status, 103);
+    tc::tc_fence_after();
+    const int row = m0 + q * 32 + lane;
+    const bool pad = P.t_pad > 0 && (row % P.t_pad) >= P.seq;
+    if (ok) {
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t r[32];
+        tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + c0, r);
+        tc::tmem_ld_wait();
+        const int n = n0 + c0;
+        if (row < P.m && n < P.n) {
+          const long long off = ((long long)(n / 64) * P.c_rpad + row) * 64 + (n % 64);
+          uint4 resv[4];
+          if (P.residual) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) resv[j] = *reinterpret_cast<const uint4*>(P.residual + off + 8 * j);
+          }
+          const __nv_bfloat16* rb = reinterpret_cast<const __nv_bfloat16*>(resv);
+          uint4 outv[4];
+          uint32_t* ow = reinterpret_cast<uint32_t*>(outv);
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float v0 = __uint_as_float(r[j]), v1 = __uint_as_float(r[j + 1]);
+            if (P.bias) { v0 += P.bias[n + j]; v1 += P.bias[n + j + 1]; }
+            if (P.residual) { v0 += __bfloat162float(rb[j]); v1 += __bfloat162float(rb[j + 1]); }
+            if (pad) { v0 = 0.f; v1 = 0.f; }
+            ow[j / 2] = tc::pack_bf16(v0, v1);
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(P.c + off + 8 * j) = outv[j];
+        }
+      }
+    }
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tc::tmem_dealloc(tmem_base, BN);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+constexpr int BN_DEFAULT = 128, STAGES_DEFAULT = 6;
+
+}  // namespace
+
+bool fbl_encode_rtile_map(CUtensorMap* map, const void* base, int64_t r_pad, int panels, int box_rows, int box_panels) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {64, (cuuint64_t)r_pad, (cuuint64_t)panels};
+  cuuint64_t strides[2] = {128, (cuuint64_t)r_pad * 128};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_panels};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g) {
+  if (p->d.dtype != FBL_DTYPE_BF16) return false;
+  if (g.n % 64 != 0 || g.n < BN_DEFAULT || g.m < BM) return false;
+  for (int t = 0; t < g.n_terms; ++t) {
+    const GemmTerm& tm = g.t[t];
+    // a box must fit inside its tensor: rows of every operand cover one tile, K-major reduction axes are whole panels
+    if (tm.a_trans ? (tm.k < BK || g.m % 64 != 0) : (tm.k % BK != 0)) return false;
+    if (tm.b_trans ? (tm.k % BK != 0) : (tm.k < BK)) return false;
+    if (tm.a_rpad < 128 || tm.b_rpad < 128) return false;
+  }
+  return true;
+}
+
+cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
+  if (count < 1 || count > MAX_PROBLEMS) return cudaErrorInvalidValue;
+  TcGroup G;
+  memset(&G, 0, sizeof(G));
+  G.count = count;
+  G.status = status;
+  int max_m = 0, max_n = 0;
+  for (int i = 0; i < count; ++i) {
+    const GemmArgs& g = gs[i];
+    TcProblem& P = G.p[i];
+    P.n_terms = g.n_terms;
+    for (int t = 0; t < g.n_terms; ++t) {
+      const GemmTerm& tm = g.t[t];
+      P.kblocks[t] = (tm.k + BK - 1) / BK;
+      P.a_mn[t] = tm.a_trans ? 1 : 0;     // stored [k rows][m cols]: rows are K indices
+      P.b_mn[t] = tm.b_trans ? 0 : 1;     // stored [k rows][n cols]: rows are K indices
+      bool ok;
+      if (tm.a_trans) ok = fbl_encode_rtile_map(&P.ta[t], tm.a, tm.a_rpad, g.m / 64, BK, BM / 64);
+      else ok = fbl_encode_rtile_map(&P.ta[t], tm.a, tm.a_rpad, tm.k / 64, BM, 1);
+      if (!ok) return cudaErrorInvalidValue;
+      if (tm.b_trans) ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, tm.k / 64, BN_DEFAULT, 1);
+      else ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, g.n / 64, BK, BN_DEFAULT / 64);
+      if (!ok) return cudaErrorInvalidValue;
+    }
+    P.m = g.m; P.n = g.n;
+    P.c = (__nv_bfloat16*)g.c; P.c_rpad = g.c_rpad;
+    P.bias = g.bias; P.residual = (const __nv_bfloat16*)g.residual;
+    P.seq = g.seq; P.t_pad = g.t_pad;
+    max_m = g.m > max_m ? g.m : max_m;
+    max_n = g.n > max_n ? g.n : max_n;
+  }
+  using SP = SmemPlan<BN_DEFAULT, STAGES_DEFAULT>;
+  auto k = gemm_tc_kernel<BN_DEFAULT, STAGES_DEFAULT>;
+  cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
+  if (attr_err != cudaSuccess) return attr_err;
+  dim3 grid((max_n + BN_DEFAULT - 1) / BN_DEFAULT, (max_m + BM - 1) / BM, count);
+  k<<<grid, 192, SP::TOTAL, st>>>(G);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_tc(const fbl_plan* p, const GemmArgs& g, void*, size_t, int32_t* status, cudaStream_t st) {
+  return launch_gemm_tc_group(p, &g, 1, status, st);
+}
