@@ -96,6 +96,9 @@ cudaError_t launch_attn_fwd_simt(const fbl_plan* p, const void* Q, const void* K
 cudaError_t launch_attn_bwd_simt(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* A,
                                  const void* dA, const float* lse, float* dvec, float* dqacc, void* dQ, void* dK,
                                  void* dV, cudaStream_t st);
+cudaError_t launch_attn_bwd_pre(const fbl_plan* p, const void* A, const void* dA, float* dvec, float* dqacc,
+                                cudaStream_t st);
+cudaError_t launch_attn_bwd_post(const fbl_plan* p, const float* dqacc, void* dQ, cudaStream_t st);
 cudaError_t launch_attn_fwd_tc(const fbl_plan* p, const void* Q, const void* K, const void* V, void* A, float* lse,
                                int32_t* status, cudaStream_t st);
 cudaError_t launch_attn_bwd_tc(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* A,

@@ -406,9 +406,8 @@ cudaError_t launch_attn_fwd_simt(const fbl_plan* p, const void* Q, const void* K
   return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_attn_bwd_simt(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* A,
-                                 const void* dA, const float* lse, float* dvec, float* dqacc, void* dQ, void* dK,
-                                 void* dV, cudaStream_t st) {
+cudaError_t launch_attn_bwd_pre(const fbl_plan* p, const void* A, const void* dA, float* dvec, float* dqacc,
+                                cudaStream_t st) {
   const int hd = p->d.head_dim;
   const int64_t total = p->n_pad * p->d.n_q_heads;
   const int64_t nq = p->n_pad * p->dq;
@@ -421,7 +420,22 @@ cudaError_t launch_attn_bwd_simt(const fbl_plan* p, const void* Q, const void* K
   else
     rowdot_kernel<__nv_bfloat16><<<rb, 256, 0, st>>>((const __nv_bfloat16*)dA, (const __nv_bfloat16*)A, dvec, p->n_pad,
                                                      p->t_pad, p->d.n_q_heads, hd, total);
-  e = cudaGetLastError();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attn_bwd_post(const fbl_plan* p, const float* dqacc, void* dQ, cudaStream_t st) {
+  const int64_t nq = p->n_pad * p->dq;
+  const int blocks = (int)min((int64_t)148 * 8, (nq + 255) / 256);
+  if (p->d.dtype == FBL_DTYPE_FP32) convert_f32_kernel<float><<<blocks, 256, 0, st>>>(dqacc, (float*)dQ, nq);
+  else convert_f32_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(dqacc, (__nv_bfloat16*)dQ, nq);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attn_bwd_simt(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* A,
+                                 const void* dA, const float* lse, float* dvec, float* dqacc, void* dQ, void* dK,
+                                 void* dV, cudaStream_t st) {
+  const int hd = p->d.head_dim;
+  cudaError_t e = launch_attn_bwd_pre(p, A, dA, dvec, dqacc, st);
   if (e != cudaSuccess) return e;
   e = cudaErrorInvalidValue;
   if (p->d.dtype == FBL_DTYPE_FP32) {
@@ -433,8 +447,5 @@ cudaError_t launch_attn_bwd_simt(const fbl_plan* p, const void* Q, const void* K
     else if (hd == 128) e = attn_bwd_launch<__nv_bfloat16, 128>(p, Q, K, V, dA, lse, dvec, dqacc, dK, dV, st);
   }
   if (e != cudaSuccess) return e;
-  const int blocks = (int)min((int64_t)148 * 8, (nq + 255) / 256);
-  if (p->d.dtype == FBL_DTYPE_FP32) convert_f32_kernel<float><<<blocks, 256, 0, st>>>(dqacc, (float*)dQ, nq);
-  else convert_f32_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(dqacc, (__nv_bfloat16*)dQ, nq);
-  return cudaGetLastError();
+  return launch_attn_bwd_post(p, dqacc, dQ, st);
 }

@@ -266,12 +266,299 @@ cudaError_t fwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   return cudaGetLastError();
 }
 
+
+// ---------------------------------------------------------------------------------------------------
+// Backward: one block per (128-key tile, KV head, batch).  For every query head of the group and every
+// query tile it recomputes the transposed scores S^T = K Q^T and dP^T = V dO^T on the tensor pipe (so
+// the rows a thread owns are keys), forms P^T = exp(S^T - LSE) and dS^T = P^T * (dP^T - D) in registers,
+// and writes both once to swizzled shared memory.  Those two tiles then feed three products:
+//   dV += P^T dO  and  dK += dS^T Q   (sequence-axis reductions; accumulators stay in TMEM over the
+//                                      whole query loop and over the G heads of the group), and
+//   dQ  = dS K    (the same dS^T bytes read MN-major, i.e. transposed by descriptor), a key-axis
+//                  reduction across blocks, added to an fp32 buffer with vector red operations.
+// ---------------------------------------------------------------------------------------------------
+struct alignas(64) AttnBwdParams {
+  CUtensorMap tq, tk, tv, tdo;
+  const float* lse;      // [B, Hq, t_pad]
+  const float* dvec;     // [B, Hq, t_pad]   D = rowsum(dO * O)
+  float* dqacc;          // fp32 [n_pad, dq] in the bf16 tile order
+  __nv_bfloat16* dk;
+  __nv_bfloat16* dv;
+  long long n_pad;
+  int seq, t_pad, hq, group, causal, dkv;
+  float scale;
+  int32_t* status;
+};
+
+template <int HD>
+struct BwdSmem {
+  static constexpr uint32_t PANELS = HD / 64;
+  static constexpr uint32_t TILE = PANELS * 16384;
+  static constexpr uint32_t K_OFF = 0, V_OFF = TILE, Q_OFF = 2 * TILE, DO_OFF = 3 * TILE;
+  static constexpr uint32_t P_OFF = 4 * TILE, DS_OFF = P_OFF + 32768;
+  static constexpr uint32_t LSE_OFF = DS_OFF + 32768;        // 2 buffers x (128 floats LSE*log2e, 128 floats D)
+  static constexpr uint32_t BAR_OFF = LSE_OFF + 2048;
+  static constexpr uint32_t N_BARS = 8;
+  static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16 + 1024;
+};
+
+enum { BB_KVFULL = 0, BB_QDOFULL, BB_QDOEMPTY, BB_SFULL, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY };
+
+template <int HD>
+__global__ void __launch_bounds__(192, 1) attn_bwd_tc_kernel(const __grid_constant__ AttnBwdParams P) {
+  using SM = BwdSmem<HD>;
+  constexpr uint32_t PANELS = SM::PANELS;
+  constexpr uint32_t S_COL = 0, DP_COL = 128, DV_COL = 256, DK_COL = 384, DQ_COL = 0, TMEM_COLS = 512;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = base + SM::BAR_OFF;
+  const uint32_t slot = bars + 8 * SM::N_BARS;
+  auto bar = [&](int i) { return bars + 8u * i; };
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int j0 = blockIdx.x * BKV, g = blockIdx.y, b = blockIdx.z;
+  const int row0 = b * P.t_pad;
+  const int n_qt = (P.seq + BQ - 1) / BQ;
+  const int qt_begin = P.causal ? j0 / BQ : 0;
+  const int n_it = P.group * (n_qt - qt_begin);
+  int32_t* status = P.status;
+
+  if (threadIdx.x == 0) {
+    tc::mbar_init(bar(BB_KVFULL), 1);
+    tc::mbar_init(bar(BB_QDOFULL), 1);
+    tc::mbar_init(bar(BB_QDOEMPTY), 1);
+    tc::mbar_init(bar(BB_SFULL), 1);
+    tc::mbar_init(bar(BB_PDSFULL), 128);
+    tc::mbar_init(bar(BB_DQFULL), 1);
+    tc::mbar_init(bar(BB_DQDRAINED), 128);
+    tc::mbar_init(bar(BB_LSEREADY), 128);
+    tc::fence_barrier_init();
+  }
+  if (warp == 1) {
+    tc::tmem_alloc(slot, TMEM_COLS);
+    tc::tmem_relinquish();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  uint32_t tmem_base;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
+
+  if (warp == 0 && lane == 0) {
+    // ---- TMA producer ------------------------------------------------------------------------
+    tc::mbar_expect_tx(bar(BB_KVFULL), 2 * SM::TILE);
+    tc::tma_load_3d(base + SM::K_OFF, &P.tk, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
+    tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
+    int it = 0;
+    for (int hh = 0; hh < P.group; ++hh) {
+      const int h = g * P.group + hh;
+      for (int qt = qt_begin; qt < n_qt; ++qt, ++it) {
+        if (!tc::mbar_wait(bar(BB_QDOEMPTY), (it & 1) ^ 1, status, 301)) { hh = P.group; break; }
+        tc::mbar_expect_tx(bar(BB_QDOFULL), 2 * SM::TILE);
+        tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(BB_QDOFULL), 0, row0 + qt * BQ, h * (int)PANELS);
+        tc::tma_load_3d(base + SM::DO_OFF, &P.tdo, bar(BB_QDOFULL), 0, row0 + qt * BQ, h * (int)PANELS);
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---- MMA issuer --------------------------------------------------------------------------
+    const uint32_t idesc_s = tc::idesc_bf16(BKV, BQ, 0, 0);
+    const uint32_t idesc_kv = tc::idesc_bf16(BKV, HD, 0, 1);
+    const uint32_t idesc_dq = tc::idesc_bf16(BQ, HD, 1, 1);
+    bool ok = tc::mbar_wait(bar(BB_KVFULL), 0, status, 302);
+    for (int it = 0; it < n_it && ok; ++it) {
+      if (!tc::mbar_wait(bar(BB_QDOFULL), it & 1, status, 303)) { ok = false; break; }
+      if (it > 0 && !tc::mbar_wait(bar(BB_DQDRAINED), (it - 1) & 1, status, 304)) { ok = false; break; }
+      tc::tc_fence_after();
+#pragma unroll
+      for (uint32_t kk = 0; kk < HD / 16; ++kk) {
+        const uint32_t o = (kk / 4) * 16384 + (kk % 4) * 32;
+        tc::mma_bf16_ss(tmem_base + S_COL, tc::smem_desc_sw128(base + SM::K_OFF + o, 16, 1024),
+                        tc::smem_desc_sw128(base + SM::Q_OFF + o, 16, 1024), idesc_s, kk > 0);
+      }
+#pragma unroll
+      for (uint32_t kk = 0; kk < HD / 16; ++kk) {
+        const uint32_t o = (kk / 4) * 16384 + (kk % 4) * 32;
+        tc::mma_bf16_ss(tmem_base + DP_COL, tc::smem_desc_sw128(base + SM::V_OFF + o, 16, 1024),
+                        tc::smem_desc_sw128(base + SM::DO_OFF + o, 16, 1024), idesc_s, kk > 0);
+      }
+      tc::mma_commit(bar(BB_SFULL));
+      if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
+      tc::tc_fence_after();
+#pragma unroll
+      for (uint32_t kk = 0; kk < BQ / 16; ++kk) {
+        const uint32_t ao = (kk / 4) * 16384 + (kk % 4) * 32;      // P^T / dS^T: K-major, reduction over queries
+        const uint32_t bo = kk * 2048;                             // dO / Q: MN-major, 16 query rows per step
+        tc::mma_bf16_ss(tmem_base + DV_COL, tc::smem_desc_sw128(base + SM::P_OFF + ao, 16, 1024),
+                        tc::smem_desc_sw128(base + SM::DO_OFF + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
+      }
+#pragma unroll
+      for (uint32_t kk = 0; kk < BQ / 16; ++kk) {
+        const uint32_t ao = (kk / 4) * 16384 + (kk % 4) * 32;
+        const uint32_t bo = kk * 2048;
+        tc::mma_bf16_ss(tmem_base + DK_COL, tc::smem_desc_sw128(base + SM::DS_OFF + ao, 16, 1024),
+                        tc::smem_desc_sw128(base + SM::Q_OFF + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
+      }
+#pragma unroll
+      for (uint32_t kk = 0; kk < BKV / 16; ++kk) {
+        const uint32_t o = kk * 2048;                              // both operands MN-major: 16 key rows per step
+        tc::mma_bf16_ss(tmem_base + DQ_COL, tc::smem_desc_sw128(base + SM::DS_OFF + o, 16384, 1024),
+                        tc::smem_desc_sw128(base + SM::K_OFF + o, 16384, 1024), idesc_dq, kk > 0);
+      }
+      tc::mma_commit(bar(BB_DQFULL));
+      tc::mma_commit(bar(BB_QDOEMPTY));
+    }
+  } else if (warp >= 2) {
+    // ---- softmax / reduction warps: one key row (then one query row of dQ) per thread ----------
+    const int q = warp % 4;
+    const int r = q * 32 + lane;
+    const int t = threadIdx.x - 64;                 // 0..127
+    const int gj = j0 + r;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+    const float c = P.scale * LOG2E;
+    float* s_stage = reinterpret_cast<float*>(smem_raw + (base - tc::smem_u32(smem_raw)) + SM::LSE_OFF);
+    bool ok = true;
+    int it = 0;
+    for (int hh = 0; hh < P.group && ok; ++hh) {
+      const int h = g * P.group + hh;
+      for (int qt = qt_begin; qt < n_qt && ok; ++qt, ++it) {
+        const int i0 = qt * BQ;
+        // LSE and D of this query tile, staged in shared memory (two buffers by iteration parity: every
+        // reader of the buffer's previous use arrived at PDSFULL two iterations ago)
+        float* s_lse = s_stage + (it & 1) * 256;
+        float* s_d = s_lse + 128;
+        {
+          const int gi = i0 + t;
+          const bool live = gi < P.seq;
+          const long long o = ((long long)b * P.hq + h) * P.t_pad + gi;
+          s_lse[t] = live ? P.lse[o] * LOG2E : INFINITY;
+          s_d[t] = live ? P.dvec[o] : 0.f;
+        }
+        tc::mbar_arrive(bar(BB_LSEREADY));
+        if (!tc::mbar_wait(bar(BB_LSEREADY), it & 1, status, 308)) { ok = false; break; }
+        if (!tc::mbar_wait(bar(BB_SFULL), it & 1, status, 306)) { ok = false; break; }
+        tc::tc_fence_after();
+        const bool diag = P.causal && (i0 < j0 + BKV - 1);
+#pragma unroll 1
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t sv[32], dpv[32];
+          tc::tmem_ld32(lane_addr + S_COL + cc * 32, sv);
+          tc::tmem_ld32(lane_addr + DP_COL + cc * 32, dpv);
+          tc::tmem_ld_wait();
+          uint32_t pp[16], dd[16];
+#pragma unroll
+          for (int k = 0; k < 32; k += 2) {
+            float pv[2], dv[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const int col = cc * 32 + k + u;
+              float p = tc::fast_exp2(fmaf(__uint_as_float(sv[k + u]), c, -s_lse[col]));
+              if (gj >= P.seq || (diag && i0 + col < gj)) p = 0.f;
+              pv[u] = p;
+              dv[u] = p * (__uint_as_float(dpv[k + u]) - s_d[col]);
+            }
+            pp[k / 2] = tc::pack_bf16(pv[0], pv[1]);
+            dd[k / 2] = tc::pack_bf16(dv[0], dv[1]);
+          }
+          // 32 query columns = 64 bytes = 4 swizzled 16-byte chunks of this key row, in panel cc/2
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
+            const uint32_t chunk = (cc % 2) * 4 + ch;
+            const uint32_t off = (cc / 2) * 16384 + r * 128 + ((chunk ^ (r & 7)) * 16);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + SM::P_OFF + off), "r"(pp[ch * 4]),
+                         "r"(pp[ch * 4 + 1]), "r"(pp[ch * 4 + 2]), "r"(pp[ch * 4 + 3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + SM::DS_OFF + off), "r"(dd[ch * 4]),
+                         "r"(dd[ch * 4 + 1]), "r"(dd[ch * 4 + 2]), "r"(dd[ch * 4 + 3]) : "memory");
+          }
+        }
+        tc::fence_proxy_async();
+        tc::tc_fence_before();
+        tc::mbar_arrive(bar(BB_PDSFULL));
+        // dQ tile of this (key tile, query tile): row r is query i0 + r; add it to the fp32 accumulator
+        if (!tc::mbar_wait(bar(BB_DQFULL), it & 1, status, 307)) { ok = false; break; }
+        tc::tc_fence_after();
+        const int gi = i0 + r;
+#pragma unroll 1
+        for (int cc = 0; cc < HD / 32; ++cc) {
+          uint32_t o[32];
+          tc::tmem_ld32(lane_addr + DQ_COL + cc * 32, o);
+          tc::tmem_ld_wait();
+          if (gi < P.seq) {
+            const int col = h * HD + cc * 32;
+            float* dst = P.dqacc + ((long long)(col / 64) * P.n_pad + row0 + gi) * 64 + (col % 64);
+#pragma unroll
+            for (int k = 0; k < 32; k += 4) {
+              asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + k),
+                           "f"(__uint_as_float(o[k]) * P.scale), "f"(__uint_as_float(o[k + 1]) * P.scale),
+                           "f"(__uint_as_float(o[k + 2]) * P.scale), "f"(__uint_as_float(o[k + 3]) * P.scale)
+                           : "memory");
+            }
+          }
+        }
+        tc::tc_fence_before();
+        tc::mbar_arrive(bar(BB_DQDRAINED));
+      }
+    }
+    // dK, dV of this key tile: every MMA has completed (the last dQ wait covered them)
+    if (ok && n_it > 0) {
+      const bool live = gj < P.seq;
+#pragma unroll 1
+      for (int which = 0; which < 2; ++which) {
+        __nv_bfloat16* out = which ? P.dk : P.dv;
+        const float f = live ? (which ? P.scale : 1.f) : 0.f;
+#pragma unroll 1
+        for (int cc = 0; cc < HD / 32; ++cc) {
+          uint32_t o[32];
+          tc::tmem_ld32(lane_addr + (which ? DK_COL : DV_COL) + cc * 32, o);   // warp-collective: no lane may skip it
+          tc::tmem_ld_wait();
+          if (gj < P.t_pad) {
+            const int col = g * HD + cc * 32;
+            __nv_bfloat16* dst = out + ((long long)(col / 64) * P.n_pad + row0 + gj) * 64 + (col % 64);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              uint4 v;
+              v.x = tc::pack_bf16(__uint_as_float(o[k * 8 + 0]) * f, __uint_as_float(o[k * 8 + 1]) * f);
+              v.y = tc::pack_bf16(__uint_as_float(o[k * 8 + 2]) * f, __uint_as_float(o[k * 8 + 3]) * f);
+              v.z = tc::pack_bf16(__uint_as_float(o[k * 8 + 4]) * f, __uint_as_float(o[k * 8 + 5]) * f);
+              v.w = tc::pack_bf16(__uint_as_float(o[k * 8 + 6]) * f, __uint_as_float(o[k * 8 + 7]) * f);
+              *reinterpret_cast<uint4*>(dst + 8 * k) = v;
+            }
+          }
+        }
+      }
+    }
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tc::tmem_dealloc(tmem_base, TMEM_COLS);
+}
+
+template <int HD>
+cudaError_t bwd_launch(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* dA,
+                       const float* lse, const float* dvec, float* dqacc, void* dK, void* dV, int32_t* status,
+                       cudaStream_t st) {
+  AttnBwdParams P;
+  memset(&P, 0, sizeof(P));
+  const int panels = HD / 64;
+  if (!fbl_encode_rtile_map(&P.tq, Q, p->n_pad, p->dq / 64, BQ, panels)) return cudaErrorInvalidValue;
+  if (!fbl_encode_rtile_map(&P.tdo, dA, p->n_pad, p->dq / 64, BQ, panels)) return cudaErrorInvalidValue;
+  if (!fbl_encode_rtile_map(&P.tk, K, p->n_pad, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
+  if (!fbl_encode_rtile_map(&P.tv, V, p->n_pad, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
+  P.lse = lse; P.dvec = dvec; P.dqacc = dqacc; P.dk = (__nv_bfloat16*)dK; P.dv = (__nv_bfloat16*)dV;
+  P.n_pad = p->n_pad; P.seq = p->d.seq; P.t_pad = p->t_pad; P.hq = p->d.n_q_heads; P.group = p->group;
+  P.causal = p->d.causal; P.dkv = p->dkv; P.scale = p->scale; P.status = status;
+  auto k = attn_bwd_tc_kernel<HD>;
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdSmem<HD>::TOTAL);
+  if (e != cudaSuccess) return e;
+  dim3 grid((p->t_pad + BKV - 1) / BKV, p->d.n_kv_heads, p->d.batch);
+  k<<<grid, 192, BwdSmem<HD>::TOTAL, st>>>(P);
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 bool attn_fwd_tc_supported(const fbl_plan* p) {
   return p->d.dtype == FBL_DTYPE_BF16 && (p->d.head_dim == 64 || p->d.head_dim == 128) && p->n_pad >= 128;
 }
-bool attn_bwd_tc_supported(const fbl_plan*) { return false; }
+bool attn_bwd_tc_supported(const fbl_plan* p) { return attn_fwd_tc_supported(p); }
 
 cudaError_t launch_attn_fwd_tc(const fbl_plan* p, const void* Q, const void* K, const void* V, void* A, float* lse,
                                int32_t* status, cudaStream_t st) {
@@ -280,7 +567,14 @@ cudaError_t launch_attn_fwd_tc(const fbl_plan* p, const void* Q, const void* K, 
   return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_attn_bwd_tc(const fbl_plan*, const void*, const void*, const void*, const void*, const void*,
-                               const float*, float*, float*, void*, void*, void*, int32_t*, cudaStream_t) {
-  return cudaErrorNotSupported;
+cudaError_t launch_attn_bwd_tc(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* A,
+                               const void* dA, const float* lse, float* dvec, float* dqacc, void* dQ, void* dK,
+                               void* dV, int32_t* status, cudaStream_t st) {
+  cudaError_t e = launch_attn_bwd_pre(p, A, dA, dvec, dqacc, st);     // D = rowsum(dO * O); dQ accumulator := 0
+  if (e != cudaSuccess) return e;
+  if (p->d.head_dim == 64) e = bwd_launch<64>(p, Q, K, V, dA, lse, dvec, dqacc, dK, dV, status, st);
+  else if (p->d.head_dim == 128) e = bwd_launch<128>(p, Q, K, V, dA, lse, dvec, dqacc, dK, dV, status, st);
+  else e = cudaErrorInvalidValue;
+  if (e != cudaSuccess) return e;
+  return launch_attn_bwd_post(p, dqacc, dQ, st);                      // fp32 accumulator -> storage dtype
 }
