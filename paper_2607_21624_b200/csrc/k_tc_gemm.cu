@@ -39,33 +39,61 @@ struct SmemPlan {
   static constexpr uint32_t B_BYTES = BN * 128;
   static constexpr uint32_t STAGE = A_BYTES + B_BYTES;
   static constexpr uint32_t BAR_OFF = STAGES * STAGE;
-  static constexpr uint32_t TOTAL = BAR_OFF + 8 * (2 * STAGES + 2) + 1024;   // + alignment slack
+  static constexpr uint32_t N_BARS = 2 * STAGES + 4;     // full[], empty[], acc_full[2], acc_empty[2]
+  static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16 + 1024;   // + TMEM slot + alignment slack
 };
 
+// Work list of a launch: output tiles of all problems, numbered problem by problem with the M tile index
+// fastest (blocks that run together then share the B tiles of one weight column block through L2).
+struct TileCoord { int prob, m0, n0; };
+
+template <int BN>
+__device__ __forceinline__ bool tile_at(const TcGroup& G, int w, TileCoord* tc_out) {
+  for (int p = 0; p < G.count; ++p) {
+    const int tm = (G.p[p].m + BM - 1) / BM, tn = (G.p[p].n + BN - 1) / BN;
+    if (w < tm * tn) {
+      tc_out->prob = p;
+      tc_out->m0 = (w % tm) * BM;
+      tc_out->n0 = (w / tm) * BN;
+      return true;
+    }
+    w -= tm * tn;
+  }
+  return false;
+}
+
+// Persistent kernel: one block per SM walks the work list with stride gridDim.x.  Warp 0 feeds the
+// shared-memory ring by TMA, warp 1 issues the MMAs into one of two TMEM accumulators, warps 2-5 drain the
+// other accumulator (bias, residual, padding-row mask, bf16 rows in R-Tile order), so the epilogue of
+// one tile overlaps the main loop of the next.
 template <int BN, int STAGES>
 __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__ TcGroup G) {
   using SP = SmemPlan<BN, STAGES>;
   extern __shared__ uint8_t smem_raw[];
-  const TcProblem& P = G.p[blockIdx.z];
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  if (m0 >= P.m || n0 >= P.n) return;          // uniform per block: problems of a group differ in size
   const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = base + SP::BAR_OFF;
-  const uint32_t bar_acc = bars + 16 * STAGES;
-  const uint32_t slot = bar_acc + 8;
+  auto full = [&](int s) { return bars + 8u * s; };
+  auto empty = [&](int s) { return bars + 8u * (STAGES + s); };
+  auto acc_full = [&](int a) { return bars + 8u * (2 * STAGES + a); };
+  auto acc_empty = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
+  const uint32_t slot = bars + 8 * SP::N_BARS;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   int32_t* status = G.status;
+  constexpr uint32_t TMEM_COLS = 2 * BN;                 // two fp32 accumulators of BN columns
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      tc::mbar_init(bars + 8 * s, 1);                 // full[s]: one producer arrival + transaction bytes
-      tc::mbar_init(bars + 8 * (STAGES + s), 1);      // empty[s]: one tcgen05.commit arrival
+      tc::mbar_init(full(s), 1);                 // one producer arrival + transaction bytes
+      tc::mbar_init(empty(s), 1);                // one tcgen05.commit arrival
     }
-    tc::mbar_init(bar_acc, 1);
+    for (int a = 0; a < 2; ++a) {
+      tc::mbar_init(acc_full(a), 1);
+      tc::mbar_init(acc_empty(a), 128);
+    }
     tc::fence_barrier_init();
   }
   if (warp == 1) {
-    tc::tmem_alloc(slot, BN);                         // BN fp32 columns x 128 lanes
+    tc::tmem_alloc(slot, TMEM_COLS);
     tc::tmem_relinquish();
   }
   tc::tc_fence_before();
@@ -78,62 +106,78 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
     // ---- TMA producer ----------------------------------------------------------------------
     int it = 0;
     bool ok = true;
-    for (int t = 0; t < P.n_terms && ok; ++t) {
-      tc::tma_prefetch_desc(&P.ta[t]);
-      tc::tma_prefetch_desc(&P.tb[t]);
-      for (int kb = 0; kb < P.kblocks[t]; ++kb, ++it) {
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1;
-        if (!tc::mbar_wait(bars + 8 * (STAGES + s), ph ^ 1, status, 101)) { ok = false; break; }
-        const uint32_t full = bars + 8 * s;
-        const uint32_t sa = base + s * SP::STAGE, sb = sa + SP::A_BYTES;
-        tc::mbar_expect_tx(full, SP::STAGE);
-        if (P.a_mn[t]) tc::tma_load_3d(sa, &P.ta[t], full, 0, kb * BK, m0 / 64);
-        else tc::tma_load_3d(sa, &P.ta[t], full, 0, m0, kb);
-        if (P.b_mn[t]) tc::tma_load_3d(sb, &P.tb[t], full, 0, kb * BK, n0 / 64);
-        else tc::tma_load_3d(sb, &P.tb[t], full, 0, n0, kb);
+    TileCoord tcd;
+    for (int w = blockIdx.x; ok && tile_at<BN>(G, w, &tcd); w += gridDim.x) {
+      const TcProblem& P = G.p[tcd.prob];
+      for (int t = 0; t < P.n_terms && ok; ++t) {
+        for (int kb = 0; kb < P.kblocks[t]; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!tc::mbar_wait(empty(s), ph ^ 1, status, 101)) { ok = false; break; }
+          const uint32_t sa = base + s * SP::STAGE, sb = sa + SP::A_BYTES;
+          tc::mbar_expect_tx(full(s), SP::STAGE);
+          if (P.a_mn[t]) tc::tma_load_3d(sa, &P.ta[t], full(s), 0, kb * BK, tcd.m0 / 64);
+          else tc::tma_load_3d(sa, &P.ta[t], full(s), 0, tcd.m0, kb);
+          if (P.b_mn[t]) tc::tma_load_3d(sb, &P.tb[t], full(s), 0, kb * BK, tcd.n0 / 64);
+          else tc::tma_load_3d(sb, &P.tb[t], full(s), 0, tcd.n0, kb);
+        }
       }
     }
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer ------------------------------------------------------------------------
-    int it = 0;
+    int it = 0, ti = 0;
     bool ok = true;
-    for (int t = 0; t < P.n_terms && ok; ++t) {
-      const uint32_t idesc = tc::idesc_bf16(BM, BN, P.a_mn[t], P.b_mn[t]);
-      // K-major: 8-row groups 1024 B apart, 16 K elements = 32 B along the row.
-      // MN-major: 64-wide M/N blocks 8 KiB apart (64 K rows x 128 B), 16 K rows = 2 KiB.
-      const uint32_t a_lbo = P.a_mn[t] ? 8192u : 16u, a_step = P.a_mn[t] ? 2048u : 32u;
-      const uint32_t b_lbo = P.b_mn[t] ? 8192u : 16u, b_step = P.b_mn[t] ? 2048u : 32u;
-      for (int kb = 0; kb < P.kblocks[t]; ++kb, ++it) {
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1;
-        if (!tc::mbar_wait(bars + 8 * s, ph, status, 102)) { ok = false; break; }
-        tc::tc_fence_after();
-        const uint32_t sa = base + s * SP::STAGE, sb = sa + SP::A_BYTES;
+    TileCoord tcd;
+    for (int w = blockIdx.x; ok && tile_at<BN>(G, w, &tcd); w += gridDim.x, ++ti) {
+      const TcProblem& P = G.p[tcd.prob];
+      const int ab = ti & 1;
+      if (!tc::mbar_wait(acc_empty(ab), ((ti >> 1) & 1) ^ 1, status, 104)) { ok = false; break; }
+      tc::tc_fence_after();
+      const uint32_t d_tmem = tmem_base + ab * BN;
+      bool first = true;
+      for (int t = 0; t < P.n_terms && ok; ++t) {
+        const uint32_t idesc = tc::idesc_bf16(BM, BN, P.a_mn[t], P.b_mn[t]);
+        // K-major: 8-row groups 1024 B apart, 16 K elements = 32 B along the row.
+        // MN-major: 64-wide M/N blocks 8 KiB apart (64 K rows x 128 B), 16 K rows = 2 KiB.
+        const uint32_t a_lbo = P.a_mn[t] ? 8192u : 16u, a_step = P.a_mn[t] ? 2048u : 32u;
+        const uint32_t b_lbo = P.b_mn[t] ? 8192u : 16u, b_step = P.b_mn[t] ? 2048u : 32u;
+        for (int kb = 0; kb < P.kblocks[t]; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!tc::mbar_wait(full(s), ph, status, 102)) { ok = false; break; }
+          tc::tc_fence_after();
+          const uint32_t sa = base + s * SP::STAGE, sb = sa + SP::A_BYTES;
 #pragma unroll
-        for (int kk = 0; kk < BK / 16; ++kk) {
-          const uint64_t da = tc::smem_desc_sw128(sa + kk * a_step, a_lbo, 1024);
-          const uint64_t db = tc::smem_desc_sw128(sb + kk * b_step, b_lbo, 1024);
-          tc::mma_bf16_ss(tmem_base, da, db, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            const uint64_t da = tc::smem_desc_sw128(sa + kk * a_step, a_lbo, 1024);
+            const uint64_t db = tc::smem_desc_sw128(sb + kk * b_step, b_lbo, 1024);
+            tc::mma_bf16_ss(d_tmem, da, db, idesc, (first && kk == 0) ? 0u : 1u);
+          }
+          first = false;
+          tc::mma_commit(empty(s));              // frees the stage once these MMAs have read it
         }
-        tc::mma_commit(bars + 8 * (STAGES + s));      // frees the stage once these MMAs have read it
       }
+      if (ok) tc::mma_commit(acc_full(ab));
     }
-    if (ok) tc::mma_commit(bar_acc);
   } else if (warp >= 2) {
     // ---- epilogue: TMEM -> registers -> R-Tile rows (each thread owns one output row) -----------
     const int q = warp % 4;                           // the TMEM lane quarter this warp may access
-    const bool ok = tc::mbar_wait(bar_acc, 0, status, 103);
-    tc::tc_fence_after();
-    const int row = m0 + q * 32 + lane;
-    const bool pad = P.t_pad > 0 && (row % P.t_pad) >= P.seq;
-    if (ok) {
+    int ti = 0;
+    bool ok = true;
+    TileCoord tcd;
+    for (int w = blockIdx.x; ok && tile_at<BN>(G, w, &tcd); w += gridDim.x, ++ti) {
+      const TcProblem& P = G.p[tcd.prob];
+      const int ab = ti & 1;
+      if (!tc::mbar_wait(acc_full(ab), (ti >> 1) & 1, status, 103)) { ok = false; break; }
+      tc::tc_fence_after();
+      const int row = tcd.m0 + q * 32 + lane;
+      const bool pad = P.t_pad > 0 && (row % P.t_pad) >= P.seq;
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         uint32_t r[32];
-        tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + c0, r);
+        tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + c0, r);
         tc::tmem_ld_wait();
-        const int n = n0 + c0;
+        const int n = tcd.n0 + c0;
         if (row < P.m && n < P.n) {
           const long long off = ((long long)(n / 64) * P.c_rpad + row) * 64 + (n % 64);
           uint4 resv[4];
@@ -156,11 +200,13 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
           for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(P.c + off + 8 * j) = outv[j];
         }
       }
+      tc::tc_fence_before();
+      tc::mbar_arrive(acc_empty(ab));             // this accumulator may be overwritten by the tile after next
     }
   }
   tc::tc_fence_before();
   __syncthreads();
-  if (warp == 1) tc::tmem_dealloc(tmem_base, BN);
+  if (warp == 1) tc::tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -180,7 +226,7 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-constexpr int BN_DEFAULT = 128, STAGES_DEFAULT = 6;
+constexpr int BN_SMALL = 128;
 
 }  // namespace
 
@@ -198,7 +244,7 @@ bool fbl_encode_rtile_map(CUtensorMap* map, const void* base, int64_t r_pad, int
 
 bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g) {
   if (p->d.dtype != FBL_DTYPE_BF16) return false;
-  if (g.n % 64 != 0 || g.n < BN_DEFAULT || g.m < BM) return false;
+  if (g.n % 64 != 0 || g.n < BN_SMALL || g.m < BM) return false;
   for (int t = 0; t < g.n_terms; ++t) {
     const GemmTerm& tm = g.t[t];
     // a box must fit inside its tensor: rows of every operand cover one tile, K-major reduction axes are whole panels
@@ -209,13 +255,13 @@ bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g) {
   return true;
 }
 
-cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
-  if (count < 1 || count > MAX_PROBLEMS) return cudaErrorInvalidValue;
+template <int BN, int STAGES>
+cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
   TcGroup G;
   memset(&G, 0, sizeof(G));
   G.count = count;
   G.status = status;
-  int max_m = 0, max_n = 0;
+  int tiles = 0;
   for (int i = 0; i < count; ++i) {
     const GemmArgs& g = gs[i];
     TcProblem& P = G.p[i];
@@ -229,24 +275,35 @@ cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int coun
       if (tm.a_trans) ok = fbl_encode_rtile_map(&P.ta[t], tm.a, tm.a_rpad, g.m / 64, BK, BM / 64);
       else ok = fbl_encode_rtile_map(&P.ta[t], tm.a, tm.a_rpad, tm.k / 64, BM, 1);
       if (!ok) return cudaErrorInvalidValue;
-      if (tm.b_trans) ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, tm.k / 64, BN_DEFAULT, 1);
-      else ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, g.n / 64, BK, BN_DEFAULT / 64);
+      if (tm.b_trans) ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, tm.k / 64, BN, 1);
+      else ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, g.n / 64, BK, BN / 64);
       if (!ok) return cudaErrorInvalidValue;
     }
     P.m = g.m; P.n = g.n;
     P.c = (__nv_bfloat16*)g.c; P.c_rpad = g.c_rpad;
     P.bias = g.bias; P.residual = (const __nv_bfloat16*)g.residual;
     P.seq = g.seq; P.t_pad = g.t_pad;
-    max_m = g.m > max_m ? g.m : max_m;
-    max_n = g.n > max_n ? g.n : max_n;
+    tiles += ((g.m + BM - 1) / BM) * ((g.n + BN - 1) / BN);
   }
-  using SP = SmemPlan<BN_DEFAULT, STAGES_DEFAULT>;
-  auto k = gemm_tc_kernel<BN_DEFAULT, STAGES_DEFAULT>;
+  using SP = SmemPlan<BN, STAGES>;
+  auto k = gemm_tc_kernel<BN, STAGES>;
   cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
   if (attr_err != cudaSuccess) return attr_err;
-  dim3 grid((max_n + BN_DEFAULT - 1) / BN_DEFAULT, (max_m + BM - 1) / BM, count);
+  const int grid = tiles < p->sm_count ? tiles : p->sm_count;
   k<<<grid, 192, SP::TOTAL, st>>>(G);
   return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
+  if (count < 1 || count > MAX_PROBLEMS) return cudaErrorInvalidValue;
+  bool wide = true;                       // 128 x 256 tiles when every problem's N is whole 256-column blocks
+  for (int i = 0; i < count; ++i) {
+    wide = wide && gs[i].n % 256 == 0;
+    for (int t = 0; t < gs[i].n_terms; ++t)
+      if (gs[i].t[t].b_trans && gs[i].t[t].b_rpad < 256) wide = false;
+  }
+  if (wide) return launch_group_bn<256, 4>(p, gs, count, status, st);
+  return launch_group_bn<128, 6>(p, gs, count, status, st);
 }
 
 cudaError_t launch_gemm_tc(const fbl_plan* p, const GemmArgs& g, void*, size_t, int32_t* status, cudaStream_t st) {
