@@ -161,12 +161,17 @@ def main():
     ap.add_argument("--path", type=int, default=0, help="0 default kernels, 1 FFMA kernels only")
     ap.add_argument("--no-graph", action="store_true", help="enqueue kernels directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling captures)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "fblayout" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     cfg = get_config(args.config)
+    if args.seq or args.batch:
+        from fbl_inputs import scaled_config
+        cfg = scaled_config(cfg, name=cfg.name + "-scaled", seq=args.seq or cfg.seq, batch=args.batch or cfg.batch)
     if args.impl == "reference":
         run_reference(args, cfg, rank)
         return

@@ -290,27 +290,37 @@ struct alignas(64) AttnBwdParams {
   int32_t* status;
 };
 
+// HD = 64 has room (shared memory and TMEM) to pipeline: Q/dO and P^T/dS^T are double-buffered and dQ has
+// its own TMEM columns, so the tensor pipe computes the next tile's S^T / dP^T and this tile's dV, dK, dQ
+// while the softmax warps are busy.  HD = 128 fills TMEM (S^T, dP^T, dV, dK = 512 columns): dQ reuses the
+// S^T columns and the steps of one tile run back to back.
 template <int HD>
 struct BwdSmem {
+  static constexpr bool PIPE = HD == 64;
+  static constexpr uint32_t NQ = PIPE ? 2 : 1, NP = PIPE ? 2 : 1;
   static constexpr uint32_t PANELS = HD / 64;
   static constexpr uint32_t TILE = PANELS * 16384;
-  static constexpr uint32_t K_OFF = 0, V_OFF = TILE, Q_OFF = 2 * TILE, DO_OFF = 3 * TILE;
-  static constexpr uint32_t P_OFF = 4 * TILE, DS_OFF = P_OFF + 32768;
-  static constexpr uint32_t LSE_OFF = DS_OFF + 32768;        // 2 buffers x (128 floats LSE*log2e, 128 floats D)
+  static constexpr uint32_t K_OFF = 0, V_OFF = TILE, Q_OFF = 2 * TILE, DO_OFF = Q_OFF + NQ * TILE;
+  static constexpr uint32_t P_OFF = DO_OFF + NQ * TILE, DS_OFF = P_OFF + NP * 32768;
+  static constexpr uint32_t LSE_OFF = DS_OFF + NP * 32768;   // 2 buffers x (128 floats LSE*log2e, 128 floats D)
   static constexpr uint32_t BAR_OFF = LSE_OFF + 2048;
-  static constexpr uint32_t N_BARS = 8;
-  static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16 + 1024;
+  static constexpr uint32_t N_BARS = 10;
+  static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16;
 };
 
-enum { BB_KVFULL = 0, BB_QDOFULL, BB_QDOEMPTY, BB_SFULL, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY };
+enum { BB_KVFULL = 0, BB_QDOFULL = 1, BB_QDOEMPTY = 3, BB_SFULL = 5, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY };
+
+constexpr int BWD_THREADS = 320;     // warp 0 TMA, warp 1 MMA, warps 2-9 softmax / reduction (two per TMEM lane quarter)
 
 template <int HD>
-__global__ void __launch_bounds__(192, 1) attn_bwd_tc_kernel(const __grid_constant__ AttnBwdParams P) {
+__global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __grid_constant__ AttnBwdParams P) {
   using SM = BwdSmem<HD>;
-  constexpr uint32_t PANELS = SM::PANELS;
-  constexpr uint32_t S_COL = 0, DP_COL = 128, DV_COL = 256, DK_COL = 384, DQ_COL = 0, TMEM_COLS = 512;
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+  constexpr bool PIPE = SM::PIPE;
+  constexpr uint32_t PANELS = SM::PANELS, NQ = SM::NQ, NP = SM::NP;
+  constexpr uint32_t S_COL = 0, DP_COL = 128, DV_COL = 256, DK_COL = 256 + HD;
+  constexpr uint32_t DQ_COL = PIPE ? 384 : 0, TMEM_COLS = 512;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t base = tc::smem_u32(smem_raw);
   const uint32_t bars = base + SM::BAR_OFF;
   const uint32_t slot = bars + 8 * SM::N_BARS;
   auto bar = [&](int i) { return bars + 8u * i; };
@@ -319,18 +329,25 @@ __global__ void __launch_bounds__(192, 1) attn_bwd_tc_kernel(const __grid_consta
   const int row0 = b * P.t_pad;
   const int n_qt = (P.seq + BQ - 1) / BQ;
   const int qt_begin = P.causal ? j0 / BQ : 0;
-  const int n_it = P.group * (n_qt - qt_begin);
+  const int per_head = n_qt - qt_begin;
+  const int n_it = P.group * per_head;
   int32_t* status = P.status;
+  if ((base & 1023u) != 0) {                    // the swizzled tiles need a 1024-byte aligned window
+    if (threadIdx.x == 0) atomicCAS(status, 0, 399);
+    return;
+  }
 
   if (threadIdx.x == 0) {
     tc::mbar_init(bar(BB_KVFULL), 1);
-    tc::mbar_init(bar(BB_QDOFULL), 1);
-    tc::mbar_init(bar(BB_QDOEMPTY), 1);
+    for (int s = 0; s < 2; ++s) {
+      tc::mbar_init(bar(BB_QDOFULL + s), 1);
+      tc::mbar_init(bar(BB_QDOEMPTY + s), 1);
+    }
     tc::mbar_init(bar(BB_SFULL), 1);
-    tc::mbar_init(bar(BB_PDSFULL), 128);
+    tc::mbar_init(bar(BB_PDSFULL), 256);
     tc::mbar_init(bar(BB_DQFULL), 1);
-    tc::mbar_init(bar(BB_DQDRAINED), 128);
-    tc::mbar_init(bar(BB_LSEREADY), 128);
+    tc::mbar_init(bar(BB_DQDRAINED), 256);
+    tc::mbar_init(bar(BB_LSEREADY), 256);
     tc::fence_barrier_init();
   }
   if (warp == 1) {
@@ -348,155 +365,192 @@ __global__ void __launch_bounds__(192, 1) attn_bwd_tc_kernel(const __grid_consta
     tc::mbar_expect_tx(bar(BB_KVFULL), 2 * SM::TILE);
     tc::tma_load_3d(base + SM::K_OFF, &P.tk, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
     tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
-    int it = 0;
-    for (int hh = 0; hh < P.group; ++hh) {
-      const int h = g * P.group + hh;
-      for (int qt = qt_begin; qt < n_qt; ++qt, ++it) {
-        if (!tc::mbar_wait(bar(BB_QDOEMPTY), (it & 1) ^ 1, status, 301)) { hh = P.group; break; }
-        tc::mbar_expect_tx(bar(BB_QDOFULL), 2 * SM::TILE);
-        tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(BB_QDOFULL), 0, row0 + qt * BQ, h * (int)PANELS);
-        tc::tma_load_3d(base + SM::DO_OFF, &P.tdo, bar(BB_QDOFULL), 0, row0 + qt * BQ, h * (int)PANELS);
-      }
+    for (int it = 0; it < n_it; ++it) {
+      const int h = g * P.group + it / per_head, qt = qt_begin + it % per_head;
+      const uint32_t s = it % NQ, ph = (it / NQ) & 1;
+      if (!tc::mbar_wait(bar(BB_QDOEMPTY + s), ph ^ 1, status, 301)) break;
+      tc::mbar_expect_tx(bar(BB_QDOFULL + s), 2 * SM::TILE);
+      tc::tma_load_3d(base + SM::Q_OFF + s * SM::TILE, &P.tq, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
+      tc::tma_load_3d(base + SM::DO_OFF + s * SM::TILE, &P.tdo, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
     }
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer --------------------------------------------------------------------------
     const uint32_t idesc_s = tc::idesc_bf16(BKV, BQ, 0, 0);
     const uint32_t idesc_kv = tc::idesc_bf16(BKV, HD, 0, 1);
     const uint32_t idesc_dq = tc::idesc_bf16(BQ, HD, 1, 1);
-    bool ok = tc::mbar_wait(bar(BB_KVFULL), 0, status, 302);
-    for (int it = 0; it < n_it && ok; ++it) {
-      if (!tc::mbar_wait(bar(BB_QDOFULL), it & 1, status, 303)) { ok = false; break; }
-      if (it > 0 && !tc::mbar_wait(bar(BB_DQDRAINED), (it - 1) & 1, status, 304)) { ok = false; break; }
-      tc::tc_fence_after();
+    auto issue_sdp = [&](int it) {            // S^T = K Q^T and dP^T = V dO^T of tile `it`
+      const uint32_t qs = base + SM::Q_OFF + (it % NQ) * SM::TILE, dos = base + SM::DO_OFF + (it % NQ) * SM::TILE;
 #pragma unroll
       for (uint32_t kk = 0; kk < HD / 16; ++kk) {
         const uint32_t o = (kk / 4) * 16384 + (kk % 4) * 32;
         tc::mma_bf16_ss(tmem_base + S_COL, tc::smem_desc_sw128(base + SM::K_OFF + o, 16, 1024),
-                        tc::smem_desc_sw128(base + SM::Q_OFF + o, 16, 1024), idesc_s, kk > 0);
+                        tc::smem_desc_sw128(qs + o, 16, 1024), idesc_s, kk > 0);
       }
 #pragma unroll
       for (uint32_t kk = 0; kk < HD / 16; ++kk) {
         const uint32_t o = (kk / 4) * 16384 + (kk % 4) * 32;
         tc::mma_bf16_ss(tmem_base + DP_COL, tc::smem_desc_sw128(base + SM::V_OFF + o, 16, 1024),
-                        tc::smem_desc_sw128(base + SM::DO_OFF + o, 16, 1024), idesc_s, kk > 0);
+                        tc::smem_desc_sw128(dos + o, 16, 1024), idesc_s, kk > 0);
       }
       tc::mma_commit(bar(BB_SFULL));
-      if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
-      tc::tc_fence_after();
+    };
+    auto issue_grads = [&](int it) {          // dV += P^T dO, dK += dS^T Q, dQ = dS K of tile `it`
+      const uint32_t qs = base + SM::Q_OFF + (it % NQ) * SM::TILE, dos = base + SM::DO_OFF + (it % NQ) * SM::TILE;
+      const uint32_t ps = base + SM::P_OFF + (it % NP) * 32768, dss = base + SM::DS_OFF + (it % NP) * 32768;
 #pragma unroll
       for (uint32_t kk = 0; kk < BQ / 16; ++kk) {
         const uint32_t ao = (kk / 4) * 16384 + (kk % 4) * 32;      // P^T / dS^T: K-major, reduction over queries
         const uint32_t bo = kk * 2048;                             // dO / Q: MN-major, 16 query rows per step
-        tc::mma_bf16_ss(tmem_base + DV_COL, tc::smem_desc_sw128(base + SM::P_OFF + ao, 16, 1024),
-                        tc::smem_desc_sw128(base + SM::DO_OFF + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
+        tc::mma_bf16_ss(tmem_base + DV_COL, tc::smem_desc_sw128(ps + ao, 16, 1024),
+                        tc::smem_desc_sw128(dos + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
       }
 #pragma unroll
       for (uint32_t kk = 0; kk < BQ / 16; ++kk) {
         const uint32_t ao = (kk / 4) * 16384 + (kk % 4) * 32;
         const uint32_t bo = kk * 2048;
-        tc::mma_bf16_ss(tmem_base + DK_COL, tc::smem_desc_sw128(base + SM::DS_OFF + ao, 16, 1024),
-                        tc::smem_desc_sw128(base + SM::Q_OFF + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
+        tc::mma_bf16_ss(tmem_base + DK_COL, tc::smem_desc_sw128(dss + ao, 16, 1024),
+                        tc::smem_desc_sw128(qs + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
       }
 #pragma unroll
       for (uint32_t kk = 0; kk < BKV / 16; ++kk) {
         const uint32_t o = kk * 2048;                              // both operands MN-major: 16 key rows per step
-        tc::mma_bf16_ss(tmem_base + DQ_COL, tc::smem_desc_sw128(base + SM::DS_OFF + o, 16384, 1024),
+        tc::mma_bf16_ss(tmem_base + DQ_COL, tc::smem_desc_sw128(dss + o, 16384, 1024),
                         tc::smem_desc_sw128(base + SM::K_OFF + o, 16384, 1024), idesc_dq, kk > 0);
       }
       tc::mma_commit(bar(BB_DQFULL));
-      tc::mma_commit(bar(BB_QDOEMPTY));
+      tc::mma_commit(bar(BB_QDOEMPTY + (it % NQ)));
+    };
+    bool ok = tc::mbar_wait(bar(BB_KVFULL), 0, status, 302);
+    if (PIPE) {
+      if (ok && n_it > 0) {
+        ok = tc::mbar_wait(bar(BB_QDOFULL), 0, status, 303);
+        if (ok) { tc::tc_fence_after(); issue_sdp(0); }
+      }
+      for (int it = 0; it < n_it && ok; ++it) {
+        if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
+        if (it + 1 < n_it) {
+          if (!tc::mbar_wait(bar(BB_QDOFULL + ((it + 1) % NQ)), ((it + 1) / NQ) & 1, status, 303)) { ok = false; break; }
+          tc::tc_fence_after();
+          issue_sdp(it + 1);
+        }
+        if (it > 0 && !tc::mbar_wait(bar(BB_DQDRAINED), (it - 1) & 1, status, 304)) { ok = false; break; }
+        tc::tc_fence_after();
+        issue_grads(it);
+      }
+    } else {
+      for (int it = 0; it < n_it && ok; ++it) {
+        if (!tc::mbar_wait(bar(BB_QDOFULL + (it % NQ)), (it / NQ) & 1, status, 303)) { ok = false; break; }
+        if (it > 0 && !tc::mbar_wait(bar(BB_DQDRAINED), (it - 1) & 1, status, 304)) { ok = false; break; }
+        tc::tc_fence_after();
+        issue_sdp(it);
+        if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
+        tc::tc_fence_after();
+        issue_grads(it);
+      }
     }
   } else if (warp >= 2) {
-    // ---- softmax / reduction warps: one key row (then one query row of dQ) per thread ----------
-    const int q = warp % 4;
+    // ---- softmax / reduction warps: thread = (key row, half of the 128 query columns) -----------
+    const int q = warp % 4;                         // TMEM lane quarter
+    const int half = (warp - 2) / 4;                // which 64 query columns (and which half of HD later)
     const int r = q * 32 + lane;
-    const int t = threadIdx.x - 64;                 // 0..127
+    const int t = threadIdx.x - 64;                 // 0..255
     const int gj = j0 + r;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
     const float c = P.scale * LOG2E;
-    float* s_stage = reinterpret_cast<float*>(smem_raw + (base - tc::smem_u32(smem_raw)) + SM::LSE_OFF);
+    float* s_stage = reinterpret_cast<float*>(smem_raw + SM::LSE_OFF);
     bool ok = true;
-    int it = 0;
-    for (int hh = 0; hh < P.group && ok; ++hh) {
-      const int h = g * P.group + hh;
-      for (int qt = qt_begin; qt < n_qt && ok; ++qt, ++it) {
-        const int i0 = qt * BQ;
-        // LSE and D of this query tile, staged in shared memory (two buffers by iteration parity: every
-        // reader of the buffer's previous use arrived at PDSFULL two iterations ago)
-        float* s_lse = s_stage + (it & 1) * 256;
-        float* s_d = s_lse + 128;
-        {
-          const int gi = i0 + t;
-          const bool live = gi < P.seq;
-          const long long o = ((long long)b * P.hq + h) * P.t_pad + gi;
-          s_lse[t] = live ? P.lse[o] * LOG2E : INFINITY;
-          s_d[t] = live ? P.dvec[o] : 0.f;
-        }
-        tc::mbar_arrive(bar(BB_LSEREADY));
-        if (!tc::mbar_wait(bar(BB_LSEREADY), it & 1, status, 308)) { ok = false; break; }
-        if (!tc::mbar_wait(bar(BB_SFULL), it & 1, status, 306)) { ok = false; break; }
-        tc::tc_fence_after();
-        const bool diag = P.causal && (i0 < j0 + BKV - 1);
+
+    // dQ tile of iteration `dit`: row r is query i0 + r; this thread adds HD/2 of its columns
+    auto drain_dq = [&](int dit) -> bool {
+      const int h = g * P.group + dit / per_head, i0 = (qt_begin + dit % per_head) * BQ;
+      if (!tc::mbar_wait(bar(BB_DQFULL), dit & 1, status, 307)) return false;
+      tc::tc_fence_after();
+      const int gi = i0 + r;
 #pragma unroll 1
-        for (int cc = 0; cc < 4; ++cc) {
-          uint32_t sv[32], dpv[32];
-          tc::tmem_ld32(lane_addr + S_COL + cc * 32, sv);
-          tc::tmem_ld32(lane_addr + DP_COL + cc * 32, dpv);
-          tc::tmem_ld_wait();
-          uint32_t pp[16], dd[16];
+      for (int cc = 0; cc < HD / 64; ++cc) {
+        const int c0 = half * (HD / 2) + cc * 32;
+        uint32_t o[32];
+        tc::tmem_ld32(lane_addr + DQ_COL + c0, o);
+        tc::tmem_ld_wait();
+        if (gi < P.seq) {
+          const int col = h * HD + c0;
+          float* dst = P.dqacc + ((long long)(col / 64) * P.n_pad + row0 + gi) * 64 + (col % 64);
 #pragma unroll
-          for (int k = 0; k < 32; k += 2) {
-            float pv[2], dv[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-              const int col = cc * 32 + k + u;
-              float p = tc::fast_exp2(fmaf(__uint_as_float(sv[k + u]), c, -s_lse[col]));
-              if (gj >= P.seq || (diag && i0 + col < gj)) p = 0.f;
-              pv[u] = p;
-              dv[u] = p * (__uint_as_float(dpv[k + u]) - s_d[col]);
-            }
-            pp[k / 2] = tc::pack_bf16(pv[0], pv[1]);
-            dd[k / 2] = tc::pack_bf16(dv[0], dv[1]);
-          }
-          // 32 query columns = 64 bytes = 4 swizzled 16-byte chunks of this key row, in panel cc/2
-#pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {
-            const uint32_t chunk = (cc % 2) * 4 + ch;
-            const uint32_t off = (cc / 2) * 16384 + r * 128 + ((chunk ^ (r & 7)) * 16);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + SM::P_OFF + off), "r"(pp[ch * 4]),
-                         "r"(pp[ch * 4 + 1]), "r"(pp[ch * 4 + 2]), "r"(pp[ch * 4 + 3]) : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + SM::DS_OFF + off), "r"(dd[ch * 4]),
-                         "r"(dd[ch * 4 + 1]), "r"(dd[ch * 4 + 2]), "r"(dd[ch * 4 + 3]) : "memory");
+          for (int k = 0; k < 32; k += 4) {
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + k),
+                         "f"(__uint_as_float(o[k]) * P.scale), "f"(__uint_as_float(o[k + 1]) * P.scale),
+                         "f"(__uint_as_float(o[k + 2]) * P.scale), "f"(__uint_as_float(o[k + 3]) * P.scale)
+                         : "memory");
           }
         }
-        tc::fence_proxy_async();
-        tc::tc_fence_before();
-        tc::mbar_arrive(bar(BB_PDSFULL));
-        // dQ tile of this (key tile, query tile): row r is query i0 + r; add it to the fp32 accumulator
-        if (!tc::mbar_wait(bar(BB_DQFULL), it & 1, status, 307)) { ok = false; break; }
-        tc::tc_fence_after();
-        const int gi = i0 + r;
+      }
+      tc::tc_fence_before();
+      tc::mbar_arrive(bar(BB_DQDRAINED));
+      return true;
+    };
+
+    for (int it = 0; it < n_it && ok; ++it) {
+      const int h = g * P.group + it / per_head, i0 = (qt_begin + it % per_head) * BQ;
+      // LSE and D of this query tile, staged in shared memory (two buffers by iteration parity: every
+      // reader of a buffer's previous use arrived at PDSFULL two iterations ago)
+      float* s_lse = s_stage + (it & 1) * 256;
+      float* s_d = s_lse + 128;
+      {
+        const int gi = i0 + (t & 127);
+        const bool live = gi < P.seq;
+        const long long o = ((long long)b * P.hq + h) * P.t_pad + gi;
+        if (t < 128) s_lse[t] = live ? P.lse[o] * LOG2E : INFINITY;
+        else s_d[t - 128] = live ? P.dvec[o] : 0.f;
+      }
+      tc::mbar_arrive(bar(BB_LSEREADY));
+      if (!tc::mbar_wait(bar(BB_LSEREADY), it & 1, status, 308)) { ok = false; break; }
+      if (!tc::mbar_wait(bar(BB_SFULL), it & 1, status, 306)) { ok = false; break; }
+      tc::tc_fence_after();
+      const bool diag = P.causal && (i0 < j0 + BKV - 1);
+      const uint32_t ps = base + SM::P_OFF + (it % NP) * 32768 + half * 16384 + r * 128;
+      const uint32_t dss = base + SM::DS_OFF + (it % NP) * 32768 + half * 16384 + r * 128;
 #pragma unroll 1
-        for (int cc = 0; cc < HD / 32; ++cc) {
-          uint32_t o[32];
-          tc::tmem_ld32(lane_addr + DQ_COL + cc * 32, o);
-          tc::tmem_ld_wait();
-          if (gi < P.seq) {
-            const int col = h * HD + cc * 32;
-            float* dst = P.dqacc + ((long long)(col / 64) * P.n_pad + row0 + gi) * 64 + (col % 64);
+      for (int cc = 0; cc < 2; ++cc) {
+        const int c0 = half * 64 + cc * 32;
+        uint32_t sv[32], dpv[32];
+        tc::tmem_ld32(lane_addr + S_COL + c0, sv);
+        tc::tmem_ld32(lane_addr + DP_COL + c0, dpv);
+        tc::tmem_ld_wait();
+        uint32_t pp[16], dd[16];
 #pragma unroll
-            for (int k = 0; k < 32; k += 4) {
-              asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + k),
-                           "f"(__uint_as_float(o[k]) * P.scale), "f"(__uint_as_float(o[k + 1]) * P.scale),
-                           "f"(__uint_as_float(o[k + 2]) * P.scale), "f"(__uint_as_float(o[k + 3]) * P.scale)
-                           : "memory");
-            }
+        for (int k = 0; k < 32; k += 2) {
+          float pv[2], dv[2];
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int col = c0 + k + u;
+            float p = tc::fast_exp2(fmaf(__uint_as_float(sv[k + u]), c, -s_lse[col]));
+            if (gj >= P.seq || (diag && i0 + col < gj)) p = 0.f;
+            pv[u] = p;
+            dv[u] = p * (__uint_as_float(dpv[k + u]) - s_d[col]);
           }
+          pp[k / 2] = tc::pack_bf16(pv[0], pv[1]);
+          dd[k / 2] = tc::pack_bf16(dv[0], dv[1]);
         }
-        tc::tc_fence_before();
-        tc::mbar_arrive(bar(BB_DQDRAINED));
+        // 32 query columns = 4 swizzled 16-byte chunks of this key row inside the 64-query panel `half`
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          const uint32_t off = (((uint32_t)(cc * 4 + ch)) ^ (uint32_t)(r & 7)) * 16;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ps + off), "r"(pp[ch * 4]),
+                       "r"(pp[ch * 4 + 1]), "r"(pp[ch * 4 + 2]), "r"(pp[ch * 4 + 3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dss + off), "r"(dd[ch * 4]),
+                       "r"(dd[ch * 4 + 1]), "r"(dd[ch * 4 + 2]), "r"(dd[ch * 4 + 3]) : "memory");
+        }
+      }
+      tc::fence_proxy_async();
+      tc::tc_fence_before();
+      tc::mbar_arrive(bar(BB_PDSFULL));
+      if (PIPE) {
+        if (it > 0) ok = drain_dq(it - 1);
+      } else {
+        ok = drain_dq(it);
       }
     }
+    if (PIPE && ok && n_it > 0) ok = drain_dq(n_it - 1);
     // dK, dV of this key tile: every MMA has completed (the last dQ wait covered them)
     if (ok && n_it > 0) {
       const bool live = gj < P.seq;
@@ -505,12 +559,13 @@ __global__ void __launch_bounds__(192, 1) attn_bwd_tc_kernel(const __grid_consta
         __nv_bfloat16* out = which ? P.dk : P.dv;
         const float f = live ? (which ? P.scale : 1.f) : 0.f;
 #pragma unroll 1
-        for (int cc = 0; cc < HD / 32; ++cc) {
+        for (int cc = 0; cc < HD / 64; ++cc) {
+          const int c0 = half * (HD / 2) + cc * 32;
           uint32_t o[32];
-          tc::tmem_ld32(lane_addr + (which ? DK_COL : DV_COL) + cc * 32, o);   // warp-collective: no lane may skip it
+          tc::tmem_ld32(lane_addr + (which ? DK_COL : DV_COL) + c0, o);   // warp-collective: no lane may skip it
           tc::tmem_ld_wait();
           if (gj < P.t_pad) {
-            const int col = g * HD + cc * 32;
+            const int col = g * HD + c0;
             __nv_bfloat16* dst = out + ((long long)(col / 64) * P.n_pad + row0 + gj) * 64 + (col % 64);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -549,7 +604,7 @@ cudaError_t bwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdSmem<HD>::TOTAL);
   if (e != cudaSuccess) return e;
   dim3 grid((p->t_pad + BKV - 1) / BKV, p->d.n_kv_heads, p->d.batch);
-  k<<<grid, 192, BwdSmem<HD>::TOTAL, st>>>(P);
+  k<<<grid, BWD_THREADS, BwdSmem<HD>::TOTAL, st>>>(P);
   return cudaGetLastError();
 }
 
