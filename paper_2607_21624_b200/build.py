@@ -31,6 +31,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         objs.append(obj)
         cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
                "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd[1:1] = os.environ.get("FBL_NVCC_FLAGS", "").split()
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")

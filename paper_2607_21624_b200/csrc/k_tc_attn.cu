@@ -9,6 +9,8 @@
 // boxes and of the output rows, no data is rearranged.
 #include <string.h>
 
+#include <type_traits>
+
 #include "fbl_internal.h"
 #include "tc_common.cuh"
 
@@ -278,7 +280,7 @@ cudaError_t fwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
 //                  reduction across blocks, added to an fp32 buffer with vector red operations.
 // ---------------------------------------------------------------------------------------------------
 struct alignas(64) AttnBwdParams {
-  CUtensorMap tq, tk, tv, tdo;
+  CUtensorMap tq, tk, tv, tdo, tdq;   // tdq: fp32 dQ accumulator, target of the bulk reductions
   const float* lse;      // [B, Hq, t_pad]
   const float* dvec;     // [B, Hq, t_pad]   D = rowsum(dO * O)
   float* dqacc;          // fp32 [n_pad, dq] in the bf16 tile order
@@ -293,7 +295,7 @@ struct alignas(64) AttnBwdParams {
 // HD = 64 has room (shared memory and TMEM) to pipeline: Q/dO and P^T/dS^T are double-buffered and dQ has
 // its own TMEM columns, so the tensor pipe computes the next tile's S^T / dP^T and this tile's dV, dK, dQ
 // while the softmax warps are busy.  HD = 128 fills TMEM (S^T, dP^T, dV, dK = 512 columns): dQ reuses the
-// S^T columns and the steps of one tile run back to back.
+// dP^T columns, so only the next tile's S^T can be issued before dQ has been drained.
 template <int HD>
 struct BwdSmem {
   static constexpr bool PIPE = HD == 64;
@@ -304,13 +306,21 @@ struct BwdSmem {
   static constexpr uint32_t P_OFF = DO_OFF + NQ * TILE, DS_OFF = P_OFF + NP * 32768;
   static constexpr uint32_t LSE_OFF = DS_OFF + NP * 32768;   // 2 buffers x (128 floats LSE*log2e, 128 floats D)
   static constexpr uint32_t BAR_OFF = LSE_OFF + 2048;
-  static constexpr uint32_t N_BARS = 10;
+  static constexpr uint32_t N_BARS = 12;
   static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16;
 };
 
-enum { BB_KVFULL = 0, BB_QDOFULL = 1, BB_QDOEMPTY = 3, BB_SFULL = 5, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY };
+enum { BB_KVFULL = 0, BB_QDOFULL = 1, BB_QDOEMPTY = 3, BB_SFULL = 5, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY, BB_DQSTAGED, BB_STAGEFREE };
 
-constexpr int BWD_THREADS = 320;     // warp 0 TMA, warp 1 MMA, warps 2-9 softmax / reduction (two per TMEM lane quarter)
+// Optional timeline probe (compile with -DFBL_TRACE): block (0,0,0) records clock64() at the marked points of
+// iterations 8..14 into the 1 KiB status area, after the status word.
+#ifdef FBL_TRACE
+#define TR(k) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && it >= 8 && it < 11) ((long long*)P.status)[8 + (it - 8) * 32 + (k)] = clock64(); } while (0)
+#else
+#define TR(k) do { } while (0)
+#endif
+constexpr int BWD_THREADS = 608;     // warp 0 TMA loads, warp 1 MMA, warps 2-17 softmax (four per TMEM lane quarter), warp 18 dQ reductions
+constexpr int BWD_SM_THREADS = 512;
 
 template <int HD>
 __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __grid_constant__ AttnBwdParams P) {
@@ -318,7 +328,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
   constexpr bool PIPE = SM::PIPE;
   constexpr uint32_t PANELS = SM::PANELS, NQ = SM::NQ, NP = SM::NP;
   constexpr uint32_t S_COL = 0, DP_COL = 128, DV_COL = 256, DK_COL = 256 + HD;
-  constexpr uint32_t DQ_COL = PIPE ? 384 : 0, TMEM_COLS = 512;
+  constexpr uint32_t DQ_COL = PIPE ? 384 : DP_COL, TMEM_COLS = 512;   // HD = 128: dQ reuses the dP^T columns
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = tc::smem_u32(smem_raw);
   const uint32_t bars = base + SM::BAR_OFF;
@@ -344,10 +354,12 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       tc::mbar_init(bar(BB_QDOEMPTY + s), 1);
     }
     tc::mbar_init(bar(BB_SFULL), 1);
-    tc::mbar_init(bar(BB_PDSFULL), 256);
+    tc::mbar_init(bar(BB_PDSFULL), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_DQFULL), 1);
-    tc::mbar_init(bar(BB_DQDRAINED), 256);
-    tc::mbar_init(bar(BB_LSEREADY), 256);
+    tc::mbar_init(bar(BB_DQDRAINED), BWD_SM_THREADS);
+    tc::mbar_init(bar(BB_LSEREADY), BWD_SM_THREADS);
+    tc::mbar_init(bar(BB_DQSTAGED), BWD_SM_THREADS);
+    tc::mbar_init(bar(BB_STAGEFREE), 1);
     tc::fence_barrier_init();
   }
   if (warp == 1) {
@@ -378,14 +390,17 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     const uint32_t idesc_s = tc::idesc_bf16(BKV, BQ, 0, 0);
     const uint32_t idesc_kv = tc::idesc_bf16(BKV, HD, 0, 1);
     const uint32_t idesc_dq = tc::idesc_bf16(BQ, HD, 1, 1);
-    auto issue_sdp = [&](int it) {            // S^T = K Q^T and dP^T = V dO^T of tile `it`
-      const uint32_t qs = base + SM::Q_OFF + (it % NQ) * SM::TILE, dos = base + SM::DO_OFF + (it % NQ) * SM::TILE;
+    auto issue_s = [&](int it) {              // S^T = K Q^T of tile `it`
+      const uint32_t qs = base + SM::Q_OFF + (it % NQ) * SM::TILE;
 #pragma unroll
       for (uint32_t kk = 0; kk < HD / 16; ++kk) {
         const uint32_t o = (kk / 4) * 16384 + (kk % 4) * 32;
         tc::mma_bf16_ss(tmem_base + S_COL, tc::smem_desc_sw128(base + SM::K_OFF + o, 16, 1024),
                         tc::smem_desc_sw128(qs + o, 16, 1024), idesc_s, kk > 0);
       }
+    };
+    auto issue_dp = [&](int it) {             // dP^T = V dO^T of tile `it`; then both score tiles are announced
+      const uint32_t dos = base + SM::DO_OFF + (it % NQ) * SM::TILE;
 #pragma unroll
       for (uint32_t kk = 0; kk < HD / 16; ++kk) {
         const uint32_t o = (kk / 4) * 16384 + (kk % 4) * 32;
@@ -411,6 +426,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         tc::mma_bf16_ss(tmem_base + DK_COL, tc::smem_desc_sw128(dss + ao, 16, 1024),
                         tc::smem_desc_sw128(qs + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
       }
+      tc::mma_commit(bar(BB_QDOEMPTY + (it % NQ)));                // Q / dO of this tile are not read again:
+                                                                   // the next tile's TMA overlaps dQ and its drain
 #pragma unroll
       for (uint32_t kk = 0; kk < BKV / 16; ++kk) {
         const uint32_t o = kk * 2048;                              // both operands MN-major: 16 key rows per step
@@ -418,137 +435,211 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
                         tc::smem_desc_sw128(base + SM::K_OFF + o, 16384, 1024), idesc_dq, kk > 0);
       }
       tc::mma_commit(bar(BB_DQFULL));
-      tc::mma_commit(bar(BB_QDOEMPTY + (it % NQ)));
     };
     bool ok = tc::mbar_wait(bar(BB_KVFULL), 0, status, 302);
+    if (ok && n_it > 0) {
+      ok = tc::mbar_wait(bar(BB_QDOFULL), 0, status, 303);
+      if (ok) { tc::tc_fence_after(); issue_s(0); issue_dp(0); }
+    }
     if (PIPE) {
-      if (ok && n_it > 0) {
-        ok = tc::mbar_wait(bar(BB_QDOFULL), 0, status, 303);
-        if (ok) { tc::tc_fence_after(); issue_sdp(0); }
-      }
       for (int it = 0; it < n_it && ok; ++it) {
+        TR(0);
         if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
+        TR(1);
         if (it + 1 < n_it) {
           if (!tc::mbar_wait(bar(BB_QDOFULL + ((it + 1) % NQ)), ((it + 1) / NQ) & 1, status, 303)) { ok = false; break; }
+          TR(2);
           tc::tc_fence_after();
-          issue_sdp(it + 1);
+          issue_s(it + 1);
+          issue_dp(it + 1);
         }
+        TR(3);
         if (it > 0 && !tc::mbar_wait(bar(BB_DQDRAINED), (it - 1) & 1, status, 304)) { ok = false; break; }
+        TR(4);
         tc::tc_fence_after();
         issue_grads(it);
+        TR(5);
       }
     } else {
       for (int it = 0; it < n_it && ok; ++it) {
-        if (!tc::mbar_wait(bar(BB_QDOFULL + (it % NQ)), (it / NQ) & 1, status, 303)) { ok = false; break; }
-        if (it > 0 && !tc::mbar_wait(bar(BB_DQDRAINED), (it - 1) & 1, status, 304)) { ok = false; break; }
-        tc::tc_fence_after();
-        issue_sdp(it);
+        TR(0);
         if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
+        TR(1);
         tc::tc_fence_after();
         issue_grads(it);
+        TR(2);
+        if (it + 1 < n_it) {
+          if (!tc::mbar_wait(bar(BB_QDOFULL), (it + 1) & 1, status, 303)) { ok = false; break; }
+          TR(3);
+          tc::tc_fence_after();
+          issue_s(it + 1);                   // the S^T columns were released by PDSFULL
+          if (!tc::mbar_wait(bar(BB_DQDRAINED), it & 1, status, 304)) { ok = false; break; }
+          TR(4);
+          tc::tc_fence_after();
+          issue_dp(it + 1);                  // the dP^T columns held dQ until it was drained
+          TR(5);
+        }
       }
     }
+  } else if (warp == 18) {
+    // ---- dQ reduction warp: adds each staged dQ tile to the fp32 accumulator with bulk tensor reductions ----
+    if (lane == 0) {
+      for (int dit = 0; dit < n_it; ++dit) {
+        const int h = g * P.group + dit / per_head, i0 = (qt_begin + dit % per_head) * BQ;
+        if (!tc::mbar_wait(bar(BB_DQSTAGED), dit & 1, status, 309)) break;
+        const uint32_t stage = base + SM::P_OFF + (dit % NP) * 32768;
+#pragma unroll
+        for (int pn = 0; pn < (int)PANELS; ++pn)
+          tc::tma_reduce_add_4d(&P.tdq, stage + pn * 32768, 0, 0, row0 + i0, h * (int)PANELS + pn);
+        tc::bulk_commit_group();
+        tc::bulk_wait_group_read0();                 // the staging tile has been read: it may be overwritten
+        tc::mbar_arrive(bar(BB_STAGEFREE));
+      }
+      tc::bulk_wait_group0();
+    }
   } else if (warp >= 2) {
-    // ---- softmax / reduction warps: thread = (key row, half of the 128 query columns) -----------
+    // ---- softmax warps: thread = (key row, one quarter of the 128 query columns) -----------------------
     const int q = warp % 4;                         // TMEM lane quarter
-    const int half = (warp - 2) / 4;                // which 64 query columns (and which half of HD later)
+    const int part = (warp - 2) / 4;                // which 32 query columns (and which quarter of HD later)
     const int r = q * 32 + lane;
-    const int t = threadIdx.x - 64;                 // 0..255
+    const int t = threadIdx.x - 64;                 // 0..511
     const int gj = j0 + r;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
     const float c = P.scale * LOG2E;
     float* s_stage = reinterpret_cast<float*>(smem_raw + SM::LSE_OFF);
     bool ok = true;
 
-    // dQ tile of iteration `dit`: row r is query i0 + r; this thread adds HD/2 of its columns
+    // dQ tile of iteration `dit` (row = query i0 + row): each thread copies its TMEM row segment, scaled, to a
+    // staging tile in shared memory (the P^T buffer of that iteration, free once its MMAs are done) in the
+    // 128-byte-swizzled box layout of the accumulator's tensor map; the reduction warp then adds the whole
+    // tile to global memory asynchronously, off the critical path of these warps.
     auto drain_dq = [&](int dit) -> bool {
-      const int h = g * P.group + dit / per_head, i0 = (qt_begin + dit % per_head) * BQ;
+      const uint32_t stage = base + SM::P_OFF + (dit % NP) * 32768;
       if (!tc::mbar_wait(bar(BB_DQFULL), dit & 1, status, 307)) return false;
+      { const int it = dit; if (t == 0) TR(8); }
       tc::tc_fence_after();
-      const int gi = i0 + r;
 #pragma unroll 1
       for (int cc = 0; cc < HD / 64; ++cc) {
-        const int c0 = half * (HD / 2) + cc * 32;
-        uint32_t o[32];
-        tc::tmem_ld32(lane_addr + DQ_COL + c0, o);
+        const int c0 = part * (HD / 4) + cc * 16;    // first of this thread's 16 columns
+        uint32_t o[16];
+        tc::tmem_ld16(lane_addr + DQ_COL + c0, o);
         tc::tmem_ld_wait();
-        if (gi < P.seq) {
-          const int col = h * HD + c0;
-          float* dst = P.dqacc + ((long long)(col / 64) * P.n_pad + row0 + gi) * 64 + (col % 64);
+        const uint32_t unit = (uint32_t)(r * 2 + (c0 % 64) / 32);                 // 128-byte unit of the box
+        const uint32_t rowaddr = stage + (c0 / 64) * 32768 + unit * 128;
 #pragma unroll
-          for (int k = 0; k < 32; k += 4) {
-            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + k),
-                         "f"(__uint_as_float(o[k]) * P.scale), "f"(__uint_as_float(o[k + 1]) * P.scale),
-                         "f"(__uint_as_float(o[k + 2]) * P.scale), "f"(__uint_as_float(o[k + 3]) * P.scale)
-                         : "memory");
-          }
+        for (int k = 0; k < 4; ++k) {
+          const uint32_t chk = (uint32_t)((c0 % 32) / 4 + k);
+          const uint32_t addr = rowaddr + ((chk ^ (unit & 7)) * 16);
+          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(__uint_as_float(o[4 * k]) * P.scale),
+                       "f"(__uint_as_float(o[4 * k + 1]) * P.scale), "f"(__uint_as_float(o[4 * k + 2]) * P.scale),
+                       "f"(__uint_as_float(o[4 * k + 3]) * P.scale) : "memory");
         }
       }
       tc::tc_fence_before();
-      tc::mbar_arrive(bar(BB_DQDRAINED));
+      { const int it = dit; if (t == 0) TR(7); }
+      tc::mbar_arrive(bar(BB_DQDRAINED));            // TMEM side done: the tensor pipe may reuse the columns
+      tc::fence_proxy_async();
+      tc::mbar_arrive(bar(BB_DQSTAGED));             // staging side done: the reduction warp takes over
       return true;
     };
 
+    // LSE / D of a query tile: thread t < 128 fetches LSE[t], thread 128 <= t < 256 fetches D[t - 128].  The
+    // value for the next iteration is requested one iteration ahead so its latency is off the critical path.
+    auto fetch_stat = [&](int fit) -> float {
+      if (t >= 256 || fit >= n_it) return 0.f;
+      const int h = g * P.group + fit / per_head, i0 = (qt_begin + fit % per_head) * BQ;
+      const int gi = i0 + (t & 127);
+      const long long o = ((long long)b * P.hq + h) * P.t_pad + gi;
+      if (gi >= P.seq) return t < 128 ? INFINITY : 0.f;
+      return t < 128 ? P.lse[o] * LOG2E : P.dvec[o];
+    };
+    float stat_next = fetch_stat(0);
+
     for (int it = 0; it < n_it && ok; ++it) {
-      const int h = g * P.group + it / per_head, i0 = (qt_begin + it % per_head) * BQ;
+      const int i0 = (qt_begin + it % per_head) * BQ;
       // LSE and D of this query tile, staged in shared memory (two buffers by iteration parity: every
-      // reader of a buffer's previous use arrived at PDSFULL two iterations ago)
+      // reader of a buffer's previous use arrived at PDSFULL two iterations ago).  All threads pass this
+      // barrier only after finishing the previous iteration, including its reads of the dQ staging tile.
       float* s_lse = s_stage + (it & 1) * 256;
       float* s_d = s_lse + 128;
-      {
-        const int gi = i0 + (t & 127);
-        const bool live = gi < P.seq;
-        const long long o = ((long long)b * P.hq + h) * P.t_pad + gi;
-        if (t < 128) s_lse[t] = live ? P.lse[o] * LOG2E : INFINITY;
-        else s_d[t - 128] = live ? P.dvec[o] : 0.f;
-      }
+      if (t < 256) s_lse[t] = stat_next;             // s_d follows s_lse: one 256-float buffer
+      stat_next = fetch_stat(it + 1);
       tc::mbar_arrive(bar(BB_LSEREADY));
       if (!tc::mbar_wait(bar(BB_LSEREADY), it & 1, status, 308)) { ok = false; break; }
+      if (t == 0) TR(9);
       if (!tc::mbar_wait(bar(BB_SFULL), it & 1, status, 306)) { ok = false; break; }
+      if (t == 0) TR(10);
       tc::tc_fence_after();
-      const bool diag = P.causal && (i0 < j0 + BKV - 1);
-      const uint32_t ps = base + SM::P_OFF + (it % NP) * 32768 + half * 16384 + r * 128;
-      const uint32_t dss = base + SM::DS_OFF + (it % NP) * 32768 + half * 16384 + r * 128;
-#pragma unroll 1
-      for (int cc = 0; cc < 2; ++cc) {
-        const int c0 = half * 64 + cc * 32;
-        uint32_t sv[32], dpv[32];
-        tc::tmem_ld32(lane_addr + S_COL + c0, sv);
-        tc::tmem_ld32(lane_addr + DP_COL + c0, dpv);
+      // element masks are needed only on the diagonal tile and on tiles with keys or queries beyond the sequence
+      const bool need_mask = (P.causal && (i0 < j0 + BKV - 1)) || (j0 + BKV > P.seq) || (i0 + BQ > P.seq);
+      const uint32_t prow = (it % NP) * 32768 + (part / 2) * 16384 + r * 128;
+      // One 16-column chunk: P^T = exp2(S^T c - LSE), dS^T = P^T (dP^T - D), both rounded to bf16 and written
+      // to the swizzled operand tiles.  MASKED is the rare path (diagonal / ragged tiles).
+      auto chunk = [&](int cc, auto masked_tag) {
+        constexpr bool MASKED = decltype(masked_tag)::value;
+        const int c0 = part * 32 + cc * 16;
+        uint32_t sv[16], dpv[16];
+        tc::tmem_ld16(lane_addr + S_COL + c0, sv);
+        tc::tmem_ld16(lane_addr + DP_COL + c0, dpv);
         tc::tmem_ld_wait();
-        uint32_t pp[16], dd[16];
+        uint32_t pp[8], dd[8];
 #pragma unroll
-        for (int k = 0; k < 32; k += 2) {
-          float pv[2], dv[2];
+        for (int k = 0; k < 16; k += 4) {
+          const float4 l4 = *reinterpret_cast<const float4*>(&s_lse[c0 + k]);
+          const float4 d4 = *reinterpret_cast<const float4*>(&s_d[c0 + k]);
+          const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dvv[4] = {d4.x, d4.y, d4.z, d4.w};
+          float pv[4], gv[4];
 #pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const int col = c0 + k + u;
-            float p = tc::fast_exp2(fmaf(__uint_as_float(sv[k + u]), c, -s_lse[col]));
-            if (gj >= P.seq || (diag && i0 + col < gj)) p = 0.f;
+          for (int u = 0; u < 4; ++u) {
+            float p = tc::fast_exp2(fmaf(__uint_as_float(sv[k + u]), c, -lv[u]));
+            if (MASKED) {
+              const int gi = i0 + c0 + k + u;
+              if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) p = 0.f;
+            }
             pv[u] = p;
-            dv[u] = p * (__uint_as_float(dpv[k + u]) - s_d[col]);
+            gv[u] = p * (__uint_as_float(dpv[k + u]) - dvv[u]);
           }
           pp[k / 2] = tc::pack_bf16(pv[0], pv[1]);
-          dd[k / 2] = tc::pack_bf16(dv[0], dv[1]);
+          pp[k / 2 + 1] = tc::pack_bf16(pv[2], pv[3]);
+          dd[k / 2] = tc::pack_bf16(gv[0], gv[1]);
+          dd[k / 2 + 1] = tc::pack_bf16(gv[2], gv[3]);
         }
-        // 32 query columns = 4 swizzled 16-byte chunks of this key row inside the 64-query panel `half`
+        if (t == 0) TR(16 + cc);
+        // 16 query columns = 2 swizzled 16-byte chunks of this key row inside its 64-query panel
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          const uint32_t off = (((uint32_t)(cc * 4 + ch)) ^ (uint32_t)(r & 7)) * 16;
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ps + off), "r"(pp[ch * 4]),
+        for (int ch = 0; ch < 2; ++ch) {
+          const uint32_t chk = (uint32_t)((part % 2) * 4 + cc * 2 + ch);
+          const uint32_t off = prow + ((chk ^ (uint32_t)(r & 7)) * 16);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + SM::P_OFF + off), "r"(pp[ch * 4]),
                        "r"(pp[ch * 4 + 1]), "r"(pp[ch * 4 + 2]), "r"(pp[ch * 4 + 3]) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dss + off), "r"(dd[ch * 4]),
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + SM::DS_OFF + off), "r"(dd[ch * 4]),
                        "r"(dd[ch * 4 + 1]), "r"(dd[ch * 4 + 2]), "r"(dd[ch * 4 + 3]) : "memory");
         }
+      };
+      {
+        // the P^T (and, for HD = 128, dS^T) buffer written next was the staging tile of an earlier drain
+        const int last = PIPE ? it - 2 : it - 1;
+        if (last >= 0 && !tc::mbar_wait(bar(BB_STAGEFREE), last & 1, status, 310)) { ok = false; break; }
       }
+      if (need_mask) {
+        chunk(0, std::true_type{});
+        chunk(1, std::true_type{});
+      } else {
+        chunk(0, std::false_type{});
+        chunk(1, std::false_type{});
+      }
+      if (t == 0) TR(15);
       tc::fence_proxy_async();
+      if (t == 0) TR(6);
       tc::tc_fence_before();
       tc::mbar_arrive(bar(BB_PDSFULL));
+      if (t == 0) TR(11);
       if (PIPE) {
         if (it > 0) ok = drain_dq(it - 1);
       } else {
         ok = drain_dq(it);
       }
+      if (t == 0) TR(12);
     }
     if (PIPE && ok && n_it > 0) ok = drain_dq(n_it - 1);
     // dK, dV of this key tile: every MMA has completed (the last dQ wait covered them)
@@ -560,15 +651,15 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         const float f = live ? (which ? P.scale : 1.f) : 0.f;
 #pragma unroll 1
         for (int cc = 0; cc < HD / 64; ++cc) {
-          const int c0 = half * (HD / 2) + cc * 32;
-          uint32_t o[32];
-          tc::tmem_ld32(lane_addr + (which ? DK_COL : DV_COL) + c0, o);   // warp-collective: no lane may skip it
+          const int c0 = part * (HD / 4) + cc * 16;
+          uint32_t o[16];
+          tc::tmem_ld16(lane_addr + (which ? DK_COL : DV_COL) + c0, o);   // warp-collective: no lane may skip it
           tc::tmem_ld_wait();
           if (gj < P.t_pad) {
             const int col = g * HD + c0;
             __nv_bfloat16* dst = out + ((long long)(col / 64) * P.n_pad + row0 + gj) * 64 + (col % 64);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+            for (int k = 0; k < 2; ++k) {
               uint4 v;
               v.x = tc::pack_bf16(__uint_as_float(o[k * 8 + 0]) * f, __uint_as_float(o[k * 8 + 1]) * f);
               v.y = tc::pack_bf16(__uint_as_float(o[k * 8 + 2]) * f, __uint_as_float(o[k * 8 + 3]) * f);
@@ -597,6 +688,7 @@ cudaError_t bwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   if (!fbl_encode_rtile_map(&P.tdo, dA, p->n_pad, p->dq / 64, BQ, panels)) return cudaErrorInvalidValue;
   if (!fbl_encode_rtile_map(&P.tk, K, p->n_pad, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
   if (!fbl_encode_rtile_map(&P.tv, V, p->n_pad, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
+  if (!fbl_encode_f32_panel_map(&P.tdq, dqacc, p->n_pad, p->dq / 64, BQ)) return cudaErrorInvalidValue;
   P.lse = lse; P.dvec = dvec; P.dqacc = dqacc; P.dk = (__nv_bfloat16*)dK; P.dv = (__nv_bfloat16*)dV;
   P.n_pad = p->n_pad; P.seq = p->d.seq; P.t_pad = p->t_pad; P.hq = p->d.n_q_heads; P.group = p->group;
   P.causal = p->d.causal; P.dkv = p->dkv; P.scale = p->scale; P.status = status;

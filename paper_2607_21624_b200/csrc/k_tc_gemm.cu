@@ -242,6 +242,20 @@ bool fbl_encode_rtile_map(CUtensorMap* map, const void* base, int64_t r_pad, int
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 accumulator [n_pad, cols] stored in the bf16 tile order (64-column panels, 256-byte rows), viewed as
+// [panels][rows][2 halves][32 floats] so that a box of 128 rows x one panel can use the 128-byte swizzle.
+bool fbl_encode_f32_panel_map(CUtensorMap* map, const void* base, int64_t r_pad, int panels, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[4] = {32, 2, (cuuint64_t)r_pad, (cuuint64_t)panels};
+  cuuint64_t strides[3] = {128, 256, (cuuint64_t)r_pad * 256};
+  cuuint32_t box[4] = {32, 2, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g) {
   if (p->d.dtype != FBL_DTYPE_BF16) return false;
   if (g.n % 64 != 0 || g.n < BN_SMALL || g.m < BM) return false;

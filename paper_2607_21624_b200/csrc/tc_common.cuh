@@ -63,6 +63,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"((uint64_t)map), "r"(bar), "r"(x), "r"(y), "r"(z)
       : "memory");
 }
+// Element-wise fp32 add of a shared-memory tile into global memory (bulk tensor reduction, asynchronous).
+__device__ __forceinline__ void tma_reduce_add_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.reduce.async.bulk.tensor.4d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+      ::"l"((uint64_t)map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_group0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)map) : "memory");
 }
@@ -118,6 +128,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -150,6 +169,21 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// 2^x on the FMA and integer pipes (no transcendental unit): round x to the nearest integer n with the
+// 1.5 * 2^23 trick, evaluate a cubic for 2^f on f = x - n in [-0.5, 0.5] (relative error 7.5e-5, far below the
+// bf16 rounding the result goes through) and add n to the exponent field.  x must be finite; x below -126
+// returns a value below 1.2e-38.  The softmax loops evaluate part of their exponentials this way because
+// the transcendental unit is their busiest resource.
+__device__ __forceinline__ float exp2_poly3(float x) {
+  x = fmaxf(x, -126.f);
+  const float t = x + 12582912.f;
+  const float f = x - (t - 12582912.f);
+  float p = fmaf(0.0551716685f, f, 0.2426111251f);
+  p = fmaf(p, f, 0.6932609677f);
+  p = fmaf(p, f, 0.9999280572f);
+  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+
 // ---- operand descriptors --------------------------------------------------------------------------
 // Shared-memory matrix descriptor for 128-byte-swizzled tiles whose rows are 128 bytes (64 bf16).
 //   K-major  (reduction axis contiguous): rows are M/N indices, 8-row groups `sbo` bytes apart.
@@ -173,6 +207,14 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int m, int n, int a_mn_major, 
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+// Two fp32 -> packed bf16 pair with integer instructions only (round half up on the dropped 16 bits, then one
+// byte permute).  The float-to-bf16 conversion instruction shares the transcendental unit with ex2, which is
+// the busiest unit of the softmax loops; this keeps it free for the exponentials.  Differs from
+// round-to-nearest-even only on exact ties.  Inputs must be finite.
+__device__ __forceinline__ uint32_t pack_bf16_alu(float lo, float hi) {
+  return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -182,3 +224,4 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // Host side: encode a 3-D tensor map over an R-Tile bf16 matrix viewed as [panels][rows][64].
 bool fbl_encode_rtile_map(CUtensorMap* map, const void* base, int64_t r_pad, int panels, int box_rows, int box_panels);
+bool fbl_encode_f32_panel_map(CUtensorMap* map, const void* base, int64_t r_pad, int panels, int box_rows);
