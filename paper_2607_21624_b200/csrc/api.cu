@@ -130,7 +130,7 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   p->saved_bytes = o;
 
   // partial-sum area: column-sum slabs or split-K slices, whichever is larger
-  size_t part = colsum_scratch_bytes(p->n_pad, d.d_model > p->dq ? d.d_model : p->dq);
+  size_t part = colsum_scratch_bytes(p->n_pad, (int64_t)d.d_model + p->dq + 2 * p->dkv);
   const size_t splitk = (size_t)p->sm_count * 128 * 256 * sizeof(float) * 2;
   if (splitk > part) part = splitk;
   p->part_bytes = fbl_align_up(part, FBL_ALIGN);
@@ -385,40 +385,34 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
 
   FBL_CUDA(cudaMemsetAsync(status, 0, FBL_ALIGN, st));
   FBL_PROF_BEGIN();
-  {  // dA = dY Wo^T : Wo's tiles read with the roles of its two axes swapped
-    GemmArgs g = {};
-    g.m = n; g.n = p->dq; g.n_terms = 1;
-    g.t[0] = {dY, p->n_pad, 0, Wo, p->dq, 1, D};
-    g.c = dA; g.c_rpad = p->n_pad; g.seq = p->d.seq; g.t_pad = p->t_pad;
-    FBL_STEP("dA", 1, run_gemm(p, g, part, p->part_bytes, status, st));
+  {
+    GemmArgs gs[2];
+    GemmArgs& gw = gs[0];   // dWo = A^T dY : token-axis reduction (longest reduction loop: first in the work list)
+    gw = GemmArgs{};
+    gw.m = p->dq; gw.n = D; gw.n_terms = 1;
+    gw.t[0] = {A, p->n_pad, 1, dY, p->n_pad, 0, n};
+    gw.c = dWo; gw.c_rpad = p->dq;
+    GemmArgs& ga = gs[1];   // dA = dY Wo^T : Wo's tiles read with the roles of its two axes swapped
+    ga = GemmArgs{};
+    ga.m = n; ga.n = p->dq; ga.n_terms = 1;
+    ga.t[0] = {dY, p->n_pad, 0, Wo, p->dq, 1, D};
+    ga.c = dA; ga.c_rpad = p->n_pad; ga.seq = p->d.seq; ga.t_pad = p->t_pad;
+    if (p->use_tc && gemm_tc_supported(p, gw) && gemm_tc_supported(p, ga)) {
+      FBL_STEP("dWo+dA", 1, launch_gemm_tc_group(p, gs, 2, status, st));
+    } else {
+      FBL_STEP("dA", 1, run_gemm(p, ga, part, p->part_bytes, status, st));
+      FBL_STEP("dWo", 1, run_gemm(p, gw, part, p->part_bytes, status, st));
+    }
   }
-  {  // dWo = A^T dY : token-axis reduction
-    GemmArgs g = {};
-    g.m = p->dq; g.n = D; g.n_terms = 1;
-    g.t[0] = {A, p->n_pad, 1, dY, p->n_pad, 0, n};
-    g.c = dWo; g.c_rpad = p->dq;
-    FBL_STEP("dWo", 1, run_gemm(p, g, part, p->part_bytes, status, st));
-  }
-  if (bias) FBL_STEP("dbo", 2, launch_colsum(p->d.dtype, dY, p->n_pad, D, dbo, (float*)part, st));
   if (p->use_tc && attn_bwd_tc_supported(p)) FBL_STEP("attn_bwd", 3, launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, status, st));
   else FBL_STEP("attn_bwd", 3, launch_attn_bwd_simt(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, st));
-  {  // dXn = dQ Wq^T + dK Wk^T + dV Wv^T : one accumulator, three reduction loops
-    GemmArgs g = {};
-    g.m = n; g.n = D; g.n_terms = 3;
-    g.t[0] = {dQ, p->n_pad, 0, Wq, D, 1, p->dq};
-    g.t[1] = {dK, p->n_pad, 0, Wk, D, 1, p->dkv};
-    g.t[2] = {dV, p->n_pad, 0, Wv, D, 1, p->dkv};
-    g.c = dXn; g.c_rpad = p->n_pad; g.seq = p->d.seq; g.t_pad = p->t_pad;
-    FBL_STEP("dXn", 1, run_gemm(p, g, part, p->part_bytes, status, st));
-  }
   {
     const void* G[3] = {dQ, dK, dV};
     void* DW[3] = {dWq, dWk, dWv};
-    float* DB[3] = {dbq, dbk, dbv};
     const int cols[3] = {p->dq, p->dkv, p->dkv};
-    GemmArgs gs[3];
+    GemmArgs gs[4];
     bool tc = p->use_tc != 0;
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < 3; ++i) {   // dW* = Xn^T d* : token-axis reductions, Xn's tiles read MN-major
       GemmArgs& g = gs[i];
       g = GemmArgs{};
       g.m = D; g.n = cols[i]; g.n_terms = 1;
@@ -426,16 +420,27 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
       g.c = DW[i]; g.c_rpad = D;
       tc = tc && gemm_tc_supported(p, g);
     }
+    GemmArgs& gx = gs[3];           // dXn = dQ Wq^T + dK Wk^T + dV Wv^T : one accumulator, three reduction loops
+    gx = GemmArgs{};
+    gx.m = n; gx.n = D; gx.n_terms = 3;
+    gx.t[0] = {dQ, p->n_pad, 0, Wq, D, 1, p->dq};
+    gx.t[1] = {dK, p->n_pad, 0, Wk, D, 1, p->dkv};
+    gx.t[2] = {dV, p->n_pad, 0, Wv, D, 1, p->dkv};
+    gx.c = dXn; gx.c_rpad = p->n_pad; gx.seq = p->d.seq; gx.t_pad = p->t_pad;
+    tc = tc && gemm_tc_supported(p, gx);
     if (tc) {
-      FBL_STEP("dWqkv", 1, launch_gemm_tc_group(p, gs, 3, status, st));
+      FBL_STEP("dWqkv+dXn", 1, launch_gemm_tc_group(p, gs, 4, status, st));
     } else {
+      FBL_STEP("dXn", 1, run_gemm(p, gx, part, p->part_bytes, status, st));
       for (int i = 0; i < 3; ++i)
-        FBL_STEP(i == 0 ? "dWq" : i == 1 ? "dWk" : "dWv", 1, launch_gemm_simt(p->d.dtype, gs[i], st));
+        FBL_STEP(i == 0 ? "dWq" : i == 1 ? "dWk" : "dWv", 1, run_gemm(p, gs[i], part, p->part_bytes, status, st));
     }
-    if (bias)
-      for (int i = 0; i < 3; ++i)
-        FBL_STEP(i == 0 ? "dbq" : i == 1 ? "dbk" : "dbv", 2,
-                 launch_colsum(p->d.dtype, G[i], p->n_pad, cols[i], DB[i], (float*)part, st));
+    if (bias) {   // every bias gradient is a token-axis column sum: one pair of launches for the four of them
+      const void* M4[4] = {dY, dQ, dK, dV};
+      float* O4[4] = {dbo, dbq, dbk, dbv};
+      const int C4[4] = {D, p->dq, p->dkv, p->dkv};
+      FBL_STEP("db", 2, launch_colsum_group(p->d.dtype, 4, M4, p->n_pad, C4, O4, (float*)part, st));
+    }
   }
   FBL_STEP("norm_bwd", 1, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, st));
   return FBL_OK;

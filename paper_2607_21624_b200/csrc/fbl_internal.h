@@ -90,6 +90,8 @@ cudaError_t launch_norm_bwd(const fbl_plan* p, const void* dXn, const void* X, c
 cudaError_t launch_colsum(int dtype, const void* M, int64_t rows, int64_t cols, float* out, float* partials,
                           cudaStream_t st);
 size_t colsum_scratch_bytes(int64_t rows, int64_t cols);
+cudaError_t launch_colsum_group(int dtype, int count, const void* const* M, int64_t rows, const int* cols,
+                                float* const* out, float* partials, cudaStream_t st);
 
 cudaError_t launch_attn_fwd_simt(const fbl_plan* p, const void* Q, const void* K, const void* V, void* A, float* lse,
                                  cudaStream_t st);

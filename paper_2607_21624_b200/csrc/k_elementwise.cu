@@ -202,19 +202,185 @@ __global__ void __launch_bounds__(256) norm_bwd_kernel(const T* __restrict__ dXn
   }
 }
 
+
+// ------------------------------------------------------------------------------------------
+// Register-resident norm kernels for bf16 rows of up to 2048 columns (NV = D / 256 vectors of 16 bytes per
+// lane): one warp owns a row, lane l holds vectors l, l + 32, ... of it (each warp-level load covers four
+// whole 128-byte tile rows, one per column panel), so X (and dXn) cross HBM exactly once.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+template <int NV>
+__global__ void __launch_bounds__(256) norm_fwd_rows_kernel(const __nv_bfloat16* __restrict__ X,
+                                                            const float* __restrict__ gamma,
+                                                            const float* __restrict__ beta,
+                                                            __nv_bfloat16* __restrict__ Xn, float* __restrict__ stats,
+                                                            int64_t n_pad, int seq, int t_pad, int rms, float eps) {
+  constexpr int D = NV * 256;
+  const int lane = threadIdx.x % 32;
+  const int64_t warp0 = (int64_t)blockIdx.x * 8 + threadIdx.x / 32, nwarps = (int64_t)gridDim.x * 8;
+  for (int64_t r = warp0; r < n_pad; r += nwarps) {
+    const bool pad = (int)(r % t_pad) >= seq;
+    float x[NV][8];
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      const int v = j * 32 + lane;                         // vector index in the row: panel v / 8, chunk v % 8
+      load16(X + ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8, x[j]);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) s += x[j][i];
+    }
+    const float mean = rms ? 0.f : warp_sum(s) * (1.f / D);
+    float q = 0.f;
+#pragma unroll
+    for (int j = 0; j < NV; ++j)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { const float c = x[j][i] - mean; q += c * c; }
+    const float rstd = rsqrtf(warp_sum(q) * (1.f / D) + eps);
+    if (lane == 0) { stats[2 * r] = pad ? 0.f : mean; stats[2 * r + 1] = pad ? 0.f : rstd; }
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      const int v = j * 32 + lane;
+      const int c0 = v * 8;
+      const float4 g0 = *reinterpret_cast<const float4*>(gamma + c0), g1 = *reinterpret_cast<const float4*>(gamma + c0 + 4);
+      float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
+      if (beta) { b0 = *reinterpret_cast<const float4*>(beta + c0); b1 = *reinterpret_cast<const float4*>(beta + c0 + 4); }
+      const float gm[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+      const float bt[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+      float y[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) y[i] = pad ? 0.f : (x[j][i] - mean) * rstd * gm[i] + bt[i];
+      store16(Xn + ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8, y);
+    }
+  }
+}
+
+template <int NV>
+__global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16* __restrict__ dXn,
+                                                            const __nv_bfloat16* __restrict__ X,
+                                                            const __nv_bfloat16* __restrict__ dY,
+                                                            const float* __restrict__ stats,
+                                                            const float* __restrict__ gamma,
+                                                            __nv_bfloat16* __restrict__ dX, float* __restrict__ dgamma,
+                                                            float* __restrict__ dbeta, int64_t n_pad, int rms) {
+  constexpr int D = NV * 256;
+  __shared__ float s_dg[D];
+  __shared__ float s_db[D];
+  for (int i = threadIdx.x; i < D; i += 256) { s_dg[i] = 0.f; s_db[i] = 0.f; }
+  __syncthreads();
+  const int lane = threadIdx.x % 32;
+  const int64_t warp0 = (int64_t)blockIdx.x * 8 + threadIdx.x / 32, nwarps = (int64_t)gridDim.x * 8;
+  float gm[NV][8];
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    const int c0 = (j * 32 + lane) * 8;
+    const float4 g0 = *reinterpret_cast<const float4*>(gamma + c0), g1 = *reinterpret_cast<const float4*>(gamma + c0 + 4);
+    gm[j][0] = g0.x; gm[j][1] = g0.y; gm[j][2] = g0.z; gm[j][3] = g0.w;
+    gm[j][4] = g1.x; gm[j][5] = g1.y; gm[j][6] = g1.z; gm[j][7] = g1.w;
+  }
+  // token-axis partial sums of this warp's rows, kept in registers and folded into shared memory at the end
+  float ag[NV][8], ab[NV][8];
+#pragma unroll
+  for (int j = 0; j < NV; ++j)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { ag[j][i] = 0.f; ab[j][i] = 0.f; }
+  for (int64_t r = warp0; r < n_pad; r += nwarps) {
+    const float mean = stats[2 * r], rstd = stats[2 * r + 1];
+    float xh[NV][8], g[NV][8];
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      const int v = j * 32 + lane;
+      const int64_t off = ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8;
+      float gv[8];
+      load16(X + off, xh[j]);
+      load16(dXn + off, gv);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        xh[j][i] = (xh[j][i] - mean) * rstd;
+        ag[j][i] = fmaf(gv[i], xh[j][i], ag[j][i]);
+        ab[j][i] += gv[i];
+        g[j][i] = gv[i] * gm[j][i];
+        s1 += g[j][i];
+        s2 = fmaf(g[j][i], xh[j][i], s2);
+      }
+    }
+    s1 = rms ? 0.f : warp_sum(s1) * (1.f / D);
+    s2 = warp_sum(s2) * (1.f / D);
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      const int v = j * 32 + lane;
+      const int64_t off = ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8;
+      float o[8];
+      if (dY) load16(dY + off, o);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float dx = rstd * (g[j][i] - s1 - xh[j][i] * s2);
+        o[i] = dY ? o[i] + dx : dx;
+      }
+      store16(dX + off, o);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < NV; ++j)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int c = (j * 32 + lane) * 8 + i;
+      atomicAdd(&s_dg[c], ag[j][i]);
+      atomicAdd(&s_db[c], ab[j][i]);
+    }
+  __syncthreads();
+  for (int i = threadIdx.x; i < D; i += 256) {
+    atomicAdd(&dgamma[i], s_dg[i]);
+    if (dbeta) atomicAdd(&dbeta[i], s_db[i]);
+  }
+}
+
+template <int NV>
+void norm_fwd_rows_launch(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
+                          float* stats, int rms, cudaStream_t st) {
+  const int blocks = (int)min((int64_t)p->sm_count * 4, (p->n_pad + 7) / 8);
+  norm_fwd_rows_kernel<NV><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)X, gamma, rms ? nullptr : beta,
+                                                   (__nv_bfloat16*)Xn, stats, p->n_pad, p->d.seq, p->t_pad, rms, p->d.eps);
+}
+template <int NV>
+void norm_bwd_rows_launch(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
+                          const float* gamma, void* dX, float* dgamma, float* dbeta, int rms, cudaStream_t st) {
+  const int blocks = (int)min((int64_t)p->sm_count * 2, (p->n_pad + 7) / 8);
+  norm_bwd_rows_kernel<NV><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dXn, (const __nv_bfloat16*)X,
+                                                   (const __nv_bfloat16*)dY, stats, gamma, (__nv_bfloat16*)dX, dgamma,
+                                                   rms ? nullptr : dbeta, p->n_pad, rms);
+}
+
 // ------------------------------------------------------------------------------------------
 // Token-axis column sums, two stages over tiles: (1) one block per (panel, slab of 256 rows)
 // reduces its 32 storage tiles to one row of partials, (2) a tree over slabs.
 // ------------------------------------------------------------------------------------------
 constexpr int COLSUM_SLAB = 256;
 
+struct ColsumGroup {
+  const void* m[4];
+  float* out[4];
+  int cols[4];
+  int64_t part_off[4];      // float offset of each matrix's partials inside the scratch area
+  int count;
+};
+
 template <typename T>
-__global__ void __launch_bounds__(256) colsum_stage1(const T* __restrict__ M, int64_t rows, float* __restrict__ part,
-                                                     int cols) {
+__global__ void __launch_bounds__(256) colsum_stage1(ColsumGroup G, int64_t rows, float* __restrict__ part_base) {
   constexpr int TW = tile_w_of<T>::value;
   constexpr int V = Vec16<T>::N;
   __shared__ float red[32][TW + 1];
+  const int which = blockIdx.z;
+  const int cols = G.cols[which];
   const int p = blockIdx.x, slab = blockIdx.y;
+  if (p * TW >= cols) return;
+  const T* M = (const T*)G.m[which];
+  float* part = part_base + G.part_off[which];
   const int rr = threadIdx.x / 8, l8 = threadIdx.x % 8;
   float acc[V];
 #pragma unroll
@@ -237,12 +403,15 @@ __global__ void __launch_bounds__(256) colsum_stage1(const T* __restrict__ M, in
   }
 }
 
-__global__ void colsum_stage2(const float* __restrict__ part, int n_slabs, int cols, float* __restrict__ out) {
+__global__ void colsum_stage2(ColsumGroup G, const float* __restrict__ part_base, int n_slabs) {
+  const int which = blockIdx.y;
+  const int cols = G.cols[which];
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= cols) return;
+  const float* part = part_base + G.part_off[which];
   float s = 0.f;
   for (int k = 0; k < n_slabs; ++k) s += part[(int64_t)k * cols + c];
-  out[c] = s;
+  G.out[which][c] = s;
 }
 
 }  // namespace
@@ -267,6 +436,15 @@ cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma
                             float* stats, cudaStream_t st) {
   const int blocks = (int)((p->n_pad + 31) / 32);
   const int rms = p->d.norm == FBL_NORM_RMSNORM;
+  if (p->d.dtype == FBL_DTYPE_BF16 && p->d.d_model % 256 == 0 && p->d.d_model <= 1024) {
+    switch (p->d.d_model / 256) {
+      case 1: norm_fwd_rows_launch<1>(p, X, gamma, beta, Xn, stats, rms, st); break;
+      case 2: norm_fwd_rows_launch<2>(p, X, gamma, beta, Xn, stats, rms, st); break;
+      case 3: norm_fwd_rows_launch<3>(p, X, gamma, beta, Xn, stats, rms, st); break;
+      default: norm_fwd_rows_launch<4>(p, X, gamma, beta, Xn, stats, rms, st); break;
+    }
+    return cudaGetLastError();
+  }
   if (p->d.dtype == FBL_DTYPE_FP32)
     norm_fwd_kernel<float><<<blocks, 256, 0, st>>>((const float*)X, gamma, rms ? nullptr : beta, (float*)Xn, stats,
                                                    p->n_pad, p->d.d_model, p->d.seq, p->t_pad, rms, p->d.eps);
@@ -289,6 +467,15 @@ cudaError_t launch_norm_bwd(const fbl_plan* p, const void* dXn, const void* X, c
     e = cudaMemsetAsync(dbeta, 0, d * sizeof(float), st);
     if (e != cudaSuccess) return e;
   }
+  if (p->d.dtype == FBL_DTYPE_BF16 && d % 256 == 0 && d <= 1024) {
+    switch (d / 256) {
+      case 1: norm_bwd_rows_launch<1>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, rms, st); break;
+      case 2: norm_bwd_rows_launch<2>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, rms, st); break;
+      case 3: norm_bwd_rows_launch<3>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, rms, st); break;
+      default: norm_bwd_rows_launch<4>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, rms, st); break;
+    }
+    return cudaGetLastError();
+  }
   if (p->d.dtype == FBL_DTYPE_FP32) {
     auto k = norm_bwd_kernel<float>;
     if (sh > 48 * 1024) cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
@@ -309,20 +496,35 @@ size_t colsum_scratch_bytes(int64_t rows, int64_t cols) {
   return (size_t)(slabs * cols) * sizeof(float);
 }
 
-cudaError_t launch_colsum(int dtype, const void* M, int64_t rows, int64_t cols, float* out, float* partials,
-                          cudaStream_t st) {
+// Column sums of up to four matrices that share a row count, in one pair of launches.
+cudaError_t launch_colsum_group(int dtype, int count, const void* const* M, int64_t rows, const int* cols, float* const* out,
+                                float* partials, cudaStream_t st) {
+  if (count < 1 || count > 4) return cudaErrorInvalidValue;
   const int slabs = (int)((rows + COLSUM_SLAB - 1) / COLSUM_SLAB);
-  if (dtype == FBL_DTYPE_FP32) {
-    dim3 grid((unsigned)(cols / 32), slabs);
-    colsum_stage1<float><<<grid, 256, 0, st>>>((const float*)M, rows, partials, (int)cols);
-  } else {
-    dim3 grid((unsigned)(cols / 64), slabs);
-    colsum_stage1<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)M, rows, partials, (int)cols);
+  ColsumGroup G;
+  int max_cols = 0;
+  int64_t off = 0;
+  for (int i = 0; i < count; ++i) {
+    G.m[i] = M[i]; G.out[i] = out[i]; G.cols[i] = cols[i]; G.part_off[i] = off;
+    off += (int64_t)slabs * cols[i];
+    max_cols = cols[i] > max_cols ? cols[i] : max_cols;
   }
+  G.count = count;
+  const int tw = dtype == FBL_DTYPE_FP32 ? 32 : 64;
+  dim3 grid((unsigned)(max_cols / tw), slabs, count);
+  if (dtype == FBL_DTYPE_FP32) colsum_stage1<float><<<grid, 256, 0, st>>>(G, rows, partials);
+  else colsum_stage1<__nv_bfloat16><<<grid, 256, 0, st>>>(G, rows, partials);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  colsum_stage2<<<(unsigned)((cols + 127) / 128), 128, 0, st>>>(partials, slabs, (int)cols, out);
+  dim3 grid2((unsigned)((max_cols + 127) / 128), count);
+  colsum_stage2<<<grid2, 128, 0, st>>>(G, partials, slabs);
   return cudaGetLastError();
+}
+
+cudaError_t launch_colsum(int dtype, const void* M, int64_t rows, int64_t cols, float* out, float* partials,
+                          cudaStream_t st) {
+  const int c = (int)cols;
+  return launch_colsum_group(dtype, 1, &M, rows, &c, &out, partials, st);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -195,19 +195,25 @@ __global__ void __launch_bounds__(256) attn_fwd_simt_kernel(const T* __restrict_
   }
 }
 
-// D_i = sum_d dO[i,d] * O[i,d] per (batch, head, query): one thread per (row, head).
+// D_i = sum_d dO[i,d] * O[i,d] per (batch, head, query): one thread per (row, head), 16-byte loads; consecutive
+// threads take consecutive rows, i.e. consecutive 128-byte tile rows of the head's column panel.
 template <typename T>
 __global__ void rowdot_kernel(const T* __restrict__ dA, const T* __restrict__ A, float* __restrict__ dvec,
                               int64_t n_pad, int t_pad, int hq, int hd, int64_t total) {
   constexpr int TW = tile_w_of<T>::value;
+  constexpr int V = 16 / (int)sizeof(T);
   const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
   if (i >= total) return;
   const int64_t r = i % n_pad;
   const int h = (int)(i / n_pad);
   float s = 0.f;
-  for (int d = 0; d < hd; ++d) {
+  for (int d = 0; d < hd; d += V) {
     const int64_t off = rt_off<TW>(n_pad, r, h * hd + d);
-    s = fmaf(to_f(dA[off]), to_f(A[off]), s);
+    const uint4 ra = *reinterpret_cast<const uint4*>(dA + off), rb = *reinterpret_cast<const uint4*>(A + off);
+    const T* ea = reinterpret_cast<const T*>(&ra);
+    const T* eb = reinterpret_cast<const T*>(&rb);
+#pragma unroll
+    for (int k = 0; k < V; ++k) s = fmaf(to_f(ea[k]), to_f(eb[k]), s);
   }
   const int64_t b = r / t_pad, t = r % t_pad;
   dvec[(b * hq + h) * t_pad + t] = s;
@@ -353,8 +359,11 @@ __global__ void __launch_bounds__(256) attn_bwd_simt_kernel(const T* __restrict_
 
 template <typename T>
 __global__ void convert_f32_kernel(const float* __restrict__ src, T* __restrict__ dst, int64_t n) {
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
-    dst[i] = from_f<T>(src[i]);
+  // n is a multiple of 4 (whole tile rows)
+  for (int64_t i = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) * 4; i < n; i += (int64_t)gridDim.x * blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(src + i);
+    dst[i] = from_f<T>(v.x); dst[i + 1] = from_f<T>(v.y); dst[i + 2] = from_f<T>(v.z); dst[i + 3] = from_f<T>(v.w);
+  }
 }
 
 template <typename T, int HD>
@@ -425,7 +434,7 @@ cudaError_t launch_attn_bwd_pre(const fbl_plan* p, const void* A, const void* dA
 
 cudaError_t launch_attn_bwd_post(const fbl_plan* p, const float* dqacc, void* dQ, cudaStream_t st) {
   const int64_t nq = p->n_pad * p->dq;
-  const int blocks = (int)min((int64_t)148 * 8, (nq + 255) / 256);
+  const int blocks = (int)min((int64_t)148 * 8, (nq / 4 + 255) / 256);
   if (p->d.dtype == FBL_DTYPE_FP32) convert_f32_kernel<float><<<blocks, 256, 0, st>>>(dqacc, (float*)dQ, nq);
   else convert_f32_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(dqacc, (__nv_bfloat16*)dQ, nq);
   return cudaGetLastError();

@@ -13,7 +13,7 @@
 namespace {
 
 constexpr int BM = 128, BK = 64;
-constexpr int MAX_TERMS = 3, MAX_PROBLEMS = 3;
+constexpr int MAX_TERMS = 3, MAX_PROBLEMS = 4;
 
 struct alignas(64) TcProblem {
   CUtensorMap ta[MAX_TERMS], tb[MAX_TERMS];
@@ -311,11 +311,15 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
 cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
   if (count < 1 || count > MAX_PROBLEMS) return cudaErrorInvalidValue;
   bool wide = true;                       // 128 x 256 tiles when every problem's N is whole 256-column blocks
+  int tiles_wide = 0;
   for (int i = 0; i < count; ++i) {
     wide = wide && gs[i].n % 256 == 0;
     for (int t = 0; t < gs[i].n_terms; ++t)
       if (gs[i].t[t].b_trans && gs[i].t[t].b_rpad < 256) wide = false;
+    tiles_wide += ((gs[i].m + BM - 1) / BM) * ((gs[i].n + 255) / 256);
   }
+  // with too few wide tiles to occupy the SMs, narrower tiles (twice as many) finish sooner
+  if (wide && tiles_wide * 3 < p->sm_count * 2) wide = false;
   if (wide) return launch_group_bn<256, 4>(p, gs, count, status, st);
   return launch_group_bn<128, 6>(p, gs, count, status, st);
 }

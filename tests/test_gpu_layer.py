@@ -95,3 +95,9 @@ def test_padding_slots_are_zero_and_padded_equals_unpadded():
 
 def test_config4_reduced_batch():
     run_and_compare(scaled_config(get_config(4), batch=1, seq=1024))
+
+
+@pytest.mark.parametrize("i", [4, 5])
+def test_full_configs_4_and_5(i):
+    # the float64 oracle needs about half a minute (workload 4) and a few minutes (workload 5) on the host cores
+    run_and_compare(get_config(i))
