@@ -3,8 +3,8 @@
 // Forward: one block per (128-query tile, head, batch).  S = Q K^T goes to TMEM (two buffers, so the
 // tensor pipe computes the next score tile while the softmax warps work on the current one); the
 // softmax warps own one query row per thread, keep the running max / sum, and hand P (bf16) to the
-// tensor pipe through 128-byte-swizzled shared memory; O accumulates in TMEM and is rescaled in place
-// only when a row's running max moved.  K/V tiles of the group's KV head are addressed by the head map
+// tensor pipe in tensor memory, over the score columns it was computed from; O accumulates in TMEM and is
+// rescaled in place only when a row's running max moved.  K/V tiles of the group's KV head are addressed by the head map
 // g = h / G; the head split of Q, K, V and the merge of O are column-panel coordinates of the TMA
 // boxes and of the output rows, no data is rearranged.
 #include <string.h>
@@ -36,8 +36,7 @@ struct FwdSmem {
   static constexpr uint32_t Q_OFF = 0;
   static constexpr uint32_t K_OFF = TILE;                   // 2 stages
   static constexpr uint32_t V_OFF = 3 * TILE;               // 2 stages
-  static constexpr uint32_t P_OFF = 5 * TILE;               // 128 x 128 bf16
-  static constexpr uint32_t BAR_OFF = P_OFF + 32768;
+  static constexpr uint32_t BAR_OFF = 5 * TILE;
   static constexpr uint32_t N_BARS = 16;
   static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16 + 1024;
 };
@@ -106,7 +105,7 @@ __global__ void __launch_bounds__(192, 1) attn_fwd_tc_kernel(const __grid_consta
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer --------------------------------------------------------------------------
     const uint32_t idesc_s = tc::idesc_bf16(BQ, BKV, 0, 0);          // Q K-major, K K-major
-    const uint32_t idesc_o = tc::idesc_bf16(BQ, HD, 0, 1);           // P K-major, V MN-major (rows are keys)
+    const uint32_t idesc_o = tc::idesc_bf16(BQ, HD, 0, 1);           // P from TMEM, V MN-major (rows are keys)
     auto issue_s = [&](int j) {
       const uint32_t ksm = base + SM::K_OFF + (j & 1) * SM::TILE;
 #pragma unroll
@@ -135,9 +134,9 @@ __global__ void __launch_bounds__(192, 1) attn_fwd_tc_kernel(const __grid_consta
       const uint32_t vsm = base + SM::V_OFF + (j & 1) * SM::TILE;
 #pragma unroll
       for (uint32_t kk = 0; kk < BKV / 16; ++kk) {
-        const uint64_t da = tc::smem_desc_sw128(base + SM::P_OFF + (kk / 4) * 16384 + (kk % 4) * 32, 16, 1024);
         const uint64_t db = tc::smem_desc_sw128(vsm + kk * 2048, 16384, 1024);
-        tc::mma_bf16_ss(tmem_base + O_COL, da, db, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+        // A operand from tensor memory: the packed bf16 P row of each lane, 16 keys = 8 columns per step
+        tc::mma_bf16_ts(tmem_base + O_COL, tmem_base + S_COL + (j & 1) * 128 + kk * 8, db, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
       }
       tc::mma_commit(bar(B_PVDONE));
       tc::mma_commit(bar(B_VEMPTY + (j & 1)));
@@ -201,18 +200,16 @@ __global__ void __launch_bounds__(192, 1) attn_fwd_tc_kernel(const __grid_consta
           tc::tmem_st_wait();
         }
       }
-      // P row -> shared memory in the 128-byte-swizzled K-major operand layout (two 64-key panels)
+      // P row -> tensor memory, packed two bf16 per column over the first 64 columns of this S buffer (the
+      // thread owns the lane, so nobody else's scores are overwritten); P never goes through shared memory
 #pragma unroll
-      for (int ch = 0; ch < 16; ++ch) {
-        uint4 v;
-        v.x = tc::pack_bf16(s[ch * 8 + 0], s[ch * 8 + 1]);
-        v.y = tc::pack_bf16(s[ch * 8 + 2], s[ch * 8 + 3]);
-        v.z = tc::pack_bf16(s[ch * 8 + 4], s[ch * 8 + 5]);
-        v.w = tc::pack_bf16(s[ch * 8 + 6], s[ch * 8 + 7]);
-        const uint32_t addr = base + SM::P_OFF + (ch / 8) * 16384 + r * 128 + (((ch % 8) ^ (r & 7)) * 16);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) pk[k] = tc::pack_bf16(s[cc * 32 + 2 * k], s[cc * 32 + 2 * k + 1]);
+        tc::tmem_st16(lane_addr + S_COL + (j & 1) * 128 + cc * 16, pk);
       }
-      tc::fence_proxy_async();
+      tc::tmem_st_wait();
       tc::tc_fence_before();
       tc::mbar_arrive(bar(B_PFULL));
     }
@@ -292,25 +289,28 @@ struct alignas(64) AttnBwdParams {
   int32_t* status;
 };
 
-// HD = 64 has room (shared memory and TMEM) to pipeline: Q/dO and P^T/dS^T are double-buffered and dQ has
-// its own TMEM columns, so the tensor pipe computes the next tile's S^T / dP^T and this tile's dV, dK, dQ
-// while the softmax warps are busy.  HD = 128 fills TMEM (S^T, dP^T, dV, dK = 512 columns): dQ reuses the
-// dP^T columns, so only the next tile's S^T can be issued before dQ has been drained.
+// P^T never touches shared memory: the softmax warps store it (bf16, two per column) over the S^T columns
+// in tensor memory once every warp has read them, and dV += P^T dO takes its A operand from there.  HD = 64
+// has spare TMEM columns for dQ and shared memory to double-buffer Q/dO and dS^T, so the tensor pipe computes
+// the next tile's S^T / dP^T and this tile's dK, dQ while the softmax warps are busy.  HD = 128 fills TMEM
+// (S^T, dP^T, dV, dK = 512 columns): dQ reuses the dP^T columns, so only the next S^T can be issued before dQ
+// has been drained.  Both keep a separate staging area for the asynchronous dQ reduction.
 template <int HD>
 struct BwdSmem {
   static constexpr bool PIPE = HD == 64;
-  static constexpr uint32_t NQ = PIPE ? 2 : 1, NP = PIPE ? 2 : 1;
+  static constexpr uint32_t NQ = PIPE ? 2 : 1, NP = PIPE ? 2 : 1;      // stages of Q/dO and of dS^T / staging
   static constexpr uint32_t PANELS = HD / 64;
   static constexpr uint32_t TILE = PANELS * 16384;
+  static constexpr uint32_t STAGE_BYTES = 128 * HD * 4;               // one fp32 dQ tile
   static constexpr uint32_t K_OFF = 0, V_OFF = TILE, Q_OFF = 2 * TILE, DO_OFF = Q_OFF + NQ * TILE;
-  static constexpr uint32_t P_OFF = DO_OFF + NQ * TILE, DS_OFF = P_OFF + NP * 32768;
-  static constexpr uint32_t LSE_OFF = DS_OFF + NP * 32768;   // 2 buffers x (128 floats LSE*log2e, 128 floats D)
+  static constexpr uint32_t DS_OFF = DO_OFF + NQ * TILE, STAGE_OFF = DS_OFF + NP * 32768;
+  static constexpr uint32_t LSE_OFF = STAGE_OFF + NP * STAGE_BYTES;    // 2 buffers x (128 floats LSE*log2e, 128 floats D)
   static constexpr uint32_t BAR_OFF = LSE_OFF + 2048;
-  static constexpr uint32_t N_BARS = 12;
+  static constexpr uint32_t N_BARS = 14;
   static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16;
 };
 
-enum { BB_KVFULL = 0, BB_QDOFULL = 1, BB_QDOEMPTY = 3, BB_SFULL = 5, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY, BB_DQSTAGED, BB_STAGEFREE };
+enum { BB_KVFULL = 0, BB_QDOFULL = 1, BB_QDOEMPTY = 3, BB_SFULL = 5, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY, BB_DQSTAGED, BB_STAGEFREE, BB_SREAD = BB_STAGEFREE + 2 };
 
 // Optional timeline probe (compile with -DFBL_TRACE): block (0,0,0) records clock64() at the marked points of
 // iterations 8..14 into the 1 KiB status area, after the status word.
@@ -328,7 +328,9 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
   constexpr bool PIPE = SM::PIPE;
   constexpr uint32_t PANELS = SM::PANELS, NQ = SM::NQ, NP = SM::NP;
   constexpr uint32_t S_COL = 0, DP_COL = 128, DV_COL = 256, DK_COL = 256 + HD;
-  constexpr uint32_t DQ_COL = PIPE ? 384 : DP_COL, TMEM_COLS = 512;   // HD = 128: dQ reuses the dP^T columns
+  constexpr uint32_t DQ_COL = PIPE ? 384 : DP_COL;   // HD = 128: dQ reuses the dP^T columns
+  constexpr uint32_t P_COL = S_COL;                  // P^T (64 packed columns) overwrites S^T in place
+  constexpr uint32_t TMEM_COLS = 512;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = tc::smem_u32(smem_raw);
   const uint32_t bars = base + SM::BAR_OFF;
@@ -360,6 +362,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     tc::mbar_init(bar(BB_LSEREADY), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_DQSTAGED), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_STAGEFREE), 1);
+    tc::mbar_init(bar(BB_STAGEFREE + 1), 1);
+    tc::mbar_init(bar(BB_SREAD), BWD_SM_THREADS);
     tc::fence_barrier_init();
   }
   if (warp == 1) {
@@ -409,25 +413,27 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       }
       tc::mma_commit(bar(BB_SFULL));
     };
-    auto issue_grads = [&](int it) {          // dV += P^T dO, dK += dS^T Q, dQ = dS K of tile `it`
-      const uint32_t qs = base + SM::Q_OFF + (it % NQ) * SM::TILE, dos = base + SM::DO_OFF + (it % NQ) * SM::TILE;
-      const uint32_t ps = base + SM::P_OFF + (it % NP) * 32768, dss = base + SM::DS_OFF + (it % NP) * 32768;
+    auto issue_dv = [&](int it) {             // dV += P^T dO, P^T read from tensor memory
+      const uint32_t dos = base + SM::DO_OFF + (it % NQ) * SM::TILE;
 #pragma unroll
       for (uint32_t kk = 0; kk < BQ / 16; ++kk) {
-        const uint32_t ao = (kk / 4) * 16384 + (kk % 4) * 32;      // P^T / dS^T: K-major, reduction over queries
-        const uint32_t bo = kk * 2048;                             // dO / Q: MN-major, 16 query rows per step
-        tc::mma_bf16_ss(tmem_base + DV_COL, tc::smem_desc_sw128(ps + ao, 16, 1024),
+        const uint32_t bo = kk * 2048;                             // dO: MN-major, 16 query rows per step
+        tc::mma_bf16_ts(tmem_base + DV_COL, tmem_base + P_COL + kk * 8,   // 16 queries = 8 packed columns
                         tc::smem_desc_sw128(dos + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
       }
+    };
+    auto issue_dk_dq = [&](int it) {          // dK += dS^T Q, dQ = dS K
+      const uint32_t qs = base + SM::Q_OFF + (it % NQ) * SM::TILE;
+      const uint32_t dss = base + SM::DS_OFF + (it % NP) * 32768;
 #pragma unroll
       for (uint32_t kk = 0; kk < BQ / 16; ++kk) {
-        const uint32_t ao = (kk / 4) * 16384 + (kk % 4) * 32;
-        const uint32_t bo = kk * 2048;
+        const uint32_t ao = (kk / 4) * 16384 + (kk % 4) * 32;      // dS^T: K-major, reduction over queries
+        const uint32_t bo = kk * 2048;                             // Q: MN-major, 16 query rows per step
         tc::mma_bf16_ss(tmem_base + DK_COL, tc::smem_desc_sw128(dss + ao, 16, 1024),
                         tc::smem_desc_sw128(qs + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
       }
       tc::mma_commit(bar(BB_QDOEMPTY + (it % NQ)));                // Q / dO of this tile are not read again:
-                                                                   // the next tile's TMA overlaps dQ and its drain
+                                                                   // the next TMA load overlaps dQ and its drain
 #pragma unroll
       for (uint32_t kk = 0; kk < BKV / 16; ++kk) {
         const uint32_t o = kk * 2048;                              // both operands MN-major: 16 key rows per step
@@ -442,23 +448,21 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       if (ok) { tc::tc_fence_after(); issue_s(0); issue_dp(0); }
     }
     if (PIPE) {
+      // dV first (it frees the S^T columns that hold P^T), then the next tile's scores, then dK and dQ: the
+      // softmax warps start on tile it + 1 while the tensor pipe is still busy with dK, dQ of tile it
       for (int it = 0; it < n_it && ok; ++it) {
-        TR(0);
         if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
-        TR(1);
+        tc::tc_fence_after();
+        issue_dv(it);
         if (it + 1 < n_it) {
           if (!tc::mbar_wait(bar(BB_QDOFULL + ((it + 1) % NQ)), ((it + 1) / NQ) & 1, status, 303)) { ok = false; break; }
-          TR(2);
           tc::tc_fence_after();
           issue_s(it + 1);
           issue_dp(it + 1);
         }
-        TR(3);
         if (it > 0 && !tc::mbar_wait(bar(BB_DQDRAINED), (it - 1) & 1, status, 304)) { ok = false; break; }
-        TR(4);
         tc::tc_fence_after();
-        issue_grads(it);
-        TR(5);
+        issue_dk_dq(it);
       }
     } else {
       for (int it = 0; it < n_it && ok; ++it) {
@@ -466,13 +470,14 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
         TR(1);
         tc::tc_fence_after();
-        issue_grads(it);
+        issue_dv(it);
+        issue_dk_dq(it);
         TR(2);
         if (it + 1 < n_it) {
           if (!tc::mbar_wait(bar(BB_QDOFULL), (it + 1) & 1, status, 303)) { ok = false; break; }
           TR(3);
           tc::tc_fence_after();
-          issue_s(it + 1);                   // the S^T columns were released by PDSFULL
+          issue_s(it + 1);                   // the S^T columns (P^T by now) were last read by dV above
           if (!tc::mbar_wait(bar(BB_DQDRAINED), it & 1, status, 304)) { ok = false; break; }
           TR(4);
           tc::tc_fence_after();
@@ -487,13 +492,14 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       for (int dit = 0; dit < n_it; ++dit) {
         const int h = g * P.group + dit / per_head, i0 = (qt_begin + dit % per_head) * BQ;
         if (!tc::mbar_wait(bar(BB_DQSTAGED), dit & 1, status, 309)) break;
-        const uint32_t stage = base + SM::P_OFF + (dit % NP) * 32768;
+        const uint32_t stage = base + SM::STAGE_OFF + (dit % NP) * SM::STAGE_BYTES;
 #pragma unroll
         for (int pn = 0; pn < (int)PANELS; ++pn)
           tc::tma_reduce_add_4d(&P.tdq, stage + pn * 32768, 0, 0, row0 + i0, h * (int)PANELS + pn);
         tc::bulk_commit_group();
         tc::bulk_wait_group_read0();                 // the staging tile has been read: it may be overwritten
-        tc::mbar_arrive(bar(BB_STAGEFREE));
+        tc::mbar_arrive(bar(BB_STAGEFREE + (dit % NP)));     // one barrier per staging buffer: a waiter is never
+                                                             // more than one phase behind
       }
       tc::bulk_wait_group0();
     }
@@ -510,12 +516,13 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     bool ok = true;
 
     // dQ tile of iteration `dit` (row = query i0 + row): each thread copies its TMEM row segment, scaled, to a
-    // staging tile in shared memory (the P^T buffer of that iteration, free once its MMAs are done) in the
-    // 128-byte-swizzled box layout of the accumulator's tensor map; the reduction warp then adds the whole
-    // tile to global memory asynchronously, off the critical path of these warps.
+    // staging tile in shared memory in the 128-byte-swizzled box layout of the accumulator's tensor map; the
+    // reduction warp then adds the whole tile to global memory asynchronously, off the critical path.
     auto drain_dq = [&](int dit) -> bool {
-      const uint32_t stage = base + SM::P_OFF + (dit % NP) * 32768;
+      const uint32_t stage = base + SM::STAGE_OFF + (dit % NP) * SM::STAGE_BYTES;
       if (!tc::mbar_wait(bar(BB_DQFULL), dit & 1, status, 307)) return false;
+      // the staging buffer's previous tile must have been read by its bulk reduction
+      if (dit >= (int)NP && !tc::mbar_wait(bar(BB_STAGEFREE + (dit % NP)), (dit / (int)NP - 1) & 1, status, 310)) return false;
       { const int it = dit; if (t == 0) TR(8); }
       tc::tc_fence_after();
 #pragma unroll 1
@@ -572,14 +579,22 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       tc::tc_fence_after();
       // element masks are needed only on the diagonal tile and on tiles with keys or queries beyond the sequence
       const bool need_mask = (P.causal && (i0 < j0 + BKV - 1)) || (j0 + BKV > P.seq) || (i0 + BQ > P.seq);
-      const uint32_t prow = (it % NP) * 32768 + (part / 2) * 16384 + r * 128;
-      // One 16-column chunk: P^T = exp2(S^T c - LSE), dS^T = P^T (dP^T - D), both rounded to bf16 and written
-      // to the swizzled operand tiles.  MASKED is the rare path (diagonal / ragged tiles).
+      const uint32_t dsrow = base + SM::DS_OFF + (it % NP) * 32768 + (part / 2) * 16384 + r * 128;
+      // this thread's 32 score columns first: the packed P^T overwrites S^T columns that belong to other warps
+      // of the same lane quarter, so every warp must have read its scores before any P^T store
+      uint32_t sv[32];
+      tc::tmem_ld32(lane_addr + S_COL + part * 32, sv);
+      tc::tmem_ld_wait();
+      tc::tc_fence_before();
+      tc::mbar_arrive(bar(BB_SREAD));
+      if (!tc::mbar_wait(bar(BB_SREAD), it & 1, status, 311)) { ok = false; break; }
+      tc::tc_fence_after();
+      // One 16-column chunk: P^T = exp2(S^T c - LSE) to tensor memory, dS^T = P^T (dP^T - D) to the swizzled
+      // shared-memory operand tile, both rounded to bf16.  MASKED is the rare path (diagonal / ragged tiles).
       auto chunk = [&](int cc, auto masked_tag) {
         constexpr bool MASKED = decltype(masked_tag)::value;
         const int c0 = part * 32 + cc * 16;
-        uint32_t sv[16], dpv[16];
-        tc::tmem_ld16(lane_addr + S_COL + c0, sv);
+        uint32_t dpv[16];
         tc::tmem_ld16(lane_addr + DP_COL + c0, dpv);
         tc::tmem_ld_wait();
         uint32_t pp[8], dd[8];
@@ -591,7 +606,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
           float pv[4], gv[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
-            float p = tc::fast_exp2(fmaf(__uint_as_float(sv[k + u]), c, -lv[u]));
+            float p = tc::fast_exp2(fmaf(__uint_as_float(sv[cc * 16 + k + u]), c, -lv[u]));
             if (MASKED) {
               const int gi = i0 + c0 + k + u;
               if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) p = 0.f;
@@ -605,22 +620,15 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
           dd[k / 2 + 1] = tc::pack_bf16(gv[2], gv[3]);
         }
         if (t == 0) TR(16 + cc);
+        tc::tmem_st8(lane_addr + P_COL + c0 / 2, pp);
         // 16 query columns = 2 swizzled 16-byte chunks of this key row inside its 64-query panel
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
           const uint32_t chk = (uint32_t)((part % 2) * 4 + cc * 2 + ch);
-          const uint32_t off = prow + ((chk ^ (uint32_t)(r & 7)) * 16);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + SM::P_OFF + off), "r"(pp[ch * 4]),
-                       "r"(pp[ch * 4 + 1]), "r"(pp[ch * 4 + 2]), "r"(pp[ch * 4 + 3]) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + SM::DS_OFF + off), "r"(dd[ch * 4]),
-                       "r"(dd[ch * 4 + 1]), "r"(dd[ch * 4 + 2]), "r"(dd[ch * 4 + 3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dsrow + ((chk ^ (uint32_t)(r & 7)) * 16)),
+                       "r"(dd[ch * 4]), "r"(dd[ch * 4 + 1]), "r"(dd[ch * 4 + 2]), "r"(dd[ch * 4 + 3]) : "memory");
         }
       };
-      {
-        // the P^T (and, for HD = 128, dS^T) buffer written next was the staging tile of an earlier drain
-        const int last = PIPE ? it - 2 : it - 1;
-        if (last >= 0 && !tc::mbar_wait(bar(BB_STAGEFREE), last & 1, status, 310)) { ok = false; break; }
-      }
       if (need_mask) {
         chunk(0, std::true_type{});
         chunk(1, std::true_type{});
@@ -628,6 +636,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         chunk(0, std::false_type{});
         chunk(1, std::false_type{});
       }
+      tc::tmem_st_wait();
       if (t == 0) TR(15);
       tc::fence_proxy_async();
       if (t == 0) TR(6);
