@@ -19,12 +19,27 @@ namespace {
 constexpr int BQ = 128, BKV = 128;
 constexpr float LOG2E = 1.4426950408889634f;
 
+// Optional timeline probe (compile with -DFBL_TRACE): block (0,0,0) records clock64() at the marked points of
+// iterations 8..14 into the 1 KiB status area, after the status word.
+#ifdef FBL_TRACE
+#ifndef FBL_TRACE_FIRST
+#define FBL_TRACE_FIRST 8
+#endif
+#ifndef FBL_TRACE_BLOCK
+#define FBL_TRACE_BLOCK 0
+#endif
+#define TR(k) do { if (blockIdx.x == FBL_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && it >= FBL_TRACE_FIRST && it < FBL_TRACE_FIRST + 3) ((long long*)P.status)[8 + (it - FBL_TRACE_FIRST) * 32 + (k)] = clock64(); } while (0)
+#else
+#define TR(k) do { } while (0)
+#endif
+
 struct alignas(64) AttnFwdParams {
   CUtensorMap tq, tk, tv;
   __nv_bfloat16* a;      // merged-head output [n_pad, dq] in R-Tile order
   float* lse;            // [B, Hq, t_pad]
   long long n_pad;
   int seq, t_pad, hq, group, causal;
+  int pair;              // 1: each block owns two adjacent query tiles, one per softmax warp group
   float scale;
   int32_t* status;
 };
@@ -33,34 +48,53 @@ template <int HD>
 struct FwdSmem {
   static constexpr uint32_t PANELS = HD / 64;
   static constexpr uint32_t TILE = PANELS * 16384;          // 128 rows x HD bf16
-  static constexpr uint32_t Q_OFF = 0;
-  static constexpr uint32_t K_OFF = TILE;                   // 2 stages
-  static constexpr uint32_t V_OFF = 3 * TILE;               // 2 stages
-  static constexpr uint32_t BAR_OFF = 5 * TILE;
+  static constexpr uint32_t Q_OFF = 0;                      // 2 query tiles
+  static constexpr uint32_t K_OFF = 2 * TILE;               // 2 stages
+  static constexpr uint32_t V_OFF = 4 * TILE;               // 2 stages
+  static constexpr uint32_t BAR_OFF = 6 * TILE;
   static constexpr uint32_t N_BARS = 16;
-  static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16 + 1024;
+  static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16;
 };
 
-enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_PVDONE = 12 };
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_PVDONE = 13 };
+
+constexpr int FWD_THREADS = 320;      // warp 0 TMA, warp 1 MMA, warps 2-5 and 6-9: one softmax warp group per query tile
+
+// A row's running max is only raised (and O rescaled) when the new max exceeds it by more than this many
+// powers of two; until then the probabilities are computed against the stale max and stay below 2^8.
+constexpr float RESCALE_LOG2 = 8.f;
 
 template <int HD>
-__global__ void __launch_bounds__(192, 1) attn_fwd_tc_kernel(const __grid_constant__ AttnFwdParams P) {
+__global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __grid_constant__ AttnFwdParams P) {
   using SM = FwdSmem<HD>;
   constexpr uint32_t PANELS = SM::PANELS;
-  constexpr uint32_t S_COL = 0, O_COL = 256, TMEM_COLS = 512;
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+  constexpr uint32_t O_COL = 256, TMEM_COLS = 512;          // S of tile g at 128 g, O of tile g at 256 + HD g
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t base = tc::smem_u32(smem_raw);
   const uint32_t bars = base + SM::BAR_OFF;
   const uint32_t slot = bars + 8 * SM::N_BARS;
   auto bar = [&](int i) { return bars + 8u * i; };
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int n_qt = (P.seq + BQ - 1) / BQ;
-  const int qt = n_qt - 1 - (int)blockIdx.x;                 // heaviest (latest) causal tiles first
-  const int i0 = qt * BQ, h = blockIdx.y, b = blockIdx.z, g = h / P.group;
+  const int h = blockIdx.y, b = blockIdx.z, g = h / P.group;
   const int row0 = b * P.t_pad;
-  const int kv_end = P.causal ? min(P.seq, i0 + BQ) : P.seq;
-  const int n_kv = (kv_end + BKV - 1) / BKV;
   int32_t* status = P.status;
+  // query tiles of this block: with pairing, tile x and its mirror n_qt-1-x (equal causal work in every block)
+  // heaviest causal tiles first; with pairing a block owns two adjacent tiles, whose key ranges differ by one tile,
+  // so both warp groups stay busy for the whole loop
+  const int slot_x = (int)gridDim.x - 1 - (int)blockIdx.x;
+  const int qt0 = P.pair ? min(2 * slot_x + 1, n_qt - 1) : slot_x;
+  const int qt1 = (P.pair && 2 * slot_x + 1 < n_qt) ? 2 * slot_x : -1;   // odd tile count: the last block has one tile
+  auto kv_tiles = [&](int t) {
+    const int kv_end = t < 0 ? 0 : (P.causal ? min(P.seq, (t + 1) * BQ) : P.seq);
+    return (kv_end + BKV - 1) / BKV;
+  };
+  const int n_kv0 = kv_tiles(qt0), n_kv1 = kv_tiles(qt1);
+  const int n_kv_max = max(n_kv0, n_kv1);
+  if ((base & 1023u) != 0) {
+    if (threadIdx.x == 0) atomicCAS(status, 0, 299);
+    return;
+  }
 
   if (threadIdx.x == 0) {
     tc::mbar_init(bar(B_QFULL), 1);
@@ -70,9 +104,9 @@ __global__ void __launch_bounds__(192, 1) attn_fwd_tc_kernel(const __grid_consta
       tc::mbar_init(bar(B_VFULL + s), 1);
       tc::mbar_init(bar(B_VEMPTY + s), 1);
       tc::mbar_init(bar(B_SFULL + s), 1);
+      tc::mbar_init(bar(B_PFULL + s), 128);
+      tc::mbar_init(bar(B_PVDONE + s), 1);
     }
-    tc::mbar_init(bar(B_PFULL), 128);
-    tc::mbar_init(bar(B_PVDONE), 1);
     tc::fence_barrier_init();
   }
   if (warp == 1) {
@@ -90,9 +124,10 @@ __global__ void __launch_bounds__(192, 1) attn_fwd_tc_kernel(const __grid_consta
     tc::tma_prefetch_desc(&P.tq);
     tc::tma_prefetch_desc(&P.tk);
     tc::tma_prefetch_desc(&P.tv);
-    tc::mbar_expect_tx(bar(B_QFULL), SM::TILE);
-    tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(B_QFULL), 0, row0 + i0, h * (int)PANELS);
-    for (int j = 0; j < n_kv; ++j) {
+    tc::mbar_expect_tx(bar(B_QFULL), (qt1 >= 0 ? 2u : 1u) * SM::TILE);
+    tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(B_QFULL), 0, row0 + qt0 * BQ, h * (int)PANELS);
+    if (qt1 >= 0) tc::tma_load_3d(base + SM::Q_OFF + SM::TILE, &P.tq, bar(B_QFULL), 0, row0 + qt1 * BQ, h * (int)PANELS);
+    for (int j = 0; j < n_kv_max; ++j) {
       const int s = j & 1;
       const uint32_t ph = (j >> 1) & 1;
       if (!tc::mbar_wait(bar(B_KEMPTY + s), ph ^ 1, status, 201)) break;
@@ -104,124 +139,161 @@ __global__ void __launch_bounds__(192, 1) attn_fwd_tc_kernel(const __grid_consta
     }
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer --------------------------------------------------------------------------
+    // Per key tile j: [P0(j) ready] PV0(j), S0(j+1), [P1(j) ready] PV1(j), S1(j+1): while one warp group works
+    // on its scores the tensor pipe serves the other one.  S and P of a query tile share TMEM columns, so
+    // S(j+1) is issued after PV(j), which reads P(j) (the tensor pipe executes in issue order).
     const uint32_t idesc_s = tc::idesc_bf16(BQ, BKV, 0, 0);          // Q K-major, K K-major
     const uint32_t idesc_o = tc::idesc_bf16(BQ, HD, 0, 1);           // P from TMEM, V MN-major (rows are keys)
-    auto issue_s = [&](int j) {
-      const uint32_t ksm = base + SM::K_OFF + (j & 1) * SM::TILE;
+    auto issue_s = [&](int w, int j) {
+      const uint32_t qsm = base + SM::Q_OFF + w * SM::TILE, ksm = base + SM::K_OFF + (j & 1) * SM::TILE;
 #pragma unroll
       for (uint32_t kk = 0; kk < HD / 16; ++kk) {
         const uint32_t o = (kk / 4) * 16384 + (kk % 4) * 32;
-        tc::mma_bf16_ss(tmem_base + S_COL + (j & 1) * 128, tc::smem_desc_sw128(base + SM::Q_OFF + o, 16, 1024),
+        tc::mma_bf16_ss(tmem_base + w * 128, tc::smem_desc_sw128(qsm + o, 16, 1024),
                         tc::smem_desc_sw128(ksm + o, 16, 1024), idesc_s, kk > 0);
       }
-      tc::mma_commit(bar(B_SFULL + (j & 1)));
-      tc::mma_commit(bar(B_KEMPTY + (j & 1)));
+      tc::mma_commit(bar(B_SFULL + w));
+    };
+    auto issue_pv = [&](int w, int j) {
+      const uint32_t vsm = base + SM::V_OFF + (j & 1) * SM::TILE;
+#pragma unroll
+      for (uint32_t kk = 0; kk < BKV / 16; ++kk) {
+        // A operand from tensor memory: the packed bf16 P row of each lane, 16 keys = 8 columns per step
+        tc::mma_bf16_ts(tmem_base + O_COL + w * HD, tmem_base + w * 128 + kk * 8,
+                        tc::smem_desc_sw128(vsm + kk * 2048, 16384, 1024), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+      }
+      tc::mma_commit(bar(B_PVDONE + w));
     };
     bool ok = tc::mbar_wait(bar(B_QFULL), 0, status, 203) && tc::mbar_wait(bar(B_KFULL), 0, status, 204);
     if (ok) {
       tc::tc_fence_after();
-      issue_s(0);
+      if (n_kv0 > 0) issue_s(0, 0);
+      if (n_kv1 > 0) issue_s(1, 0);
     }
-    for (int j = 0; j < n_kv && ok; ++j) {
-      if (j + 1 < n_kv) {
-        if (!tc::mbar_wait(bar(B_KFULL + ((j + 1) & 1)), ((j + 1) >> 1) & 1, status, 205)) { ok = false; break; }
-        tc::tc_fence_after();
-        issue_s(j + 1);
-      }
-      if (!tc::mbar_wait(bar(B_PFULL), j & 1, status, 206)) { ok = false; break; }
+    for (int j = 0; j < n_kv_max && ok; ++j) {
+      const bool next = j + 1 < n_kv_max;
+      { const int it = j; TR(0); }
       if (!tc::mbar_wait(bar(B_VFULL + (j & 1)), (j >> 1) & 1, status, 207)) { ok = false; break; }
-      tc::tc_fence_after();
-      const uint32_t vsm = base + SM::V_OFF + (j & 1) * SM::TILE;
+      if (next && !tc::mbar_wait(bar(B_KFULL + ((j + 1) & 1)), ((j + 1) >> 1) & 1, status, 205)) { ok = false; break; }
 #pragma unroll
-      for (uint32_t kk = 0; kk < BKV / 16; ++kk) {
-        const uint64_t db = tc::smem_desc_sw128(vsm + kk * 2048, 16384, 1024);
-        // A operand from tensor memory: the packed bf16 P row of each lane, 16 keys = 8 columns per step
-        tc::mma_bf16_ts(tmem_base + O_COL, tmem_base + S_COL + (j & 1) * 128 + kk * 8, db, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+      for (int w = 0; w < 2; ++w) {
+        const int nk = w ? n_kv1 : n_kv0;
+        if (ok && j < nk) {
+          { const int it = j; TR(1 + 3 * w); }
+          if (!tc::mbar_wait(bar(B_PFULL + w), j & 1, status, 206)) { ok = false; }
+          else { { const int it = j; TR(2 + 3 * w); } tc::tc_fence_after(); issue_pv(w, j); }
+        }
+        if (ok && j + 1 < nk) issue_s(w, j + 1);
+        { const int it = j; TR(3 + 3 * w); }
       }
-      tc::mma_commit(bar(B_PVDONE));
-      tc::mma_commit(bar(B_VEMPTY + (j & 1)));
+      if (!ok) break;
+      tc::mma_commit(bar(B_VEMPTY + (j & 1)));              // both P V products of this stage are behind us
+      if (next) tc::mma_commit(bar(B_KEMPTY + ((j + 1) & 1)));   // ... and both score products of the next stage
+      if (j == 0) tc::mma_commit(bar(B_KEMPTY));            // stage 0 scores were issued before the loop
     }
   } else if (warp >= 2) {
-    // ---- softmax warps: one query row per thread ----------------------------------------------
+    // ---- softmax warp groups: group w owns query tile qt[w], one query row per thread --------------
+    const int w = (warp - 2) / 4;
     const int q = warp % 4;
     const int r = q * 32 + lane;
+    const int n_kvw = w ? n_kv1 : n_kv0;
+    const int i0 = (w ? qt1 : qt0) * BQ;
     const int gi = i0 + r;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+    const uint32_t s_addr = lane_addr + w * 128, o_addr = lane_addr + O_COL + w * HD;
     const float c = P.scale * LOG2E;
+    const float tau = RESCALE_LOG2 / c;              // the same threshold in raw score units
     float m = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int j = 0; j < n_kv && ok; ++j) {
+    for (int j = 0; j < n_kvw && ok; ++j) {
       const int j0 = j * BKV;
-      if (!tc::mbar_wait(bar(B_SFULL + (j & 1)), (j >> 1) & 1, status, 208)) { ok = false; break; }
+      { const int it = j; if (r == 0) TR(8 + 8 * w); }
+      if (!tc::mbar_wait(bar(B_SFULL + w), j & 1, status, 208)) { ok = false; break; }
+      { const int it = j; if (r == 0) TR(9 + 8 * w); }
       tc::tc_fence_after();
-      uint32_t sr[128];
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) tc::tmem_ld32(lane_addr + S_COL + (j & 1) * 128 + cc * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[cc * 32]));
-      tc::tmem_ld_wait();
-      float* s = reinterpret_cast<float*>(sr);
       const bool need_mask = (j0 + BKV > P.seq) || (P.causal && j0 + BKV - 1 > i0);
-      if (need_mask) {
+      // pass 1 over the 128 scores of this row (four 32-column loads): the row maximum
+      auto mask_chunk = [&](float* s, int cc) {
 #pragma unroll
-        for (int k = 0; k < 128; ++k) {
-          const int gj = j0 + k;
+        for (int k = 0; k < 32; ++k) {
+          const int gj = j0 + cc * 32 + k;
           if (gj >= P.seq || (P.causal && gj > gi)) s[k] = -INFINITY;
         }
-      }
-      float mx = s[0];
+      };
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t sr[32];
+        tc::tmem_ld32(s_addr + cc * 32, sr);
+        tc::tmem_ld_wait();
+        float* s = reinterpret_cast<float*>(sr);
+        if (need_mask) mask_chunk(s, cc);
 #pragma unroll
-      for (int k = 1; k < 128; ++k) mx = fmaxf(mx, s[k]);
-      const float m_new = fmaxf(m, mx);
-      const bool moved = m_new > m;
-      const float alpha = (m == -INFINITY) ? 0.f : tc::fast_exp2((m - m_new) * c);
-      const float mc = (m_new == -INFINITY) ? 0.f : m_new * c;
-      float sum = 0.f;
-#pragma unroll
-      for (int k = 0; k < 128; ++k) {
-        s[k] = tc::fast_exp2(fmaf(s[k], c, -mc));
-        sum += s[k];
-      }
-      l = l * alpha + sum;
-      m = m_new;
-      if (j > 0) {
-        // the previous P V product must have finished before P is overwritten or O is touched
-        if (!tc::mbar_wait(bar(B_PVDONE), (j - 1) & 1, status, 209)) { ok = false; break; }
-        tc::tc_fence_after();
-        if (__any_sync(0xffffffffu, moved)) {
-          const float a = moved ? alpha : 1.f;
-#pragma unroll
-          for (int cc = 0; cc < HD / 32; ++cc) {
-            uint32_t o[32];
-            tc::tmem_ld32(lane_addr + O_COL + cc * 32, o);
-            tc::tmem_ld_wait();
-#pragma unroll
-            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * a);
-            tc::tmem_st32(lane_addr + O_COL + cc * 32, o);
-          }
-          tc::tmem_st_wait();
+        for (int k = 0; k < 32; k += 4) {
+          mx0 = fmaxf(mx0, s[k]); mx1 = fmaxf(mx1, s[k + 1]); mx2 = fmaxf(mx2, s[k + 2]); mx3 = fmaxf(mx3, s[k + 3]);
         }
       }
-      // P row -> tensor memory, packed two bf16 per column over the first 64 columns of this S buffer (the
-      // thread owns the lane, so nobody else's scores are overwritten); P never goes through shared memory
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      { const int it = j; if (r == 0) TR(10 + 8 * w); }
+      // lazy running max: move it only when the tile's max beats it by more than the threshold
+      const bool moved = mx > m + tau || m == -INFINITY;
+      const float m_new = moved ? fmaxf(m, mx) : m;
+      const float alpha = (m == -INFINITY) ? 0.f : tc::fast_exp2((m - m_new) * c);
+      const float mc = (m_new == -INFINITY) ? 0.f : m_new * c;
+      m = m_new;
+      if (j > 0 && __any_sync(0xffffffffu, moved)) {
+        // O is rescaled in place: the previous P V product must have finished
+        if (!tc::mbar_wait(bar(B_PVDONE + w), (j - 1) & 1, status, 209)) { ok = false; break; }
+        tc::tc_fence_after();
+        const float a = moved ? alpha : 1.f;
+#pragma unroll 1
+        for (int cc = 0; cc < HD / 32; ++cc) {
+          uint32_t o[32];
+          tc::tmem_ld32(o_addr + cc * 32, o);
+          tc::tmem_ld_wait();
 #pragma unroll
+          for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * a);
+          tc::tmem_st32(o_addr + cc * 32, o);
+        }
+      }
+      { const int it = j; if (r == 0) TR(11 + 8 * w); }
+      // pass 2: P = exp2(S c - m c), its row sum, and P packed to bf16 over the score columns already consumed
+      // (32 scores become 16 packed columns; the thread owns the lane, so nobody else's data is overwritten)
+      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+#pragma unroll 1
       for (int cc = 0; cc < 4; ++cc) {
+        uint32_t sr[32];
+        tc::tmem_ld32(s_addr + cc * 32, sr);
+        tc::tmem_ld_wait();
+        float* s = reinterpret_cast<float*>(sr);
+        if (need_mask) mask_chunk(s, cc);
         uint32_t pk[16];
 #pragma unroll
-        for (int k = 0; k < 16; ++k) pk[k] = tc::pack_bf16(s[cc * 32 + 2 * k], s[cc * 32 + 2 * k + 1]);
-        tc::tmem_st16(lane_addr + S_COL + (j & 1) * 128 + cc * 16, pk);
+        for (int k = 0; k < 32; k += 4) {
+          const float p0 = tc::fast_exp2(fmaf(s[k], c, -mc)), p1 = tc::fast_exp2(fmaf(s[k + 1], c, -mc));
+          const float p2 = tc::fast_exp2(fmaf(s[k + 2], c, -mc)), p3 = tc::fast_exp2(fmaf(s[k + 3], c, -mc));
+          sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+          pk[k / 2] = tc::pack_bf16(p0, p1);
+          pk[k / 2 + 1] = tc::pack_bf16(p2, p3);
+        }
+        tc::tmem_st16(s_addr + cc * 16, pk);
       }
+      if (moved) l *= alpha;
+      l += (sum0 + sum1) + (sum2 + sum3);
       tc::tmem_st_wait();
       tc::tc_fence_before();
-      tc::mbar_arrive(bar(B_PFULL));
+      tc::mbar_arrive(bar(B_PFULL + w));
+      { const int it = j; if (r == 0) TR(12 + 8 * w); }
     }
-    if (ok && n_kv > 0) ok = tc::mbar_wait(bar(B_PVDONE), (n_kv - 1) & 1, status, 210);
+    if (ok && n_kvw > 0) ok = tc::mbar_wait(bar(B_PVDONE + w), (n_kvw - 1) & 1, status, 210);
     tc::tc_fence_after();
-    if (ok) {
+    if (ok && n_kvw > 0) {
       const bool live = gi < P.seq;
       const float inv = live ? 1.f / l : 0.f;
 #pragma unroll
       for (int cc = 0; cc < HD / 32; ++cc) {
         uint32_t o[32];
-        tc::tmem_ld32(lane_addr + O_COL + cc * 32, o);
+        tc::tmem_ld32(o_addr + cc * 32, o);
         tc::tmem_ld_wait();
         if (gi < P.t_pad) {
           const int col = h * HD + cc * 32;
@@ -257,14 +329,16 @@ cudaError_t fwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   P.a = (__nv_bfloat16*)A; P.lse = lse; P.n_pad = p->n_pad;
   P.seq = p->d.seq; P.t_pad = p->t_pad; P.hq = p->d.n_q_heads; P.group = p->group; P.causal = p->d.causal;
   P.scale = p->scale; P.status = status;
+  const int n_qt = (p->d.seq + BQ - 1) / BQ;
+  // two query tiles per block when that still leaves at least one block per SM
+  P.pair = (n_qt >= 2 && (long long)((n_qt + 1) / 2) * p->d.n_q_heads * p->d.batch >= p->sm_count) ? 1 : 0;
   auto k = attn_fwd_tc_kernel<HD>;
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FwdSmem<HD>::TOTAL);
   if (e != cudaSuccess) return e;
-  dim3 grid((p->d.seq + BQ - 1) / BQ, p->d.n_q_heads, p->d.batch);
-  k<<<grid, 192, FwdSmem<HD>::TOTAL, st>>>(P);
+  dim3 grid(P.pair ? (n_qt + 1) / 2 : n_qt, p->d.n_q_heads, p->d.batch);
+  k<<<grid, FWD_THREADS, FwdSmem<HD>::TOTAL, st>>>(P);
   return cudaGetLastError();
 }
-
 
 // ---------------------------------------------------------------------------------------------------
 // Backward: one block per (128-key tile, KV head, batch).  For every query head of the group and every
@@ -312,13 +386,6 @@ struct BwdSmem {
 
 enum { BB_KVFULL = 0, BB_QDOFULL = 1, BB_QDOEMPTY = 3, BB_SFULL = 5, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY, BB_DQSTAGED, BB_STAGEFREE, BB_SREAD = BB_STAGEFREE + 2 };
 
-// Optional timeline probe (compile with -DFBL_TRACE): block (0,0,0) records clock64() at the marked points of
-// iterations 8..14 into the 1 KiB status area, after the status word.
-#ifdef FBL_TRACE
-#define TR(k) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && it >= 8 && it < 11) ((long long*)P.status)[8 + (it - 8) * 32 + (k)] = clock64(); } while (0)
-#else
-#define TR(k) do { } while (0)
-#endif
 constexpr int BWD_THREADS = 608;     // warp 0 TMA loads, warp 1 MMA, warps 2-17 softmax (four per TMEM lane quarter), warp 18 dQ reductions
 constexpr int BWD_SM_THREADS = 512;
 
