@@ -204,8 +204,8 @@ __global__ void __launch_bounds__(256) norm_bwd_kernel(const T* __restrict__ dXn
 
 
 // ------------------------------------------------------------------------------------------
-// Register-resident norm kernels for bf16 rows of up to 2048 columns (NV = D / 256 vectors of 16 bytes per
-// lane): one warp owns a row, lane l holds vectors l, l + 32, ... of it (each warp-level load covers four
+// Register-resident norm kernels for bf16 rows (NV vectors of 16 bytes per lane, WPR warps per row, d_model =
+// 256 NV WPR up to 4096): a warp owns a row or a contiguous part of it, lane l holds vectors l, l + 32, ... of it (each warp-level load covers four
 // whole 128-byte tile rows, one per column panel), so X (and dXn) cross HBM exactly once.
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ float warp_sum(float v) {
@@ -214,37 +214,54 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-template <int NV>
+// WPR warps share a row (d_model = NV * 256 * WPR columns): the row statistics are combined through shared memory.
+template <int WPR>
+__device__ __forceinline__ float row_sum(float v, float* s_part, int slot, int part) {
+  v = warp_sum(v);
+  if (WPR == 1) return v;
+  __syncthreads();                                   // previous use of s_part is over
+  if ((threadIdx.x & 31) == 0) s_part[slot * WPR + part] = v;
+  __syncthreads();
+  float t = 0.f;
+#pragma unroll
+  for (int i = 0; i < WPR; ++i) t += s_part[slot * WPR + i];
+  return t;
+}
+
+template <int NV, int WPR>
 __global__ void __launch_bounds__(256) norm_fwd_rows_kernel(const __nv_bfloat16* __restrict__ X,
                                                             const float* __restrict__ gamma,
                                                             const float* __restrict__ beta,
                                                             __nv_bfloat16* __restrict__ Xn, float* __restrict__ stats,
                                                             int64_t n_pad, int seq, int t_pad, int rms, float eps) {
-  constexpr int D = NV * 256;
-  const int lane = threadIdx.x % 32;
-  const int64_t warp0 = (int64_t)blockIdx.x * 8 + threadIdx.x / 32, nwarps = (int64_t)gridDim.x * 8;
-  for (int64_t r = warp0; r < n_pad; r += nwarps) {
+  constexpr int D = NV * 256 * WPR;
+  constexpr int RPB = 8 / WPR;                       // rows per block pass
+  __shared__ float s_part[8];
+  const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
+  const int slot = wib / WPR, part = wib % WPR;
+  // n_pad is a multiple of 8, so every warp of a block sees the same number of rows (block-wide barriers)
+  for (int64_t r = (int64_t)blockIdx.x * RPB + slot; r < n_pad; r += (int64_t)gridDim.x * RPB) {
     const bool pad = (int)(r % t_pad) >= seq;
     float x[NV][8];
     float s = 0.f;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      const int v = j * 32 + lane;                         // vector index in the row: panel v / 8, chunk v % 8
+      const int v = (part * NV + j) * 32 + lane;           // vector index in the row: panel v / 8, chunk v % 8
       load16(X + ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8, x[j]);
 #pragma unroll
       for (int i = 0; i < 8; ++i) s += x[j][i];
     }
-    const float mean = rms ? 0.f : warp_sum(s) * (1.f / D);
+    const float mean = rms ? 0.f : row_sum<WPR>(s, s_part, slot, part) * (1.f / D);
     float q = 0.f;
 #pragma unroll
     for (int j = 0; j < NV; ++j)
 #pragma unroll
       for (int i = 0; i < 8; ++i) { const float c = x[j][i] - mean; q += c * c; }
-    const float rstd = rsqrtf(warp_sum(q) * (1.f / D) + eps);
-    if (lane == 0) { stats[2 * r] = pad ? 0.f : mean; stats[2 * r + 1] = pad ? 0.f : rstd; }
+    const float rstd = rsqrtf(row_sum<WPR>(q, s_part, slot, part) * (1.f / D) + eps);
+    if (lane == 0 && part == 0) { stats[2 * r] = pad ? 0.f : mean; stats[2 * r + 1] = pad ? 0.f : rstd; }
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      const int v = j * 32 + lane;
+      const int v = (part * NV + j) * 32 + lane;
       const int c0 = v * 8;
       const float4 g0 = *reinterpret_cast<const float4*>(gamma + c0), g1 = *reinterpret_cast<const float4*>(gamma + c0 + 4);
       float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
@@ -259,7 +276,7 @@ __global__ void __launch_bounds__(256) norm_fwd_rows_kernel(const __nv_bfloat16*
   }
 }
 
-template <int NV>
+template <int NV, int WPR>
 __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16* __restrict__ dXn,
                                                             const __nv_bfloat16* __restrict__ X,
                                                             const __nv_bfloat16* __restrict__ dY,
@@ -267,17 +284,19 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
                                                             const float* __restrict__ gamma,
                                                             __nv_bfloat16* __restrict__ dX, float* __restrict__ dgamma,
                                                             float* __restrict__ dbeta, int64_t n_pad, int rms) {
-  constexpr int D = NV * 256;
+  constexpr int D = NV * 256 * WPR;
+  constexpr int RPB = 8 / WPR;
   __shared__ float s_dg[D];
   __shared__ float s_db[D];
+  __shared__ float s_part[8];
   for (int i = threadIdx.x; i < D; i += 256) { s_dg[i] = 0.f; s_db[i] = 0.f; }
   __syncthreads();
-  const int lane = threadIdx.x % 32;
-  const int64_t warp0 = (int64_t)blockIdx.x * 8 + threadIdx.x / 32, nwarps = (int64_t)gridDim.x * 8;
+  const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
+  const int slot = wib / WPR, part = wib % WPR;
   float gm[NV][8];
 #pragma unroll
   for (int j = 0; j < NV; ++j) {
-    const int c0 = (j * 32 + lane) * 8;
+    const int c0 = ((part * NV + j) * 32 + lane) * 8;
     const float4 g0 = *reinterpret_cast<const float4*>(gamma + c0), g1 = *reinterpret_cast<const float4*>(gamma + c0 + 4);
     gm[j][0] = g0.x; gm[j][1] = g0.y; gm[j][2] = g0.z; gm[j][3] = g0.w;
     gm[j][4] = g1.x; gm[j][5] = g1.y; gm[j][6] = g1.z; gm[j][7] = g1.w;
@@ -288,13 +307,13 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
   for (int j = 0; j < NV; ++j)
 #pragma unroll
     for (int i = 0; i < 8; ++i) { ag[j][i] = 0.f; ab[j][i] = 0.f; }
-  for (int64_t r = warp0; r < n_pad; r += nwarps) {
+  for (int64_t r = (int64_t)blockIdx.x * RPB + slot; r < n_pad; r += (int64_t)gridDim.x * RPB) {
     const float mean = stats[2 * r], rstd = stats[2 * r + 1];
     float xh[NV][8], g[NV][8];
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      const int v = j * 32 + lane;
+      const int v = (part * NV + j) * 32 + lane;
       const int64_t off = ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8;
       float gv[8];
       load16(X + off, xh[j]);
@@ -309,11 +328,11 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
         s2 = fmaf(g[j][i], xh[j][i], s2);
       }
     }
-    s1 = rms ? 0.f : warp_sum(s1) * (1.f / D);
-    s2 = warp_sum(s2) * (1.f / D);
+    s1 = rms ? 0.f : row_sum<WPR>(s1, s_part, slot, part) * (1.f / D);
+    s2 = row_sum<WPR>(s2, s_part, slot, part) * (1.f / D);
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      const int v = j * 32 + lane;
+      const int v = (part * NV + j) * 32 + lane;
       const int64_t off = ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8;
       float o[8];
       if (dY) load16(dY + off, o);
@@ -329,7 +348,7 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
   for (int j = 0; j < NV; ++j)
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const int c = (j * 32 + lane) * 8 + i;
+      const int c = ((part * NV + j) * 32 + lane) * 8 + i;
       atomicAdd(&s_dg[c], ag[j][i]);
       atomicAdd(&s_db[c], ab[j][i]);
     }
@@ -340,21 +359,45 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
   }
 }
 
-template <int NV>
+template <int NV, int WPR>
 void norm_fwd_rows_launch(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
                           float* stats, int rms, cudaStream_t st) {
-  const int blocks = (int)min((int64_t)p->sm_count * 4, (p->n_pad + 7) / 8);
-  norm_fwd_rows_kernel<NV><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)X, gamma, rms ? nullptr : beta,
-                                                   (__nv_bfloat16*)Xn, stats, p->n_pad, p->d.seq, p->t_pad, rms, p->d.eps);
+  const int blocks = (int)min((int64_t)p->sm_count * 4, p->n_pad / (8 / WPR));
+  norm_fwd_rows_kernel<NV, WPR><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)X, gamma, rms ? nullptr : beta,
+                                                        (__nv_bfloat16*)Xn, stats, p->n_pad, p->d.seq, p->t_pad, rms,
+                                                        p->d.eps);
 }
-template <int NV>
+template <int NV, int WPR>
 void norm_bwd_rows_launch(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
                           const float* gamma, void* dX, float* dgamma, float* dbeta, int rms, cudaStream_t st) {
-  const int blocks = (int)min((int64_t)p->sm_count * 2, (p->n_pad + 7) / 8);
-  norm_bwd_rows_kernel<NV><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dXn, (const __nv_bfloat16*)X,
-                                                   (const __nv_bfloat16*)dY, stats, gamma, (__nv_bfloat16*)dX, dgamma,
-                                                   rms ? nullptr : dbeta, p->n_pad, rms);
+  const int blocks = (int)min((int64_t)p->sm_count * 2, p->n_pad / (8 / WPR));
+  norm_bwd_rows_kernel<NV, WPR><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dXn, (const __nv_bfloat16*)X,
+                                                        (const __nv_bfloat16*)dY, stats, gamma, (__nv_bfloat16*)dX,
+                                                        dgamma, rms ? nullptr : dbeta, p->n_pad, rms);
 }
+
+// d_model -> (vectors per lane, warps per row) of the register-resident kernels; false if there is none
+bool norm_rows_shape(int d, int* nv, int* wpr) {
+  if (d % 256 != 0) return false;
+  const int v = d / 256;
+  if (v <= 4) { *nv = v; *wpr = 1; return true; }
+  if (v == 8) { *nv = 4; *wpr = 2; return true; }
+  if (v == 16) { *nv = 4; *wpr = 4; return true; }
+  if (v == 6) { *nv = 3; *wpr = 2; return true; }
+  if (v == 12) { *nv = 3; *wpr = 4; return true; }
+  return false;
+}
+
+#define FBL_NORM_DISPATCH(CALL)                                        \
+  do {                                                                 \
+    if (wpr == 1) {                                                    \
+      if (nv == 1) CALL(1, 1); else if (nv == 2) CALL(2, 1); else if (nv == 3) CALL(3, 1); else CALL(4, 1); \
+    } else if (wpr == 2) {                                             \
+      if (nv == 3) CALL(3, 2); else CALL(4, 2);                        \
+    } else {                                                           \
+      if (nv == 3) CALL(3, 4); else CALL(4, 4);                        \
+    }                                                                  \
+  } while (0)
 
 // ------------------------------------------------------------------------------------------
 // Token-axis column sums, two stages over tiles: (1) one block per (panel, slab of 256 rows)
@@ -436,13 +479,11 @@ cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma
                             float* stats, cudaStream_t st) {
   const int blocks = (int)((p->n_pad + 31) / 32);
   const int rms = p->d.norm == FBL_NORM_RMSNORM;
-  if (p->d.dtype == FBL_DTYPE_BF16 && p->d.d_model % 256 == 0 && p->d.d_model <= 1024) {
-    switch (p->d.d_model / 256) {
-      case 1: norm_fwd_rows_launch<1>(p, X, gamma, beta, Xn, stats, rms, st); break;
-      case 2: norm_fwd_rows_launch<2>(p, X, gamma, beta, Xn, stats, rms, st); break;
-      case 3: norm_fwd_rows_launch<3>(p, X, gamma, beta, Xn, stats, rms, st); break;
-      default: norm_fwd_rows_launch<4>(p, X, gamma, beta, Xn, stats, rms, st); break;
-    }
+  int nv, wpr;
+  if (p->d.dtype == FBL_DTYPE_BF16 && norm_rows_shape(p->d.d_model, &nv, &wpr)) {
+#define FBL_CALL(NV_, WPR_) norm_fwd_rows_launch<NV_, WPR_>(p, X, gamma, beta, Xn, stats, rms, st)
+    FBL_NORM_DISPATCH(FBL_CALL);
+#undef FBL_CALL
     return cudaGetLastError();
   }
   if (p->d.dtype == FBL_DTYPE_FP32)
@@ -467,13 +508,11 @@ cudaError_t launch_norm_bwd(const fbl_plan* p, const void* dXn, const void* X, c
     e = cudaMemsetAsync(dbeta, 0, d * sizeof(float), st);
     if (e != cudaSuccess) return e;
   }
-  if (p->d.dtype == FBL_DTYPE_BF16 && d % 256 == 0 && d <= 1024) {
-    switch (d / 256) {
-      case 1: norm_bwd_rows_launch<1>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, rms, st); break;
-      case 2: norm_bwd_rows_launch<2>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, rms, st); break;
-      case 3: norm_bwd_rows_launch<3>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, rms, st); break;
-      default: norm_bwd_rows_launch<4>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, rms, st); break;
-    }
+  int nv, wpr;
+  if (p->d.dtype == FBL_DTYPE_BF16 && norm_rows_shape(d, &nv, &wpr)) {
+#define FBL_CALL(NV_, WPR_) norm_bwd_rows_launch<NV_, WPR_>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, rms, st)
+    FBL_NORM_DISPATCH(FBL_CALL);
+#undef FBL_CALL
     return cudaGetLastError();
   }
   if (p->d.dtype == FBL_DTYPE_FP32) {
