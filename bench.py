@@ -53,6 +53,16 @@ def step_flops(cfg):
             "dWv": pk, "dWqkv": pq + 2 * pk, "dWqkv+dXn": 2 * (pq + 2 * pk)}
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the step kernels, from the ncu captures
+# summarised under profiles/ (workload 4, and workload 5 at sequence 2048).  Keyed by (workload name, step).
+NCU_TRAFFIC_BYTES = {
+    ("cfg4-llama1b-gqa", "attn_bwd"): 76.594e6 + 2.509e6,
+    ("cfg4-llama1b-gqa", "attn_fwd"): 25.207e6 + 0.001e6,
+    ("cfg4-llama1b-gqa", "proj_qkv"): 29.397e6 + 0.042e6,
+    ("cfg4-llama1b-gqa", "dWqkv+dXn"): 55.615e6 + 11.459e6,
+}
+
+
 def step_bytes(cfg):
     """Algorithmic HBM bytes of the bandwidth-bound steps."""
     e = 2 if cfg.dtype == "bf16" else 4
@@ -61,48 +71,82 @@ def step_bytes(cfg):
 
 
 class ClockSampler:
+    """Samples the SM clock and the throttle reasons of one GPU while the timed region runs.
+
+    Uses NVML from a background thread (every 5 ms); falls back to an `nvidia-smi -lms 100` child process.
+    Only reads: no clock, power or persistence setting is touched."""
+
+    REASONS = ((0x8, "hw_slowdown"), (0x40, "hw_thermal_slowdown"), (0x20, "sw_thermal_slowdown"), (0x4, "sw_power_cap"))
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index):
-        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        import threading
+        self.sm, self.reasons, self.max_mhz = [], set(), None
+        self.stop_flag = threading.Event()
+        self.thread = self.proc = self.f = None
         try:
-            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
-        except OSError:
-            self.p = None
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = int(visible.split(",")[gpu_index]) if visible and visible.split(",")[gpu_index].isdigit() else gpu_index
+            h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+
+            def poll():
+                while not self.stop_flag.is_set():
+                    try:
+                        self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                        mask = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+                        for bit, name in self.REASONS:
+                            if mask & bit:
+                                self.reasons.add(name)
+                    except Exception:
+                        pass
+                    time.sleep(0.005)
+
+            self.thread = threading.Thread(target=poll, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            try:
+                self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                              "-lms", "100", "-i", str(gpu_index)], stdout=self.f,
+                                             stderr=subprocess.DEVNULL)
+            except OSError:
+                self.proc = None
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.p is None:
-            return out
-        self.p.terminate()
-        try:
-            self.p.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.p.kill()
-        self.f.flush()
-        self.f.seek(0)
-        sm, reasons, mx = [], set(), None
-        for line in self.f.read().splitlines():
-            parts = [x.strip() for x in line.split(",")]
-            if len(parts) < 9:
-                continue
+        if self.thread is not None:
+            self.stop_flag.set()
+            self.thread.join(timeout=2)
+        elif self.proc is not None:
+            self.proc.terminate()
             try:
-                sm.append(float(parts[1]))
-                mx = float(parts[2])
-            except ValueError:
-                continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        os.unlink(self.f.name)
-        if sm:
-            sm.sort()
-            # the median over the whole window includes idle samples between steps; report the upper quartile too
-            out.update(sm_mhz=sm[len(sm) // 2], sm_mhz_p75=sm[(3 * len(sm)) // 4], sm_max_mhz=mx,
-                       reasons=sorted(reasons), samples=len(sm))
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.f.flush()
+            self.f.seek(0)
+            for line in self.f.read().splitlines():
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    self.sm.append(float(parts[1]))
+                    self.max_mhz = float(parts[2])
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                    if val.lower().startswith("active"):
+                        self.reasons.add(name)
+            os.unlink(self.f.name)
+        if self.sm:
+            sm = sorted(self.sm)
+            out.update(sm_mhz=sm[len(sm) // 2], sm_mhz_min=sm[0], sm_max_mhz=self.max_mhz, reasons=sorted(self.reasons),
+                       samples=len(sm))
         return out
 
 
@@ -154,7 +198,7 @@ def run_reference(args, cfg, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=2, help="1-based index into the five workloads (default: the second)")
     ap.add_argument("--impl", default="fblayout", choices=["fblayout", "reference"])
@@ -167,7 +211,6 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "fblayout" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     cfg = get_config(args.config)
     if args.seq or args.batch:
         from fbl_inputs import scaled_config
@@ -184,10 +227,9 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
     torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    from paper_2607_21624_b200.replicas import Replicas
+    rep = Replicas(backend="nccl", device=torch.device("cuda", local_rank))
+    world = rep.world
 
     # replicas only: every rank runs the same workload on its own GPU, no data-path collective
     inp = make_inputs(cfg)
@@ -215,8 +257,7 @@ def main():
 
     def barrier():
         torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
+        rep.barrier()
         torch.cuda.synchronize()
 
     launches0 = run.plan.launch_count()
@@ -305,20 +346,15 @@ def main():
     run.plan.profile_enable(False)
     kernel_ms = {k: sum(v) / len(v) for k, v in acc.items()}
 
-    # max over ranks
-    if dist is not None:
-        t = torch.tensor([ms, ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = rep.max_over_ranks([ms, ms_e2e])      # the slowest replica sets the whole-job time
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
+        rep.close()
         return
 
     peaks = measured_peaks()
     flops = cfg.flops()
-    tfl = world * flops / (ms * 1e-3) / 1e12
-    tfl_e2e = world * flops / (ms_e2e * 1e-3) / 1e12
+    tfl = rep.whole_job_rate(flops, ms) / 1e12
+    tfl_e2e = rep.whole_job_rate(flops, ms_e2e) / 1e12
     sf, sbytes = step_flops(cfg), step_bytes(cfg)
     dom = max(kernel_ms, key=kernel_ms.get)
     total_k = sum(kernel_ms.values())
@@ -336,6 +372,7 @@ def main():
         ach = sbytes.get(dom, 0.0) / (kernel_ms[dom] * 1e-3) / 1e9
         roof = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peaks["gbs"], "unit": "GB/s",
                 "frac": ach / peaks["gbs"], "traffic": None, "peak_source": peaks["source"]}
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((cfg.name, dom))
     roof["kernel_share"] = kernel_ms[dom] / total_k
     roof["kernel_ms"] = {k: round(v, 5) for k, v in sorted(kernel_ms.items(), key=lambda kv: -kv[1])}
 
@@ -358,7 +395,7 @@ def main():
         "config": {"workload": workload_name(cfg), "l2": "256 MiB flush write before every timed step",
                    "launch": "cuda graph replay" if graph is not None else "direct launches",
                    "kernel_path": "default" if args.path == 0 else "ffma", "parallelism": "replicas only"},
-        "tokens_per_s": world * cfg.n_tokens / (ms * 1e-3),
+        "tokens_per_s": rep.whole_job_rate(cfg.n_tokens, ms),
         "layer_roofline": {"t_tensor_us_at_measured_burst": t_tensor * 1e6, "frac_of_measured_burst": t_tensor / (ms * 1e-3),
                            "frac_of_nominal_2250": flops / (NOMINAL_TFLOPS * 1e12) / (ms * 1e-3)},
         "activation_bytes": {"saved": run.sizes["saved"], "scratch": max(run.sizes["scratch_fwd"], run.sizes["scratch_bwd"])},
@@ -368,8 +405,7 @@ def main():
         "clocks": clocks, "roofline": roof, "cpu_baseline": cpu, "wall_s_timed_region": t_wall,
     }
     print(json.dumps(line))
-    if dist is not None:
-        dist.destroy_process_group()
+    rep.close()
 
 
 if __name__ == "__main__":
