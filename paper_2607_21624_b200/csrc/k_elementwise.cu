@@ -3,6 +3,7 @@
 // 16-byte vector each, 4 rows per warp are 512 contiguous bytes, so every warp-level access is a
 // run of whole 128-byte lines.
 #include "fbl_internal.h"
+#include "pdl.cuh"
 
 namespace {
 
@@ -237,6 +238,8 @@ __global__ void __launch_bounds__(256) norm_fwd_rows_kernel(const __nv_bfloat16*
   constexpr int D = NV * 256 * WPR;
   constexpr int RPB = 8 / WPR;                       // rows per block pass
   __shared__ float s_part[8];
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
   const int slot = wib / WPR, part = wib % WPR;
   // n_pad is a multiple of 8, so every warp of a block sees the same number of rows (block-wide barriers)
@@ -291,6 +294,8 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
   __shared__ float s_part[8];
   for (int i = threadIdx.x; i < D; i += 256) { s_dg[i] = 0.f; s_db[i] = 0.f; }
   __syncthreads();
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
   const int slot = wib / WPR, part = wib % WPR;
   float gm[NV][8];
@@ -363,17 +368,16 @@ template <int NV, int WPR>
 void norm_fwd_rows_launch(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
                           float* stats, int rms, cudaStream_t st) {
   const int blocks = (int)min((int64_t)p->sm_count * 4, p->n_pad / (8 / WPR));
-  norm_fwd_rows_kernel<NV, WPR><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)X, gamma, rms ? nullptr : beta,
-                                                        (__nv_bfloat16*)Xn, stats, p->n_pad, p->d.seq, p->t_pad, rms,
-                                                        p->d.eps);
+  launch_pdl(norm_fwd_rows_kernel<NV, WPR>, dim3(blocks), dim3(256), 0, st, (const __nv_bfloat16*)X, gamma,
+             rms ? (const float*)nullptr : beta, (__nv_bfloat16*)Xn, stats, p->n_pad, p->d.seq, p->t_pad, rms, p->d.eps);
 }
 template <int NV, int WPR>
 void norm_bwd_rows_launch(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
                           const float* gamma, void* dX, float* dgamma, float* dbeta, int rms, cudaStream_t st) {
   const int blocks = (int)min((int64_t)p->sm_count * 2, p->n_pad / (8 / WPR));
-  norm_bwd_rows_kernel<NV, WPR><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dXn, (const __nv_bfloat16*)X,
-                                                        (const __nv_bfloat16*)dY, stats, gamma, (__nv_bfloat16*)dX,
-                                                        dgamma, rms ? nullptr : dbeta, p->n_pad, rms);
+  launch_pdl(norm_bwd_rows_kernel<NV, WPR>, dim3(blocks), dim3(256), 0, st, (const __nv_bfloat16*)dXn,
+             (const __nv_bfloat16*)X, (const __nv_bfloat16*)dY, stats, gamma, (__nv_bfloat16*)dX, dgamma,
+             rms ? (float*)nullptr : dbeta, p->n_pad, rms);
 }
 
 // d_model -> (vectors per lane, warps per row) of the register-resident kernels; false if there is none
@@ -418,6 +422,8 @@ __global__ void __launch_bounds__(256) colsum_stage1(ColsumGroup G, int64_t rows
   constexpr int TW = tile_w_of<T>::value;
   constexpr int V = Vec16<T>::N;
   __shared__ float red[32][TW + 1];
+  pdl_launch_dependents();
+  pdl_wait();
   const int which = blockIdx.z;
   const int cols = G.cols[which];
   const int p = blockIdx.x, slab = blockIdx.y;
@@ -447,6 +453,8 @@ __global__ void __launch_bounds__(256) colsum_stage1(ColsumGroup G, int64_t rows
 }
 
 __global__ void colsum_stage2(ColsumGroup G, const float* __restrict__ part_base, int n_slabs) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int which = blockIdx.y;
   const int cols = G.cols[which];
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -551,13 +559,12 @@ cudaError_t launch_colsum_group(int dtype, int count, const void* const* M, int6
   G.count = count;
   const int tw = dtype == FBL_DTYPE_FP32 ? 32 : 64;
   dim3 grid((unsigned)(max_cols / tw), slabs, count);
-  if (dtype == FBL_DTYPE_FP32) colsum_stage1<float><<<grid, 256, 0, st>>>(G, rows, partials);
-  else colsum_stage1<__nv_bfloat16><<<grid, 256, 0, st>>>(G, rows, partials);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e;
+  if (dtype == FBL_DTYPE_FP32) e = launch_pdl(colsum_stage1<float>, grid, dim3(256), 0, st, G, rows, partials);
+  else e = launch_pdl(colsum_stage1<__nv_bfloat16>, grid, dim3(256), 0, st, G, rows, partials);
   if (e != cudaSuccess) return e;
   dim3 grid2((unsigned)((max_cols + 127) / 128), count);
-  colsum_stage2<<<grid2, 128, 0, st>>>(G, partials, slabs);
-  return cudaGetLastError();
+  return launch_pdl(colsum_stage2, grid2, dim3(128), 0, st, G, (const float*)partials, slabs);
 }
 
 cudaError_t launch_colsum(int dtype, const void* M, int64_t rows, int64_t cols, float* out, float* partials,

@@ -3,6 +3,7 @@
 // hold a 1e-4 relative bound) and accept bf16 storage too.  Every operand is addressed through the
 // R-Tile element map; "transposed" operands are the same tiles read with swapped index roles.
 #include "fbl_internal.h"
+#include "pdl.cuh"
 
 namespace {
 
@@ -202,6 +203,8 @@ __global__ void rowdot_kernel(const T* __restrict__ dA, const T* __restrict__ A,
                               int64_t n_pad, int t_pad, int hq, int hd, int64_t total) {
   constexpr int TW = tile_w_of<T>::value;
   constexpr int V = 16 / (int)sizeof(T);
+  pdl_launch_dependents();
+  pdl_wait();
   const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
   if (i >= total) return;
   const int64_t r = i % n_pad;
@@ -360,6 +363,8 @@ __global__ void __launch_bounds__(256) attn_bwd_simt_kernel(const T* __restrict_
 template <typename T>
 __global__ void convert_f32_kernel(const float* __restrict__ src, T* __restrict__ dst, int64_t n) {
   // n is a multiple of 4 (whole tile rows)
+  pdl_launch_dependents();
+  pdl_wait();
   for (int64_t i = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) * 4; i < n; i += (int64_t)gridDim.x * blockDim.x * 4) {
     const float4 v = *reinterpret_cast<const float4*>(src + i);
     dst[i] = from_f<T>(v.x); dst[i + 1] = from_f<T>(v.y); dst[i + 2] = from_f<T>(v.z); dst[i + 3] = from_f<T>(v.w);
@@ -424,20 +429,18 @@ cudaError_t launch_attn_bwd_pre(const fbl_plan* p, const void* A, const void* dA
   if (e != cudaSuccess) return e;
   const unsigned rb = (unsigned)((total + 255) / 256);
   if (p->d.dtype == FBL_DTYPE_FP32)
-    rowdot_kernel<float><<<rb, 256, 0, st>>>((const float*)dA, (const float*)A, dvec, p->n_pad, p->t_pad,
-                                             p->d.n_q_heads, hd, total);
-  else
-    rowdot_kernel<__nv_bfloat16><<<rb, 256, 0, st>>>((const __nv_bfloat16*)dA, (const __nv_bfloat16*)A, dvec, p->n_pad,
-                                                     p->t_pad, p->d.n_q_heads, hd, total);
-  return cudaGetLastError();
+    return launch_pdl(rowdot_kernel<float>, dim3(rb), dim3(256), 0, st, (const float*)dA, (const float*)A, dvec, p->n_pad,
+                      p->t_pad, p->d.n_q_heads, hd, total);
+  return launch_pdl(rowdot_kernel<__nv_bfloat16>, dim3(rb), dim3(256), 0, st, (const __nv_bfloat16*)dA,
+                    (const __nv_bfloat16*)A, dvec, p->n_pad, p->t_pad, p->d.n_q_heads, hd, total);
 }
 
 cudaError_t launch_attn_bwd_post(const fbl_plan* p, const float* dqacc, void* dQ, cudaStream_t st) {
   const int64_t nq = p->n_pad * p->dq;
   const int blocks = (int)min((int64_t)148 * 8, (nq / 4 + 255) / 256);
-  if (p->d.dtype == FBL_DTYPE_FP32) convert_f32_kernel<float><<<blocks, 256, 0, st>>>(dqacc, (float*)dQ, nq);
-  else convert_f32_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(dqacc, (__nv_bfloat16*)dQ, nq);
-  return cudaGetLastError();
+  if (p->d.dtype == FBL_DTYPE_FP32)
+    return launch_pdl(convert_f32_kernel<float>, dim3(blocks), dim3(256), 0, st, dqacc, (float*)dQ, nq);
+  return launch_pdl(convert_f32_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, dqacc, (__nv_bfloat16*)dQ, nq);
 }
 
 cudaError_t launch_attn_bwd_simt(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* A,

@@ -12,6 +12,7 @@
 #include <type_traits>
 
 #include "fbl_internal.h"
+#include "pdl.cuh"
 #include "tc_common.cuh"
 
 namespace {
@@ -118,6 +119,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __gri
   tc::tc_fence_after();
   uint32_t tmem_base;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
+  pdl_launch_dependents();
+  pdl_wait();                                    // the set-up above overlapped the previous kernel's tail
 
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ------------------------------------------------------------------------
@@ -336,8 +339,7 @@ cudaError_t fwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FwdSmem<HD>::TOTAL);
   if (e != cudaSuccess) return e;
   dim3 grid(P.pair ? (n_qt + 1) / 2 : n_qt, p->d.n_q_heads, p->d.batch);
-  k<<<grid, FWD_THREADS, FwdSmem<HD>::TOTAL, st>>>(P);
-  return cudaGetLastError();
+  return launch_pdl(k, grid, dim3(FWD_THREADS), FwdSmem<HD>::TOTAL, st, P);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -442,6 +444,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
   tc::tc_fence_after();
   uint32_t tmem_base;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
+  pdl_launch_dependents();
+  pdl_wait();                                    // the set-up above overlapped the previous kernel's tail
 
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ------------------------------------------------------------------------
@@ -772,8 +776,7 @@ cudaError_t bwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdSmem<HD>::TOTAL);
   if (e != cudaSuccess) return e;
   dim3 grid((p->t_pad + BKV - 1) / BKV, p->d.n_kv_heads, p->d.batch);
-  k<<<grid, BWD_THREADS, BwdSmem<HD>::TOTAL, st>>>(P);
-  return cudaGetLastError();
+  return launch_pdl(k, grid, dim3(BWD_THREADS), BwdSmem<HD>::TOTAL, st, P);
 }
 
 }  // namespace

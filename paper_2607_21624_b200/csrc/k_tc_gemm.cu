@@ -8,6 +8,7 @@
 #include <mutex>
 
 #include "fbl_internal.h"
+#include "pdl.cuh"
 #include "tc_common.cuh"
 
 namespace {
@@ -101,6 +102,8 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
   tc::tc_fence_after();
   uint32_t tmem_base;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
+  pdl_launch_dependents();
+  pdl_wait();                                    // everything above overlapped the previous kernel's tail
 
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ----------------------------------------------------------------------
@@ -304,8 +307,7 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
   cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
   if (attr_err != cudaSuccess) return attr_err;
   const int grid = tiles < p->sm_count ? tiles : p->sm_count;
-  k<<<grid, 192, SP::TOTAL, st>>>(G);
-  return cudaGetLastError();
+  return launch_pdl(k, dim3(grid), dim3(192), SP::TOTAL, st, G);
 }
 
 cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {

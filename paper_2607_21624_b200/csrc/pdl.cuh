@@ -1,0 +1,26 @@
+// Programmatic dependent launch: a kernel launched through launch_pdl may start (block scheduling, barrier
+// and tensor-memory set-up, descriptor prefetch) while the kernel before it on the stream is still draining;
+// pdl_wait() then blocks until that kernel has completed and its memory is visible.  Nothing before
+// pdl_wait() may touch global memory written by earlier kernels.  Outside such a launch both calls are no-ops.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <utility>
+
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
