@@ -334,6 +334,7 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
       g = GemmArgs{};
       g.m = n; g.n = cols[i]; g.n_terms = 1;
       g.t[0] = {Xn, p->n_pad, 0, W[i], D, 0, D};
+      g.b_static = 1;
       g.c = O[i]; g.c_rpad = p->n_pad; g.bias = bias ? B[i] : nullptr;
       g.seq = p->d.seq; g.t_pad = p->t_pad;
       tc = tc && gemm_tc_supported(p, g);
@@ -351,6 +352,7 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
     GemmArgs g = {};
     g.m = n; g.n = D; g.n_terms = 1;
     g.t[0] = {A, p->n_pad, 0, Wo, p->dq, 0, p->dq};
+    g.b_static = 1;
     g.c = Y; g.c_rpad = p->n_pad; g.bias = bias ? bo : nullptr;
     g.residual = p->d.residual ? X : nullptr;
     g.seq = p->d.seq; g.t_pad = p->t_pad;
@@ -396,6 +398,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
     ga = GemmArgs{};
     ga.m = n; ga.n = p->dq; ga.n_terms = 1;
     ga.t[0] = {dY, p->n_pad, 0, Wo, p->dq, 1, D};
+    ga.b_static = 1;
     ga.c = dA; ga.c_rpad = p->n_pad; ga.seq = p->d.seq; ga.t_pad = p->t_pad;
     if (p->use_tc && gemm_tc_supported(p, gw) && gemm_tc_supported(p, ga)) {
       FBL_STEP("dWo+dA", 1, launch_gemm_tc_group(p, gs, 2, status, st));
@@ -424,6 +427,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
     gx = GemmArgs{};
     gx.m = n; gx.n = D; gx.n_terms = 3;
     gx.t[0] = {dQ, p->n_pad, 0, Wq, D, 1, p->dq};
+    gx.b_static = 1;
     gx.t[1] = {dK, p->n_pad, 0, Wk, D, 1, p->dkv};
     gx.t[2] = {dV, p->n_pad, 0, Wv, D, 1, p->dkv};
     gx.c = dXn; gx.c_rpad = p->n_pad; gx.seq = p->d.seq; gx.t_pad = p->t_pad;

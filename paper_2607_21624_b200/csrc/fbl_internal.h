@@ -70,6 +70,7 @@ struct GemmArgs {
   const float* bias;              // per output column, or nullptr
   const void* residual;           // same layout as C, or nullptr
   int seq, t_pad;                 // if t_pad > 0: rows with (row % t_pad) >= seq are written as zero
+  int b_static;                   // 1: the first term's B operand is an input of the whole step (a weight)
 };
 
 cudaError_t launch_gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);

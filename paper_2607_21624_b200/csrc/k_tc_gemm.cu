@@ -17,8 +17,10 @@ constexpr int BM = 128, BK = 64;
 constexpr int MAX_TERMS = 3, MAX_PROBLEMS = 4;
 
 struct alignas(64) TcProblem {
-  CUtensorMap ta[MAX_TERMS], tb[MAX_TERMS];
+  CUtensorMap ta[MAX_TERMS], tb[MAX_TERMS], tc;     // tc: the output, for the epilogue's bulk stores
   int n_terms;
+  int b_static;                                        // 1: the first term's B operand is an input of the whole
+                                                       // step (a weight), not written by an earlier kernel
   int kblocks[MAX_TERMS];
   int a_mn[MAX_TERMS], b_mn[MAX_TERMS];   // 1: operand is MN-major in shared memory (its rows are K indices)
   int m, n;
@@ -39,8 +41,9 @@ struct SmemPlan {
   static constexpr uint32_t A_BYTES = BM * 128;
   static constexpr uint32_t B_BYTES = BN * 128;
   static constexpr uint32_t STAGE = A_BYTES + B_BYTES;
-  static constexpr uint32_t BAR_OFF = STAGES * STAGE;
-  static constexpr uint32_t N_BARS = 2 * STAGES + 4;     // full[], empty[], acc_full[2], acc_empty[2]
+  static constexpr uint32_t STG_OFF = STAGES * STAGE;    // two 128 x 64 bf16 output staging tiles
+  static constexpr uint32_t BAR_OFF = STG_OFF + 2 * 16384;
+  static constexpr uint32_t N_BARS = 2 * STAGES + 8;     // full[], empty[], acc_full[2], acc_empty[2], stg_full[2], stg_free[2]
   static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16 + 1024;   // + TMEM slot + alignment slack
 };
 
@@ -77,6 +80,8 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
   auto empty = [&](int s) { return bars + 8u * (STAGES + s); };
   auto acc_full = [&](int a) { return bars + 8u * (2 * STAGES + a); };
   auto acc_empty = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
+  auto stg_full = [&](int a) { return bars + 8u * (2 * STAGES + 4 + a); };
+  auto stg_free = [&](int a) { return bars + 8u * (2 * STAGES + 6 + a); };
   const uint32_t slot = bars + 8 * SP::N_BARS;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   int32_t* status = G.status;
@@ -90,6 +95,8 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
     for (int a = 0; a < 2; ++a) {
       tc::mbar_init(acc_full(a), 1);
       tc::mbar_init(acc_empty(a), 128);
+      tc::mbar_init(stg_full(a), 128);
+      tc::mbar_init(stg_free(a), 1);
     }
     tc::fence_barrier_init();
   }
@@ -103,26 +110,47 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
   uint32_t tmem_base;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
   pdl_launch_dependents();
-  pdl_wait();                                    // everything above overlapped the previous kernel's tail
 
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ----------------------------------------------------------------------
     int it = 0;
     bool ok = true;
     TileCoord tcd;
+    // Weights do not depend on the kernel before this one: their tiles for the first stages of the first
+    // output tile are requested before waiting for that kernel, hiding their (cold) latency.
+    int prefilled = 0;
+    if (tile_at<BN>(G, blockIdx.x, &tcd) && G.p[tcd.prob].b_static) {
+      const TcProblem& P = G.p[tcd.prob];
+      tc::tma_prefetch_desc(&P.ta[0]);
+      tc::tma_prefetch_desc(&P.tb[0]);
+      const int n = P.kblocks[0] < STAGES ? P.kblocks[0] : STAGES;
+      for (int kb = 0; kb < n; ++kb) {
+        const uint32_t sb = base + kb * SP::STAGE + SP::A_BYTES;
+        tc::mbar_expect_tx(full(kb), SP::STAGE);
+        if (P.b_mn[0]) tc::tma_load_3d(sb, &P.tb[0], full(kb), 0, kb * BK, tcd.n0 / 64);
+        else tc::tma_load_3d(sb, &P.tb[0], full(kb), 0, tcd.n0, kb);
+      }
+      prefilled = n;
+    }
+    pdl_wait();
     for (int w = blockIdx.x; ok && tile_at<BN>(G, w, &tcd); w += gridDim.x) {
       const TcProblem& P = G.p[tcd.prob];
       for (int t = 0; t < P.n_terms && ok; ++t) {
         for (int kb = 0; kb < P.kblocks[t]; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
-          if (!tc::mbar_wait(empty(s), ph ^ 1, status, 101)) { ok = false; break; }
           const uint32_t sa = base + s * SP::STAGE, sb = sa + SP::A_BYTES;
-          tc::mbar_expect_tx(full(s), SP::STAGE);
+          const bool pre = it < prefilled;                 // this stage's barrier is armed and its B tile on its way
+          if (!pre) {
+            if (!tc::mbar_wait(empty(s), ph ^ 1, status, 101)) { ok = false; break; }
+            tc::mbar_expect_tx(full(s), SP::STAGE);
+          }
           if (P.a_mn[t]) tc::tma_load_3d(sa, &P.ta[t], full(s), 0, kb * BK, tcd.m0 / 64);
           else tc::tma_load_3d(sa, &P.ta[t], full(s), 0, tcd.m0, kb);
-          if (P.b_mn[t]) tc::tma_load_3d(sb, &P.tb[t], full(s), 0, kb * BK, tcd.n0 / 64);
-          else tc::tma_load_3d(sb, &P.tb[t], full(s), 0, tcd.n0, kb);
+          if (!pre) {
+            if (P.b_mn[t]) tc::tma_load_3d(sb, &P.tb[t], full(s), 0, kb * BK, tcd.n0 / 64);
+            else tc::tma_load_3d(sb, &P.tb[t], full(s), 0, tcd.n0, kb);
+          }
         }
       }
     }
@@ -163,9 +191,13 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
       if (ok) tc::mma_commit(acc_full(ab));
     }
   } else if (warp >= 2) {
-    // ---- epilogue: TMEM -> registers -> R-Tile rows (each thread owns one output row) -----------
+    // ---- epilogue: TMEM -> registers -> swizzled staging tile -> bulk tensor store, one 64-column panel at
+    // a time (two staging tiles: the store of one panel overlaps the conversion of the next) -------------
+    pdl_wait();                                       // the previous kernel may still be reading what we overwrite
     const int q = warp % 4;                           // the TMEM lane quarter this warp may access
-    int ti = 0;
+    const int r = q * 32 + lane;                      // row of the tile owned by this thread
+    const bool issuer = threadIdx.x == 64;
+    int ti = 0, pc = 0;                               // tiles and panels done by this block
     bool ok = true;
     TileCoord tcd;
     for (int w = blockIdx.x; ok && tile_at<BN>(G, w, &tcd); w += gridDim.x, ++ti) {
@@ -173,39 +205,60 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
       const int ab = ti & 1;
       if (!tc::mbar_wait(acc_full(ab), (ti >> 1) & 1, status, 103)) { ok = false; break; }
       tc::tc_fence_after();
-      const int row = tcd.m0 + q * 32 + lane;
+      const int row = tcd.m0 + r;
       const bool pad = P.t_pad > 0 && (row % P.t_pad) >= P.seq;
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t r[32];
-        tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + c0, r);
+      for (int pn = 0; pn < BN / 64 && ok; ++pn) {
+        const int n = tcd.n0 + pn * 64;
+        if (n >= P.n) break;                           // uniform: N is whole 64-column panels
+        uint32_t v[64];
+        tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + pn * 64, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+        tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + pn * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
         tc::tmem_ld_wait();
-        const int n = tcd.n0 + c0;
-        if (row < P.m && n < P.n) {
-          const long long off = ((long long)(n / 64) * P.c_rpad + row) * 64 + (n % 64);
-          uint4 resv[4];
-          if (P.residual) {
+        uint4 outv[8];
+        uint32_t* ow = reinterpret_cast<uint32_t*>(outv);
+        if (P.residual && row < P.m) {
+          const __nv_bfloat16* rp = P.residual + ((long long)(n / 64) * P.c_rpad + row) * 64;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) resv[j] = *reinterpret_cast<const uint4*>(P.residual + off + 8 * j);
+          for (int j = 0; j < 8; ++j) {
+            const uint4 rv = *reinterpret_cast<const uint4*>(rp + 8 * j);
+            const __nv_bfloat16* rb = reinterpret_cast<const __nv_bfloat16*>(&rv);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v[8 * j + k] = __float_as_uint(__uint_as_float(v[8 * j + k]) + __bfloat162float(rb[k]));
           }
-          const __nv_bfloat16* rb = reinterpret_cast<const __nv_bfloat16*>(resv);
-          uint4 outv[4];
-          uint32_t* ow = reinterpret_cast<uint32_t*>(outv);
-#pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            float v0 = __uint_as_float(r[j]), v1 = __uint_as_float(r[j + 1]);
-            if (P.bias) { v0 += P.bias[n + j]; v1 += P.bias[n + j + 1]; }
-            if (P.residual) { v0 += __bfloat162float(rb[j]); v1 += __bfloat162float(rb[j + 1]); }
-            if (pad) { v0 = 0.f; v1 = 0.f; }
-            ow[j / 2] = tc::pack_bf16(v0, v1);
-          }
-#pragma unroll
-          for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(P.c + off + 8 * j) = outv[j];
         }
+#pragma unroll
+        for (int j = 0; j < 64; j += 2) {
+          float v0 = __uint_as_float(v[j]), v1 = __uint_as_float(v[j + 1]);
+          if (P.bias) { v0 += P.bias[n + j]; v1 += P.bias[n + j + 1]; }
+          if (pad) { v0 = 0.f; v1 = 0.f; }
+          ow[j / 2] = tc::pack_bf16(v0, v1);
+        }
+        const int sb = pc & 1;
+        const uint32_t stg = base + SP::STG_OFF + sb * 16384;
+        // the staging tile's previous store (two panels ago) must have read it
+        if (pc >= 2 && !tc::mbar_wait(stg_free(sb), ((pc >> 1) - 1) & 1, status, 105)) { ok = false; break; }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + r * 128 + (((uint32_t)j ^ (uint32_t)(r & 7)) * 16)),
+                       "r"(outv[j].x), "r"(outv[j].y), "r"(outv[j].z), "r"(outv[j].w) : "memory");
+        tc::fence_proxy_async();
+        tc::mbar_arrive(stg_full(sb));
+        if (issuer) {
+          if (!tc::mbar_wait(stg_full(sb), (pc >> 1) & 1, status, 106)) { ok = false; break; }
+          tc::tma_store_3d(&P.tc, stg, 0, tcd.m0, n / 64);
+          tc::bulk_commit_group();
+          if (pc >= 1) {                               // at most this store in flight: the previous one has read
+            tc::bulk_wait_group_read1();               // its staging tile, which may now be overwritten
+            tc::mbar_arrive(stg_free(sb ^ 1));
+          }
+        }
+        ++pc;
       }
       tc::tc_fence_before();
       tc::mbar_arrive(acc_empty(ab));             // this accumulator may be overwritten by the tile after next
     }
+    if (issuer) tc::bulk_wait_group0();           // all output tiles are in global memory before the block exits
   }
   tc::tc_fence_before();
   __syncthreads();
@@ -297,6 +350,8 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
       if (!ok) return cudaErrorInvalidValue;
     }
     P.m = g.m; P.n = g.n;
+    if (!fbl_encode_rtile_map(&P.tc, g.c, g.c_rpad, g.n / 64, BM, 1)) return cudaErrorInvalidValue;
+    P.b_static = g.b_static;
     P.c = (__nv_bfloat16*)g.c; P.c_rpad = g.c_rpad;
     P.bias = g.bias; P.residual = (const __nv_bfloat16*)g.residual;
     P.seq = g.seq; P.t_pad = g.t_pad;
