@@ -20,6 +20,24 @@ namespace {
 constexpr int BQ = 128, BKV = 128;
 constexpr float LOG2E = 1.4426950408889634f;
 
+// Block numbering shared by both kernels.  (head, batch) pairs are taken in chunks small enough for their
+// operands to stay in L2 together; inside a chunk the causal-work index ("slot": query-tile slot forward, key
+// tile backward) varies slowest, heaviest first, so the block scheduler, which dispatches in block-id order,
+// hands out the long blocks of a chunk before its short ones.
+__device__ __forceinline__ void decode_block(int lin, int n_slots, int n_hb, int chunk, int* slot, int* hb) {
+  const int per_chunk = n_slots * chunk;
+  const int full = (n_hb / chunk) * per_chunk;
+  int c0, csize, rem;
+  if (lin < full) { c0 = (lin / per_chunk) * chunk; csize = chunk; rem = lin % per_chunk; }
+  else { c0 = (n_hb / chunk) * chunk; csize = n_hb - c0; rem = lin - full; }
+  *slot = rem / csize;
+  *hb = c0 + rem % csize;
+}
+static int chunk_for(long long bytes_per_hb, int n_hb, long long budget) {
+  long long c = budget / (bytes_per_hb > 0 ? bytes_per_hb : 1);
+  return (int)(c < 1 ? 1 : (c > n_hb ? n_hb : c));
+}
+
 // Optional timeline probe (compile with -DFBL_TRACE): block (0,0,0) records clock64() at the marked points of
 // iterations 8..14 into the 1 KiB status area, after the status word.
 #ifdef FBL_TRACE
@@ -29,7 +47,7 @@ constexpr float LOG2E = 1.4426950408889634f;
 #ifndef FBL_TRACE_BLOCK
 #define FBL_TRACE_BLOCK 0
 #endif
-#define TR(k) do { if (blockIdx.x == FBL_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && it >= FBL_TRACE_FIRST && it < FBL_TRACE_FIRST + 3) ((long long*)P.status)[8 + (it - FBL_TRACE_FIRST) * 32 + (k)] = clock64(); } while (0)
+#define TR(k) do { if (blockIdx.x == FBL_TRACE_BLOCK && it >= FBL_TRACE_FIRST && it < FBL_TRACE_FIRST + 3) ((long long*)P.status)[8 + (it - FBL_TRACE_FIRST) * 32 + (k)] = clock64(); } while (0)
 #else
 #define TR(k) do { } while (0)
 #endif
@@ -41,6 +59,7 @@ struct alignas(64) AttnFwdParams {
   long long n_pad;
   int seq, t_pad, hq, group, causal;
   int pair;              // 1: each block owns two adjacent query tiles, one per softmax warp group
+  int batch, n_slots, chunk;   // grid = n_slots * hq * batch blocks, see decode_block
   float scale;
   int32_t* status;
 };
@@ -77,13 +96,14 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __gri
   auto bar = [&](int i) { return bars + 8u * i; };
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int n_qt = (P.seq + BQ - 1) / BQ;
-  const int h = blockIdx.y, b = blockIdx.z, g = h / P.group;
+  int slot_i, hb;
+  decode_block((int)blockIdx.x, P.n_slots, P.hq * P.batch, P.chunk, &slot_i, &hb);
+  const int h = hb % P.hq, b = hb / P.hq, g = h / P.group;
   const int row0 = b * P.t_pad;
   int32_t* status = P.status;
-  // query tiles of this block: with pairing, tile x and its mirror n_qt-1-x (equal causal work in every block)
-  // heaviest causal tiles first; with pairing a block owns two adjacent tiles, whose key ranges differ by one tile,
-  // so both warp groups stay busy for the whole loop
-  const int slot_x = (int)gridDim.x - 1 - (int)blockIdx.x;
+  // with pairing a block owns two adjacent tiles, whose key ranges differ by one tile, so both warp groups stay
+  // busy for the whole loop
+  const int slot_x = P.n_slots - 1 - slot_i;                 // heaviest (latest) causal tiles first
   const int qt0 = P.pair ? min(2 * slot_x + 1, n_qt - 1) : slot_x;
   const int qt1 = (P.pair && 2 * slot_x + 1 < n_qt) ? 2 * slot_x : -1;   // odd tile count: the last block has one tile
   auto kv_tiles = [&](int t) {
@@ -338,7 +358,10 @@ cudaError_t fwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   auto k = attn_fwd_tc_kernel<HD>;
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FwdSmem<HD>::TOTAL);
   if (e != cudaSuccess) return e;
-  dim3 grid(P.pair ? (n_qt + 1) / 2 : n_qt, p->d.n_q_heads, p->d.batch);
+  P.batch = p->d.batch;
+  P.n_slots = P.pair ? (n_qt + 1) / 2 : n_qt;
+  P.chunk = chunk_for((long long)p->d.seq * HD * 4, p->d.n_q_heads * p->d.batch, 96ll << 20);   // K and V of one head
+  dim3 grid((unsigned)(P.n_slots * p->d.n_q_heads * p->d.batch));
   return launch_pdl(k, grid, dim3(FWD_THREADS), FwdSmem<HD>::TOTAL, st, P);
 }
 
@@ -361,6 +384,7 @@ struct alignas(64) AttnBwdParams {
   __nv_bfloat16* dv;
   long long n_pad;
   int seq, t_pad, hq, group, causal, dkv;
+  int batch, chunk;      // grid = key tiles * KV heads * batch blocks, see decode_block
   float scale;
   int32_t* status;
 };
@@ -382,11 +406,11 @@ struct BwdSmem {
   static constexpr uint32_t DS_OFF = DO_OFF + NQ * TILE, STAGE_OFF = DS_OFF + NP * 32768;
   static constexpr uint32_t LSE_OFF = STAGE_OFF + NP * STAGE_BYTES;    // 2 buffers x (128 floats LSE*log2e, 128 floats D)
   static constexpr uint32_t BAR_OFF = LSE_OFF + 2048;
-  static constexpr uint32_t N_BARS = 14;
+  static constexpr uint32_t N_BARS = 15;
   static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16;
 };
 
-enum { BB_KVFULL = 0, BB_QDOFULL = 1, BB_QDOEMPTY = 3, BB_SFULL = 5, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY, BB_DQSTAGED, BB_STAGEFREE, BB_SREAD = BB_STAGEFREE + 2 };
+enum { BB_KVFULL = 0, BB_QDOFULL = 1, BB_QDOEMPTY = 3, BB_SFULL = 5, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY, BB_DQSTAGED, BB_STAGEFREE, BB_SREAD = BB_STAGEFREE + 2, BB_DVDONE };
 
 constexpr int BWD_THREADS = 608;     // warp 0 TMA loads, warp 1 MMA, warps 2-17 softmax (four per TMEM lane quarter), warp 18 dQ reductions
 constexpr int BWD_SM_THREADS = 512;
@@ -398,7 +422,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
   constexpr uint32_t PANELS = SM::PANELS, NQ = SM::NQ, NP = SM::NP;
   constexpr uint32_t S_COL = 0, DP_COL = 128, DV_COL = 256, DK_COL = 256 + HD;
   constexpr uint32_t DQ_COL = PIPE ? 384 : DP_COL;   // HD = 128: dQ reuses the dP^T columns
-  constexpr uint32_t P_COL = S_COL;                  // P^T (64 packed columns) overwrites S^T in place
+  constexpr uint32_t P_COL = PIPE ? 448 : S_COL;     // HD = 64: own columns; HD = 128: P^T overwrites S^T in place
   constexpr uint32_t TMEM_COLS = 512;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = tc::smem_u32(smem_raw);
@@ -406,7 +430,11 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
   const uint32_t slot = bars + 8 * SM::N_BARS;
   auto bar = [&](int i) { return bars + 8u * i; };
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int j0 = blockIdx.x * BKV, g = blockIdx.y, b = blockIdx.z;
+  // under a causal mask key tile 0 has the most query tiles: it is slot 0
+  const int n_kvh = P.hq / P.group;
+  int slot_i, gb;
+  decode_block((int)blockIdx.x, (P.t_pad + BKV - 1) / BKV, n_kvh * P.batch, P.chunk, &slot_i, &gb);
+  const int j0 = slot_i * BKV, g = gb % n_kvh, b = gb / n_kvh;
   const int row0 = b * P.t_pad;
   const int n_qt = (P.seq + BQ - 1) / BQ;
   const int qt_begin = P.causal ? j0 / BQ : 0;
@@ -433,6 +461,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     tc::mbar_init(bar(BB_STAGEFREE), 1);
     tc::mbar_init(bar(BB_STAGEFREE + 1), 1);
     tc::mbar_init(bar(BB_SREAD), BWD_SM_THREADS);
+    tc::mbar_init(bar(BB_DVDONE), 1);
     tc::fence_barrier_init();
   }
   if (warp == 1) {
@@ -493,7 +522,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
                         tc::smem_desc_sw128(dos + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
       }
     };
-    auto issue_dk_dq = [&](int it) {          // dK += dS^T Q, dQ = dS K
+    auto issue_dk = [&](int it) {             // dK += dS^T Q
       const uint32_t qs = base + SM::Q_OFF + (it % NQ) * SM::TILE;
       const uint32_t dss = base + SM::DS_OFF + (it % NP) * 32768;
 #pragma unroll
@@ -503,8 +532,9 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         tc::mma_bf16_ss(tmem_base + DK_COL, tc::smem_desc_sw128(dss + ao, 16, 1024),
                         tc::smem_desc_sw128(qs + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
       }
-      tc::mma_commit(bar(BB_QDOEMPTY + (it % NQ)));                // Q / dO of this tile are not read again:
-                                                                   // the next TMA load overlaps dQ and its drain
+    };
+    auto issue_dq = [&](int it) {             // dQ = dS K: the dS^T tile read MN-major, i.e. transposed by descriptor
+      const uint32_t dss = base + SM::DS_OFF + (it % NP) * 32768;
 #pragma unroll
       for (uint32_t kk = 0; kk < BKV / 16; ++kk) {
         const uint32_t o = kk * 2048;                              // both operands MN-major: 16 key rows per step
@@ -519,21 +549,34 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       if (ok) { tc::tc_fence_after(); issue_s(0); issue_dp(0); }
     }
     if (PIPE) {
-      // dV first (it frees the S^T columns that hold P^T), then the next tile's scores, then dK and dQ: the
-      // softmax warps start on tile it + 1 while the tensor pipe is still busy with dK, dQ of tile it
+      // P^T has its own columns here, so the next tile's products come first and the softmax warps start on
+      // tile it + 1 while the tensor pipe works on dV, dK, dQ of tile it
       for (int it = 0; it < n_it && ok; ++it) {
-        if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
-        tc::tc_fence_after();
-        issue_dv(it);
+        TR(0);
         if (it + 1 < n_it) {
+          // S^T(it+1) as soon as every softmax warp has copied S^T(it) to registers: it is computed while
+          // they work on tile it
+          if (!tc::mbar_wait(bar(BB_SREAD), it & 1, status, 311)) { ok = false; break; }
           if (!tc::mbar_wait(bar(BB_QDOFULL + ((it + 1) % NQ)), ((it + 1) / NQ) & 1, status, 303)) { ok = false; break; }
+          TR(1);
           tc::tc_fence_after();
           issue_s(it + 1);
-          issue_dp(it + 1);
         }
-        if (it > 0 && !tc::mbar_wait(bar(BB_DQDRAINED), (it - 1) & 1, status, 304)) { ok = false; break; }
+        if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
+        TR(2);
         tc::tc_fence_after();
-        issue_dk_dq(it);
+        if (it + 1 < n_it) issue_dp(it + 1);            // dP^T(it) has been read as well: announce tile it + 1
+        TR(3);
+        issue_dv(it);
+        tc::mma_commit(bar(BB_DVDONE));                 // P^T(it) has been read: P^T(it+1) may be stored
+        TR(4);
+        if (it > 0 && !tc::mbar_wait(bar(BB_DQDRAINED), (it - 1) & 1, status, 304)) { ok = false; break; }
+        TR(5);
+        tc::tc_fence_after();
+        issue_dk(it);
+        tc::mma_commit(bar(BB_QDOEMPTY + (it % NQ)));   // Q / dO of this tile are not read again
+        issue_dq(it);
+        TR(6);
       }
     } else {
       for (int it = 0; it < n_it && ok; ++it) {
@@ -541,8 +584,12 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
         TR(1);
         tc::tc_fence_after();
+        // dQ first: its drain to shared memory (which frees the dP^T columns for the next tile) then overlaps
+        // the dV and dK products
+        issue_dq(it);
+        issue_dk(it);
         issue_dv(it);
-        issue_dk_dq(it);
+        tc::mma_commit(bar(BB_QDOEMPTY));               // Q / dO of this tile are not read again
         TR(2);
         if (it + 1 < n_it) {
           if (!tc::mbar_wait(bar(BB_QDOFULL), (it + 1) & 1, status, 303)) { ok = false; break; }
@@ -651,15 +698,21 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       // element masks are needed only on the diagonal tile and on tiles with keys or queries beyond the sequence
       const bool need_mask = (P.causal && (i0 < j0 + BKV - 1)) || (j0 + BKV > P.seq) || (i0 + BQ > P.seq);
       const uint32_t dsrow = base + SM::DS_OFF + (it % NP) * 32768 + (part / 2) * 16384 + r * 128;
-      // this thread's 32 score columns first: the packed P^T overwrites S^T columns that belong to other warps
-      // of the same lane quarter, so every warp must have read its scores before any P^T store
+      // this thread's 32 score columns first: with HD = 128 the packed P^T overwrites S^T columns that belong to
+      // other warps of the same lane quarter, so every warp must have read its scores before any P^T store
       uint32_t sv[32];
       tc::tmem_ld32(lane_addr + S_COL + part * 32, sv);
       tc::tmem_ld_wait();
       tc::tc_fence_before();
-      tc::mbar_arrive(bar(BB_SREAD));
-      if (!tc::mbar_wait(bar(BB_SREAD), it & 1, status, 311)) { ok = false; break; }
-      tc::tc_fence_after();
+      tc::mbar_arrive(bar(BB_SREAD));                   // this thread's scores are in registers
+      if (!PIPE) {
+        if (!tc::mbar_wait(bar(BB_SREAD), it & 1, status, 311)) { ok = false; break; }
+        tc::tc_fence_after();
+      } else if (it > 0) {
+        // P^T has its own columns, single-buffered: the dV product of the previous tile must have read them
+        if (!tc::mbar_wait(bar(BB_DVDONE), (it - 1) & 1, status, 312)) { ok = false; break; }
+        tc::tc_fence_after();
+      }
       // One 16-column chunk: P^T = exp2(S^T c - LSE) to tensor memory, dS^T = P^T (dP^T - D) to the swizzled
       // shared-memory operand tile, both rounded to bf16.  MASKED is the rare path (diagonal / ragged tiles).
       auto chunk = [&](int cc, auto masked_tag) {
@@ -775,7 +828,13 @@ cudaError_t bwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   auto k = attn_bwd_tc_kernel<HD>;
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdSmem<HD>::TOTAL);
   if (e != cudaSuccess) return e;
-  dim3 grid((p->t_pad + BKV - 1) / BKV, p->d.n_kv_heads, p->d.batch);
+  P.batch = p->d.batch;
+  // Q, dO (bf16) and the fp32 dQ accumulator of the query heads of one KV head.  The HD = 128 variant waits for
+  // its single-buffered Q / dO tiles on the critical path, so it keeps the blocks that share those tiles close
+  // together (small chunks: L2 hits); the pipelined HD = 64 variant hides that latency and prefers balance.
+  P.chunk = chunk_for((long long)p->group * p->d.seq * HD * 8, p->d.n_kv_heads * p->d.batch,
+                      BwdSmem<HD>::PIPE ? (96ll << 20) : (8ll << 20));
+  dim3 grid((unsigned)(((p->t_pad + BKV - 1) / BKV) * p->d.n_kv_heads * p->d.batch));
   return launch_pdl(k, grid, dim3(BWD_THREADS), BwdSmem<HD>::TOTAL, st, P);
 }
 
