@@ -56,10 +56,12 @@ def step_flops(cfg):
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the step kernels, from the ncu captures
 # summarised under profiles/ (workload 4, and workload 5 at sequence 2048).  Keyed by (workload name, step).
 NCU_TRAFFIC_BYTES = {
-    ("cfg4-llama1b-gqa", "attn_bwd"): 76.594e6 + 2.509e6,
-    ("cfg4-llama1b-gqa", "attn_fwd"): 25.207e6 + 0.001e6,
-    ("cfg4-llama1b-gqa", "proj_qkv"): 29.397e6 + 0.042e6,
-    ("cfg4-llama1b-gqa", "dWqkv+dXn"): 55.615e6 + 11.459e6,
+    ("cfg4-llama1b-gqa", "proj_qkv"): 29.4e6 + 0.4e6,
+    ("cfg4-llama1b-gqa", "attn_fwd"): 25.2e6 + 0.0e6,
+    ("cfg4-llama1b-gqa", "proj_o"): 25.2e6 + 0.0e6,
+    ("cfg4-llama1b-gqa", "dWo+dA"): 42.0e6 + 1.9e6,
+    ("cfg4-llama1b-gqa", "attn_bwd"): 76.6e6 + 3.8e6,
+    ("cfg4-llama1b-gqa", "dWqkv+dXn"): 55.9e6 + 11.8e6,
 }
 
 
