@@ -69,6 +69,11 @@ SMALL_BF16 = [
     LayerConfig("b4", 2, 130, 256, 2, 2, 128, "bf16", "rmsnorm", True, False, False, 1e-5, 24, 0.01),
     LayerConfig("b5", 1, 8, 128, 2, 2, 64, "bf16", "layernorm", True, True, False, 1e-5, 25, 0.02),
     LayerConfig("b6", 2, 1, 128, 2, 1, 64, "bf16", "rmsnorm", False, False, False, 1e-5, 26, 0.02),
+    # enough blocks for the forward kernel to pair query tiles, with an odd tile count and a ragged last tile
+    LayerConfig("b7", 10, 330, 512, 8, 2, 64, "bf16", "rmsnorm", True, False, False, 1e-5, 27, 0.02),
+    LayerConfig("b8", 20, 300, 512, 4, 4, 128, "bf16", "layernorm", False, True, True, 1e-5, 28, 0.02),
+    # sequence an exact multiple of the 128-row tiles, group of 8 query heads per KV head
+    LayerConfig("b9", 2, 256, 512, 8, 1, 64, "bf16", "layernorm", True, False, False, 1e-5, 29, 0.02),
 ]
 
 
