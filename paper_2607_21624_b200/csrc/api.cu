@@ -387,6 +387,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
 
   FBL_CUDA(cudaMemsetAsync(status, 0, FBL_ALIGN, st));
   FBL_PROF_BEGIN();
+  bool dvec_ready = false;
   {
     GemmArgs gs[2];
     GemmArgs& gw = gs[0];   // dWo = A^T dY : token-axis reduction (longest reduction loop: first in the work list)
@@ -401,13 +402,16 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
     ga.b_static = 1;
     ga.c = dA; ga.c_rpad = p->n_pad; ga.seq = p->d.seq; ga.t_pad = p->t_pad;
     if (p->use_tc && gemm_tc_supported(p, gw) && gemm_tc_supported(p, ga)) {
+      // D = rowsum(dO * O) per head comes out of the dA epilogue, from the fp32 accumulator
+      ga.dot_with = A; ga.dot_out = dvec; ga.dot_hd = p->d.head_dim; ga.dot_hq = p->d.n_q_heads;
+      dvec_ready = true;
       FBL_STEP("dWo+dA", 1, launch_gemm_tc_group(p, gs, 2, status, st));
     } else {
       FBL_STEP("dA", 1, run_gemm(p, ga, part, p->part_bytes, status, st));
       FBL_STEP("dWo", 1, run_gemm(p, gw, part, p->part_bytes, status, st));
     }
   }
-  if (p->use_tc && attn_bwd_tc_supported(p)) FBL_STEP("attn_bwd", 3, launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, status, st));
+  if (p->use_tc && attn_bwd_tc_supported(p)) FBL_STEP("attn_bwd", dvec_ready ? 2 : 3, launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, dvec_ready, status, st));
   else FBL_STEP("attn_bwd", 3, launch_attn_bwd_simt(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, st));
   {
     const void* G[3] = {dQ, dK, dV};

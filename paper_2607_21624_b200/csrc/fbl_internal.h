@@ -71,6 +71,8 @@ struct GemmArgs {
   const void* residual;           // same layout as C, or nullptr
   int seq, t_pad;                 // if t_pad > 0: rows with (row % t_pad) >= seq are written as zero
   int b_static;                   // 1: the first term's B operand is an input of the whole step (a weight)
+  // optional fused row reduction D[b,h,t] = sum_d C[row, h*hd+d] * dot_with[row, h*hd+d] (fp32 C, before rounding)
+  const void* dot_with; float* dot_out; int dot_hd, dot_hq;
 };
 
 cudaError_t launch_gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);
@@ -100,10 +102,10 @@ cudaError_t launch_attn_bwd_simt(const fbl_plan* p, const void* Q, const void* K
                                  const void* dA, const float* lse, float* dvec, float* dqacc, void* dQ, void* dK,
                                  void* dV, cudaStream_t st);
 cudaError_t launch_attn_bwd_pre(const fbl_plan* p, const void* A, const void* dA, float* dvec, float* dqacc,
-                                cudaStream_t st);
+                                bool dvec_ready, cudaStream_t st);
 cudaError_t launch_attn_bwd_post(const fbl_plan* p, const float* dqacc, void* dQ, cudaStream_t st);
 cudaError_t launch_attn_fwd_tc(const fbl_plan* p, const void* Q, const void* K, const void* V, void* A, float* lse,
                                int32_t* status, cudaStream_t st);
 cudaError_t launch_attn_bwd_tc(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* A,
                                const void* dA, const float* lse, float* dvec, float* dqacc, void* dQ, void* dK,
-                               void* dV, int32_t* status, cudaStream_t st);
+                               void* dV, bool dvec_ready, int32_t* status, cudaStream_t st);

@@ -421,12 +421,12 @@ cudaError_t launch_attn_fwd_simt(const fbl_plan* p, const void* Q, const void* K
 }
 
 cudaError_t launch_attn_bwd_pre(const fbl_plan* p, const void* A, const void* dA, float* dvec, float* dqacc,
-                                cudaStream_t st) {
+                                bool dvec_ready, cudaStream_t st) {
   const int hd = p->d.head_dim;
   const int64_t total = p->n_pad * p->d.n_q_heads;
   const int64_t nq = p->n_pad * p->dq;
   cudaError_t e = cudaMemsetAsync(dqacc, 0, (size_t)nq * sizeof(float), st);
-  if (e != cudaSuccess) return e;
+  if (e != cudaSuccess || dvec_ready) return e;
   const unsigned rb = (unsigned)((total + 255) / 256);
   if (p->d.dtype == FBL_DTYPE_FP32)
     return launch_pdl(rowdot_kernel<float>, dim3(rb), dim3(256), 0, st, (const float*)dA, (const float*)A, dvec, p->n_pad,
@@ -447,7 +447,7 @@ cudaError_t launch_attn_bwd_simt(const fbl_plan* p, const void* Q, const void* K
                                  const void* dA, const float* lse, float* dvec, float* dqacc, void* dQ, void* dK,
                                  void* dV, cudaStream_t st) {
   const int hd = p->d.head_dim;
-  cudaError_t e = launch_attn_bwd_pre(p, A, dA, dvec, dqacc, st);
+  cudaError_t e = launch_attn_bwd_pre(p, A, dA, dvec, dqacc, false, st);
   if (e != cudaSuccess) return e;
   e = cudaErrorInvalidValue;
   if (p->d.dtype == FBL_DTYPE_FP32) {

@@ -854,8 +854,9 @@ cudaError_t launch_attn_fwd_tc(const fbl_plan* p, const void* Q, const void* K, 
 
 cudaError_t launch_attn_bwd_tc(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* A,
                                const void* dA, const float* lse, float* dvec, float* dqacc, void* dQ, void* dK,
-                               void* dV, int32_t* status, cudaStream_t st) {
-  cudaError_t e = launch_attn_bwd_pre(p, A, dA, dvec, dqacc, st);     // D = rowsum(dO * O); dQ accumulator := 0
+                               void* dV, bool dvec_ready, int32_t* status, cudaStream_t st) {
+  // dQ accumulator := 0, and D = rowsum(dO * O) unless the dA GEMM's epilogue already produced it
+  cudaError_t e = launch_attn_bwd_pre(p, A, dA, dvec, dqacc, dvec_ready, st);
   if (e != cudaSuccess) return e;
   if (p->d.head_dim == 64) e = bwd_launch<64>(p, Q, K, V, dA, lse, dvec, dqacc, dK, dV, status, st);
   else if (p->d.head_dim == 128) e = bwd_launch<128>(p, Q, K, V, dA, lse, dvec, dqacc, dK, dV, status, st);

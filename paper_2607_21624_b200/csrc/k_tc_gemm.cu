@@ -2,7 +2,7 @@
 // R-Tile order fetched by TMA.  One kernel serves all six projection steps and their transposed forms:
 // each operand is declared K-major or MN-major in the descriptors, so W / W^T and X / X^T are the same
 // tiles in HBM and in shared memory.  Up to three reduction loops feed one accumulator (dXn), and up
-// to three problems that share a launch are selected by blockIdx.z (Q/K/V projections, dWq/dWk/dWv).
+// to four problems share one persistent launch (Q/K/V projections; dWo with dA; dWq/dWk/dWv with dXn).
 #include <string.h>
 
 #include <mutex>
@@ -29,6 +29,9 @@ struct alignas(64) TcProblem {
   const float* bias;
   const __nv_bfloat16* residual;
   int seq, t_pad;
+  const __nv_bfloat16* dot_with;   // fused D = rowsum(C * dot_with) per head (the attention backward's D), or nullptr
+  float* dot_out;
+  int dot_hd, dot_hq;
 };
 struct alignas(64) TcGroup {
   TcProblem p[MAX_PROBLEMS];
@@ -207,6 +210,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
       tc::tc_fence_after();
       const int row = tcd.m0 + r;
       const bool pad = P.t_pad > 0 && (row % P.t_pad) >= P.seq;
+      float dot_acc = 0.f;
 #pragma unroll 1
       for (int pn = 0; pn < BN / 64 && ok; ++pn) {
         const int n = tcd.n0 + pn * 64;
@@ -233,6 +237,27 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
           if (P.bias) { v0 += P.bias[n + j]; v1 += P.bias[n + j + 1]; }
           if (pad) { v0 = 0.f; v1 = 0.f; }
           ow[j / 2] = tc::pack_bf16(v0, v1);
+        }
+        if (P.dot_with && row < P.m) {
+          // Row reduction over this head's columns, on the ROUNDED values the attention backward will read:
+          // sum_j dS_ij = 0 (softmax shift invariance) holds only if D matches the dP that kernel forms.
+          const __nv_bfloat16* ap = P.dot_with + ((long long)(n / 64) * P.c_rpad + row) * 64;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint4 av = *reinterpret_cast<const uint4*>(ap + 8 * j);
+            const __nv_bfloat16* ab16 = reinterpret_cast<const __nv_bfloat16*>(&av);
+#pragma unroll
+            for (int k = 0; k < 8; k += 2) {
+              const uint32_t w2 = ow[4 * j + k / 2];        // two bf16: low half = even column
+              dot_acc = fmaf(__uint_as_float(w2 << 16), __bfloat162float(ab16[k]), dot_acc);
+              dot_acc = fmaf(__uint_as_float(w2 & 0xffff0000u), __bfloat162float(ab16[k + 1]), dot_acc);
+            }
+          }
+          if ((n + 64) % P.dot_hd == 0) {                 // last panel of a head
+            const int hh = n / P.dot_hd, bb = row / P.t_pad, tt = row % P.t_pad;
+            P.dot_out[((long long)bb * P.dot_hq + hh) * P.t_pad + tt] = dot_acc;
+            dot_acc = 0.f;
+          }
         }
         const int sb = pc & 1;
         const uint32_t stg = base + SP::STG_OFF + sb * 16384;
@@ -355,6 +380,7 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
     P.c = (__nv_bfloat16*)g.c; P.c_rpad = g.c_rpad;
     P.bias = g.bias; P.residual = (const __nv_bfloat16*)g.residual;
     P.seq = g.seq; P.t_pad = g.t_pad;
+    P.dot_with = (const __nv_bfloat16*)g.dot_with; P.dot_out = g.dot_out; P.dot_hd = g.dot_hd; P.dot_hq = g.dot_hq;
     tiles += ((g.m + BM - 1) / BM) * ((g.n + BN - 1) / BN);
   }
   using SP = SmemPlan<BN, STAGES>;

@@ -185,21 +185,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-// 2^x on the FMA and integer pipes (no transcendental unit): round x to the nearest integer n with the
-// 1.5 * 2^23 trick, evaluate a cubic for 2^f on f = x - n in [-0.5, 0.5] (relative error 7.5e-5, far below the
-// bf16 rounding the result goes through) and add n to the exponent field.  x must be finite; x below -126
-// returns a value below 1.2e-38.  The softmax loops evaluate part of their exponentials this way because
-// the transcendental unit is their busiest resource.
-__device__ __forceinline__ float exp2_poly3(float x) {
-  x = fmaxf(x, -126.f);
-  const float t = x + 12582912.f;
-  const float f = x - (t - 12582912.f);
-  float p = fmaf(0.0551716685f, f, 0.2426111251f);
-  p = fmaf(p, f, 0.6932609677f);
-  p = fmaf(p, f, 0.9999280572f);
-  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
-}
-
 // ---- operand descriptors --------------------------------------------------------------------------
 // Shared-memory matrix descriptor for 128-byte-swizzled tiles whose rows are 128 bytes (64 bf16).
 //   K-major  (reduction axis contiguous): rows are M/N indices, 8-row groups `sbo` bytes apart.
@@ -221,14 +206,6 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
 __host__ __device__ constexpr uint32_t idesc_bf16(int m, int n, int a_mn_major, int b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-}
-
-// Two fp32 -> packed bf16 pair with integer instructions only (round half up on the dropped 16 bits, then one
-// byte permute).  The float-to-bf16 conversion instruction shares the transcendental unit with ex2, which is
-// the busiest unit of the softmax loops; this keeps it free for the exponentials.  Differs from
-// round-to-nearest-even only on exact ties.  Inputs must be finite.
-__device__ __forceinline__ uint32_t pack_bf16_alu(float lo, float hi) {
-  return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
