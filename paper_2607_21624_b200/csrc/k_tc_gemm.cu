@@ -37,16 +37,36 @@ struct alignas(64) TcGroup {
   TcProblem p[MAX_PROBLEMS];
   int count;
   int32_t* status;
+  int trace_slot;
 };
+
+#ifdef FBL_TRACE
+int g_trace_launch = 0;
+#endif
+// Optional timeline probe (compile with -DFBL_TRACE): one block records clock64() at the marked points of its
+// first output tile into the words after the status word; slot = index of the GEMM launch within the pass.
+#ifdef FBL_TRACE
+#ifndef FBL_TRACE_BLOCK
+#define FBL_TRACE_BLOCK 0
+#endif
+__device__ long long g_gemm_trace[2 * 256];
+#define GTR(k) do { if (blockIdx.x == FBL_TRACE_BLOCK) ((long long*)G.status)[8 + G.trace_slot * 24 + (k)] = clock64(); } while (0)
+#define GTK(k) do { if (blockIdx.x == FBL_TRACE_BLOCK && (k) < 256) g_gemm_trace[G.trace_slot * 256 + (k)] = clock64(); } while (0)
+#define GTRG(k) do { if (blockIdx.x == FBL_TRACE_BLOCK) { unsigned long long g_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_)); ((long long*)G.status)[8 + G.trace_slot * 24 + (k)] = (long long)g_; } } while (0)
+#else
+#define GTR(k) do { } while (0)
+#define GTRG(k) do { } while (0)
+#define GTK(k) do { } while (0)
+#endif
 
 template <int BN, int STAGES>
 struct SmemPlan {
   static constexpr uint32_t A_BYTES = BM * 128;
   static constexpr uint32_t B_BYTES = BN * 128;
   static constexpr uint32_t STAGE = A_BYTES + B_BYTES;
-  static constexpr uint32_t STG_OFF = STAGES * STAGE;    // two 128 x 64 bf16 output staging tiles
+  static constexpr uint32_t STG_OFF = STAGES * STAGE;    // per epilogue warp two 32 x 64 bf16 output staging tiles
   static constexpr uint32_t BAR_OFF = STG_OFF + 2 * 16384;
-  static constexpr uint32_t N_BARS = 2 * STAGES + 8;     // full[], empty[], acc_full[2], acc_empty[2], stg_full[2], stg_free[2]
+  static constexpr uint32_t N_BARS = 2 * STAGES + 4;     // full[], empty[], acc_full[2], acc_empty[2]
   static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16 + 1024;   // + TMEM slot + alignment slack
 };
 
@@ -83,14 +103,13 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
   auto empty = [&](int s) { return bars + 8u * (STAGES + s); };
   auto acc_full = [&](int a) { return bars + 8u * (2 * STAGES + a); };
   auto acc_empty = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
-  auto stg_full = [&](int a) { return bars + 8u * (2 * STAGES + 4 + a); };
-  auto stg_free = [&](int a) { return bars + 8u * (2 * STAGES + 6 + a); };
   const uint32_t slot = bars + 8 * SP::N_BARS;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   int32_t* status = G.status;
   constexpr uint32_t TMEM_COLS = 2 * BN;                 // two fp32 accumulators of BN columns
 
   if (threadIdx.x == 0) {
+    GTR(0); GTRG(8);
     for (int s = 0; s < STAGES; ++s) {
       tc::mbar_init(full(s), 1);                 // one producer arrival + transaction bytes
       tc::mbar_init(empty(s), 1);                // one tcgen05.commit arrival
@@ -98,8 +117,6 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
     for (int a = 0; a < 2; ++a) {
       tc::mbar_init(acc_full(a), 1);
       tc::mbar_init(acc_empty(a), 128);
-      tc::mbar_init(stg_full(a), 128);
-      tc::mbar_init(stg_free(a), 1);
     }
     tc::fence_barrier_init();
   }
@@ -113,6 +130,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
   uint32_t tmem_base;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
   pdl_launch_dependents();
+  if (threadIdx.x == 0) GTR(1);
 
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ----------------------------------------------------------------------
@@ -136,6 +154,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
       prefilled = n;
     }
     pdl_wait();
+    GTR(2);
     for (int w = blockIdx.x; ok && tile_at<BN>(G, w, &tcd); w += gridDim.x) {
       const TcProblem& P = G.p[tcd.prob];
       for (int t = 0; t < P.n_terms && ok; ++t) {
@@ -148,96 +167,142 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
             if (!tc::mbar_wait(empty(s), ph ^ 1, status, 101)) { ok = false; break; }
             tc::mbar_expect_tx(full(s), SP::STAGE);
           }
+          if (it < 64) GTK(it);
+#ifdef FBL_NO_LOADS
+          asm volatile("mbarrier.complete_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(full(s)), "r"(pre ? SP::A_BYTES : SP::STAGE) : "memory");
+#else
           if (P.a_mn[t]) tc::tma_load_3d(sa, &P.ta[t], full(s), 0, kb * BK, tcd.m0 / 64);
           else tc::tma_load_3d(sa, &P.ta[t], full(s), 0, tcd.m0, kb);
           if (!pre) {
             if (P.b_mn[t]) tc::tma_load_3d(sb, &P.tb[t], full(s), 0, kb * BK, tcd.n0 / 64);
             else tc::tma_load_3d(sb, &P.tb[t], full(s), 0, tcd.n0, kb);
           }
+#endif
         }
       }
     }
   } else if (warp == 1 && lane == 0) {
-    // ---- MMA issuer ------------------------------------------------------------------------
-    int it = 0, ti = 0;
+    // ---- MMA issuer: one thread.  Descriptor words are formed once per reduction loop; per instruction only
+    // the start-address field moves.  (The loop is not the limit: with 128 x 256 tiles a k-block's 48 KB of
+    // operands take longer to arrive from L2, at about 64 B/clk per SM, than its four MMAs take to run.) ------
+    int s = 0, ti = 0;
+    uint32_t ph = 0;
     bool ok = true;
     TileCoord tcd;
+    const uint32_t hi = tc::smem_desc_hi(1024);
     for (int w = blockIdx.x; ok && tile_at<BN>(G, w, &tcd); w += gridDim.x, ++ti) {
       const TcProblem& P = G.p[tcd.prob];
       const int ab = ti & 1;
       if (!tc::mbar_wait(acc_empty(ab), ((ti >> 1) & 1) ^ 1, status, 104)) { ok = false; break; }
       tc::tc_fence_after();
       const uint32_t d_tmem = tmem_base + ab * BN;
-      bool first = true;
+      uint32_t acc = 0;
       for (int t = 0; t < P.n_terms && ok; ++t) {
         const uint32_t idesc = tc::idesc_bf16(BM, BN, P.a_mn[t], P.b_mn[t]);
         // K-major: 8-row groups 1024 B apart, 16 K elements = 32 B along the row.
         // MN-major: 64-wide M/N blocks 8 KiB apart (64 K rows x 128 B), 16 K rows = 2 KiB.
-        const uint32_t a_lbo = P.a_mn[t] ? 8192u : 16u, a_step = P.a_mn[t] ? 2048u : 32u;
-        const uint32_t b_lbo = P.b_mn[t] ? 8192u : 16u, b_step = P.b_mn[t] ? 2048u : 32u;
-        for (int kb = 0; kb < P.kblocks[t]; ++kb, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
+        const uint32_t a_lo0 = tc::smem_desc_lo(base, P.a_mn[t] ? 8192u : 16u), a_step = P.a_mn[t] ? 128u : 2u;
+        const uint32_t b_lo0 = tc::smem_desc_lo(base + SP::A_BYTES, P.b_mn[t] ? 8192u : 16u), b_step = P.b_mn[t] ? 128u : 2u;
+        const int nkb = P.kblocks[t];
+        for (int kb = 0; kb < nkb; ++kb) {
           if (!tc::mbar_wait(full(s), ph, status, 102)) { ok = false; break; }
+          if (ti == 0 && t == 0 && kb == 0) GTR(3);
           tc::tc_fence_after();
-          const uint32_t sa = base + s * SP::STAGE, sb = sa + SP::A_BYTES;
+          uint32_t a_lo = a_lo0 + (uint32_t)s * (SP::STAGE >> 4), b_lo = b_lo0 + (uint32_t)s * (SP::STAGE >> 4);
 #pragma unroll
           for (int kk = 0; kk < BK / 16; ++kk) {
-            const uint64_t da = tc::smem_desc_sw128(sa + kk * a_step, a_lbo, 1024);
-            const uint64_t db = tc::smem_desc_sw128(sb + kk * b_step, b_lbo, 1024);
-            tc::mma_bf16_ss(d_tmem, da, db, idesc, (first && kk == 0) ? 0u : 1u);
+            tc::mma_bf16_ss_w(d_tmem, a_lo, hi, b_lo, hi, idesc, acc);
+            acc = 1;
+            a_lo += a_step; b_lo += b_step;
           }
-          first = false;
           tc::mma_commit(empty(s));              // frees the stage once these MMAs have read it
+          if (++s == STAGES) { s = 0; ph ^= 1; }
         }
       }
       if (ok) tc::mma_commit(acc_full(ab));
+      if (ti == 0) GTR(4);
     }
   } else if (warp >= 2) {
-    // ---- epilogue: TMEM -> registers -> swizzled staging tile -> bulk tensor store, one 64-column panel at
-    // a time (two staging tiles: the store of one panel overlaps the conversion of the next) -------------
+    // ---- epilogue: TMEM -> registers -> swizzled staging -> bulk tensor store.  Each warp owns the 32 rows of
+    // its TMEM lane quarter and two 32 x 64 staging tiles, and issues its own stores: no block-wide hand-off per
+    // panel, and the store of one panel overlaps the conversion of the next. ---------------------------------
     pdl_wait();                                       // the previous kernel may still be reading what we overwrite
     const int q = warp % 4;                           // the TMEM lane quarter this warp may access
     const int r = q * 32 + lane;                      // row of the tile owned by this thread
-    const bool issuer = threadIdx.x == 64;
-    int ti = 0, pc = 0;                               // tiles and panels done by this block
+    const bool tracer = threadIdx.x == 64;
+    int ti = 0, pc = 0;                               // tiles and panels done by this warp
     bool ok = true;
     TileCoord tcd;
     for (int w = blockIdx.x; ok && tile_at<BN>(G, w, &tcd); w += gridDim.x, ++ti) {
       const TcProblem& P = G.p[tcd.prob];
       const int ab = ti & 1;
-      if (!tc::mbar_wait(acc_full(ab), (ti >> 1) & 1, status, 103)) { ok = false; break; }
-      tc::tc_fence_after();
       const int row = tcd.m0 + r;
       const bool pad = P.t_pad > 0 && (row % P.t_pad) >= P.seq;
+      const bool has_res = P.residual && row < P.m;
+      uint4 rv[8];                                    // residual values of the next panel, requested a panel ahead
+      if (has_res) {
+        const __nv_bfloat16* rp = P.residual + ((long long)(tcd.n0 / 64) * P.c_rpad + row) * 64;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) rv[j] = *reinterpret_cast<const uint4*>(rp + 8 * j);
+      }
+      const float* bias = P.bias;
+      float bl[BN / 32];                              // this tile's bias: lane l holds columns l*BN/32 ... (requested
+      if (bias) {                                     // while the MMAs run, handed out by shuffles below)
+#pragma unroll
+        for (int k = 0; k < BN / 32; ++k) {
+          const int c = tcd.n0 + lane * (BN / 32) + k;
+          bl[k] = c < P.n ? bias[c] : 0.f;
+        }
+      }
+      if (!tc::mbar_wait(acc_full(ab), (ti >> 1) & 1, status, 103)) { ok = false; break; }
+      tc::tc_fence_after();
+      if (tracer && ti == 0) GTR(5);
       float dot_acc = 0.f;
 #pragma unroll 1
-      for (int pn = 0; pn < BN / 64 && ok; ++pn) {
+      for (int pn = 0; pn < BN / 64; ++pn) {
         const int n = tcd.n0 + pn * 64;
         if (n >= P.n) break;                           // uniform: N is whole 64-column panels
         uint32_t v[64];
         tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + pn * 64, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
         tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + pn * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
         tc::tmem_ld_wait();
+        if (tracer && ti == 0 && pn < 2) GTR(10 + 2 * pn);
         uint4 outv[8];
         uint32_t* ow = reinterpret_cast<uint32_t*>(outv);
-        if (P.residual && row < P.m) {
-          const __nv_bfloat16* rp = P.residual + ((long long)(n / 64) * P.c_rpad + row) * 64;
+#ifdef FBL_TRACE
+        asm volatile("" ::"r"(v[0]), "r"(v[31]), "r"(v[32]), "r"(v[63]));
+        if (tracer && ti == 0 && pn == 1) GTR(18);
+#endif
+        if (has_res) {
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            const uint4 rv = *reinterpret_cast<const uint4*>(rp + 8 * j);
-            const __nv_bfloat16* rb = reinterpret_cast<const __nv_bfloat16*>(&rv);
+            const __nv_bfloat16* rb = reinterpret_cast<const __nv_bfloat16*>(&rv[j]);
 #pragma unroll
             for (int k = 0; k < 8; ++k) v[8 * j + k] = __float_as_uint(__uint_as_float(v[8 * j + k]) + __bfloat162float(rb[k]));
           }
-        }
+          if (pn + 1 < BN / 64 && n + 64 < P.n) {
+            const __nv_bfloat16* rp = P.residual + ((long long)(n / 64 + 1) * P.c_rpad + row) * 64;
 #pragma unroll
-        for (int j = 0; j < 64; j += 2) {
-          float v0 = __uint_as_float(v[j]), v1 = __uint_as_float(v[j + 1]);
-          if (P.bias) { v0 += P.bias[n + j]; v1 += P.bias[n + j + 1]; }
-          if (pad) { v0 = 0.f; v1 = 0.f; }
-          ow[j / 2] = tc::pack_bf16(v0, v1);
+            for (int j = 0; j < 8; ++j) rv[j] = *reinterpret_cast<const uint4*>(rp + 8 * j);
+          }
         }
+        if (bias) {
+#pragma unroll
+          for (int j = 0; j < 64; j += 2) {
+            // column pn*64 + j is register (j % (BN/32)) of lane (pn*64 + j) / (BN/32)
+            const float b0 = __shfl_sync(0xffffffffu, bl[j % (BN / 32)], (pn * 64 + j) / (BN / 32));
+            const float b1 = __shfl_sync(0xffffffffu, bl[(j + 1) % (BN / 32)], (pn * 64 + j + 1) / (BN / 32));
+            ow[j / 2] = tc::pack_bf16(pad ? 0.f : __uint_as_float(v[j]) + b0, pad ? 0.f : __uint_as_float(v[j + 1]) + b1);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 64; j += 2)
+            ow[j / 2] = tc::pack_bf16(pad ? 0.f : __uint_as_float(v[j]), pad ? 0.f : __uint_as_float(v[j + 1]));
+        }
+#ifdef FBL_TRACE
+        asm volatile("" ::"r"(ow[0]), "r"(ow[15]), "r"(ow[16]), "r"(ow[31]));
+        if (tracer && ti == 0 && pn == 1) GTR(19);
+#endif
         if (P.dot_with && row < P.m) {
           // Row reduction over this head's columns, on the ROUNDED values the attention backward will read:
           // sum_j dS_ij = 0 (softmax shift invariance) holds only if D matches the dP that kernel forms.
@@ -259,31 +324,35 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
             dot_acc = 0.f;
           }
         }
-        const int sb = pc & 1;
-        const uint32_t stg = base + SP::STG_OFF + sb * 16384;
-        // the staging tile's previous store (two panels ago) must have read it
-        if (pc >= 2 && !tc::mbar_wait(stg_free(sb), ((pc >> 1) - 1) & 1, status, 105)) { ok = false; break; }
+        // Staging tile (pc & 1) of this warp: its previous store (two panels ago) has been read, since lane 0
+        // waited for that after committing the store of the panel before this one.
+        const uint32_t stg = base + SP::STG_OFF + (uint32_t)(q * 2 + (pc & 1)) * 4096u;
+        if (tracer && ti == 0 && pn == 1) GTR(13);
+        __syncwarp();
+        if (tracer && ti == 0 && pn == 1) GTR(14);
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + r * 128 + (((uint32_t)j ^ (uint32_t)(r & 7)) * 16)),
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + (((uint32_t)j ^ (uint32_t)(lane & 7)) * 16)),
                        "r"(outv[j].x), "r"(outv[j].y), "r"(outv[j].z), "r"(outv[j].w) : "memory");
+        if (tracer && ti == 0 && pn == 1) GTR(15);
         tc::fence_proxy_async();
-        tc::mbar_arrive(stg_full(sb));
-        if (issuer) {
-          if (!tc::mbar_wait(stg_full(sb), (pc >> 1) & 1, status, 106)) { ok = false; break; }
-          tc::tma_store_3d(&P.tc, stg, 0, tcd.m0, n / 64);
+        if (tracer && ti == 0 && pn == 1) GTR(16);
+        __syncwarp();
+        if (tracer && ti == 0 && pn == 1) GTR(17);
+        if (lane == 0) {
+          tc::tma_store_3d(&P.tc, stg, 0, tcd.m0 + q * 32, n / 64);
           tc::bulk_commit_group();
-          if (pc >= 1) {                               // at most this store in flight: the previous one has read
-            tc::bulk_wait_group_read1();               // its staging tile, which may now be overwritten
-            tc::mbar_arrive(stg_free(sb ^ 1));
-          }
+          tc::bulk_wait_group_read1();                 // the store before this one has read its staging tile
         }
+        if (tracer && ti == 0 && pn < 1) GTR(11 + 2 * pn);
         ++pc;
       }
+      if (tracer && ti == 0) GTR(6);
       tc::tc_fence_before();
       tc::mbar_arrive(acc_empty(ab));             // this accumulator may be overwritten by the tile after next
     }
-    if (issuer) tc::bulk_wait_group0();           // all output tiles are in global memory before the block exits
+    if (lane == 0) tc::bulk_wait_group0();        // all output tiles are in global memory before the block exits
+    if (tracer) { GTR(7); GTRG(9); }
   }
   tc::tc_fence_before();
   __syncthreads();
@@ -337,6 +406,12 @@ bool fbl_encode_f32_panel_map(CUtensorMap* map, const void* base, int64_t r_pad,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+#ifdef FBL_TRACE
+extern "C" int fbl_debug_gemm_trace(long long* host_dst) {
+  return (int)cudaMemcpyFromSymbol(host_dst, g_gemm_trace, sizeof(long long) * 512);
+}
+#endif
+
 bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g) {
   if (p->d.dtype != FBL_DTYPE_BF16) return false;
   if (g.n % 64 != 0 || g.n < BN_SMALL || g.m < BM) return false;
@@ -356,6 +431,9 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
   memset(&G, 0, sizeof(G));
   G.count = count;
   G.status = status;
+#ifdef FBL_TRACE
+  G.trace_slot = (g_trace_launch++) & 1;      // two GEMM launches per pass
+#endif
   int tiles = 0;
   for (int i = 0; i < count; ++i) {
     const GemmArgs& g = gs[i];
@@ -375,7 +453,7 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
       if (!ok) return cudaErrorInvalidValue;
     }
     P.m = g.m; P.n = g.n;
-    if (!fbl_encode_rtile_map(&P.tc, g.c, g.c_rpad, g.n / 64, BM, 1)) return cudaErrorInvalidValue;
+    if (!fbl_encode_rtile_map(&P.tc, g.c, g.c_rpad, g.n / 64, 32, 1)) return cudaErrorInvalidValue;   // one warp's rows
     P.b_static = g.b_static;
     P.c = (__nv_bfloat16*)g.c; P.c_rpad = g.c_rpad;
     P.bias = g.bias; P.residual = (const __nv_bfloat16*)g.residual;
