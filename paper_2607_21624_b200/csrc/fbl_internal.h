@@ -89,7 +89,8 @@ cudaError_t launch_pack(int dtype, int unpack, const void* src, void* dst, int64
 cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
                             float* stats, cudaStream_t st);
 cudaError_t launch_norm_bwd(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
-                            const float* gamma, void* dX, float* dgamma, float* dbeta, cudaStream_t st);
+                            const float* gamma, void* dX, float* dgamma, float* dbeta, float* part,
+                            cudaStream_t st);
 cudaError_t launch_colsum(int dtype, const void* M, int64_t rows, int64_t cols, float* out, float* partials,
                           cudaStream_t st);
 size_t colsum_scratch_bytes(int64_t rows, int64_t cols);

@@ -285,8 +285,8 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
                                                             const __nv_bfloat16* __restrict__ dY,
                                                             const float* __restrict__ stats,
                                                             const float* __restrict__ gamma,
-                                                            __nv_bfloat16* __restrict__ dX, float* __restrict__ dgamma,
-                                                            float* __restrict__ dbeta, int64_t n_pad, int rms) {
+                                                            __nv_bfloat16* __restrict__ dX, float* __restrict__ partials,
+                                                            int64_t n_pad, int rms) {
   constexpr int D = NV * 256 * WPR;
   constexpr int RPB = 8 / WPR;
   __shared__ float s_dg[D];
@@ -295,10 +295,9 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
   for (int i = threadIdx.x; i < D; i += 256) { s_dg[i] = 0.f; s_db[i] = 0.f; }
   __syncthreads();
   pdl_launch_dependents();
-  pdl_wait();
   const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
   const int slot = wib / WPR, part = wib % WPR;
-  float gm[NV][8];
+  float gm[NV][8];                           // gamma is an input of the step: read before waiting for the GEMM
 #pragma unroll
   for (int j = 0; j < NV; ++j) {
     const int c0 = ((part * NV + j) * 32 + lane) * 8;
@@ -306,6 +305,7 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
     gm[j][0] = g0.x; gm[j][1] = g0.y; gm[j][2] = g0.z; gm[j][3] = g0.w;
     gm[j][4] = g1.x; gm[j][5] = g1.y; gm[j][6] = g1.z; gm[j][7] = g1.w;
   }
+  pdl_wait();
   // token-axis partial sums of this warp's rows, kept in registers and folded into shared memory at the end
   float ag[NV][8], ab[NV][8];
 #pragma unroll
@@ -316,6 +316,14 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
     const float mean = stats[2 * r], rstd = stats[2 * r + 1];
     float xh[NV][8], g[NV][8];
     float s1 = 0.f, s2 = 0.f;
+    uint4 yraw[NV];                          // the residual's gradient, requested together with the other two rows
+    if (dY) {
+#pragma unroll
+      for (int j = 0; j < NV; ++j) {
+        const int v = (part * NV + j) * 32 + lane;
+        yraw[j] = *reinterpret_cast<const uint4*>(dY + ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8);
+      }
+    }
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
       const int v = (part * NV + j) * 32 + lane;
@@ -340,27 +348,63 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
       const int v = (part * NV + j) * 32 + lane;
       const int64_t off = ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8;
       float o[8];
-      if (dY) load16(dY + off, o);
+      const __nv_bfloat16* ye = reinterpret_cast<const __nv_bfloat16*>(&yraw[j]);
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const float dx = rstd * (g[j][i] - s1 - xh[j][i] * s2);
-        o[i] = dY ? o[i] + dx : dx;
+        o[i] = dY ? __bfloat162float(ye[i]) + dx : dx;
       }
       store16(dX + off, o);
     }
   }
+  // Fold the warps' sums in shared memory.  Slot (k, lane) with k = (part*NV + j)*8 + i holds column
+  // ((part*NV + j)*32 + lane)*8 + i: consecutive lanes hit consecutive banks.
 #pragma unroll
   for (int j = 0; j < NV; ++j)
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const int c = ((part * NV + j) * 32 + lane) * 8 + i;
-      atomicAdd(&s_dg[c], ag[j][i]);
-      atomicAdd(&s_db[c], ab[j][i]);
+      const int k = ((part * NV + j) * 8 + i) * 32 + lane;
+      atomicAdd(&s_dg[k], ag[j][i]);
+      if (!rms) atomicAdd(&s_db[k], ab[j][i]);
     }
   __syncthreads();
-  for (int i = threadIdx.x; i < D; i += 256) {
-    atomicAdd(&dgamma[i], s_dg[i]);
-    if (dbeta) atomicAdd(&dbeta[i], s_db[i]);
+  // this block's token-axis partial sums: row blockIdx.x of partials[blocks][2][D]; a second kernel adds the rows
+  float* mine = partials + (int64_t)blockIdx.x * 2 * D;
+  for (int c = threadIdx.x; c < D; c += 256) {
+    const int k = ((c / 256) * 8 + c % 8) * 32 + (c / 8) % 32;
+    mine[c] = s_dg[k];
+    if (!rms) mine[D + c] = s_db[k];
+  }
+}
+
+// dgamma[c] (y = 0) or dbeta[c] (y = 1) = sum over the first kernel's blocks of their partial rows.
+__global__ void __launch_bounds__(256) norm_bwd_reduce_kernel(const float* __restrict__ part, int blocks, int d,
+                                                              float* __restrict__ dgamma, float* __restrict__ dbeta) {
+  __shared__ float red[8][33];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
+  const int c = blockIdx.x * 32 + tx;
+  float s = 0.f;
+  if (c < d) {
+    const float* col = part + (int64_t)blockIdx.y * d + c;
+    const int64_t stride = 2 * (int64_t)d;
+    int b = ty;
+    for (; b + 56 < blocks; b += 64) {          // eight independent loads in flight per thread
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = col[(b + 8 * u) * stride];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) s += v[u];
+    }
+    for (; b < blocks; b += 8) s += col[b * stride];
+  }
+  red[ty][tx] = s;
+  __syncthreads();
+  if (ty == 0 && c < d) {
+#pragma unroll
+    for (int k = 1; k < 8; ++k) s += red[k][tx];
+    (blockIdx.y == 0 ? dgamma : dbeta)[c] = s;
   }
 }
 
@@ -373,11 +417,13 @@ void norm_fwd_rows_launch(const fbl_plan* p, const void* X, const float* gamma, 
 }
 template <int NV, int WPR>
 void norm_bwd_rows_launch(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
-                          const float* gamma, void* dX, float* dgamma, float* dbeta, int rms, cudaStream_t st) {
+                          const float* gamma, void* dX, float* dgamma, float* dbeta, float* part, int rms,
+                          cudaStream_t st) {
   const int blocks = (int)min((int64_t)p->sm_count * 2, p->n_pad / (8 / WPR));
   launch_pdl(norm_bwd_rows_kernel<NV, WPR>, dim3(blocks), dim3(256), 0, st, (const __nv_bfloat16*)dXn,
-             (const __nv_bfloat16*)X, (const __nv_bfloat16*)dY, stats, gamma, (__nv_bfloat16*)dX, dgamma,
-             rms ? (float*)nullptr : dbeta, p->n_pad, rms);
+             (const __nv_bfloat16*)X, (const __nv_bfloat16*)dY, stats, gamma, (__nv_bfloat16*)dX, part, p->n_pad, rms);
+  launch_pdl(norm_bwd_reduce_kernel, dim3((p->d.d_model + 31) / 32, rms ? 1 : 2), dim3(256), 0, st, (const float*)part,
+             blocks, p->d.d_model, dgamma, dbeta);
 }
 
 // d_model -> (vectors per lane, warps per row) of the register-resident kernels; false if there is none
@@ -435,6 +481,7 @@ __global__ void __launch_bounds__(256) colsum_stage1(ColsumGroup G, int64_t rows
 #pragma unroll
   for (int i = 0; i < V; ++i) acc[i] = 0.f;
   const int64_t r_end = min((int64_t)(slab + 1) * COLSUM_SLAB, rows);
+#pragma unroll 8                              // a slab is eight 32-row steps: all their loads in flight together
   for (int64_t r = (int64_t)slab * COLSUM_SLAB + rr; r < r_end; r += 32) {
     float v[V];
     load16(M + ((int64_t)p * rows + r) * TW + l8 * V, v);
@@ -461,6 +508,7 @@ __global__ void colsum_stage2(ColsumGroup G, const float* __restrict__ part_base
   if (c >= cols) return;
   const float* part = part_base + G.part_off[which];
   float s = 0.f;
+#pragma unroll 8
   for (int k = 0; k < n_slabs; ++k) s += part[(int64_t)k * cols + c];
   G.out[which][c] = s;
 }
@@ -505,23 +553,25 @@ cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma
 }
 
 cudaError_t launch_norm_bwd(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
-                            const float* gamma, void* dX, float* dgamma, float* dbeta, cudaStream_t st) {
+                            const float* gamma, void* dX, float* dgamma, float* dbeta, float* part,
+                            cudaStream_t st) {
   const int blocks = (int)((p->n_pad + 31) / 32);
   const int d = p->d.d_model;
   const int rms = p->d.norm == FBL_NORM_RMSNORM;
   const size_t sh = 2 * (size_t)d * sizeof(float);
+  int nv, wpr;
+  if (p->d.dtype == FBL_DTYPE_BF16 && norm_rows_shape(d, &nv, &wpr)) {
+    // token-axis sums in two steps over `part` (no atomics: the result does not depend on block order)
+#define FBL_CALL(NV_, WPR_) norm_bwd_rows_launch<NV_, WPR_>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, part, rms, st)
+    FBL_NORM_DISPATCH(FBL_CALL);
+#undef FBL_CALL
+    return cudaGetLastError();
+  }
   cudaError_t e = cudaMemsetAsync(dgamma, 0, d * sizeof(float), st);
   if (e != cudaSuccess) return e;
   if (dbeta) {
     e = cudaMemsetAsync(dbeta, 0, d * sizeof(float), st);
     if (e != cudaSuccess) return e;
-  }
-  int nv, wpr;
-  if (p->d.dtype == FBL_DTYPE_BF16 && norm_rows_shape(d, &nv, &wpr)) {
-#define FBL_CALL(NV_, WPR_) norm_bwd_rows_launch<NV_, WPR_>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, rms, st)
-    FBL_NORM_DISPATCH(FBL_CALL);
-#undef FBL_CALL
-    return cudaGetLastError();
   }
   if (p->d.dtype == FBL_DTYPE_FP32) {
     auto k = norm_bwd_kernel<float>;
