@@ -167,23 +167,26 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __gri
     // S(j+1) is issued after PV(j), which reads P(j) (the tensor pipe executes in issue order).
     const uint32_t idesc_s = tc::idesc_bf16(BQ, BKV, 0, 0);          // Q K-major, K K-major
     const uint32_t idesc_o = tc::idesc_bf16(BQ, HD, 0, 1);           // P from TMEM, V MN-major (rows are keys)
+    // Descriptor words are formed once; per instruction only the start-address field of the low word moves.
+    const uint32_t hi = tc::smem_desc_hi(1024);
+    const uint32_t q_lo = tc::smem_desc_lo(base + SM::Q_OFF, 16), k_lo = tc::smem_desc_lo(base + SM::K_OFF, 16);
+    const uint32_t v_lo = tc::smem_desc_lo(base + SM::V_OFF, 16384);
     auto issue_s = [&](int w, int j) {
-      const uint32_t qsm = base + SM::Q_OFF + w * SM::TILE, ksm = base + SM::K_OFF + (j & 1) * SM::TILE;
+      const uint32_t ql = q_lo + w * (SM::TILE >> 4), kl = k_lo + (j & 1) * (SM::TILE >> 4);
 #pragma unroll
       for (uint32_t kk = 0; kk < HD / 16; ++kk) {
-        const uint32_t o = (kk / 4) * 16384 + (kk % 4) * 32;
-        tc::mma_bf16_ss(tmem_base + w * 128, tc::smem_desc_sw128(qsm + o, 16, 1024),
-                        tc::smem_desc_sw128(ksm + o, 16, 1024), idesc_s, kk > 0);
+        const uint32_t o = (kk / 4) * 1024 + (kk % 4) * 2;            // 16-byte units: 64-column panel, 16-element step
+        tc::mma_bf16_ss_w(tmem_base + w * 128, ql + o, hi, kl + o, hi, idesc_s, kk > 0);
       }
       tc::mma_commit(bar(B_SFULL + w));
     };
     auto issue_pv = [&](int w, int j) {
-      const uint32_t vsm = base + SM::V_OFF + (j & 1) * SM::TILE;
+      const uint32_t vl = v_lo + (j & 1) * (SM::TILE >> 4);
 #pragma unroll
       for (uint32_t kk = 0; kk < BKV / 16; ++kk) {
         // A operand from tensor memory: the packed bf16 P row of each lane, 16 keys = 8 columns per step
-        tc::mma_bf16_ts(tmem_base + O_COL + w * HD, tmem_base + w * 128 + kk * 8,
-                        tc::smem_desc_sw128(vsm + kk * 2048, 16384, 1024), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+        tc::mma_bf16_ts_w(tmem_base + O_COL + w * HD, tmem_base + w * 128 + kk * 8, vl + kk * 128, hi, idesc_o,
+                          (j > 0 || kk > 0) ? 1u : 0u);
       }
       tc::mma_commit(bar(B_PVDONE + w));
     };
@@ -235,26 +238,25 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __gri
       { const int it = j; if (r == 0) TR(9 + 8 * w); }
       tc::tc_fence_after();
       const bool need_mask = (j0 + BKV > P.seq) || (P.causal && j0 + BKV - 1 > i0);
-      // pass 1 over the 128 scores of this row (four 32-column loads): the row maximum
-      auto mask_chunk = [&](float* s, int cc) {
+      // The row's 128 scores come into registers with one wait (one block per SM: a thread may hold them all):
+      // the maximum, the exponentials and the packing then run without touching tensor memory again until
+      // the packed P row is stored over the score columns.
+      uint32_t sr[128];
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
-          const int gj = j0 + cc * 32 + k;
-          if (gj >= P.seq || (P.causal && gj > gi)) s[k] = -INFINITY;
+      for (int cc = 0; cc < 4; ++cc) tc::tmem_ld32(s_addr + cc * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[cc * 32]));
+      tc::tmem_ld_wait();
+      float* sv = reinterpret_cast<float*>(sr);
+      if (need_mask) {
+#pragma unroll
+        for (int k = 0; k < 128; ++k) {
+          const int gj = j0 + k;
+          if (gj >= P.seq || (P.causal && gj > gi)) sv[k] = -INFINITY;
         }
-      };
+      }
       float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t sr[32];
-        tc::tmem_ld32(s_addr + cc * 32, sr);
-        tc::tmem_ld_wait();
-        float* s = reinterpret_cast<float*>(sr);
-        if (need_mask) mask_chunk(s, cc);
 #pragma unroll
-        for (int k = 0; k < 32; k += 4) {
-          mx0 = fmaxf(mx0, s[k]); mx1 = fmaxf(mx1, s[k + 1]); mx2 = fmaxf(mx2, s[k + 2]); mx3 = fmaxf(mx3, s[k + 3]);
-        }
+      for (int k = 0; k < 128; k += 4) {
+        mx0 = fmaxf(mx0, sv[k]); mx1 = fmaxf(mx1, sv[k + 1]); mx2 = fmaxf(mx2, sv[k + 2]); mx3 = fmaxf(mx3, sv[k + 3]);
       }
       const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
       { const int it = j; if (r == 0) TR(10 + 8 * w); }
@@ -280,27 +282,18 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __gri
         }
       }
       { const int it = j; if (r == 0) TR(11 + 8 * w); }
-      // pass 2: P = exp2(S c - m c), its row sum, and P packed to bf16 over the score columns already consumed
-      // (32 scores become 16 packed columns; the thread owns the lane, so nobody else's data is overwritten)
+      // P = exp2(S c - m c), its row sum, and P packed to bf16 (128 scores become 64 packed columns)
       float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-#pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t sr[32];
-        tc::tmem_ld32(s_addr + cc * 32, sr);
-        tc::tmem_ld_wait();
-        float* s = reinterpret_cast<float*>(sr);
-        if (need_mask) mask_chunk(s, cc);
-        uint32_t pk[16];
 #pragma unroll
-        for (int k = 0; k < 32; k += 4) {
-          const float p0 = tc::fast_exp2(fmaf(s[k], c, -mc)), p1 = tc::fast_exp2(fmaf(s[k + 1], c, -mc));
-          const float p2 = tc::fast_exp2(fmaf(s[k + 2], c, -mc)), p3 = tc::fast_exp2(fmaf(s[k + 3], c, -mc));
-          sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
-          pk[k / 2] = tc::pack_bf16(p0, p1);
-          pk[k / 2 + 1] = tc::pack_bf16(p2, p3);
-        }
-        tc::tmem_st16(s_addr + cc * 16, pk);
+      for (int k = 0; k < 128; k += 4) {
+        const float p0 = tc::fast_exp2(fmaf(sv[k], c, -mc)), p1 = tc::fast_exp2(fmaf(sv[k + 1], c, -mc));
+        const float p2 = tc::fast_exp2(fmaf(sv[k + 2], c, -mc)), p3 = tc::fast_exp2(fmaf(sv[k + 3], c, -mc));
+        sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+        sr[k / 2] = tc::pack_bf16(p0, p1);
+        sr[k / 2 + 1] = tc::pack_bf16(p2, p3);
       }
+      tc::tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+      tc::tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
       if (moved) l *= alpha;
       l += (sum0 + sum1) + (sum2 + sum3);
       tc::tmem_st_wait();
@@ -494,53 +487,53 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     const uint32_t idesc_s = tc::idesc_bf16(BKV, BQ, 0, 0);
     const uint32_t idesc_kv = tc::idesc_bf16(BKV, HD, 0, 1);
     const uint32_t idesc_dq = tc::idesc_bf16(BQ, HD, 1, 1);
+    // Descriptor words are formed once; per instruction only the start-address field of the low word moves
+    // (offsets below are in 16-byte units: a 64-column panel is 1024, a 16-element step along a row 2, 16 rows 128).
+    const uint32_t hi = tc::smem_desc_hi(1024);
+    const uint32_t k_km = tc::smem_desc_lo(base + SM::K_OFF, 16), k_mn = tc::smem_desc_lo(base + SM::K_OFF, 16384);
+    const uint32_t v_km = tc::smem_desc_lo(base + SM::V_OFF, 16);
+    const uint32_t q_km = tc::smem_desc_lo(base + SM::Q_OFF, 16), q_mn = tc::smem_desc_lo(base + SM::Q_OFF, 16384);
+    const uint32_t do_km = tc::smem_desc_lo(base + SM::DO_OFF, 16), do_mn = tc::smem_desc_lo(base + SM::DO_OFF, 16384);
+    const uint32_t ds_km = tc::smem_desc_lo(base + SM::DS_OFF, 16), ds_mn = tc::smem_desc_lo(base + SM::DS_OFF, 16384);
     auto issue_s = [&](int it) {              // S^T = K Q^T of tile `it`
-      const uint32_t qs = base + SM::Q_OFF + (it % NQ) * SM::TILE;
+      const uint32_t qs = q_km + (it % NQ) * (SM::TILE >> 4);
 #pragma unroll
       for (uint32_t kk = 0; kk < HD / 16; ++kk) {
-        const uint32_t o = (kk / 4) * 16384 + (kk % 4) * 32;
-        tc::mma_bf16_ss(tmem_base + S_COL, tc::smem_desc_sw128(base + SM::K_OFF + o, 16, 1024),
-                        tc::smem_desc_sw128(qs + o, 16, 1024), idesc_s, kk > 0);
+        const uint32_t o = (kk / 4) * 1024 + (kk % 4) * 2;
+        tc::mma_bf16_ss_w(tmem_base + S_COL, k_km + o, hi, qs + o, hi, idesc_s, kk > 0);
       }
     };
     auto issue_dp = [&](int it) {             // dP^T = V dO^T of tile `it`; then both score tiles are announced
-      const uint32_t dos = base + SM::DO_OFF + (it % NQ) * SM::TILE;
+      const uint32_t dos = do_km + (it % NQ) * (SM::TILE >> 4);
 #pragma unroll
       for (uint32_t kk = 0; kk < HD / 16; ++kk) {
-        const uint32_t o = (kk / 4) * 16384 + (kk % 4) * 32;
-        tc::mma_bf16_ss(tmem_base + DP_COL, tc::smem_desc_sw128(base + SM::V_OFF + o, 16, 1024),
-                        tc::smem_desc_sw128(dos + o, 16, 1024), idesc_s, kk > 0);
+        const uint32_t o = (kk / 4) * 1024 + (kk % 4) * 2;
+        tc::mma_bf16_ss_w(tmem_base + DP_COL, v_km + o, hi, dos + o, hi, idesc_s, kk > 0);
       }
       tc::mma_commit(bar(BB_SFULL));
     };
     auto issue_dv = [&](int it) {             // dV += P^T dO, P^T read from tensor memory
-      const uint32_t dos = base + SM::DO_OFF + (it % NQ) * SM::TILE;
+      const uint32_t dos = do_mn + (it % NQ) * (SM::TILE >> 4);
 #pragma unroll
-      for (uint32_t kk = 0; kk < BQ / 16; ++kk) {
-        const uint32_t bo = kk * 2048;                             // dO: MN-major, 16 query rows per step
-        tc::mma_bf16_ts(tmem_base + DV_COL, tmem_base + P_COL + kk * 8,   // 16 queries = 8 packed columns
-                        tc::smem_desc_sw128(dos + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
-      }
+      for (uint32_t kk = 0; kk < BQ / 16; ++kk)                      // dO: MN-major, 16 query rows per step;
+        tc::mma_bf16_ts_w(tmem_base + DV_COL, tmem_base + P_COL + kk * 8,   // 16 queries = 8 packed columns
+                          dos + kk * 128, hi, idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
     };
     auto issue_dk = [&](int it) {             // dK += dS^T Q
-      const uint32_t qs = base + SM::Q_OFF + (it % NQ) * SM::TILE;
-      const uint32_t dss = base + SM::DS_OFF + (it % NP) * 32768;
+      const uint32_t qs = q_mn + (it % NQ) * (SM::TILE >> 4);
+      const uint32_t dss = ds_km + (it % NP) * 2048;
 #pragma unroll
       for (uint32_t kk = 0; kk < BQ / 16; ++kk) {
-        const uint32_t ao = (kk / 4) * 16384 + (kk % 4) * 32;      // dS^T: K-major, reduction over queries
-        const uint32_t bo = kk * 2048;                             // Q: MN-major, 16 query rows per step
-        tc::mma_bf16_ss(tmem_base + DK_COL, tc::smem_desc_sw128(dss + ao, 16, 1024),
-                        tc::smem_desc_sw128(qs + bo, 16384, 1024), idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
+        const uint32_t ao = (kk / 4) * 1024 + (kk % 4) * 2;        // dS^T: K-major, reduction over queries
+        tc::mma_bf16_ss_w(tmem_base + DK_COL, dss + ao, hi, qs + kk * 128, hi, idesc_kv,   // Q: MN-major, 16 query rows
+                          (it > 0 || kk > 0) ? 1u : 0u);
       }
     };
     auto issue_dq = [&](int it) {             // dQ = dS K: the dS^T tile read MN-major, i.e. transposed by descriptor
-      const uint32_t dss = base + SM::DS_OFF + (it % NP) * 32768;
+      const uint32_t dss = ds_mn + (it % NP) * 2048;
 #pragma unroll
-      for (uint32_t kk = 0; kk < BKV / 16; ++kk) {
-        const uint32_t o = kk * 2048;                              // both operands MN-major: 16 key rows per step
-        tc::mma_bf16_ss(tmem_base + DQ_COL, tc::smem_desc_sw128(dss + o, 16384, 1024),
-                        tc::smem_desc_sw128(base + SM::K_OFF + o, 16384, 1024), idesc_dq, kk > 0);
-      }
+      for (uint32_t kk = 0; kk < BKV / 16; ++kk)                     // both operands MN-major: 16 key rows per step
+        tc::mma_bf16_ss_w(tmem_base + DQ_COL, dss + kk * 128, hi, k_mn + kk * 128, hi, idesc_dq, kk > 0);
       tc::mma_commit(bar(BB_DQFULL));
     };
     bool ok = tc::mbar_wait(bar(BB_KVFULL), 0, status, 302);

@@ -40,12 +40,12 @@ struct alignas(64) TcGroup {
   int trace_slot;
 };
 
-#ifdef FBL_TRACE
+#ifdef FBL_TRACE_GEMM
 int g_trace_launch = 0;
 #endif
-// Optional timeline probe (compile with -DFBL_TRACE): one block records clock64() at the marked points of its
+// Optional timeline probe (compile with -DFBL_TRACE_GEMM): one block records clock64() at the marked points of its
 // first output tile into the words after the status word; slot = index of the GEMM launch within the pass.
-#ifdef FBL_TRACE
+#ifdef FBL_TRACE_GEMM
 #ifndef FBL_TRACE_BLOCK
 #define FBL_TRACE_BLOCK 0
 #endif
@@ -269,7 +269,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
         if (tracer && ti == 0 && pn < 2) GTR(10 + 2 * pn);
         uint4 outv[8];
         uint32_t* ow = reinterpret_cast<uint32_t*>(outv);
-#ifdef FBL_TRACE
+#ifdef FBL_TRACE_GEMM
         asm volatile("" ::"r"(v[0]), "r"(v[31]), "r"(v[32]), "r"(v[63]));
         if (tracer && ti == 0 && pn == 1) GTR(18);
 #endif
@@ -299,7 +299,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
           for (int j = 0; j < 64; j += 2)
             ow[j / 2] = tc::pack_bf16(pad ? 0.f : __uint_as_float(v[j]), pad ? 0.f : __uint_as_float(v[j + 1]));
         }
-#ifdef FBL_TRACE
+#ifdef FBL_TRACE_GEMM
         asm volatile("" ::"r"(ow[0]), "r"(ow[15]), "r"(ow[16]), "r"(ow[31]));
         if (tracer && ti == 0 && pn == 1) GTR(19);
 #endif
@@ -406,7 +406,7 @@ bool fbl_encode_f32_panel_map(CUtensorMap* map, const void* base, int64_t r_pad,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-#ifdef FBL_TRACE
+#ifdef FBL_TRACE_GEMM
 extern "C" int fbl_debug_gemm_trace(long long* host_dst) {
   return (int)cudaMemcpyFromSymbol(host_dst, g_gemm_trace, sizeof(long long) * 512);
 }
@@ -431,7 +431,7 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
   memset(&G, 0, sizeof(G));
   G.count = count;
   G.status = status;
-#ifdef FBL_TRACE
+#ifdef FBL_TRACE_GEMM
   G.trace_slot = (g_trace_launch++) & 1;      // two GEMM launches per pass
 #endif
   int tiles = 0;
