@@ -216,71 +216,109 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 // WPR warps share a row (d_model = NV * 256 * WPR columns): the row statistics are combined through shared memory.
+// The warps of a row meet at a named barrier of their own (rows of one block do not wait for each other), and
+// successive reductions alternate between two exchange buffers: a warp that writes buffer b again has passed the
+// barrier of the reduction in between, which every reader of the earlier value reached after reading it.
 template <int WPR>
-__device__ __forceinline__ float row_sum(float v, float* s_part, int slot, int part) {
+__device__ __forceinline__ float row_sum(float v, float* s_part, int slot, int part, int& buf) {
   v = warp_sum(v);
   if (WPR == 1) return v;
-  __syncthreads();                                   // previous use of s_part is over
-  if ((threadIdx.x & 31) == 0) s_part[slot * WPR + part] = v;
-  __syncthreads();
+  float* ex = s_part + buf * 8;
+  buf ^= 1;
+  if ((threadIdx.x & 31) == 0) ex[slot * WPR + part] = v;
+  asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "r"(WPR * 32) : "memory");
   float t = 0.f;
 #pragma unroll
-  for (int i = 0; i < WPR; ++i) t += s_part[slot * WPR + i];
+  for (int i = 0; i < WPR; ++i) t += ex[slot * WPR + i];
   return t;
 }
 
+// Two sums in one exchange.
+template <int WPR>
+__device__ __forceinline__ void row_sum2(float& a, float& b, float* s_part, int slot, int part, int& buf) {
+  a = warp_sum(a);
+  b = warp_sum(b);
+  if (WPR == 1) return;
+  float* ex = s_part + buf * 16;
+  buf ^= 1;
+  if ((threadIdx.x & 31) == 0) { ex[(slot * WPR + part) * 2] = a; ex[(slot * WPR + part) * 2 + 1] = b; }
+  asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "r"(WPR * 32) : "memory");
+  a = 0.f; b = 0.f;
+#pragma unroll
+  for (int i = 0; i < WPR; ++i) { a += ex[(slot * WPR + i) * 2]; b += ex[(slot * WPR + i) * 2 + 1]; }
+}
+
 template <int NV, int WPR>
-__global__ void __launch_bounds__(256) norm_fwd_rows_kernel(const __nv_bfloat16* __restrict__ X,
+__global__ void __launch_bounds__(256, 2) norm_fwd_rows_kernel(const __nv_bfloat16* __restrict__ X,
                                                             const float* __restrict__ gamma,
                                                             const float* __restrict__ beta,
                                                             __nv_bfloat16* __restrict__ Xn, float* __restrict__ stats,
                                                             int64_t n_pad, int seq, int t_pad, int rms, float eps) {
   constexpr int D = NV * 256 * WPR;
   constexpr int RPB = 8 / WPR;                       // rows per block pass
-  __shared__ float s_part[8];
-  pdl_launch_dependents();
-  pdl_wait();
+  __shared__ float s_part[16];
   const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
   const int slot = wib / WPR, part = wib % WPR;
-  // n_pad is a multiple of 8, so every warp of a block sees the same number of rows (block-wide barriers)
-  for (int64_t r = (int64_t)blockIdx.x * RPB + slot; r < n_pad; r += (int64_t)gridDim.x * RPB) {
+  int buf = 0;
+  pdl_launch_dependents();
+  // gamma and beta are inputs of the step: in registers before waiting for the previous kernel
+  float gm[NV][8], bt[NV][8];
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    const int c0 = ((part * NV + j) * 32 + lane) * 8;
+    const float4 g0 = *reinterpret_cast<const float4*>(gamma + c0), g1 = *reinterpret_cast<const float4*>(gamma + c0 + 4);
+    float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
+    if (beta) { b0 = *reinterpret_cast<const float4*>(beta + c0); b1 = *reinterpret_cast<const float4*>(beta + c0 + 4); }
+    gm[j][0] = g0.x; gm[j][1] = g0.y; gm[j][2] = g0.z; gm[j][3] = g0.w; gm[j][4] = g1.x; gm[j][5] = g1.y; gm[j][6] = g1.z; gm[j][7] = g1.w;
+    bt[j][0] = b0.x; bt[j][1] = b0.y; bt[j][2] = b0.z; bt[j][3] = b0.w; bt[j][4] = b1.x; bt[j][5] = b1.y; bt[j][6] = b1.z; bt[j][7] = b1.w;
+  }
+  pdl_wait();
+  const int64_t stride = (int64_t)gridDim.x * RPB;
+  // lane's vectors of a row: vector index v -> panel v / 8, chunk v % 8
+  auto vec_off = [&](int j, int64_t r) {
+    const int v = (part * NV + j) * 32 + lane;
+    return ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8;
+  };
+  int64_t r = (int64_t)blockIdx.x * RPB + slot;
+  uint4 nxt[NV];                                     // the next row is requested before this one is reduced
+  if (r < n_pad) {
+#pragma unroll
+    for (int j = 0; j < NV; ++j) nxt[j] = *reinterpret_cast<const uint4*>(X + vec_off(j, r));
+  }
+  for (; r < n_pad; r += stride) {
     const bool pad = (int)(r % t_pad) >= seq;
     float x[NV][8];
     float s = 0.f;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      const int v = (part * NV + j) * 32 + lane;           // vector index in the row: panel v / 8, chunk v % 8
-      load16(X + ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8, x[j]);
+      const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&nxt[j]);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) s += x[j][i];
+      for (int i = 0; i < 8; ++i) { x[j][i] = __bfloat162float(e[i]); s += x[j][i]; }
     }
-    const float mean = rms ? 0.f : row_sum<WPR>(s, s_part, slot, part) * (1.f / D);
+    if (r + stride < n_pad) {
+#pragma unroll
+      for (int j = 0; j < NV; ++j) nxt[j] = *reinterpret_cast<const uint4*>(X + vec_off(j, r + stride));
+    }
+    const float mean = rms ? 0.f : row_sum<WPR>(s, s_part, slot, part, buf) * (1.f / D);
     float q = 0.f;
 #pragma unroll
     for (int j = 0; j < NV; ++j)
 #pragma unroll
       for (int i = 0; i < 8; ++i) { const float c = x[j][i] - mean; q += c * c; }
-    const float rstd = rsqrtf(row_sum<WPR>(q, s_part, slot, part) * (1.f / D) + eps);
+    const float rstd = rsqrtf(row_sum<WPR>(q, s_part, slot, part, buf) * (1.f / D) + eps);
     if (lane == 0 && part == 0) { stats[2 * r] = pad ? 0.f : mean; stats[2 * r + 1] = pad ? 0.f : rstd; }
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      const int v = (part * NV + j) * 32 + lane;
-      const int c0 = v * 8;
-      const float4 g0 = *reinterpret_cast<const float4*>(gamma + c0), g1 = *reinterpret_cast<const float4*>(gamma + c0 + 4);
-      float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
-      if (beta) { b0 = *reinterpret_cast<const float4*>(beta + c0); b1 = *reinterpret_cast<const float4*>(beta + c0 + 4); }
-      const float gm[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-      const float bt[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
       float y[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) y[i] = pad ? 0.f : (x[j][i] - mean) * rstd * gm[i] + bt[i];
-      store16(Xn + ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8, y);
+      for (int i = 0; i < 8; ++i) y[i] = pad ? 0.f : (x[j][i] - mean) * rstd * gm[j][i] + bt[j][i];
+      store16(Xn + vec_off(j, r), y);
     }
   }
 }
 
 template <int NV, int WPR>
-__global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16* __restrict__ dXn,
+__global__ void __launch_bounds__(256, 2) norm_bwd_rows_kernel(const __nv_bfloat16* __restrict__ dXn,
                                                             const __nv_bfloat16* __restrict__ X,
                                                             const __nv_bfloat16* __restrict__ dY,
                                                             const float* __restrict__ stats,
@@ -291,7 +329,8 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
   constexpr int RPB = 8 / WPR;
   __shared__ float s_dg[D];
   __shared__ float s_db[D];
-  __shared__ float s_part[8];
+  __shared__ float s_part[32];
+  int buf = 0;
   for (int i = threadIdx.x; i < D; i += 256) { s_dg[i] = 0.f; s_db[i] = 0.f; }
   __syncthreads();
   pdl_launch_dependents();
@@ -341,8 +380,9 @@ __global__ void __launch_bounds__(256) norm_bwd_rows_kernel(const __nv_bfloat16*
         s2 = fmaf(g[j][i], xh[j][i], s2);
       }
     }
-    s1 = rms ? 0.f : row_sum<WPR>(s1, s_part, slot, part) * (1.f / D);
-    s2 = row_sum<WPR>(s2, s_part, slot, part) * (1.f / D);
+    row_sum2<WPR>(s1, s2, s_part, slot, part, buf);
+    s1 = rms ? 0.f : s1 * (1.f / D);
+    s2 *= (1.f / D);
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
       const int v = (part * NV + j) * 32 + lane;
@@ -411,7 +451,7 @@ __global__ void __launch_bounds__(256) norm_bwd_reduce_kernel(const float* __res
 template <int NV, int WPR>
 void norm_fwd_rows_launch(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
                           float* stats, int rms, cudaStream_t st) {
-  const int blocks = (int)min((int64_t)p->sm_count * 4, p->n_pad / (8 / WPR));
+  const int blocks = (int)min((int64_t)p->sm_count * 2, p->n_pad / (8 / WPR));
   launch_pdl(norm_fwd_rows_kernel<NV, WPR>, dim3(blocks), dim3(256), 0, st, (const __nv_bfloat16*)X, gamma,
              rms ? (const float*)nullptr : beta, (__nv_bfloat16*)Xn, stats, p->n_pad, p->d.seq, p->t_pad, rms, p->d.eps);
 }
@@ -426,26 +466,33 @@ void norm_bwd_rows_launch(const fbl_plan* p, const void* dXn, const void* X, con
              blocks, p->d.d_model, dgamma, dbeta);
 }
 
-// d_model -> (vectors per lane, warps per row) of the register-resident kernels; false if there is none
+// d_model -> (vectors per lane, warps per row) of the register-resident kernels; false if there is none.  At most
+// three vectors per lane: the backward keeps five values per column in registers, and two blocks should fit an SM.
 bool norm_rows_shape(int d, int* nv, int* wpr) {
   if (d % 256 != 0) return false;
-  const int v = d / 256;
-  if (v <= 4) { *nv = v; *wpr = 1; return true; }
-  if (v == 8) { *nv = 4; *wpr = 2; return true; }
-  if (v == 16) { *nv = 4; *wpr = 4; return true; }
-  if (v == 6) { *nv = 3; *wpr = 2; return true; }
-  if (v == 12) { *nv = 3; *wpr = 4; return true; }
-  return false;
+  switch (d / 256) {
+    case 1: *nv = 1; *wpr = 1; return true;
+    case 2: *nv = 2; *wpr = 1; return true;
+    case 3: *nv = 3; *wpr = 1; return true;
+    case 4: *nv = 2; *wpr = 2; return true;
+    case 6: *nv = 3; *wpr = 2; return true;
+    case 8: *nv = 2; *wpr = 4; return true;
+    case 12: *nv = 3; *wpr = 4; return true;
+    case 16: *nv = 2; *wpr = 8; return true;
+    default: return false;
+  }
 }
 
 #define FBL_NORM_DISPATCH(CALL)                                        \
   do {                                                                 \
     if (wpr == 1) {                                                    \
-      if (nv == 1) CALL(1, 1); else if (nv == 2) CALL(2, 1); else if (nv == 3) CALL(3, 1); else CALL(4, 1); \
+      if (nv == 1) CALL(1, 1); else if (nv == 2) CALL(2, 1); else CALL(3, 1); \
     } else if (wpr == 2) {                                             \
-      if (nv == 3) CALL(3, 2); else CALL(4, 2);                        \
+      if (nv == 2) CALL(2, 2); else CALL(3, 2);                        \
+    } else if (wpr == 4) {                                             \
+      if (nv == 2) CALL(2, 4); else CALL(3, 4);                        \
     } else {                                                           \
-      if (nv == 3) CALL(3, 4); else CALL(4, 4);                        \
+      CALL(2, 8);                                                      \
     }                                                                  \
   } while (0)
 
