@@ -139,7 +139,25 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   p->sf_part = o; o += p->part_bytes;
   p->scratch_fwd_bytes = o;
 
-  o = FBL_ALIGN;
+  // weight-gradient GEMMs: few output tiles, reduction over all tokens; slice the reduction when that balances the SMs
+  p->ksplit_o = p->ksplit_qkv = 1;
+  if (p->use_tc) {
+    const int kb_tok = (int)((p->n_pad + 63) / 64);
+    const GemmShape go[2] = {{p->dq, d.d_model, kb_tok, 1}, {p->n_pad, p->dq, (d.d_model + 63) / 64, 0}};
+    p->ksplit_o = gemm_tc_choose_split(p->sm_count, go, 2);
+    const GemmShape gq[4] = {{d.d_model, p->dq, kb_tok, 1}, {d.d_model, p->dkv, kb_tok, 1}, {d.d_model, p->dkv, kb_tok, 1},
+                             {p->n_pad, d.d_model, (p->dq + 2 * p->dkv + 63) / 64, 0}};
+    p->ksplit_qkv = gemm_tc_choose_split(p->sm_count, gq, 4);
+  }
+  if (p->use_tc && getenv("FBL_KSPLIT_O")) p->ksplit_o = atoi(getenv("FBL_KSPLIT_O"));          // tuning knobs
+  if (p->use_tc && getenv("FBL_KSPLIT_QKV")) p->ksplit_qkv = atoi(getenv("FBL_KSPLIT_QKV"));
+  if (getenv("FBL_VERBOSE")) fprintf(stderr, "fblayout: reduction slices dWo %d, dWq/dWk/dWv %d\n", p->ksplit_o, p->ksplit_qkv);
+  o = FBL_ALIGN;  // status word, then the fp32 accumulation areas
+  p->sb_acc_o = o;
+  if (p->ksplit_o > 1) o += fbl_align_up((size_t)up8(p->dq) * d.d_model * sizeof(float), FBL_ALIGN);
+  p->sb_acc_qkv = o;
+  if (p->ksplit_qkv > 1) o += fbl_align_up((size_t)up8(d.d_model) * (p->dq + 2 * p->dkv) * sizeof(float), FBL_ALIGN);
+  p->acc_bytes = o - FBL_ALIGN;
   p->sb_da = o;    o += mat(p->dq);
   p->sb_dvec = o;  o += fbl_align_up(rows_bh * sizeof(float), FBL_ALIGN);
   p->sb_dqacc = o; o += fbl_align_up(n * p->dq * sizeof(float), FBL_ALIGN);
@@ -385,7 +403,9 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
   const bool bias = p->d.has_bias;
   const int n = (int)p->n_pad, D = p->d.d_model;
 
-  FBL_CUDA(cudaMemsetAsync(status, 0, FBL_ALIGN, st));
+  // the status word and, behind it, the fp32 accumulation areas of sliced weight-gradient GEMMs: one fill
+  const bool split_o = p->use_tc && p->ksplit_o > 1, split_qkv = p->use_tc && p->ksplit_qkv > 1;
+  FBL_CUDA(cudaMemsetAsync(status, 0, FBL_ALIGN + ((split_o || split_qkv) ? p->acc_bytes : 0), st));
   FBL_PROF_BEGIN();
   bool dvec_ready = false;
   {
@@ -405,7 +425,13 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
       // D = rowsum(dO * O) per head comes out of the dA epilogue, from the fp32 accumulator
       ga.dot_with = A; ga.dot_out = dvec; ga.dot_hd = p->d.head_dim; ga.dot_hq = p->d.n_q_heads;
       dvec_ready = true;
+      if (split_o) { gw.ksplit = p->ksplit_o; gw.acc = (float*)(sc + p->sb_acc_o); }
       FBL_STEP("dWo+dA", 1, launch_gemm_tc_group(p, gs, 2, status, st));
+      if (split_o) {
+        ConvertGroup cg = {};
+        cg.src[0] = gw.acc; cg.dst[0] = dWo; cg.n[0] = up8(p->dq) * (int64_t)D; cg.count = 1;
+        FBL_STEP("dWo round", 1, launch_convert_f32_group(cg, st));
+      }
     } else {
       FBL_STEP("dA", 1, run_gemm(p, ga, part, p->part_bytes, status, st));
       FBL_STEP("dWo", 1, run_gemm(p, gw, part, p->part_bytes, status, st));
@@ -437,7 +463,18 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
     gx.c = dXn; gx.c_rpad = p->n_pad; gx.seq = p->d.seq; gx.t_pad = p->t_pad;
     tc = tc && gemm_tc_supported(p, gx);
     if (tc) {
+      ConvertGroup cg = {};
+      if (split_qkv) {
+        float* acc = (float*)(sc + p->sb_acc_qkv);
+        for (int i = 0; i < 3; ++i) {
+          gs[i].ksplit = p->ksplit_qkv; gs[i].acc = acc;
+          cg.src[i] = acc; cg.dst[i] = DW[i]; cg.n[i] = up8(D) * (int64_t)cols[i];
+          acc += cg.n[i];
+        }
+        cg.count = 3;
+      }
       FBL_STEP("dWqkv+dXn", 1, launch_gemm_tc_group(p, gs, 4, status, st));
+      if (split_qkv) FBL_STEP("dWqkv round", 1, launch_convert_f32_group(cg, st));
     } else {
       FBL_STEP("dXn", 1, run_gemm(p, gx, part, p->part_bytes, status, st));
       for (int i = 0; i < 3; ++i)

@@ -46,6 +46,10 @@ struct fbl_plan {
   size_t sb_da, sb_dvec, sb_dqacc, sb_dq, sb_dk, sb_dv, sb_dxn, sb_part, scratch_bwd_bytes;
   size_t sf_part, scratch_fwd_bytes;
   size_t part_bytes;
+  // reduction-loop slicing of the weight-gradient GEMMs (1: none) and their fp32 accumulation areas, which
+  // follow the status word so that one fill zeroes both
+  int ksplit_o, ksplit_qkv;
+  size_t sb_acc_o, sb_acc_qkv, acc_bytes;
   // bookkeeping: kernels enqueued so far, optional per-step event timing
   int64_t launches;
   int prof_on, prof_n;
@@ -73,6 +77,9 @@ struct GemmArgs {
   int b_static;                   // 1: the first term's B operand is an input of the whole step (a weight)
   // optional fused row reduction D[b,h,t] = sum_d C[row, h*hd+d] * dot_with[row, h*hd+d] (fp32 C, before rounding)
   const void* dot_with; float* dot_out; int dot_hd, dot_hq;
+  // reduction loop cut into ksplit slices whose fp32 partial tiles are added into `acc` (zeroed by the caller, same
+  // element order as C with 4-byte elements); C itself is then produced from acc by launch_convert_f32_group
+  int ksplit; float* acc;
 };
 
 cudaError_t launch_gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);
@@ -80,6 +87,8 @@ cudaError_t launch_gemm_tc(const fbl_plan* p, const GemmArgs& g, void* splitk_sc
                            int32_t* status, cudaStream_t st);
 bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g);
 cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st);
+struct GemmShape { int64_t m; int n; int kblocks; int splittable; };
+int gemm_tc_choose_split(int sm_count, const GemmShape* sh, int count);
 bool attn_fwd_tc_supported(const fbl_plan* p);
 bool attn_bwd_tc_supported(const fbl_plan* p);
 void fbl_note_cuda_error(cudaError_t e, const char* where);
@@ -104,6 +113,8 @@ cudaError_t launch_attn_bwd_simt(const fbl_plan* p, const void* Q, const void* K
                                  void* dV, cudaStream_t st);
 cudaError_t launch_attn_bwd_pre(const fbl_plan* p, const void* A, const void* dA, float* dvec, float* dqacc,
                                 bool dvec_ready, cudaStream_t st);
+struct ConvertGroup { const float* src[4]; void* dst[4]; int64_t n[4]; int count; };
+cudaError_t launch_convert_f32_group(const ConvertGroup& g, cudaStream_t st);   // bf16 destinations, n multiples of 4
 cudaError_t launch_attn_bwd_post(const fbl_plan* p, const float* dqacc, void* dQ, cudaStream_t st);
 cudaError_t launch_attn_fwd_tc(const fbl_plan* p, const void* Q, const void* K, const void* V, void* A, float* lse,
                                int32_t* status, cudaStream_t st);

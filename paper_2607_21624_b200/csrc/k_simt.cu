@@ -371,6 +371,22 @@ __global__ void convert_f32_kernel(const float* __restrict__ src, T* __restrict_
   }
 }
 
+// Up to four fp32 buffers rounded to bf16 in one launch (blockIdx.y picks the buffer).
+__global__ void convert_f32_group_kernel(ConvertGroup g) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const float* __restrict__ src = g.src[blockIdx.y];
+  __nv_bfloat16* __restrict__ dst = (__nv_bfloat16*)g.dst[blockIdx.y];
+  const int64_t n = g.n[blockIdx.y];
+  for (int64_t i = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) * 4; i < n; i += (int64_t)gridDim.x * blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(src + i);
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 o;
+    o.x = *reinterpret_cast<uint32_t*>(&lo); o.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(dst + i) = o;
+  }
+}
+
 template <typename T, int HD>
 cudaError_t attn_fwd_launch(const fbl_plan* p, const void* Q, const void* K, const void* V, void* A, float* lse,
                             cudaStream_t st) {
@@ -441,6 +457,13 @@ cudaError_t launch_attn_bwd_post(const fbl_plan* p, const float* dqacc, void* dQ
   if (p->d.dtype == FBL_DTYPE_FP32)
     return launch_pdl(convert_f32_kernel<float>, dim3(blocks), dim3(256), 0, st, dqacc, (float*)dQ, nq);
   return launch_pdl(convert_f32_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, dqacc, (__nv_bfloat16*)dQ, nq);
+}
+
+cudaError_t launch_convert_f32_group(const ConvertGroup& g, cudaStream_t st) {
+  int64_t mx = 0;
+  for (int i = 0; i < g.count; ++i) mx = g.n[i] > mx ? g.n[i] : mx;
+  const int blocks = (int)min((int64_t)148 * 4, (mx / 4 + 255) / 256);
+  return launch_pdl(convert_f32_group_kernel, dim3(blocks > 0 ? blocks : 1, g.count), dim3(256), 0, st, g);
 }
 
 cudaError_t launch_attn_bwd_simt(const fbl_plan* p, const void* Q, const void* K, const void* V, const void* A,

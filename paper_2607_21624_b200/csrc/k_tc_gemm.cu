@@ -32,6 +32,11 @@ struct alignas(64) TcProblem {
   const __nv_bfloat16* dot_with;   // fused D = rowsum(C * dot_with) per head (the attention backward's D), or nullptr
   float* dot_out;
   int dot_hd, dot_hq;
+  // Reduction loop cut into `ksplit` slices, each a work unit of its own (a problem with few output tiles and a
+  // long reduction): slices add their fp32 partial tiles into `tacc`'s buffer with bulk tensor reductions, and a
+  // later kernel rounds the sums to bf16.  Single-term problems without epilogue extras only.
+  int ksplit;
+  CUtensorMap tacc;
 };
 struct alignas(64) TcGroup {
   TcProblem p[MAX_PROBLEMS];
@@ -72,19 +77,25 @@ struct SmemPlan {
 
 // Work list of a launch: output tiles of all problems, numbered problem by problem with the M tile index
 // fastest (blocks that run together then share the B tiles of one weight column block through L2).
-struct TileCoord { int prob, m0, n0; };
+struct TileCoord { int prob, m0, n0, kb0, kb1; };     // kb0..kb1: k-block range of term 0 (split problems)
 
 template <int BN>
 __device__ __forceinline__ bool tile_at(const TcGroup& G, int w, TileCoord* tc_out) {
   for (int p = 0; p < G.count; ++p) {
-    const int tm = (G.p[p].m + BM - 1) / BM, tn = (G.p[p].n + BN - 1) / BN;
-    if (w < tm * tn) {
+    const TcProblem& P = G.p[p];
+    const int tm = (P.m + BM - 1) / BM, tn = (P.n + BN - 1) / BN;
+    const int units = tm * tn * P.ksplit;
+    if (w < units) {
+      const int slice = w % P.ksplit, t = w / P.ksplit;        // slices of one tile are neighbours in the list
       tc_out->prob = p;
-      tc_out->m0 = (w % tm) * BM;
-      tc_out->n0 = (w / tm) * BN;
+      tc_out->m0 = (t % tm) * BM;
+      tc_out->n0 = (t / tm) * BN;
+      const int per = (P.kblocks[0] + P.ksplit - 1) / P.ksplit;
+      tc_out->kb0 = slice * per;
+      tc_out->kb1 = min(P.kblocks[0], (slice + 1) * per);
       return true;
     }
-    w -= tm * tn;
+    w -= units;
   }
   return false;
 }
@@ -140,7 +151,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
     // Weights do not depend on the kernel before this one: their tiles for the first stages of the first
     // output tile are requested before waiting for that kernel, hiding their (cold) latency.
     int prefilled = 0;
-    if (tile_at<BN>(G, blockIdx.x, &tcd) && G.p[tcd.prob].b_static) {
+    if (tile_at<BN>(G, blockIdx.x, &tcd) && G.p[tcd.prob].b_static && G.p[tcd.prob].ksplit == 1) {
       const TcProblem& P = G.p[tcd.prob];
       tc::tma_prefetch_desc(&P.ta[0]);
       tc::tma_prefetch_desc(&P.tb[0]);
@@ -158,7 +169,8 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
     for (int w = blockIdx.x; ok && tile_at<BN>(G, w, &tcd); w += gridDim.x) {
       const TcProblem& P = G.p[tcd.prob];
       for (int t = 0; t < P.n_terms && ok; ++t) {
-        for (int kb = 0; kb < P.kblocks[t]; ++kb, ++it) {
+        const int kb_begin = t == 0 ? tcd.kb0 : 0, kb_end = t == 0 ? tcd.kb1 : P.kblocks[t];
+        for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           const uint32_t sa = base + s * SP::STAGE, sb = sa + SP::A_BYTES;
@@ -203,7 +215,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
         // MN-major: 64-wide M/N blocks 8 KiB apart (64 K rows x 128 B), 16 K rows = 2 KiB.
         const uint32_t a_lo0 = tc::smem_desc_lo(base, P.a_mn[t] ? 8192u : 16u), a_step = P.a_mn[t] ? 128u : 2u;
         const uint32_t b_lo0 = tc::smem_desc_lo(base + SP::A_BYTES, P.b_mn[t] ? 8192u : 16u), b_step = P.b_mn[t] ? 128u : 2u;
-        const int nkb = P.kblocks[t];
+        const int nkb = t == 0 ? tcd.kb1 - tcd.kb0 : P.kblocks[t];
         for (int kb = 0; kb < nkb; ++kb) {
           if (!tc::mbar_wait(full(s), ph, status, 102)) { ok = false; break; }
           if (ti == 0 && t == 0 && kb == 0) GTR(3);
@@ -267,6 +279,29 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
         tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + pn * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
         tc::tmem_ld_wait();
         if (tracer && ti == 0 && pn < 2) GTR(10 + 2 * pn);
+        if (P.ksplit > 1) {
+          // partial sums of a reduction slice: two 32-column halves of the panel, fp32, added to the accumulation
+          // buffer by bulk tensor reductions (same staging tiles and swizzle as the bf16 rows below)
+#pragma unroll 1
+          for (int hf = 0; hf < 2; ++hf) {
+            const uint32_t stg = base + SP::STG_OFF + (uint32_t)(q * 2 + (pc & 1)) * 4096u;
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + (((uint32_t)j ^ (uint32_t)(lane & 7)) * 16)),
+                           "r"(hf ? v[32 + 4 * j] : v[4 * j]), "r"(hf ? v[33 + 4 * j] : v[4 * j + 1]),
+                           "r"(hf ? v[34 + 4 * j] : v[4 * j + 2]), "r"(hf ? v[35 + 4 * j] : v[4 * j + 3]) : "memory");
+            tc::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tc::tma_reduce_add_4d(&P.tacc, stg, 0, hf, tcd.m0 + q * 32, n / 64);
+              tc::bulk_commit_group();
+              tc::bulk_wait_group_read1();
+            }
+            ++pc;
+          }
+          continue;
+        }
         uint4 outv[8];
         uint32_t* ow = reinterpret_cast<uint32_t*>(outv);
 #ifdef FBL_TRACE_GEMM
@@ -394,12 +429,12 @@ bool fbl_encode_rtile_map(CUtensorMap* map, const void* base, int64_t r_pad, int
 
 // fp32 accumulator [n_pad, cols] stored in the bf16 tile order (64-column panels, 256-byte rows), viewed as
 // [panels][rows][2 halves][32 floats] so that a box of 128 rows x one panel can use the 128-byte swizzle.
-bool fbl_encode_f32_panel_map(CUtensorMap* map, const void* base, int64_t r_pad, int panels, int box_rows) {
+bool fbl_encode_f32_panel_map(CUtensorMap* map, const void* base, int64_t r_pad, int panels, int box_rows, int box_halves) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[4] = {32, 2, (cuuint64_t)r_pad, (cuuint64_t)panels};
   cuuint64_t strides[3] = {128, 256, (cuuint64_t)r_pad * 256};
-  cuuint32_t box[4] = {32, 2, (cuuint32_t)box_rows, 1};
+  cuuint32_t box[4] = {32, (cuuint32_t)box_halves, (cuuint32_t)box_rows, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -459,7 +494,14 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
     P.bias = g.bias; P.residual = (const __nv_bfloat16*)g.residual;
     P.seq = g.seq; P.t_pad = g.t_pad;
     P.dot_with = (const __nv_bfloat16*)g.dot_with; P.dot_out = g.dot_out; P.dot_hd = g.dot_hd; P.dot_hq = g.dot_hq;
-    tiles += ((g.m + BM - 1) / BM) * ((g.n + BN - 1) / BN);
+    P.ksplit = 1;
+    if (g.ksplit > 1) {
+      if (g.n_terms != 1 || g.bias || g.residual || g.dot_with || g.t_pad > 0 || !g.acc) return cudaErrorInvalidValue;
+      const int per = (P.kblocks[0] + g.ksplit - 1) / g.ksplit;        // no empty slice
+      P.ksplit = (P.kblocks[0] + per - 1) / per;
+      if (!fbl_encode_f32_panel_map(&P.tacc, g.acc, g.c_rpad, g.n / 64, 32, 1)) return cudaErrorInvalidValue;
+    }
+    tiles += ((g.m + BM - 1) / BM) * ((g.n + BN - 1) / BN) * P.ksplit;
   }
   using SP = SmemPlan<BN, STAGES>;
   auto k = gemm_tc_kernel<BN, STAGES>;
@@ -477,12 +519,57 @@ cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int coun
     wide = wide && gs[i].n % 256 == 0;
     for (int t = 0; t < gs[i].n_terms; ++t)
       if (gs[i].t[t].b_trans && gs[i].t[t].b_rpad < 256) wide = false;
-    tiles_wide += ((gs[i].m + BM - 1) / BM) * ((gs[i].n + 255) / 256);
+    tiles_wide += ((gs[i].m + BM - 1) / BM) * ((gs[i].n + 255) / 256) * (gs[i].ksplit > 1 ? gs[i].ksplit : 1);
   }
   // with too few wide tiles to occupy the SMs, narrower tiles (twice as many) finish sooner
   if (wide && tiles_wide * 3 < p->sm_count * 2) wide = false;
   if (wide) return launch_group_bn<256, 4>(p, gs, count, status, st);
   return launch_group_bn<128, 6>(p, gs, count, status, st);
+}
+
+// How many slices to cut the reduction loops of the splittable problems of a group into (the same number for all
+// of them).  The persistent kernel deals work units to its blocks round-robin, so a few long units beside many
+// short ones leave most SMs idle: this replays the dealing for each candidate and keeps the one whose longest
+// block finishes first, charging the fp32 detour (zero-fill, bulk reductions, rounding pass) as extra k-blocks.
+int gemm_tc_choose_split(int sm_count, const GemmShape* sh, int count) {
+  static const int cand[] = {1, 2, 3, 4, 6, 8, 12, 16};
+  double base_cost = 0.0, best_cost = 0.0;
+  int best = 1;
+  for (int ci = 0; ci < (int)(sizeof(cand) / sizeof(cand[0])); ++ci) {
+    const int S = cand[ci];
+    bool wide = true;
+    long long tiles_wide = 0;
+    bool any_split = false;
+    for (int i = 0; i < count; ++i) {
+      wide = wide && sh[i].n % 256 == 0;
+      const int s_i = (sh[i].splittable && S > 1) ? S : 1;
+      if (s_i > 1 && sh[i].kblocks / s_i < 8) { any_split = false; tiles_wide = -1; break; }   // slices too short
+      any_split = any_split || s_i > 1;
+      tiles_wide += (long long)((sh[i].m + BM - 1) / BM) * ((sh[i].n + 255) / 256) * s_i;
+    }
+    if (tiles_wide < 0 || (S > 1 && !any_split)) continue;
+    if (wide && tiles_wide * 3 < (long long)sm_count * 2) wide = false;
+    const int bn = wide ? 256 : 128;
+    const double per_kb = wide ? 1.32 : 1.0;               // a k-block of a 128 x 256 tile takes about 660 clk, of 128 x 128 about 500
+    long long units = 0;
+    for (int i = 0; i < count; ++i)
+      units += (long long)((sh[i].m + BM - 1) / BM) * ((sh[i].n + bn - 1) / bn) * ((sh[i].splittable && S > 1) ? S : 1);
+    const int grid = (int)(units < sm_count ? units : sm_count);
+    double load[256] = {0};
+    long long w = 0;
+    for (int i = 0; i < count; ++i) {
+      const int s_i = (sh[i].splittable && S > 1) ? S : 1;
+      const long long n_i = (long long)((sh[i].m + BM - 1) / BM) * ((sh[i].n + bn - 1) / bn) * s_i;
+      const double len = ((sh[i].kblocks + s_i - 1) / s_i + (s_i > 1 ? 2 : 0) + 3) * per_kb;   // + pipeline fill and epilogue
+      for (long long u = 0; u < n_i; ++u, ++w) load[w % grid] += len;
+    }
+    double mk = 0;
+    for (int b = 0; b < grid; ++b) mk = load[b] > mk ? load[b] : mk;
+    if (S > 1) mk += 16;                                   // zero-fill and rounding pass
+    if (ci == 0) { base_cost = mk; best_cost = mk; }
+    else if (mk < 0.85 * base_cost && mk < best_cost) { best = S; best_cost = mk; }   // worth it only with a clear gain
+  }
+  return best;
 }
 
 cudaError_t launch_gemm_tc(const fbl_plan* p, const GemmArgs& g, void*, size_t, int32_t* status, cudaStream_t st) {

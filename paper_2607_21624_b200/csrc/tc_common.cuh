@@ -248,4 +248,4 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // Host side: encode a 3-D tensor map over an R-Tile bf16 matrix viewed as [panels][rows][64].
 bool fbl_encode_rtile_map(CUtensorMap* map, const void* base, int64_t r_pad, int panels, int box_rows, int box_panels);
-bool fbl_encode_f32_panel_map(CUtensorMap* map, const void* base, int64_t r_pad, int panels, int box_rows);
+bool fbl_encode_f32_panel_map(CUtensorMap* map, const void* base, int64_t r_pad, int panels, int box_rows, int box_halves = 2);
