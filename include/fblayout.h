@@ -95,7 +95,11 @@ typedef struct fbl_plan fbl_plan; /* opaque: padded sizes, index-map constants, 
 
 /* Host only.  Validates the description against the tile-propagation legality checks of section 4.3
  * (head_dim and d_model multiples of tile_w, n_q_heads a multiple of n_kv_heads) and the kernels'
- * limits, then builds the plan.  *out is owned by the caller; release with fbl_plan_destroy. */
+ * limits, then builds the plan.  *out is owned by the caller; release with fbl_plan_destroy.
+ * The plan also fixes, from the shapes alone, into how many slices the token-axis reductions of the weight
+ * gradients are cut (1 for all but layers with few weight tiles and many tokens).  Environment variables
+ * read here, for tuning and tests only: FBL_KSPLIT_O and FBL_KSPLIT_QKV override those slice counts,
+ * FBL_VERBOSE prints the ones chosen to stderr. */
 int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out);
 void fbl_plan_destroy(fbl_plan* plan);
 

@@ -83,6 +83,17 @@ def test_bf16_small(cfg, path):
     run_and_compare(cfg, affine_noise=True, path=path)
 
 
+@pytest.mark.parametrize("slices", [(3, 4), (19, 2)], ids=["o3-qkv4", "o19-qkv2"])
+def test_sliced_weight_gradient_reductions(slices, monkeypatch):
+    # The plan slices the token-axis reduction of dWo / dWq, dWk, dWv only when the replayed work dealing gains
+    # from it (workload 3 does); the tuning knobs force it here on a shape with 19 k-blocks of tokens (ragged
+    # last slice; one k-block per slice) and with biases, so that the sliced path is compared at a small size too.
+    monkeypatch.setenv("FBL_KSPLIT_O", str(slices[0]))
+    monkeypatch.setenv("FBL_KSPLIT_QKV", str(slices[1]))
+    run_and_compare(LayerConfig("s1", 6, 197, 256, 4, 2, 64, "bf16", "layernorm", True, True, True, 1e-5, 31, 0.02),
+                    affine_noise=True)
+
+
 @pytest.mark.parametrize("i", [2, 3])
 def test_full_configs_2_and_3(i):
     run_and_compare(get_config(i))
