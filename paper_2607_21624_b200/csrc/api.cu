@@ -158,9 +158,10 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   p->sb_acc_qkv = o;
   if (p->ksplit_qkv > 1) o += fbl_align_up((size_t)up8(d.d_model) * (p->dq + 2 * p->dkv) * sizeof(float), FBL_ALIGN);
   p->acc_bytes = o - FBL_ALIGN;
+  p->sb_dqacc = o; o += fbl_align_up(n * p->dq * sizeof(float), FBL_ALIGN);   // zero-filled with the areas before it
+  p->zero_bytes = o;
   p->sb_da = o;    o += mat(p->dq);
   p->sb_dvec = o;  o += fbl_align_up(rows_bh * sizeof(float), FBL_ALIGN);
-  p->sb_dqacc = o; o += fbl_align_up(n * p->dq * sizeof(float), FBL_ALIGN);
   p->sb_dq = o;    o += mat(p->dq);
   p->sb_dk = o;    o += mat(p->dkv);
   p->sb_dv = o;    o += mat(p->dkv);
@@ -337,9 +338,9 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
   const bool bias = p->d.has_bias;
   const int n = (int)p->n_pad, D = p->d.d_model;
 
-  FBL_CUDA(cudaMemsetAsync(status, 0, FBL_ALIGN, st));
+  if (!norm_fwd_resets_status(p)) FBL_CUDA(cudaMemsetAsync(status, 0, FBL_ALIGN, st));
   FBL_PROF_BEGIN();
-  FBL_STEP("norm_fwd", 1, launch_norm_fwd(p, X, gamma, beta, Xn, stats, st));
+  FBL_STEP("norm_fwd", 1, launch_norm_fwd(p, X, gamma, beta, Xn, stats, status, st));
   {
     const void* W[3] = {Wq, Wk, Wv};
     void* O[3] = {Q, K, V};
@@ -403,9 +404,11 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
   const bool bias = p->d.has_bias;
   const int n = (int)p->n_pad, D = p->d.d_model;
 
-  // the status word and, behind it, the fp32 accumulation areas of sliced weight-gradient GEMMs: one fill
+  // One fill zeroes the status word and, behind it, every fp32 area the step adds into: the accumulation areas
+  // of sliced weight-gradient GEMMs and the dQ accumulator.  No fill then separates later kernels of the step,
+  // so each can start (programmatic dependent launch) while its predecessor drains.
   const bool split_o = p->use_tc && p->ksplit_o > 1, split_qkv = p->use_tc && p->ksplit_qkv > 1;
-  FBL_CUDA(cudaMemsetAsync(status, 0, FBL_ALIGN + ((split_o || split_qkv) ? p->acc_bytes : 0), st));
+  FBL_CUDA(cudaMemsetAsync(status, 0, p->zero_bytes, st));
   FBL_PROF_BEGIN();
   bool dvec_ready = false;
   {
@@ -437,7 +440,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
       FBL_STEP("dWo", 1, run_gemm(p, gw, part, p->part_bytes, status, st));
     }
   }
-  if (p->use_tc && attn_bwd_tc_supported(p)) FBL_STEP("attn_bwd", dvec_ready ? 2 : 3, launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, dvec_ready, status, st));
+  if (p->use_tc && attn_bwd_tc_supported(p)) FBL_STEP("attn_bwd", dvec_ready ? 2 : 3, launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, dvec_ready, status, st));   // dqacc: zero already
   else FBL_STEP("attn_bwd", 3, launch_attn_bwd_simt(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, st));
   {
     const void* G[3] = {dQ, dK, dV};

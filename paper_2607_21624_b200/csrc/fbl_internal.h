@@ -50,6 +50,7 @@ struct fbl_plan {
   // follow the status word so that one fill zeroes both
   int ksplit_o, ksplit_qkv;
   size_t sb_acc_o, sb_acc_qkv, acc_bytes;
+  size_t zero_bytes;        // leading part of the backward scratch that every step starts by zero-filling
   // bookkeeping: kernels enqueued so far, optional per-step event timing
   int64_t launches;
   int prof_on, prof_n;
@@ -95,8 +96,9 @@ void fbl_note_cuda_error(cudaError_t e, const char* where);
 
 cudaError_t launch_pack(int dtype, int unpack, const void* src, void* dst, int64_t outer, int64_t rows,
                         int64_t rows_pad, int cols, cudaStream_t st);
+bool norm_fwd_resets_status(const fbl_plan* p);   // the forward norm kernel for this plan zeroes the status word itself
 cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
-                            float* stats, cudaStream_t st);
+                            float* stats, int32_t* status, cudaStream_t st);
 cudaError_t launch_norm_bwd(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
                             const float* gamma, void* dX, float* dgamma, float* dbeta, float* part,
                             cudaStream_t st);

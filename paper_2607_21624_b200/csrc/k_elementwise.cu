@@ -253,10 +253,14 @@ __global__ void __launch_bounds__(256, 2) norm_fwd_rows_kernel(const __nv_bfloat
                                                             const float* __restrict__ gamma,
                                                             const float* __restrict__ beta,
                                                             __nv_bfloat16* __restrict__ Xn, float* __restrict__ stats,
-                                                            int64_t n_pad, int seq, int t_pad, int rms, float eps) {
+                                                            int64_t n_pad, int seq, int t_pad, int rms, float eps,
+                                                            int32_t* __restrict__ status) {
   constexpr int D = NV * 256 * WPR;
   constexpr int RPB = 8 / WPR;                       // rows per block pass
   __shared__ float s_part[16];
+  // First kernel of the forward pass: it resets the pass's status word (later kernels only write it after a
+  // bounded wait of about a second has expired), which saves a fill node in front of the pass.
+  if (status && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;
   const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
   const int slot = wib / WPR, part = wib % WPR;
   int buf = 0;
@@ -450,10 +454,10 @@ __global__ void __launch_bounds__(256) norm_bwd_reduce_kernel(const float* __res
 
 template <int NV, int WPR>
 void norm_fwd_rows_launch(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
-                          float* stats, int rms, cudaStream_t st) {
+                          float* stats, int rms, int32_t* status, cudaStream_t st) {
   const int blocks = (int)min((int64_t)p->sm_count * 2, p->n_pad / (8 / WPR));
   launch_pdl(norm_fwd_rows_kernel<NV, WPR>, dim3(blocks), dim3(256), 0, st, (const __nv_bfloat16*)X, gamma,
-             rms ? (const float*)nullptr : beta, (__nv_bfloat16*)Xn, stats, p->n_pad, p->d.seq, p->t_pad, rms, p->d.eps);
+             rms ? (const float*)nullptr : beta, (__nv_bfloat16*)Xn, stats, p->n_pad, p->d.seq, p->t_pad, rms, p->d.eps, status);
 }
 template <int NV, int WPR>
 void norm_bwd_rows_launch(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
@@ -578,13 +582,18 @@ cudaError_t launch_pack(int dtype, int unpack, const void* src, void* dst, int64
   return cudaGetLastError();
 }
 
+bool norm_fwd_resets_status(const fbl_plan* p) {
+  int nv, wpr;
+  return p->d.dtype == FBL_DTYPE_BF16 && norm_rows_shape(p->d.d_model, &nv, &wpr);
+}
+
 cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
-                            float* stats, cudaStream_t st) {
+                            float* stats, int32_t* status, cudaStream_t st) {
   const int blocks = (int)((p->n_pad + 31) / 32);
   const int rms = p->d.norm == FBL_NORM_RMSNORM;
   int nv, wpr;
   if (p->d.dtype == FBL_DTYPE_BF16 && norm_rows_shape(p->d.d_model, &nv, &wpr)) {
-#define FBL_CALL(NV_, WPR_) norm_fwd_rows_launch<NV_, WPR_>(p, X, gamma, beta, Xn, stats, rms, st)
+#define FBL_CALL(NV_, WPR_) norm_fwd_rows_launch<NV_, WPR_>(p, X, gamma, beta, Xn, stats, rms, status, st)
     FBL_NORM_DISPATCH(FBL_CALL);
 #undef FBL_CALL
     return cudaGetLastError();
