@@ -1,0 +1,75 @@
+"""Edge cases of the layer step on the GPU: degenerate shapes, refusals at the C boundary, repeatability."""
+import numpy as np
+import pytest
+
+from fbl_inputs import LayerConfig, make_inputs
+from tests.test_gpu_layer import run_and_compare
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("cfg", [
+    # one token per sequence: softmax over a single key (P = 1, dS = 0), every tile a ragged tail
+    LayerConfig("e1", 3, 1, 128, 2, 2, 64, "bf16", "layernorm", True, True, True, 1e-5, 41, 0.02),
+    LayerConfig("e2", 2, 1, 64, 2, 1, 32, "fp32", "rmsnorm", False, False, False, 1e-5, 42, 0.02),
+    # sequence one short of / one past a 128-row tile, many sequences: tile tails at both ends
+    LayerConfig("e3", 5, 127, 256, 4, 4, 64, "bf16", "rmsnorm", True, False, True, 1e-5, 43, 0.02),
+    LayerConfig("e4", 5, 129, 256, 2, 1, 128, "bf16", "layernorm", False, True, False, 1e-6, 44, 0.02),
+], ids=lambda c: c.name)
+def test_degenerate_and_tail_shapes(cfg):
+    run_and_compare(cfg, affine_noise=True)
+
+
+def test_single_token_closed_form():
+    # T = 1: attention is the identity on V, so Y = (Xn Wv + bv) Wo + bo (+ X) whatever Q and K are
+    from oracle.layer import layer_fwd_bwd
+    cfg = LayerConfig("e5", 4, 1, 128, 2, 2, 64, "bf16", "layernorm", True, True, True, 1e-5, 45, 0.02)
+    inp = make_inputs(cfg, affine_noise=True)
+    run = run_and_compare(cfg, affine_noise=True)
+    got = run.fetch("Y")
+    x = inp["X"][:, 0, :]
+    mu = x.mean(-1, keepdims=True)
+    xn = (x - mu) / np.sqrt(((x - mu) ** 2).mean(-1, keepdims=True) + cfg.eps) * inp["gamma"] + inp["beta"]
+    y = (xn @ inp["Wv"] + inp["bv"]) @ inp["Wo"] + inp["bo"] + x
+    assert np.abs(got[:, 0, :] - y).max() <= 1e-2 + 2e-2 * np.abs(y).max()
+
+
+def test_boundary_refuses_bad_arguments_without_touching_the_device():
+    import torch
+    from paper_2607_21624_b200 import LayerRunner
+    from paper_2607_21624_b200.binding import FblError
+    cfg = LayerConfig("e6", 1, 64, 128, 2, 2, 64, "bf16", "layernorm", True, False, False, 1e-5, 46, 0.02)
+    run = LayerRunner(cfg)
+    run.load_inputs(make_inputs(cfg))
+    good = run.buf["X"]
+    # a matrix pointer that is not 1024-byte aligned
+    run.buf["X"] = good[16:]
+    with pytest.raises(FblError):
+        run.forward()
+    run.buf["X"] = good
+    # a required vector missing
+    gamma = run.vec["gamma"]
+    class Null:
+        def data_ptr(self):
+            return None
+    run.vec["gamma"] = Null()
+    with pytest.raises(FblError):
+        run.forward()
+    run.vec["gamma"] = gamma
+    run.step()
+    assert run.status() == 0
+    torch.cuda.synchronize()
+
+
+def test_two_steps_give_identical_bits_except_dq_order():
+    # Everything except the fp32 dQ accumulation (bulk reductions arrive in any order) is order-free; dX, dWq depend
+    # on dQ, so they may differ in the last bf16 bit between runs.  Y, dWo, dgamma of the forward-only chain must not.
+    from paper_2607_21624_b200 import LayerRunner
+    cfg = LayerConfig("e7", 2, 300, 256, 4, 2, 64, "bf16", "layernorm", True, True, True, 1e-5, 47, 0.02)
+    run = LayerRunner(cfg)
+    run.load_inputs(make_inputs(cfg, affine_noise=True))
+    run.step()
+    a = {n: run.fetch(n) for n in ("Y", "dWo", "dbo", "dWv", "dbv")}
+    run.step()
+    for n, v in a.items():
+        assert np.array_equal(v, run.fetch(n)), n
