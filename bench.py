@@ -56,12 +56,23 @@ def step_flops(cfg):
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the step kernels, from the ncu captures
 # summarised under profiles/ (workload 4, and workload 5 at sequence 2048).  Keyed by (workload name, step).
 NCU_TRAFFIC_BYTES = {
-    ("cfg4-llama1b-gqa", "proj_qkv"): 29.4e6 + 0.4e6,
+    # workload 2 (the default): every kernel of a step, profiles/ncu_full_workload2_gpt2small_hd64.md
+    ("cfg2-gpt2-small", "norm_fwd"): 3.2e6 + 0.0e6,
+    ("cfg2-gpt2-small", "proj_qkv"): 6.8e6 + 0.0e6,
+    ("cfg2-gpt2-small", "attn_fwd"): 9.5e6 + 0.0e6,
+    ("cfg2-gpt2-small", "proj_o"): 4.4e6 + 0.0e6,
+    ("cfg2-gpt2-small", "dWo+dA"): 7.5e6 + 0.0e6,
+    ("cfg2-gpt2-small", "attn_bwd"): 19.1e6 + 0.3e6 + 6.3e6,      # main kernel + rounding of the fp32 dQ
+    ("cfg2-gpt2-small", "dWqkv+dXn"): 16.2e6 + 0.0e6,
+    ("cfg2-gpt2-small", "db"): 12.6e6 + 12.5e6 + 0.1e6,           # the write is the previous kernel's dirty lines
+    ("cfg2-gpt2-small", "norm_bwd"): 6.3e6 + 8.2e6 + 1.6e6,
+    # workload 4, profiles/ncu_full_workload4_llama1b_gqa_hd64.md
+    ("cfg4-llama1b-gqa", "proj_qkv"): 29.4e6 + 0.3e6,
     ("cfg4-llama1b-gqa", "attn_fwd"): 25.2e6 + 0.0e6,
     ("cfg4-llama1b-gqa", "proj_o"): 25.2e6 + 0.0e6,
-    ("cfg4-llama1b-gqa", "dWo+dA"): 42.0e6 + 1.9e6,
+    ("cfg4-llama1b-gqa", "dWo+dA"): 42.5e6 + 2.6e6,
     ("cfg4-llama1b-gqa", "attn_bwd"): 76.6e6 + 3.8e6,
-    ("cfg4-llama1b-gqa", "dWqkv+dXn"): 55.9e6 + 11.8e6,
+    ("cfg4-llama1b-gqa", "dWqkv+dXn"): 56.3e6 + 11.7e6,
 }
 
 
