@@ -663,9 +663,13 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
 
     // LSE / D of a query tile: thread t < 128 fetches LSE[t], thread 128 <= t < 256 fetches D[t - 128].  The
     // value for the next iteration is requested one iteration ahead so its latency is off the critical path.
+    // (head, query tile) of the tile being fetched and of the tile being processed advance by counting: an
+    // integer division per thread and iteration is a noticeable share of this loop's instructions
+    int f_h = 0, f_q = 0;                           // fetch position: head within the group, query tile within the head
     auto fetch_stat = [&](int fit) -> float {
+      const int h = g * P.group + f_h, i0 = (qt_begin + f_q) * BQ;
+      if (++f_q == per_head) { f_q = 0; ++f_h; }
       if (t >= 256 || fit >= n_it) return 0.f;
-      const int h = g * P.group + fit / per_head, i0 = (qt_begin + fit % per_head) * BQ;
       const int gi = i0 + (t & 127);
       const long long o = ((long long)b * P.hq + h) * P.t_pad + gi;
       if (gi >= P.seq) return t < 128 ? INFINITY : 0.f;
@@ -673,8 +677,10 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     };
     float stat_next = fetch_stat(0);
 
+    int c_q = 0;                                    // query tile within the head of the tile being processed
     for (int it = 0; it < n_it && ok; ++it) {
-      const int i0 = (qt_begin + it % per_head) * BQ;
+      const int i0 = (qt_begin + c_q) * BQ;
+      if (++c_q == per_head) c_q = 0;
       // LSE and D of this query tile, staged in shared memory (two buffers by iteration parity: every
       // reader of a buffer's previous use arrived at PDSFULL two iterations ago).  All threads pass this
       // barrier only after finishing the previous iteration, including its reads of the dQ staging tile.
