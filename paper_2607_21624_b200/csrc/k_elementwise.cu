@@ -277,46 +277,62 @@ __global__ void __launch_bounds__(256, 2) norm_fwd_rows_kernel(const __nv_bfloat
     bt[j][0] = b0.x; bt[j][1] = b0.y; bt[j][2] = b0.z; bt[j][3] = b0.w; bt[j][4] = b1.x; bt[j][5] = b1.y; bt[j][6] = b1.z; bt[j][7] = b1.w;
   }
   pdl_wait();
-  const int64_t stride = (int64_t)gridDim.x * RPB;
+  // Each block owns a contiguous range of rows and walks it in order: the PF rows in flight are then neighbours,
+  // i.e. in every 64-column panel PF adjacent 128-byte pieces (with a grid-stride walk every piece stood alone).
+  constexpr int64_t stride = RPB;
+  const int64_t per_block = ((n_pad + gridDim.x - 1) / gridDim.x + RPB - 1) / RPB * RPB;
+  const int64_t r_end = min(n_pad, ((int64_t)blockIdx.x + 1) * per_block);
   // lane's vectors of a row: vector index v -> panel v / 8, chunk v % 8
   auto vec_off = [&](int j, int64_t r) {
     const int v = (part * NV + j) * 32 + lane;
     return ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8;
   };
-  int64_t r = (int64_t)blockIdx.x * RPB + slot;
-  uint4 nxt[NV];                                     // the next row is requested before this one is reduced
-  if (r < n_pad) {
+  // PF rows ahead are in flight per warp (raw vectors in registers): with one row ahead a block waited ~1.4 us
+  // per row on the load of the next one; HBM needs about 10 MB in flight across the GPU
+  constexpr int PF = NV == 3 ? 3 : 4;
+  int64_t r = (int64_t)blockIdx.x * per_block + slot;
+  uint4 ring[PF][NV];
 #pragma unroll
-    for (int j = 0; j < NV; ++j) nxt[j] = *reinterpret_cast<const uint4*>(X + vec_off(j, r));
+  for (int k = 0; k < PF; ++k) {
+    if (r + k * stride < r_end) {
+#pragma unroll
+      for (int j = 0; j < NV; ++j) ring[k][j] = *reinterpret_cast<const uint4*>(X + vec_off(j, r + k * stride));
+    }
   }
-  for (; r < n_pad; r += stride) {
-    const bool pad = (int)(r % t_pad) >= seq;
-    float x[NV][8];
-    float s = 0.f;
+  bool more = r < r_end;
+  while (more) {
 #pragma unroll
-    for (int j = 0; j < NV; ++j) {
-      const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&nxt[j]);
+    for (int k = 0; k < PF; ++k) {
+      if (r >= r_end) { more = false; break; }
+      const bool pad = (int)(r % t_pad) >= seq;
+      float x[NV][8];
+      float s = 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { x[j][i] = __bfloat162float(e[i]); s += x[j][i]; }
-    }
-    if (r + stride < n_pad) {
+      for (int j = 0; j < NV; ++j) {
+        const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&ring[k][j]);
 #pragma unroll
-      for (int j = 0; j < NV; ++j) nxt[j] = *reinterpret_cast<const uint4*>(X + vec_off(j, r + stride));
-    }
-    const float mean = rms ? 0.f : row_sum<WPR>(s, s_part, slot, part, buf) * (1.f / D);
-    float q = 0.f;
+        for (int i = 0; i < 8; ++i) { x[j][i] = __bfloat162float(e[i]); s += x[j][i]; }
+      }
+      if (r + PF * stride < r_end) {
 #pragma unroll
-    for (int j = 0; j < NV; ++j)
+        for (int j = 0; j < NV; ++j) ring[k][j] = *reinterpret_cast<const uint4*>(X + vec_off(j, r + PF * stride));
+      }
+      const float mean = rms ? 0.f : row_sum<WPR>(s, s_part, slot, part, buf) * (1.f / D);
+      float q = 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { const float c = x[j][i] - mean; q += c * c; }
-    const float rstd = rsqrtf(row_sum<WPR>(q, s_part, slot, part, buf) * (1.f / D) + eps);
-    if (lane == 0 && part == 0) { stats[2 * r] = pad ? 0.f : mean; stats[2 * r + 1] = pad ? 0.f : rstd; }
+      for (int j = 0; j < NV; ++j)
 #pragma unroll
-    for (int j = 0; j < NV; ++j) {
-      float y[8];
+        for (int i = 0; i < 8; ++i) { const float c = x[j][i] - mean; q += c * c; }
+      const float rstd = rsqrtf(row_sum<WPR>(q, s_part, slot, part, buf) * (1.f / D) + eps);
+      if (lane == 0 && part == 0) { stats[2 * r] = pad ? 0.f : mean; stats[2 * r + 1] = pad ? 0.f : rstd; }
 #pragma unroll
-      for (int i = 0; i < 8; ++i) y[i] = pad ? 0.f : (x[j][i] - mean) * rstd * gm[j][i] + bt[j][i];
-      store16(Xn + vec_off(j, r), y);
+      for (int j = 0; j < NV; ++j) {
+        float y[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) y[i] = pad ? 0.f : (x[j][i] - mean) * rstd * gm[j][i] + bt[j][i];
+        store16(Xn + vec_off(j, r), y);
+      }
+      r += stride;
     }
   }
 }
@@ -355,7 +371,10 @@ __global__ void __launch_bounds__(256, 2) norm_bwd_rows_kernel(const __nv_bfloat
   for (int j = 0; j < NV; ++j)
 #pragma unroll
     for (int i = 0; i < 8; ++i) { ag[j][i] = 0.f; ab[j][i] = 0.f; }
-  for (int64_t r = (int64_t)blockIdx.x * RPB + slot; r < n_pad; r += (int64_t)gridDim.x * RPB) {
+  // each block owns a contiguous range of rows (neighbouring 128-byte pieces in every panel)
+  const int64_t per_block = ((n_pad + gridDim.x - 1) / gridDim.x + RPB - 1) / RPB * RPB;
+  const int64_t r_end = min(n_pad, ((int64_t)blockIdx.x + 1) * per_block);
+  for (int64_t r = (int64_t)blockIdx.x * per_block + slot; r < r_end; r += RPB) {
     const float mean = stats[2 * r], rstd = stats[2 * r + 1];
     float xh[NV][8], g[NV][8];
     float s1 = 0.f, s2 = 0.f;
