@@ -3,6 +3,7 @@
 // each operand is declared K-major or MN-major in the descriptors, so W / W^T and X / X^T are the same
 // tiles in HBM and in shared memory.  Up to three reduction loops feed one accumulator (dXn), and up
 // to four problems share one persistent launch (Q/K/V projections; dWo with dA; dWq/dWk/dWv with dXn).
+#include <stdlib.h>
 #include <string.h>
 
 #include <mutex>
@@ -394,6 +395,279 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
   if (warp == 1) tc::tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
+// ---------------------------------------------------------------------------------------------------
+// CTA-pair variant (tcgen05 cta_group::2): two SMs share a 256 x 256 output tile.  Each CTA loads its 128 rows of
+// A and its 128 columns of B (32 KB per k-block instead of 48 KB for a 128 x 256 tile of its own: operand
+// delivery from L2, about 64 B/clk per SM, is what bounds the single-CTA kernel), the leader (cluster rank 0)
+// issues MMAs of M = 256, N = 256 that read both CTAs' shared memory and write 128 accumulator rows into each
+// CTA's tensor memory, and each CTA drains its own rows.  Barriers: full[] lives in the leader and counts the
+// bytes of both CTAs' loads; empty[] and acc_full[] exist in both and get their arrivals from one commit that
+// signals both CTAs; acc_empty[] lives in the leader and takes the arrivals of both CTAs' epilogue threads.
+// ---------------------------------------------------------------------------------------------------
+constexpr int PAIR_BN = 256, PAIR_STAGES = 6;
+struct PairSmem {
+  static constexpr uint32_t A_BYTES = 128 * 128, B_BYTES = 128 * 128, STAGE = A_BYTES + B_BYTES;
+  static constexpr uint32_t STG_OFF = PAIR_STAGES * STAGE;
+  static constexpr uint32_t BAR_OFF = STG_OFF + 2 * 16384;
+  static constexpr uint32_t N_BARS = 2 * PAIR_STAGES + 4;
+  static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16 + 1024;
+};
+
+// work list in 256 x 256 tiles (ksplit slices as in tile_at); m0 / n0 are the pair's
+__device__ __forceinline__ bool pair_tile_at(const TcGroup& G, int w, TileCoord* tc_out) {
+  for (int p = 0; p < G.count; ++p) {
+    const TcProblem& P = G.p[p];
+    const int tm = (P.m + 255) / 256, tn = (P.n + 255) / 256;
+    const int units = tm * tn * P.ksplit;
+    if (w < units) {
+      const int slice = w % P.ksplit, t = w / P.ksplit;
+      tc_out->prob = p;
+      tc_out->m0 = (t % tm) * 256;
+      tc_out->n0 = (t / tm) * 256;
+      const int per = (P.kblocks[0] + P.ksplit - 1) / P.ksplit;
+      tc_out->kb0 = slice * per;
+      tc_out->kb1 = min(P.kblocks[0], (slice + 1) * per);
+      return true;
+    }
+    w -= units;
+  }
+  return false;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1) gemm_tc_pair_kernel(const __grid_constant__ TcGroup G) {
+  using SP = PairSmem;
+  constexpr int STAGES = PAIR_STAGES, BN = PAIR_BN;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = base + SP::BAR_OFF;
+  auto full = [&](int s) { return bars + 8u * s; };
+  auto empty = [&](int s) { return bars + 8u * (STAGES + s); };
+  auto acc_full = [&](int a) { return bars + 8u * (2 * STAGES + a); };
+  auto acc_empty = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
+  const uint32_t slot = bars + 8 * SP::N_BARS;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const uint32_t rank = tc::cluster_ctarank();
+  const int pair_id = blockIdx.x / 2, n_pairs = gridDim.x / 2;
+  int32_t* status = G.status;
+  constexpr uint32_t TMEM_COLS = 2 * BN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      tc::mbar_init(full(s), 1);                 // leader: its producer's arrival + both CTAs' transaction bytes
+      tc::mbar_init(empty(s), 1);                // one commit arrival (sent to both CTAs)
+    }
+    for (int a = 0; a < 2; ++a) {
+      tc::mbar_init(acc_full(a), 1);
+      tc::mbar_init(acc_empty(a), 256);          // leader: the epilogue threads of both CTAs
+    }
+    tc::fence_barrier_init();
+  }
+  if (warp == 1) {
+    tc::tmem_alloc2(slot, TMEM_COLS);
+    tc::tmem_relinquish2();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::cluster_sync_all();                        // the peer's barriers exist before anything signals them
+  tc::tc_fence_after();
+  uint32_t tmem_base;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
+  pdl_launch_dependents();
+
+  if (warp == 0 && lane == 0) {
+    // ---- TMA producer (both CTAs): own A rows, own half of B's columns; bytes counted on the leader's barrier ----
+    int it = 0;
+    bool ok = true;
+    TileCoord tcd;
+    pdl_wait();
+    for (int w = pair_id; ok && pair_tile_at(G, w, &tcd); w += n_pairs) {
+      const TcProblem& P = G.p[tcd.prob];
+      const int m0 = tcd.m0 + (int)rank * 128, n0 = tcd.n0 + (int)rank * 128;
+      for (int t = 0; t < P.n_terms && ok; ++t) {
+        const int kb_begin = t == 0 ? tcd.kb0 : 0, kb_end = t == 0 ? tcd.kb1 : P.kblocks[t];
+        for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          const uint32_t sa = base + s * SP::STAGE, sb = sa + SP::A_BYTES;
+          if (!tc::mbar_wait(empty(s), ph ^ 1, status, 111)) { ok = false; break; }
+          if (rank == 0) tc::mbar_expect_tx(full(s), 2 * SP::STAGE);
+          const uint32_t fb = tc::map_to_cta(full(s), 0);
+          if (P.a_mn[t]) tc::tma_load_3d_pair(sa, &P.ta[t], fb, 0, kb * BK, m0 / 64);
+          else tc::tma_load_3d_pair(sa, &P.ta[t], fb, 0, m0, kb);
+          if (P.b_mn[t]) tc::tma_load_3d_pair(sb, &P.tb[t], fb, 0, kb * BK, n0 / 64);
+          else tc::tma_load_3d_pair(sb, &P.tb[t], fb, 0, n0, kb);
+        }
+      }
+    }
+  } else if (warp == 1 && lane == 0 && rank == 0) {
+    // ---- MMA issuer (leader only) --------------------------------------------------------------
+    int s = 0, ti = 0;
+    uint32_t ph = 0;
+    bool ok = true;
+    TileCoord tcd;
+    const uint32_t hi = tc::smem_desc_hi(1024);
+    for (int w = pair_id; ok && pair_tile_at(G, w, &tcd); w += n_pairs, ++ti) {
+      const TcProblem& P = G.p[tcd.prob];
+      const int ab = ti & 1;
+      if (!tc::mbar_wait(acc_empty(ab), ((ti >> 1) & 1) ^ 1, status, 114)) { ok = false; break; }
+      tc::tc_fence_after();
+      const uint32_t d_tmem = tmem_base + ab * BN;
+      uint32_t acc = 0;
+      for (int t = 0; t < P.n_terms && ok; ++t) {
+        const uint32_t idesc = tc::idesc_bf16(256, BN, P.a_mn[t], P.b_mn[t]);
+        const uint32_t a_lo0 = tc::smem_desc_lo(base, P.a_mn[t] ? 8192u : 16u), a_step = P.a_mn[t] ? 128u : 2u;
+        const uint32_t b_lo0 = tc::smem_desc_lo(base + SP::A_BYTES, P.b_mn[t] ? 8192u : 16u), b_step = P.b_mn[t] ? 128u : 2u;
+        const int nkb = t == 0 ? tcd.kb1 - tcd.kb0 : P.kblocks[t];
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!tc::mbar_wait(full(s), ph, status, 112)) { ok = false; break; }
+          tc::tc_fence_after();
+          uint32_t a_lo = a_lo0 + (uint32_t)s * (SP::STAGE >> 4), b_lo = b_lo0 + (uint32_t)s * (SP::STAGE >> 4);
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            tc::mma_bf16_ss_w2(d_tmem, a_lo, hi, b_lo, hi, idesc, acc);
+            acc = 1;
+            a_lo += a_step; b_lo += b_step;
+          }
+          tc::mma_commit2_both(empty(s));        // frees the stage in both CTAs once these MMAs have read it
+          if (++s == STAGES) { s = 0; ph ^= 1; }
+        }
+      }
+      if (ok) tc::mma_commit2_both(acc_full(ab));
+    }
+  } else if (warp >= 2) {
+    // ---- epilogue (both CTAs): this CTA's 128 accumulator rows, as in the single-CTA kernel -------------
+    pdl_wait();
+    const int q = warp % 4;
+    const int r = q * 32 + lane;
+    int ti = 0, pc = 0;
+    bool ok = true;
+    TileCoord tcd;
+    for (int w = pair_id; ok && pair_tile_at(G, w, &tcd); w += n_pairs, ++ti) {
+      const TcProblem& P = G.p[tcd.prob];
+      const int ab = ti & 1;
+      const int m0 = tcd.m0 + (int)rank * 128;
+      const int row = m0 + r;
+      const bool pad = P.t_pad > 0 && (row % P.t_pad) >= P.seq;
+      const bool has_res = P.residual && row < P.m;
+      uint4 rv[8];
+      if (has_res) {
+        const __nv_bfloat16* rp = P.residual + ((long long)(tcd.n0 / 64) * P.c_rpad + row) * 64;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) rv[j] = *reinterpret_cast<const uint4*>(rp + 8 * j);
+      }
+      const float* bias = P.bias;
+      float bl[BN / 32];
+      if (bias) {
+#pragma unroll
+        for (int k = 0; k < BN / 32; ++k) {
+          const int c = tcd.n0 + lane * (BN / 32) + k;
+          bl[k] = c < P.n ? bias[c] : 0.f;
+        }
+      }
+      if (!tc::mbar_wait(acc_full(ab), (ti >> 1) & 1, status, 113)) { ok = false; break; }
+      tc::tc_fence_after();
+      float dot_acc = 0.f;
+#pragma unroll 1
+      for (int pn = 0; pn < BN / 64; ++pn) {
+        const int n = tcd.n0 + pn * 64;
+        if (n >= P.n) break;
+        uint32_t v[64];
+        tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + pn * 64, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+        tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + pn * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+        tc::tmem_ld_wait();
+        if (P.ksplit > 1) {
+#pragma unroll 1
+          for (int hf = 0; hf < 2; ++hf) {
+            const uint32_t stg = base + SP::STG_OFF + (uint32_t)(q * 2 + (pc & 1)) * 4096u;
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + (((uint32_t)j ^ (uint32_t)(lane & 7)) * 16)),
+                           "r"(hf ? v[32 + 4 * j] : v[4 * j]), "r"(hf ? v[33 + 4 * j] : v[4 * j + 1]),
+                           "r"(hf ? v[34 + 4 * j] : v[4 * j + 2]), "r"(hf ? v[35 + 4 * j] : v[4 * j + 3]) : "memory");
+            tc::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tc::tma_reduce_add_4d(&P.tacc, stg, 0, hf, m0 + q * 32, n / 64);
+              tc::bulk_commit_group();
+              tc::bulk_wait_group_read1();
+            }
+            ++pc;
+          }
+          continue;
+        }
+        uint4 outv[8];
+        uint32_t* ow = reinterpret_cast<uint32_t*>(outv);
+        if (has_res) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const __nv_bfloat16* rb = reinterpret_cast<const __nv_bfloat16*>(&rv[j]);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v[8 * j + k] = __float_as_uint(__uint_as_float(v[8 * j + k]) + __bfloat162float(rb[k]));
+          }
+          if (pn + 1 < BN / 64 && n + 64 < P.n) {
+            const __nv_bfloat16* rp = P.residual + ((long long)(n / 64 + 1) * P.c_rpad + row) * 64;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) rv[j] = *reinterpret_cast<const uint4*>(rp + 8 * j);
+          }
+        }
+        if (bias) {
+#pragma unroll
+          for (int j = 0; j < 64; j += 2) {
+            const float b0 = __shfl_sync(0xffffffffu, bl[j % (BN / 32)], (pn * 64 + j) / (BN / 32));
+            const float b1 = __shfl_sync(0xffffffffu, bl[(j + 1) % (BN / 32)], (pn * 64 + j + 1) / (BN / 32));
+            ow[j / 2] = tc::pack_bf16(pad ? 0.f : __uint_as_float(v[j]) + b0, pad ? 0.f : __uint_as_float(v[j + 1]) + b1);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 64; j += 2)
+            ow[j / 2] = tc::pack_bf16(pad ? 0.f : __uint_as_float(v[j]), pad ? 0.f : __uint_as_float(v[j + 1]));
+        }
+        if (P.dot_with && row < P.m) {
+          const __nv_bfloat16* ap = P.dot_with + ((long long)(n / 64) * P.c_rpad + row) * 64;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint4 av = *reinterpret_cast<const uint4*>(ap + 8 * j);
+            const __nv_bfloat16* ab16 = reinterpret_cast<const __nv_bfloat16*>(&av);
+#pragma unroll
+            for (int k = 0; k < 8; k += 2) {
+              const uint32_t w2 = ow[4 * j + k / 2];
+              dot_acc = fmaf(__uint_as_float(w2 << 16), __bfloat162float(ab16[k]), dot_acc);
+              dot_acc = fmaf(__uint_as_float(w2 & 0xffff0000u), __bfloat162float(ab16[k + 1]), dot_acc);
+            }
+          }
+          if ((n + 64) % P.dot_hd == 0) {
+            const int hh = n / P.dot_hd, bb = row / P.t_pad, tt = row % P.t_pad;
+            P.dot_out[((long long)bb * P.dot_hq + hh) * P.t_pad + tt] = dot_acc;
+            dot_acc = 0.f;
+          }
+        }
+        const uint32_t stg = base + SP::STG_OFF + (uint32_t)(q * 2 + (pc & 1)) * 4096u;
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + (((uint32_t)j ^ (uint32_t)(lane & 7)) * 16)),
+                       "r"(outv[j].x), "r"(outv[j].y), "r"(outv[j].z), "r"(outv[j].w) : "memory");
+        tc::fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          tc::tma_store_3d(&P.tc, stg, 0, m0 + q * 32, n / 64);
+          tc::bulk_commit_group();
+          tc::bulk_wait_group_read1();
+        }
+        ++pc;
+      }
+      tc::tc_fence_before();
+      tc::mbar_arrive_cluster(tc::map_to_cta(acc_empty(ab), 0));     // the leader's barrier, from either CTA
+    }
+    if (lane == 0) tc::bulk_wait_group0();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::cluster_sync_all();                        // neither CTA frees tensor memory or leaves while its peer may still
+  if (warp == 1) tc::tmem_dealloc2(tmem_base, TMEM_COLS);   // read its shared memory or signal its barriers
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -511,6 +785,56 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
   return launch_pdl(k, dim3(grid), dim3(192), SP::TOTAL, st, G);
 }
 
+cudaError_t launch_group_pair(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
+  TcGroup G;
+  memset(&G, 0, sizeof(G));
+  G.count = count;
+  G.status = status;
+#ifdef FBL_TRACE_GEMM
+  G.trace_slot = (g_trace_launch++) & 1;      // two GEMM launches per pass
+#endif
+  int tiles = 0;
+  for (int i = 0; i < count; ++i) {
+    const GemmArgs& g = gs[i];
+    TcProblem& P = G.p[i];
+    P.n_terms = g.n_terms;
+    for (int t = 0; t < g.n_terms; ++t) {
+      const GemmTerm& tm = g.t[t];
+      P.kblocks[t] = (tm.k + BK - 1) / BK;
+      P.a_mn[t] = tm.a_trans ? 1 : 0;     // stored [k rows][m cols]: rows are K indices
+      P.b_mn[t] = tm.b_trans ? 0 : 1;     // stored [k rows][n cols]: rows are K indices
+      bool ok;
+      if (tm.a_trans) ok = fbl_encode_rtile_map(&P.ta[t], tm.a, tm.a_rpad, g.m / 64, BK, BM / 64);
+      else ok = fbl_encode_rtile_map(&P.ta[t], tm.a, tm.a_rpad, tm.k / 64, BM, 1);
+      if (!ok) return cudaErrorInvalidValue;
+      if (tm.b_trans) ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, tm.k / 64, 128, 1);
+      else ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, g.n / 64, BK, 2);
+      if (!ok) return cudaErrorInvalidValue;
+    }
+    P.m = g.m; P.n = g.n;
+    if (!fbl_encode_rtile_map(&P.tc, g.c, g.c_rpad, g.n / 64, 32, 1)) return cudaErrorInvalidValue;   // one warp's rows
+    P.b_static = g.b_static;
+    P.c = (__nv_bfloat16*)g.c; P.c_rpad = g.c_rpad;
+    P.bias = g.bias; P.residual = (const __nv_bfloat16*)g.residual;
+    P.seq = g.seq; P.t_pad = g.t_pad;
+    P.dot_with = (const __nv_bfloat16*)g.dot_with; P.dot_out = g.dot_out; P.dot_hd = g.dot_hd; P.dot_hq = g.dot_hq;
+    P.ksplit = 1;
+    if (g.ksplit > 1) {
+      if (g.n_terms != 1 || g.bias || g.residual || g.dot_with || g.t_pad > 0 || !g.acc) return cudaErrorInvalidValue;
+      const int per = (P.kblocks[0] + g.ksplit - 1) / g.ksplit;        // no empty slice
+      P.ksplit = (P.kblocks[0] + per - 1) / per;
+      if (!fbl_encode_f32_panel_map(&P.tacc, g.acc, g.c_rpad, g.n / 64, 32, 1)) return cudaErrorInvalidValue;
+    }
+    tiles += ((g.m + 255) / 256) * ((g.n + 255) / 256) * P.ksplit;
+  }
+  using SP = PairSmem;
+  auto k = gemm_tc_pair_kernel;
+  cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
+  if (attr_err != cudaSuccess) return attr_err;
+  const int pairs = tiles < p->sm_count / 2 ? tiles : p->sm_count / 2;
+  return launch_pdl(k, dim3(2 * pairs), dim3(192), SP::TOTAL, st, G);
+}
+
 cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
   if (count < 1 || count > MAX_PROBLEMS) return cudaErrorInvalidValue;
   bool wide = true;                       // 128 x 256 tiles when every problem's N is whole 256-column blocks
@@ -521,8 +845,19 @@ cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int coun
       if (gs[i].t[t].b_trans && gs[i].t[t].b_rpad < 256) wide = false;
     tiles_wide += ((gs[i].m + BM - 1) / BM) * ((gs[i].n + 255) / 256) * (gs[i].ksplit > 1 ? gs[i].ksplit : 1);
   }
+  const bool wide_legal = wide;
   // with too few wide tiles to occupy the SMs, narrower tiles (twice as many) finish sooner
   if (wide && tiles_wide * 3 < p->sm_count * 2) wide = false;
+  // CTA pairs on 256 x 256 tiles for large problems (several rounds of tiles per SM pair): measured 2-6 % faster
+  // on the workload 5 GEMMs, no gain or a loss below that
+  const int pair_mode = getenv("FBL_GEMM_PAIR") ? atoi(getenv("FBL_GEMM_PAIR")) : -1;   // tuning knob: 0 never, 1 whenever legal
+  if (pair_mode == 1 && wide_legal) return launch_group_pair(p, gs, count, status, st);
+  if (wide && pair_mode != 0) {
+    long long pair_tiles = 0;
+    for (int i = 0; i < count; ++i)
+      pair_tiles += (long long)((gs[i].m + 255) / 256) * (gs[i].n / 256) * (gs[i].ksplit > 1 ? gs[i].ksplit : 1);
+    if (pair_tiles >= 4 * (p->sm_count / 2)) return launch_group_pair(p, gs, count, status, st);
+  }
   if (wide) return launch_group_bn<256, 4>(p, gs, count, status, st);
   return launch_group_bn<128, 6>(p, gs, count, status, st);
 }

@@ -96,6 +96,17 @@ def test_sliced_weight_gradient_reductions(slices, monkeypatch):
                     affine_noise=True)
 
 
+@pytest.mark.parametrize("cfg", [c for c in SMALL_BF16 if c.name in ("b1", "b4", "b8")] + [
+    LayerConfig("p1", 3, 333, 512, 8, 4, 64, "bf16", "layernorm", True, True, True, 1e-5, 33, 0.02)], ids=lambda c: c.name)
+def test_cta_pair_gemm_forced(cfg, monkeypatch):
+    # Large layers run their GEMMs on CTA pairs (256 x 256 tiles, tcgen05 cta_group::2); workload 5 covers that at
+    # full size.  The knob forces the pair kernel wherever its tile shape is legal, so that bias, residual, padding
+    # rows, the fused row reduction, odd tile counts and tiles whose second half lies beyond the matrix are
+    # compared at small sizes too.
+    monkeypatch.setenv("FBL_GEMM_PAIR", "1")
+    run_and_compare(cfg, affine_noise=True)
+
+
 @pytest.mark.parametrize("i", [2, 3])
 def test_full_configs_2_and_3(i):
     run_and_compare(get_config(i))
