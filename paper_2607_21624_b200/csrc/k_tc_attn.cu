@@ -476,11 +476,23 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
     for (int it = 0; it < n_it; ++it) {
       const int h = g * P.group + it / per_head, qt = qt_begin + it % per_head;
-      const uint32_t s = it % NQ, ph = (it / NQ) & 1;
-      if (!tc::mbar_wait(bar(BB_QDOEMPTY + s), ph ^ 1, status, 301)) break;
-      tc::mbar_expect_tx(bar(BB_QDOFULL + s), 2 * SM::TILE);
-      tc::tma_load_3d(base + SM::Q_OFF + s * SM::TILE, &P.tq, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
-      tc::tma_load_3d(base + SM::DO_OFF + s * SM::TILE, &P.tdo, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
+      if (PIPE) {
+        const uint32_t s = it % NQ, ph = (it / NQ) & 1;
+        if (!tc::mbar_wait(bar(BB_QDOEMPTY + s), ph ^ 1, status, 301)) break;
+        tc::mbar_expect_tx(bar(BB_QDOFULL + s), 2 * SM::TILE);
+        tc::tma_load_3d(base + SM::Q_OFF + s * SM::TILE, &P.tq, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
+        tc::tma_load_3d(base + SM::DO_OFF + s * SM::TILE, &P.tdo, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
+      } else {
+        // single buffers: Q and dO have a barrier pair each (slot 0: Q, slot 1: dO), since Q is free after the dK
+        // product and dO only after the dV product, and the next score tile needs Q alone
+        const uint32_t ph = it & 1;
+        if (!tc::mbar_wait(bar(BB_QDOEMPTY), ph ^ 1, status, 301)) break;
+        tc::mbar_expect_tx(bar(BB_QDOFULL), SM::TILE);
+        tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(BB_QDOFULL), 0, row0 + qt * BQ, h * (int)PANELS);
+        if (!tc::mbar_wait(bar(BB_QDOEMPTY + 1), ph ^ 1, status, 313)) break;
+        tc::mbar_expect_tx(bar(BB_QDOFULL + 1), SM::TILE);
+        tc::tma_load_3d(base + SM::DO_OFF, &P.tdo, bar(BB_QDOFULL + 1), 0, row0 + qt * BQ, h * (int)PANELS);
+      }
     }
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer --------------------------------------------------------------------------
@@ -539,6 +551,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     bool ok = tc::mbar_wait(bar(BB_KVFULL), 0, status, 302);
     if (ok && n_it > 0) {
       ok = tc::mbar_wait(bar(BB_QDOFULL), 0, status, 303);
+      if (ok && !PIPE) ok = tc::mbar_wait(bar(BB_QDOFULL + 1), 0, status, 314);
       if (ok) { tc::tc_fence_after(); issue_s(0); issue_dp(0); }
     }
     if (PIPE) {
@@ -581,8 +594,9 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         // the dV and dK products
         issue_dq(it);
         issue_dk(it);
-        issue_dv(it);
-        tc::mma_commit(bar(BB_QDOEMPTY));               // Q / dO of this tile are not read again
+        tc::mma_commit(bar(BB_QDOEMPTY));               // Q of this tile is not read again: the next one is fetched
+        issue_dv(it);                                   // while dV runs
+        tc::mma_commit(bar(BB_QDOEMPTY + 1));           // ... and dO
         TR(2);
         if (it + 1 < n_it) {
           if (!tc::mbar_wait(bar(BB_QDOFULL), (it + 1) & 1, status, 303)) { ok = false; break; }
@@ -590,6 +604,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
           tc::tc_fence_after();
           issue_s(it + 1);                   // the S^T columns (P^T by now) were last read by dV above
           if (!tc::mbar_wait(bar(BB_DQDRAINED), it & 1, status, 304)) { ok = false; break; }
+          if (!tc::mbar_wait(bar(BB_QDOFULL + 1), (it + 1) & 1, status, 314)) { ok = false; break; }
           TR(4);
           tc::tc_fence_after();
           issue_dp(it + 1);                  // the dP^T columns held dQ until it was drained
