@@ -681,14 +681,17 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     // (head, query tile) of the tile being fetched and of the tile being processed advance by counting: an
     // integer division per thread and iteration is a noticeable share of this loop's instructions
     int f_h = 0, f_q = 0;                           // fetch position: head within the group, query tile within the head
+    // The value is used (scaled, stored to shared memory) only at the top of the next iteration: nothing here may
+    // depend on the load, or the thread would wait out its L2 latency before reaching the barrier below.
+    bool stat_oob = false;
     auto fetch_stat = [&](int fit) -> float {
       const int h = g * P.group + f_h, i0 = (qt_begin + f_q) * BQ;
       if (++f_q == per_head) { f_q = 0; ++f_h; }
-      if (t >= 256 || fit >= n_it) return 0.f;
       const int gi = i0 + (t & 127);
+      stat_oob = t >= 256 || fit >= n_it || gi >= P.seq;
+      if (stat_oob) return 0.f;
       const long long o = ((long long)b * P.hq + h) * P.t_pad + gi;
-      if (gi >= P.seq) return t < 128 ? INFINITY : 0.f;
-      return t < 128 ? P.lse[o] * LOG2E : P.dvec[o];
+      return __ldg((t < 128 ? P.lse : P.dvec) + o);
     };
     float stat_next = fetch_stat(0);
 
@@ -701,7 +704,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       // barrier only after finishing the previous iteration, including its reads of the dQ staging tile.
       float* s_lse = s_stage + (it & 1) * 256;
       float* s_d = s_lse + 128;
-      if (t < 256) s_lse[t] = stat_next;             // s_d follows s_lse: one 256-float buffer
+      if (t < 256) s_lse[t] = t < 128 ? (stat_oob ? INFINITY : stat_next * LOG2E) : (stat_oob ? 0.f : stat_next);   // s_d follows s_lse
       stat_next = fetch_stat(it + 1);
       tc::mbar_arrive(bar(BB_LSEREADY));
       if (!tc::mbar_wait(bar(BB_LSEREADY), it & 1, status, 308)) { ok = false; break; }
