@@ -64,31 +64,34 @@ struct alignas(64) AttnFwdParams {
   int32_t* status;
 };
 
-template <int HD>
+template <int HD, int TILES>
 struct FwdSmem {
   static constexpr uint32_t PANELS = HD / 64;
   static constexpr uint32_t TILE = PANELS * 16384;          // 128 rows x HD bf16
-  static constexpr uint32_t Q_OFF = 0;                      // 2 query tiles
-  static constexpr uint32_t K_OFF = 2 * TILE;               // 2 stages
-  static constexpr uint32_t V_OFF = 4 * TILE;               // 2 stages
-  static constexpr uint32_t BAR_OFF = 6 * TILE;
+  static constexpr uint32_t Q_OFF = 0;                      // TILES query tiles
+  static constexpr uint32_t K_OFF = TILES * TILE;           // 2 stages
+  static constexpr uint32_t V_OFF = (TILES + 2) * TILE;     // 2 stages
+  static constexpr uint32_t BAR_OFF = (TILES + 4) * TILE;
   static constexpr uint32_t N_BARS = 16;
   static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16;
 };
 
 enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_PVDONE = 13 };
 
-constexpr int FWD_THREADS = 320;      // warp 0 TMA, warp 1 MMA, warps 2-5 and 6-9: one softmax warp group per query tile
+// warp 0 TMA, warp 1 MMA, then one softmax warp group (4 warps) per query tile of the block.  TILES = 2: two
+// adjacent query tiles share the K/V tiles, one block per SM.  TILES = 1 (head_dim 64 only: its tiles leave room): a
+// block of 192 threads with one query tile, half the tensor memory and at most 128 registers per thread, so that two
+// blocks share an SM and one's set-up and epilogue overlap the other's key loop (short sequences are mostly that).
 
 // A row's running max is only raised (and O rescaled) when the new max exceeds it by more than this many
 // powers of two; until then the probabilities are computed against the stale max and stay below 2^8.
 constexpr float RESCALE_LOG2 = 8.f;
 
-template <int HD>
-__global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __grid_constant__ AttnFwdParams P) {
-  using SM = FwdSmem<HD>;
+template <int HD, int TILES>
+__global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd_tc_kernel(const __grid_constant__ AttnFwdParams P) {
+  using SM = FwdSmem<HD, TILES>;
   constexpr uint32_t PANELS = SM::PANELS;
-  constexpr uint32_t O_COL = 256, TMEM_COLS = 512;          // S of tile g at 128 g, O of tile g at 256 + HD g
+  constexpr uint32_t O_COL = 128 * TILES, TMEM_COLS = 256 * TILES;   // S of tile g at 128 g, O of tile g at O_COL + HD g
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = tc::smem_u32(smem_raw);
   const uint32_t bars = base + SM::BAR_OFF;
@@ -104,8 +107,9 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __gri
   // with pairing a block owns two adjacent tiles, whose key ranges differ by one tile, so both warp groups stay
   // busy for the whole loop
   const int slot_x = P.n_slots - 1 - slot_i;                 // heaviest (latest) causal tiles first
-  const int qt0 = P.pair ? min(2 * slot_x + 1, n_qt - 1) : slot_x;
-  const int qt1 = (P.pair && 2 * slot_x + 1 < n_qt) ? 2 * slot_x : -1;   // odd tile count: the last block has one tile
+  const bool pair = TILES == 2 && P.pair;
+  const int qt0 = pair ? min(2 * slot_x + 1, n_qt - 1) : slot_x;
+  const int qt1 = (pair && 2 * slot_x + 1 < n_qt) ? 2 * slot_x : -1;   // odd tile count: the last block has one tile
   auto kv_tiles = [&](int t) {
     const int kv_end = t < 0 ? 0 : (P.causal ? min(P.seq, (t + 1) * BQ) : P.seq);
     return (kv_end + BKV - 1) / BKV;
@@ -194,7 +198,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __gri
     if (ok) {
       tc::tc_fence_after();
       if (n_kv0 > 0) issue_s(0, 0);
-      if (n_kv1 > 0) issue_s(1, 0);
+      if (TILES == 2 && n_kv1 > 0) issue_s(1, 0);
     }
     for (int j = 0; j < n_kv_max && ok; ++j) {
       const bool next = j + 1 < n_kv_max;
@@ -202,7 +206,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __gri
       if (!tc::mbar_wait(bar(B_VFULL + (j & 1)), (j >> 1) & 1, status, 207)) { ok = false; break; }
       if (next && !tc::mbar_wait(bar(B_KFULL + ((j + 1) & 1)), ((j + 1) >> 1) & 1, status, 205)) { ok = false; break; }
 #pragma unroll
-      for (int w = 0; w < 2; ++w) {
+      for (int w = 0; w < TILES; ++w) {
         const int nk = w ? n_kv1 : n_kv0;
         if (ok && j < nk) {
           { const int it = j; TR(1 + 3 * w); }
@@ -238,62 +242,128 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __gri
       { const int it = j; if (r == 0) TR(9 + 8 * w); }
       tc::tc_fence_after();
       const bool need_mask = (j0 + BKV > P.seq) || (P.causal && j0 + BKV - 1 > i0);
-      // The row's 128 scores come into registers with one wait (one block per SM: a thread may hold them all):
-      // the maximum, the exponentials and the packing then run without touching tensor memory again until
-      // the packed P row is stored over the score columns.
-      uint32_t sr[128];
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) tc::tmem_ld32(s_addr + cc * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[cc * 32]));
-      tc::tmem_ld_wait();
-      float* sv = reinterpret_cast<float*>(sr);
-      if (need_mask) {
-#pragma unroll
-        for (int k = 0; k < 128; ++k) {
-          const int gj = j0 + k;
-          if (gj >= P.seq || (P.causal && gj > gi)) sv[k] = -INFINITY;
+      float mx, sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f, alpha, mc;
+      bool moved;
+      if constexpr (TILES == 2) {
+        // The row's 128 scores come into registers with one wait (one block per SM: a thread may hold them all):
+        // the maximum, the exponentials and the packing then run without touching tensor memory again until
+        // the packed P row is stored over the score columns.
+        uint32_t sr[128];
+  #pragma unroll
+        for (int cc = 0; cc < 4; ++cc) tc::tmem_ld32(s_addr + cc * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[cc * 32]));
+        tc::tmem_ld_wait();
+        float* sv = reinterpret_cast<float*>(sr);
+        if (need_mask) {
+  #pragma unroll
+          for (int k = 0; k < 128; ++k) {
+            const int gj = j0 + k;
+            if (gj >= P.seq || (P.causal && gj > gi)) sv[k] = -INFINITY;
+          }
         }
-      }
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+  #pragma unroll
+        for (int k = 0; k < 128; k += 4) {
+          mx0 = fmaxf(mx0, sv[k]); mx1 = fmaxf(mx1, sv[k + 1]); mx2 = fmaxf(mx2, sv[k + 2]); mx3 = fmaxf(mx3, sv[k + 3]);
+        }
+        mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        { const int it = j; if (r == 0) TR(10 + 8 * w); }
+        // lazy running max: move it only when the tile's max beats it by more than the threshold
+        moved = mx > m + tau || m == -INFINITY;
+        const float m_new = moved ? fmaxf(m, mx) : m;
+        alpha = (m == -INFINITY) ? 0.f : tc::fast_exp2((m - m_new) * c);
+        mc = (m_new == -INFINITY) ? 0.f : m_new * c;
+        m = m_new;
+        if (j > 0 && __any_sync(0xffffffffu, moved)) {
+          // O is rescaled in place: the previous P V product must have finished
+          if (!tc::mbar_wait(bar(B_PVDONE + w), (j - 1) & 1, status, 209)) { ok = false; break; }
+          tc::tc_fence_after();
+          const float a = moved ? alpha : 1.f;
+  #pragma unroll 1
+          for (int cc = 0; cc < HD / 32; ++cc) {
+            uint32_t o[32];
+            tc::tmem_ld32(o_addr + cc * 32, o);
+            tc::tmem_ld_wait();
+  #pragma unroll
+            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * a);
+            tc::tmem_st32(o_addr + cc * 32, o);
+          }
+        }
+        { const int it = j; if (r == 0) TR(11 + 8 * w); }
+        // P = exp2(S c - m c), its row sum, and P packed to bf16 (128 scores become 64 packed columns)
+  #pragma unroll
+        for (int k = 0; k < 128; k += 4) {
+          const float p0 = tc::fast_exp2(fmaf(sv[k], c, -mc)), p1 = tc::fast_exp2(fmaf(sv[k + 1], c, -mc));
+          const float p2 = tc::fast_exp2(fmaf(sv[k + 2], c, -mc)), p3 = tc::fast_exp2(fmaf(sv[k + 3], c, -mc));
+          sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+          sr[k / 2] = tc::pack_bf16(p0, p1);
+          sr[k / 2 + 1] = tc::pack_bf16(p2, p3);
+        }
+        tc::tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+        tc::tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+      } else {
+        // At most 128 registers here (two blocks per SM): two passes over the scores in tensor memory, four
+        // 32-column loads each, instead of holding the row.
+        auto mask_chunk = [&](float* sc, int cc) {
 #pragma unroll
-      for (int k = 0; k < 128; k += 4) {
-        mx0 = fmaxf(mx0, sv[k]); mx1 = fmaxf(mx1, sv[k + 1]); mx2 = fmaxf(mx2, sv[k + 2]); mx3 = fmaxf(mx3, sv[k + 3]);
-      }
-      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-      { const int it = j; if (r == 0) TR(10 + 8 * w); }
-      // lazy running max: move it only when the tile's max beats it by more than the threshold
-      const bool moved = mx > m + tau || m == -INFINITY;
-      const float m_new = moved ? fmaxf(m, mx) : m;
-      const float alpha = (m == -INFINITY) ? 0.f : tc::fast_exp2((m - m_new) * c);
-      const float mc = (m_new == -INFINITY) ? 0.f : m_new * c;
-      m = m_new;
-      if (j > 0 && __any_sync(0xffffffffu, moved)) {
-        // O is rescaled in place: the previous P V product must have finished
-        if (!tc::mbar_wait(bar(B_PVDONE + w), (j - 1) & 1, status, 209)) { ok = false; break; }
-        tc::tc_fence_after();
-        const float a = moved ? alpha : 1.f;
+          for (int k = 0; k < 32; ++k) {
+            const int gj = j0 + cc * 32 + k;
+            if (gj >= P.seq || (P.causal && gj > gi)) sc[k] = -INFINITY;
+          }
+        };
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll 1
-        for (int cc = 0; cc < HD / 32; ++cc) {
-          uint32_t o[32];
-          tc::tmem_ld32(o_addr + cc * 32, o);
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t sr[32];
+          tc::tmem_ld32(s_addr + cc * 32, sr);
           tc::tmem_ld_wait();
+          float* sc = reinterpret_cast<float*>(sr);
+          if (need_mask) mask_chunk(sc, cc);
 #pragma unroll
-          for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * a);
-          tc::tmem_st32(o_addr + cc * 32, o);
+          for (int k = 0; k < 32; k += 4) {
+            mx0 = fmaxf(mx0, sc[k]); mx1 = fmaxf(mx1, sc[k + 1]); mx2 = fmaxf(mx2, sc[k + 2]); mx3 = fmaxf(mx3, sc[k + 3]);
+          }
+        }
+        mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        moved = mx > m + tau || m == -INFINITY;
+        const float m_new = moved ? fmaxf(m, mx) : m;
+        alpha = (m == -INFINITY) ? 0.f : tc::fast_exp2((m - m_new) * c);
+        mc = (m_new == -INFINITY) ? 0.f : m_new * c;
+        m = m_new;
+        if (j > 0 && __any_sync(0xffffffffu, moved)) {
+          if (!tc::mbar_wait(bar(B_PVDONE + w), (j - 1) & 1, status, 209)) { ok = false; break; }
+          tc::tc_fence_after();
+          const float a = moved ? alpha : 1.f;
+#pragma unroll 1
+          for (int cc = 0; cc < HD / 32; ++cc) {
+            uint32_t o[32];
+            tc::tmem_ld32(o_addr + cc * 32, o);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * a);
+            tc::tmem_st32(o_addr + cc * 32, o);
+          }
+        }
+        // pass 2: P packed to bf16 over the score columns already consumed (32 scores become 16 packed columns;
+        // the thread owns the lane, so nobody else's data is overwritten)
+#pragma unroll 1
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t sr[32];
+          tc::tmem_ld32(s_addr + cc * 32, sr);
+          tc::tmem_ld_wait();
+          float* sc = reinterpret_cast<float*>(sr);
+          if (need_mask) mask_chunk(sc, cc);
+          uint32_t pk[16];
+#pragma unroll
+          for (int k = 0; k < 32; k += 4) {
+            const float p0 = tc::fast_exp2(fmaf(sc[k], c, -mc)), p1 = tc::fast_exp2(fmaf(sc[k + 1], c, -mc));
+            const float p2 = tc::fast_exp2(fmaf(sc[k + 2], c, -mc)), p3 = tc::fast_exp2(fmaf(sc[k + 3], c, -mc));
+            sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+            pk[k / 2] = tc::pack_bf16(p0, p1);
+            pk[k / 2 + 1] = tc::pack_bf16(p2, p3);
+          }
+          tc::tmem_st16(s_addr + cc * 16, pk);
         }
       }
-      { const int it = j; if (r == 0) TR(11 + 8 * w); }
-      // P = exp2(S c - m c), its row sum, and P packed to bf16 (128 scores become 64 packed columns)
-      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-#pragma unroll
-      for (int k = 0; k < 128; k += 4) {
-        const float p0 = tc::fast_exp2(fmaf(sv[k], c, -mc)), p1 = tc::fast_exp2(fmaf(sv[k + 1], c, -mc));
-        const float p2 = tc::fast_exp2(fmaf(sv[k + 2], c, -mc)), p3 = tc::fast_exp2(fmaf(sv[k + 3], c, -mc));
-        sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
-        sr[k / 2] = tc::pack_bf16(p0, p1);
-        sr[k / 2 + 1] = tc::pack_bf16(p2, p3);
-      }
-      tc::tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-      tc::tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
       if (moved) l *= alpha;
       l += (sum0 + sum1) + (sum2 + sum3);
       tc::tmem_st_wait();
@@ -333,6 +403,19 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_tc_kernel(const __gri
   if (warp == 1) tc::tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
+template <int HD, int TILES>
+cudaError_t fwd_launch_t(const fbl_plan* p, AttnFwdParams& P, int n_qt, cudaStream_t st) {
+  auto k = attn_fwd_tc_kernel<HD, TILES>;
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FwdSmem<HD, TILES>::TOTAL);
+  if (e != cudaSuccess) return e;
+  if (TILES == 1) P.pair = 0;
+  P.batch = p->d.batch;
+  P.n_slots = P.pair ? (n_qt + 1) / 2 : n_qt;
+  P.chunk = chunk_for((long long)p->d.seq * HD * 4, p->d.n_q_heads * p->d.batch, 96ll << 20);   // K and V of one head
+  dim3 grid((unsigned)(P.n_slots * p->d.n_q_heads * p->d.batch));
+  return launch_pdl(k, grid, dim3(64 + 128 * TILES), FwdSmem<HD, TILES>::TOTAL, st, P);
+}
+
 template <int HD>
 cudaError_t fwd_launch(const fbl_plan* p, const void* Q, const void* K, const void* V, void* A, float* lse,
                        int32_t* status, cudaStream_t st) {
@@ -348,14 +431,12 @@ cudaError_t fwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   const int n_qt = (p->d.seq + BQ - 1) / BQ;
   // two query tiles per block when that still leaves at least one block per SM
   P.pair = (n_qt >= 2 && (long long)((n_qt + 1) / 2) * p->d.n_q_heads * p->d.batch >= p->sm_count) ? 1 : 0;
-  auto k = attn_fwd_tc_kernel<HD>;
-  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FwdSmem<HD>::TOTAL);
-  if (e != cudaSuccess) return e;
-  P.batch = p->d.batch;
-  P.n_slots = P.pair ? (n_qt + 1) / 2 : n_qt;
-  P.chunk = chunk_for((long long)p->d.seq * HD * 4, p->d.n_q_heads * p->d.batch, 96ll << 20);   // K and V of one head
-  dim3 grid((unsigned)(P.n_slots * p->d.n_q_heads * p->d.batch));
-  return launch_pdl(k, grid, dim3(FWD_THREADS), FwdSmem<HD>::TOTAL, st, P);
+  if (HD == 64) {
+    // tuning knob: 1 = one query tile per block and two blocks per SM, 2 = two tiles per block; default by sequence length
+    const int mode = getenv("FBL_FWD_TILES") ? atoi(getenv("FBL_FWD_TILES")) : 0;
+    if (mode == 1 || (mode == 0 && n_qt <= 4)) return fwd_launch_t<64, 1>(p, P, n_qt, st);
+  }
+  return fwd_launch_t<HD, 2>(p, P, n_qt, st);
 }
 
 // ---------------------------------------------------------------------------------------------------
