@@ -64,8 +64,8 @@ NCU_TRAFFIC_BYTES = {
     ("cfg2-gpt2-small", "dWo+dA"): 7.5e6 + 0.0e6,
     ("cfg2-gpt2-small", "attn_bwd"): 19.1e6 + 0.3e6 + 6.3e6,      # main kernel + rounding of the fp32 dQ
     ("cfg2-gpt2-small", "dWqkv+dXn"): 16.2e6 + 0.0e6,
-    ("cfg2-gpt2-small", "db"): 12.6e6 + 12.5e6 + 0.1e6,           # the write is the previous kernel's dirty lines
-    ("cfg2-gpt2-small", "norm_bwd"): 6.3e6 + 8.2e6 + 1.6e6,
+    # bias column sums (first stage; its DRAM write is the previous kernel's dirty lines), norm backward, shared second stage
+    ("cfg2-gpt2-small", "db+norm_bwd"): 12.6e6 + 12.5e6 + 6.3e6 + 8.2e6 + 1.6e6,
     # workload 4, profiles/ncu_full_workload4_llama1b_gqa_hd64.md
     ("cfg4-llama1b-gqa", "proj_qkv"): 29.4e6 + 0.3e6,
     ("cfg4-llama1b-gqa", "attn_fwd"): 25.2e6 + 0.0e6,
@@ -80,7 +80,9 @@ def step_bytes(cfg):
     """Algorithmic HBM bytes of the bandwidth-bound steps."""
     e = 2 if cfg.dtype == "bf16" else 4
     nd = cfg.n_tokens * cfg.d_model * e
-    return {"norm_fwd": 2 * nd, "norm_bwd": (4 if cfg.residual else 3) * nd}
+    nb = (4 if cfg.residual else 3) * nd
+    db = (cfg.n_tokens * (cfg.d_model + cfg.d_q + 2 * cfg.d_kv) * e) if cfg.has_bias else 0
+    return {"norm_fwd": 2 * nd, "norm_bwd": nb, "db+norm_bwd": nb + db}
 
 
 class ClockSampler:

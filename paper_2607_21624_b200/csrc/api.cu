@@ -483,13 +483,17 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
       for (int i = 0; i < 3; ++i)
         FBL_STEP(i == 0 ? "dWq" : i == 1 ? "dWk" : "dWv", 1, run_gemm(p, gs[i], part, p->part_bytes, status, st));
     }
-    if (bias) {   // every bias gradient is a token-axis column sum: one pair of launches for the four of them
-      const void* M4[4] = {dY, dQ, dK, dV};
-      float* O4[4] = {dbo, dbq, dbk, dbv};
-      const int C4[4] = {D, p->dq, p->dkv, p->dkv};
-      FBL_STEP("db", 2, launch_colsum_group(p->d.dtype, 4, M4, p->n_pad, C4, O4, (float*)part, st));
-    }
   }
+  // every bias gradient is a token-axis column sum: the four of them share their launches, and the second stage
+  // shares the norm backward's second kernel where that kernel exists
+  const void* M4[4] = {dY, dQ, dK, dV};
+  float* O4[4] = {dbo, dbq, dbk, dbv};
+  const int C4[4] = {D, p->dq, p->dkv, p->dkv};
+  if (bias && norm_bwd_takes_colsums(p)) {
+    FBL_STEP("db+norm_bwd", 3, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, (float*)part, st, 4, M4, C4, O4));
+    return FBL_OK;
+  }
+  if (bias) FBL_STEP("db", 2, launch_colsum_group(p->d.dtype, 4, M4, p->n_pad, C4, O4, (float*)part, st));
   FBL_STEP("norm_bwd", 2, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, (float*)part, st));
   return FBL_OK;
 }

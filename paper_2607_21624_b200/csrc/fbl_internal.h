@@ -99,9 +99,11 @@ cudaError_t launch_pack(int dtype, int unpack, const void* src, void* dst, int64
 bool norm_fwd_resets_status(const fbl_plan* p);   // the forward norm kernel for this plan zeroes the status word itself
 cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
                             float* stats, int32_t* status, cudaStream_t st);
+bool norm_bwd_takes_colsums(const fbl_plan* p);
 cudaError_t launch_norm_bwd(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
                             const float* gamma, void* dX, float* dgamma, float* dbeta, float* part,
-                            cudaStream_t st);
+                            cudaStream_t st, int bias_count = 0, const void* const* bias_m = nullptr,
+                            const int* bias_cols = nullptr, float* const* bias_out = nullptr);
 cudaError_t launch_colsum(int dtype, const void* M, int64_t rows, int64_t cols, float* out, float* partials,
                           cudaStream_t st);
 size_t colsum_scratch_bytes(int64_t rows, int64_t cols);

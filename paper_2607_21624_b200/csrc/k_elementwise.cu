@@ -440,12 +440,38 @@ __global__ void __launch_bounds__(256, 2) norm_bwd_rows_kernel(const __nv_bfloat
   }
 }
 
-// dgamma[c] (y = 0) or dbeta[c] (y = 1) = sum over the first kernel's blocks of their partial rows.
+constexpr int COLSUM_SLAB = 256;
+
+struct ColsumGroup {
+  const void* m[4];
+  float* out[4];
+  int cols[4];
+  int64_t part_off[4];      // float offset of each matrix's partials inside the scratch area
+  int count;
+};
+
+// dgamma[c] (y = 0) or dbeta[c] (y = 1) = sum over the first kernel's blocks of their partial rows.  Blocks with
+// y >= ny_norm finish the bias column sums instead (matrix y - ny_norm: the tree over its slab partials), so that
+// the step's two small final reductions share one launch.
 __global__ void __launch_bounds__(256) norm_bwd_reduce_kernel(const float* __restrict__ part, int blocks, int d,
-                                                              float* __restrict__ dgamma, float* __restrict__ dbeta) {
+                                                              float* __restrict__ dgamma, float* __restrict__ dbeta,
+                                                              int ny_norm, ColsumGroup G, const float* __restrict__ cpart,
+                                                              int n_slabs) {
   __shared__ float red[8][33];
   pdl_launch_dependents();
   pdl_wait();
+  if ((int)blockIdx.y >= ny_norm) {
+    const int which = blockIdx.y - ny_norm;
+    const int cols = G.cols[which];
+    const float* cp = cpart + G.part_off[which];
+    for (int c = blockIdx.x * 256 + threadIdx.x; c < cols; c += gridDim.x * 256) {
+      float s = 0.f;
+#pragma unroll 8
+      for (int k = 0; k < n_slabs; ++k) s += cp[(int64_t)k * cols + c];
+      G.out[which][c] = s;
+    }
+    return;
+  }
   const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
   const int c = blockIdx.x * 32 + tx;
   float s = 0.f;
@@ -481,12 +507,13 @@ void norm_fwd_rows_launch(const fbl_plan* p, const void* X, const float* gamma, 
 template <int NV, int WPR>
 void norm_bwd_rows_launch(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
                           const float* gamma, void* dX, float* dgamma, float* dbeta, float* part, int rms,
-                          cudaStream_t st) {
+                          const ColsumGroup& cg, const float* cpart, int n_slabs, cudaStream_t st) {
   const int blocks = (int)min((int64_t)p->sm_count * 2, p->n_pad / (8 / WPR));
   launch_pdl(norm_bwd_rows_kernel<NV, WPR>, dim3(blocks), dim3(256), 0, st, (const __nv_bfloat16*)dXn,
              (const __nv_bfloat16*)X, (const __nv_bfloat16*)dY, stats, gamma, (__nv_bfloat16*)dX, part, p->n_pad, rms);
-  launch_pdl(norm_bwd_reduce_kernel, dim3((p->d.d_model + 31) / 32, rms ? 1 : 2), dim3(256), 0, st, (const float*)part,
-             blocks, p->d.d_model, dgamma, dbeta);
+  const int ny = rms ? 1 : 2;
+  launch_pdl(norm_bwd_reduce_kernel, dim3((p->d.d_model + 31) / 32, ny + cg.count), dim3(256), 0, st, (const float*)part,
+             blocks, p->d.d_model, dgamma, dbeta, ny, cg, cpart, n_slabs);
 }
 
 // d_model -> (vectors per lane, warps per row) of the register-resident kernels; false if there is none.  At most
@@ -523,16 +550,6 @@ bool norm_rows_shape(int d, int* nv, int* wpr) {
 // Token-axis column sums, two stages over tiles: (1) one block per (panel, slab of 256 rows)
 // reduces its 32 storage tiles to one row of partials, (2) a tree over slabs.
 // ------------------------------------------------------------------------------------------
-constexpr int COLSUM_SLAB = 256;
-
-struct ColsumGroup {
-  const void* m[4];
-  float* out[4];
-  int cols[4];
-  int64_t part_off[4];      // float offset of each matrix's partials inside the scratch area
-  int count;
-};
-
 template <typename T>
 __global__ void __launch_bounds__(256) colsum_stage1(ColsumGroup G, int64_t rows, float* __restrict__ part_base) {
   constexpr int TW = tile_w_of<T>::value;
@@ -627,21 +644,50 @@ cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma
   return cudaGetLastError();
 }
 
+// Norm backward, and with it (bias_count > 0, register-resident bf16 path only) the bias column sums of up to four
+// matrices: their first stage runs before the norm kernel, their second stage inside the norm's own second kernel.
+// `part` holds the column-sum slab partials first and the norm's per-block partial rows behind them.
+bool norm_bwd_takes_colsums(const fbl_plan* p) {
+  int nv, wpr;
+  return p->d.dtype == FBL_DTYPE_BF16 && norm_rows_shape(p->d.d_model, &nv, &wpr);
+}
+
 cudaError_t launch_norm_bwd(const fbl_plan* p, const void* dXn, const void* X, const void* dY, const float* stats,
                             const float* gamma, void* dX, float* dgamma, float* dbeta, float* part,
-                            cudaStream_t st) {
+                            cudaStream_t st, int bias_count, const void* const* bias_m, const int* bias_cols,
+                            float* const* bias_out) {
   const int blocks = (int)((p->n_pad + 31) / 32);
   const int d = p->d.d_model;
   const int rms = p->d.norm == FBL_NORM_RMSNORM;
   const size_t sh = 2 * (size_t)d * sizeof(float);
   int nv, wpr;
   if (p->d.dtype == FBL_DTYPE_BF16 && norm_rows_shape(d, &nv, &wpr)) {
-    // token-axis sums in two steps over `part` (no atomics: the result does not depend on block order)
-#define FBL_CALL(NV_, WPR_) norm_bwd_rows_launch<NV_, WPR_>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, part, rms, st)
+    ColsumGroup cg;
+    memset(&cg, 0, sizeof(cg));
+    const int n_slabs = (int)((p->n_pad + COLSUM_SLAB - 1) / COLSUM_SLAB);
+    float* npart = part;
+    if (bias_count > 0) {
+      if (bias_count > 4) return cudaErrorInvalidValue;
+      int max_cols = 0;
+      int64_t off = 0;
+      for (int i = 0; i < bias_count; ++i) {
+        cg.m[i] = bias_m[i]; cg.out[i] = bias_out[i]; cg.cols[i] = bias_cols[i]; cg.part_off[i] = off;
+        off += (int64_t)n_slabs * bias_cols[i];
+        max_cols = bias_cols[i] > max_cols ? bias_cols[i] : max_cols;
+      }
+      cg.count = bias_count;
+      cudaError_t e = launch_pdl(colsum_stage1<__nv_bfloat16>, dim3((unsigned)(max_cols / 64), n_slabs, bias_count), dim3(256), 0,
+                                 st, cg, p->n_pad, part);
+      if (e != cudaSuccess) return e;
+      npart = part + (off + 255) / 256 * 256;
+    }
+    // token-axis sums in two steps over `npart` (no atomics: the result does not depend on block order)
+#define FBL_CALL(NV_, WPR_) norm_bwd_rows_launch<NV_, WPR_>(p, dXn, X, dY, stats, gamma, dX, dgamma, dbeta, npart, rms, cg, part, n_slabs, st)
     FBL_NORM_DISPATCH(FBL_CALL);
 #undef FBL_CALL
     return cudaGetLastError();
   }
+  if (bias_count > 0) return cudaErrorInvalidValue;      // callers ask norm_bwd_takes_colsums first
   cudaError_t e = cudaMemsetAsync(dgamma, 0, d * sizeof(float), st);
   if (e != cudaSuccess) return e;
   if (dbeta) {
