@@ -548,13 +548,17 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
   uint32_t tmem_base;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
   pdl_launch_dependents();
-  pdl_wait();                                    // the set-up above overlapped the previous kernel's tail
-
+  // Of this kernel's inputs only dO (and D) come from the kernel before it (the dA GEMM); K, V, Q and LSE are the
+  // forward pass's.  Each role therefore waits for that kernel where it first needs it: the producer has K, V
+  // and the first Q tile on their way before it does.
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ------------------------------------------------------------------------
+    tc::tma_prefetch_desc(&P.tk); tc::tma_prefetch_desc(&P.tv); tc::tma_prefetch_desc(&P.tq);
+    tc::tma_prefetch_desc(&P.tdo); tc::tma_prefetch_desc(&P.tdq);
     tc::mbar_expect_tx(bar(BB_KVFULL), 2 * SM::TILE);
     tc::tma_load_3d(base + SM::K_OFF, &P.tk, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
     tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
+    bool waited = false;
     for (int it = 0; it < n_it; ++it) {
       const int h = g * P.group + it / per_head, qt = qt_begin + it % per_head;
       if (PIPE) {
@@ -562,6 +566,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         if (!tc::mbar_wait(bar(BB_QDOEMPTY + s), ph ^ 1, status, 301)) break;
         tc::mbar_expect_tx(bar(BB_QDOFULL + s), 2 * SM::TILE);
         tc::tma_load_3d(base + SM::Q_OFF + s * SM::TILE, &P.tq, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
+        if (!waited) { pdl_wait(); waited = true; }
         tc::tma_load_3d(base + SM::DO_OFF + s * SM::TILE, &P.tdo, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
       } else {
         // single buffers: Q and dO have a barrier pair each (slot 0: Q, slot 1: dO), since Q is free after the dK
@@ -571,6 +576,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         tc::mbar_expect_tx(bar(BB_QDOFULL), SM::TILE);
         tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(BB_QDOFULL), 0, row0 + qt * BQ, h * (int)PANELS);
         if (!tc::mbar_wait(bar(BB_QDOEMPTY + 1), ph ^ 1, status, 313)) break;
+        if (!waited) { pdl_wait(); waited = true; }
         tc::mbar_expect_tx(bar(BB_QDOFULL + 1), SM::TILE);
         tc::tma_load_3d(base + SM::DO_OFF, &P.tdo, bar(BB_QDOFULL + 1), 0, row0 + qt * BQ, h * (int)PANELS);
       }
@@ -696,6 +702,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
   } else if (warp == 18) {
     // ---- dQ reduction warp: adds each staged dQ tile to the fp32 accumulator with bulk tensor reductions ----
     if (lane == 0) {
+      pdl_wait();                                    // the accumulator's zero-fill precedes the kernel before this one
       for (int dit = 0; dit < n_it; ++dit) {
         const int h = g * P.group + dit / per_head, i0 = (qt_begin + dit % per_head) * BQ;
         if (!tc::mbar_wait(bar(BB_DQSTAGED), dit & 1, status, 309)) break;
@@ -717,6 +724,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     const int r = q * 32 + lane;
     const int t = threadIdx.x - 64;                 // 0..511
     const int gj = j0 + r;
+    pdl_wait();                                     // D is written by the kernel before this one; dK, dV may still be read by it
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
     const float c = P.scale * LOG2E;
     float* s_stage = reinterpret_cast<float*>(smem_raw + SM::LSE_OFF);
