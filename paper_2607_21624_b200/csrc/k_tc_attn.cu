@@ -537,6 +537,17 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     tc::mbar_init(bar(BB_SREAD), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_DVDONE), 1);
     tc::fence_barrier_init();
+    // This thread is the TMA producer: K, V and the first Q tile (forward-pass data) are requested right here, so
+    // that their latency overlaps the tensor-memory allocation and the block-wide barrier below.
+    tc::tma_prefetch_desc(&P.tk); tc::tma_prefetch_desc(&P.tv); tc::tma_prefetch_desc(&P.tq);
+    tc::tma_prefetch_desc(&P.tdo); tc::tma_prefetch_desc(&P.tdq);
+    tc::mbar_expect_tx(bar(BB_KVFULL), 2 * SM::TILE);
+    tc::tma_load_3d(base + SM::K_OFF, &P.tk, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
+    tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
+    if (n_it > 0) {
+      tc::mbar_expect_tx(bar(BB_QDOFULL), PIPE ? 2 * SM::TILE : SM::TILE);
+      tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(BB_QDOFULL), 0, row0 + qt_begin * BQ, g * P.group * (int)PANELS);
+    }
   }
   if (warp == 1) {
     tc::tmem_alloc(slot, TMEM_COLS);
@@ -553,28 +564,28 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
   // and the first Q tile on their way before it does.
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ------------------------------------------------------------------------
-    tc::tma_prefetch_desc(&P.tk); tc::tma_prefetch_desc(&P.tv); tc::tma_prefetch_desc(&P.tq);
-    tc::tma_prefetch_desc(&P.tdo); tc::tma_prefetch_desc(&P.tdq);
-    tc::mbar_expect_tx(bar(BB_KVFULL), 2 * SM::TILE);
-    tc::tma_load_3d(base + SM::K_OFF, &P.tk, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
-    tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
+    // (K, V and Q of the first tile were requested during set-up)
     bool waited = false;
     for (int it = 0; it < n_it; ++it) {
       const int h = g * P.group + it / per_head, qt = qt_begin + it % per_head;
       if (PIPE) {
         const uint32_t s = it % NQ, ph = (it / NQ) & 1;
-        if (!tc::mbar_wait(bar(BB_QDOEMPTY + s), ph ^ 1, status, 301)) break;
-        tc::mbar_expect_tx(bar(BB_QDOFULL + s), 2 * SM::TILE);
-        tc::tma_load_3d(base + SM::Q_OFF + s * SM::TILE, &P.tq, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
+        if (it > 0) {
+          if (!tc::mbar_wait(bar(BB_QDOEMPTY + s), ph ^ 1, status, 301)) break;
+          tc::mbar_expect_tx(bar(BB_QDOFULL + s), 2 * SM::TILE);
+          tc::tma_load_3d(base + SM::Q_OFF + s * SM::TILE, &P.tq, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
+        }
         if (!waited) { pdl_wait(); waited = true; }
         tc::tma_load_3d(base + SM::DO_OFF + s * SM::TILE, &P.tdo, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
       } else {
         // single buffers: Q and dO have a barrier pair each (slot 0: Q, slot 1: dO), since Q is free after the dK
         // product and dO only after the dV product, and the next score tile needs Q alone
         const uint32_t ph = it & 1;
-        if (!tc::mbar_wait(bar(BB_QDOEMPTY), ph ^ 1, status, 301)) break;
-        tc::mbar_expect_tx(bar(BB_QDOFULL), SM::TILE);
-        tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(BB_QDOFULL), 0, row0 + qt * BQ, h * (int)PANELS);
+        if (it > 0) {
+          if (!tc::mbar_wait(bar(BB_QDOEMPTY), ph ^ 1, status, 301)) break;
+          tc::mbar_expect_tx(bar(BB_QDOFULL), SM::TILE);
+          tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(BB_QDOFULL), 0, row0 + qt * BQ, h * (int)PANELS);
+        }
         if (!tc::mbar_wait(bar(BB_QDOEMPTY + 1), ph ^ 1, status, 313)) break;
         if (!waited) { pdl_wait(); waited = true; }
         tc::mbar_expect_tx(bar(BB_QDOFULL + 1), SM::TILE);
