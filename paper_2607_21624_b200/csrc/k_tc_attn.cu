@@ -133,6 +133,22 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
       tc::mbar_init(bar(B_PVDONE + s), 1);
     }
     tc::fence_barrier_init();
+    // This thread is the TMA producer: once the kernel before this one (which writes Q, K, V) is complete, the
+    // query tiles and the first K / V tiles are requested right here, so that their latency overlaps the
+    // tensor-memory allocation and the block-wide barrier below.
+    tc::tma_prefetch_desc(&P.tq);
+    tc::tma_prefetch_desc(&P.tk);
+    tc::tma_prefetch_desc(&P.tv);
+    pdl_wait();
+    tc::mbar_expect_tx(bar(B_QFULL), (qt1 >= 0 ? 2u : 1u) * SM::TILE);
+    tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(B_QFULL), 0, row0 + qt0 * BQ, h * (int)PANELS);
+    if (qt1 >= 0) tc::tma_load_3d(base + SM::Q_OFF + SM::TILE, &P.tq, bar(B_QFULL), 0, row0 + qt1 * BQ, h * (int)PANELS);
+    if (n_kv_max > 0) {
+      tc::mbar_expect_tx(bar(B_KFULL), SM::TILE);
+      tc::tma_load_3d(base + SM::K_OFF, &P.tk, bar(B_KFULL), 0, row0, g * (int)PANELS);
+      tc::mbar_expect_tx(bar(B_VFULL), SM::TILE);
+      tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(B_VFULL), 0, row0, g * (int)PANELS);
+    }
   }
   if (warp == 1) {
     tc::tmem_alloc(slot, TMEM_COLS);
@@ -144,17 +160,10 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
   uint32_t tmem_base;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
   pdl_launch_dependents();
-  pdl_wait();                                    // the set-up above overlapped the previous kernel's tail
 
   if (warp == 0 && lane == 0) {
-    // ---- TMA producer ------------------------------------------------------------------------
-    tc::tma_prefetch_desc(&P.tq);
-    tc::tma_prefetch_desc(&P.tk);
-    tc::tma_prefetch_desc(&P.tv);
-    tc::mbar_expect_tx(bar(B_QFULL), (qt1 >= 0 ? 2u : 1u) * SM::TILE);
-    tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(B_QFULL), 0, row0 + qt0 * BQ, h * (int)PANELS);
-    if (qt1 >= 0) tc::tma_load_3d(base + SM::Q_OFF + SM::TILE, &P.tq, bar(B_QFULL), 0, row0 + qt1 * BQ, h * (int)PANELS);
-    for (int j = 0; j < n_kv_max; ++j) {
+    // ---- TMA producer (the query tiles and key tile 0 were requested during set-up) ---------------
+    for (int j = 1; j < n_kv_max; ++j) {
       const int s = j & 1;
       const uint32_t ph = (j >> 1) & 1;
       if (!tc::mbar_wait(bar(B_KEMPTY + s), ph ^ 1, status, 201)) break;
@@ -233,6 +242,7 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
     const uint32_t s_addr = lane_addr + w * 128, o_addr = lane_addr + O_COL + w * HD;
     const float c = P.scale * LOG2E;
     const float tau = RESCALE_LOG2 / c;              // the same threshold in raw score units
+    pdl_wait();                                      // before this role writes anything
     float m = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < n_kvw && ok; ++j) {
