@@ -57,7 +57,7 @@ def step_flops(cfg):
 # summarised under profiles/ (workload 4, and workload 5 at sequence 2048).  Keyed by (workload name, step).
 NCU_TRAFFIC_BYTES = {
     # workload 2 (the default): every kernel of a step, profiles/ncu_full_workload2_gpt2small_hd64.md
-    ("cfg2-gpt2-small", "norm_fwd"): 3.2e6 + 0.0e6,
+    ("cfg2-gpt2-small", "norm_fwd"): 3.5e6 + 0.0e6,
     ("cfg2-gpt2-small", "proj_qkv"): 6.8e6 + 0.0e6,
     ("cfg2-gpt2-small", "attn_fwd"): 9.5e6 + 0.0e6,
     ("cfg2-gpt2-small", "proj_o"): 4.4e6 + 0.0e6,
@@ -65,7 +65,7 @@ NCU_TRAFFIC_BYTES = {
     ("cfg2-gpt2-small", "attn_bwd"): 19.1e6 + 0.3e6 + 6.3e6,      # main kernel + rounding of the fp32 dQ
     ("cfg2-gpt2-small", "dWqkv+dXn"): 16.2e6 + 0.0e6,
     # bias column sums (first stage; its DRAM write is the previous kernel's dirty lines), norm backward, shared second stage
-    ("cfg2-gpt2-small", "db+norm_bwd"): 12.6e6 + 12.5e6 + 6.3e6 + 8.2e6 + 1.6e6,
+    ("cfg2-gpt2-small", "db+norm_bwd"): 12.6e6 + 4.4e6 + 6.3e6 + 5.9e6 + 1.7e6,
     # workload 4, profiles/ncu_full_workload4_llama1b_gqa_hd64.md
     ("cfg4-llama1b-gqa", "proj_qkv"): 29.4e6 + 0.3e6,
     ("cfg4-llama1b-gqa", "attn_fwd"): 25.2e6 + 0.0e6,
