@@ -719,6 +719,9 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
           TR(5);
         }
       }
+      // dQ is issued first here, so its barrier does not cover the last tile's dK and dV products: one more
+      // arrival, on the barrier the pipelined variant uses for dV, tells the epilogue that they are complete
+      if (ok && n_it > 0) tc::mma_commit(bar(BB_DVDONE));
     }
   } else if (warp == 18) {
     // ---- dQ reduction warp: adds each staged dQ tile to the fp32 accumulator with bulk tensor reductions ----
@@ -902,7 +905,10 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       if (t == 0) TR(12);
     }
     if (PIPE && ok && n_it > 0) ok = drain_dq(n_it - 1);
-    // dK, dV of this key tile: every MMA has completed (the last dQ wait covered them)
+    // dK, dV of this key tile: every MMA has completed (HD = 64: dQ is the last product issued, and the wait for
+    // it is behind us; HD = 128: the extra arrival above)
+    if (!PIPE && ok && n_it > 0) ok = tc::mbar_wait(bar(BB_DVDONE), 0, status, 315);
+    tc::tc_fence_after();
     if (ok && n_it > 0) {
       const bool live = gj < P.seq;
 #pragma unroll 1
