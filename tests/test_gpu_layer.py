@@ -107,6 +107,15 @@ def test_cta_pair_gemm_forced(cfg, monkeypatch):
     run_and_compare(cfg, affine_noise=True)
 
 
+def test_forward_tile_variants_forced(monkeypatch):
+    # head_dim 64 forward: one-tile blocks (two per SM) are the default for short sequences, two-tile blocks for long
+    # ones; force each on a shape the other would get
+    for mode, cfg in (("2", LayerConfig("f1", 2, 300, 256, 4, 2, 64, "bf16", "rmsnorm", True, False, False, 1e-5, 34, 0.02)),
+                      ("1", LayerConfig("f2", 1, 700, 256, 4, 4, 64, "bf16", "layernorm", True, True, False, 1e-5, 35, 0.02))):
+        monkeypatch.setenv("FBL_FWD_TILES", mode)
+        run_and_compare(cfg, affine_noise=True)
+
+
 @pytest.mark.parametrize("i", [2, 3])
 def test_full_configs_2_and_3(i):
     run_and_compare(get_config(i))
