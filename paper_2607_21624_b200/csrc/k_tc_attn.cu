@@ -490,11 +490,11 @@ struct BwdSmem {
   static constexpr uint32_t DS_OFF = DO_OFF + NQ * TILE, STAGE_OFF = DS_OFF + NP * 32768;
   static constexpr uint32_t LSE_OFF = STAGE_OFF + NP * STAGE_BYTES;    // 2 buffers x (128 floats LSE*log2e, 128 floats D)
   static constexpr uint32_t BAR_OFF = LSE_OFF + 2048;
-  static constexpr uint32_t N_BARS = 15;
+  static constexpr uint32_t N_BARS = 16;
   static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16;
 };
 
-enum { BB_KVFULL = 0, BB_QDOFULL = 1, BB_QDOEMPTY = 3, BB_SFULL = 5, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY, BB_DQSTAGED, BB_STAGEFREE, BB_SREAD = BB_STAGEFREE + 2, BB_DVDONE };
+enum { BB_KVFULL = 0, BB_QDOFULL = 1, BB_QDOEMPTY = 3, BB_SFULL = 5, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY, BB_DQSTAGED, BB_STAGEFREE = BB_DQSTAGED + 2, BB_SREAD = BB_STAGEFREE + 2, BB_DVDONE };
 
 constexpr int BWD_THREADS = 608;     // warp 0 TMA loads, warp 1 MMA, warps 2-17 softmax (four per TMEM lane quarter), warp 18 dQ reductions
 constexpr int BWD_SM_THREADS = 512;
@@ -542,6 +542,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     tc::mbar_init(bar(BB_DQDRAINED), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_LSEREADY), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_DQSTAGED), BWD_SM_THREADS);
+    tc::mbar_init(bar(BB_DQSTAGED + 1), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_STAGEFREE), 1);
     tc::mbar_init(bar(BB_STAGEFREE + 1), 1);
     tc::mbar_init(bar(BB_SREAD), BWD_SM_THREADS);
@@ -729,7 +730,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       pdl_wait();                                    // the accumulator's zero-fill precedes the kernel before this one
       for (int dit = 0; dit < n_it; ++dit) {
         const int h = g * P.group + dit / per_head, i0 = (qt_begin + dit % per_head) * BQ;
-        if (!tc::mbar_wait(bar(BB_DQSTAGED), dit & 1, status, 309)) break;
+        if (!tc::mbar_wait(bar(BB_DQSTAGED + (dit % NP)), (dit / (int)NP) & 1, status, 309)) break;   // one per buffer, like STAGEFREE
         const uint32_t stage = base + SM::STAGE_OFF + (dit % NP) * SM::STAGE_BYTES;
 #pragma unroll
         for (int pn = 0; pn < (int)PANELS; ++pn)
@@ -785,7 +786,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       { const int it = dit; if (t == 0) TR(7); }
       tc::mbar_arrive(bar(BB_DQDRAINED));            // TMEM side done: the tensor pipe may reuse the columns
       tc::fence_proxy_async();
-      tc::mbar_arrive(bar(BB_DQSTAGED));             // staging side done: the reduction warp takes over
+      tc::mbar_arrive(bar(BB_DQSTAGED + (dit % NP)));     // staging side done: the reduction warp takes over
       return true;
     };
 
