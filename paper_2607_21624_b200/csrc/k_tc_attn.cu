@@ -72,11 +72,11 @@ struct FwdSmem {
   static constexpr uint32_t K_OFF = TILES * TILE;           // 2 stages
   static constexpr uint32_t V_OFF = (TILES + 2) * TILE;     // 2 stages
   static constexpr uint32_t BAR_OFF = (TILES + 4) * TILE;
-  static constexpr uint32_t N_BARS = 16;
+  static constexpr uint32_t N_BARS = 18;
   static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16;
 };
 
-enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_PVDONE = 13 };
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 12, B_PVDONE = 15 };   // SFULL, PFULL: one per score buffer (up to 3)
 
 // warp 0 TMA, warp 1 MMA, then one softmax warp group (4 warps) per query tile of the block.  TILES = 2: two
 // adjacent query tiles share the K/V tiles, one block per SM.  TILES = 1 (head_dim 64 only: its tiles leave room): a
@@ -91,7 +91,16 @@ template <int HD, int TILES>
 __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd_tc_kernel(const __grid_constant__ AttnFwdParams P) {
   using SM = FwdSmem<HD, TILES>;
   constexpr uint32_t PANELS = SM::PANELS;
-  constexpr uint32_t O_COL = 128 * TILES, TMEM_COLS = 256 * TILES;   // S of tile g at 128 g, O of tile g at O_COL + HD g
+  // Score buffers in tensor memory.  HD = 128 (and one-tile blocks): one per query tile, P written over S, so the
+  // next S of a tile follows its P V product.  HD = 64 with two tiles leaves room for a third buffer (3 x 128 score
+  // columns + 2 x 64 output columns = 512): the block's work items (tile, key tile), in issue order, then take the
+  // buffers in rotation, item n using buffer n % 3, and the S product of item n + 3 is issued right after the P V
+  // product of item n.  Every warp group then finds its next scores computed when it finishes a tile, instead of
+  // waiting for P V and S behind its own P.
+  constexpr bool ROT = TILES == 2 && HD == 64;
+  constexpr int NBUF = ROT ? 3 : TILES;
+  constexpr uint32_t O_COL = 128 * NBUF, TMEM_COLS = 256 * TILES;   // score buffer i at 128 i, O of tile g at O_COL + HD g
+  static_assert(O_COL + TILES * HD <= TMEM_COLS, "tensor memory columns");
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = tc::smem_u32(smem_raw);
   const uint32_t bars = base + SM::BAR_OFF;
@@ -128,9 +137,11 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
       tc::mbar_init(bar(B_KEMPTY + s), 1);
       tc::mbar_init(bar(B_VFULL + s), 1);
       tc::mbar_init(bar(B_VEMPTY + s), 1);
+      tc::mbar_init(bar(B_PVDONE + s), 1);
+    }
+    for (int s = 0; s < 3; ++s) {
       tc::mbar_init(bar(B_SFULL + s), 1);
       tc::mbar_init(bar(B_PFULL + s), 128);
-      tc::mbar_init(bar(B_PVDONE + s), 1);
     }
     tc::fence_barrier_init();
     // This thread is the TMA producer: once the kernel before this one (which writes Q, K, V) is complete, the
@@ -203,6 +214,50 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
       }
       tc::mma_commit(bar(B_PVDONE + w));
     };
+    if constexpr (ROT) {
+      // Work items in issue order: (tile 0, j), (tile 1, j) while tile 1 has key tiles, then tile 0's remaining
+      // ones (n_kv0 >= n_kv1: tile 0 is the later query tile).  Barriers of a score buffer are used once per
+      // rotation, so neither side can run more than one phase ahead on any of them.
+      const int n_items = n_kv0 + n_kv1;
+      auto item = [&](int n, int& w, int& j) {
+        if (n < 2 * n_kv1) { w = n & 1; j = n >> 1; } else { w = 0; j = n - n_kv1; }
+      };
+      auto issue_s_item = [&](int n) -> bool {
+        int w, j; item(n, w, j);
+        // tile 0 is the first user of every key tile, and the last one where tile 1 has none
+        if (w == 0 && !tc::mbar_wait(bar(B_KFULL + (j & 1)), (j >> 1) & 1, status, 205)) return false;
+        const uint32_t ql = q_lo + w * (SM::TILE >> 4), kl = k_lo + (j & 1) * (SM::TILE >> 4);
+        const uint32_t d = tmem_base + (uint32_t)(n % 3) * 128;
+#pragma unroll
+        for (uint32_t kk = 0; kk < HD / 16; ++kk) {
+          const uint32_t o = (kk / 4) * 1024 + (kk % 4) * 2;
+          tc::mma_bf16_ss_w(d, ql + o, hi, kl + o, hi, idesc_s, kk > 0);
+        }
+        tc::mma_commit(bar(B_SFULL + n % 3));
+        if (w == 1 || j >= n_kv1) tc::mma_commit(bar(B_KEMPTY + (j & 1)));
+        return true;
+      };
+      bool ok = tc::mbar_wait(bar(B_QFULL), 0, status, 203);
+      if (ok) tc::tc_fence_after();
+      for (int n = 0; n < 3 && n < n_items && ok; ++n) ok = issue_s_item(n);
+      for (int n = 0; n < n_items && ok; ++n) {
+        int w, j; item(n, w, j);
+        { const int it = j; TR(1 + 3 * w); }
+        if (w == 0 && !tc::mbar_wait(bar(B_VFULL + (j & 1)), (j >> 1) & 1, status, 207)) { ok = false; break; }
+        if (!tc::mbar_wait(bar(B_PFULL + n % 3), (n / 3) & 1, status, 206)) { ok = false; break; }
+        { const int it = j; TR(2 + 3 * w); }
+        tc::tc_fence_after();
+        const uint32_t vl = v_lo + (j & 1) * (SM::TILE >> 4);
+        const uint32_t pa = tmem_base + (uint32_t)(n % 3) * 128, od = tmem_base + O_COL + w * HD;
+#pragma unroll
+        for (uint32_t kk = 0; kk < BKV / 16; ++kk)
+          tc::mma_bf16_ts_w(od, pa + kk * 8, vl + kk * 128, hi, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+        tc::mma_commit(bar(B_PVDONE + w));
+        if (w == 1 || j >= n_kv1) tc::mma_commit(bar(B_VEMPTY + (j & 1)));
+        if (n + 3 < n_items) ok = issue_s_item(n + 3);     // into the buffer whose P the product above has just read
+        { const int it = j; TR(3 + 3 * w); }
+      }
+    } else {
     bool ok = tc::mbar_wait(bar(B_QFULL), 0, status, 203) && tc::mbar_wait(bar(B_KFULL), 0, status, 204);
     if (ok) {
       tc::tc_fence_after();
@@ -230,6 +285,7 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
       if (next) tc::mma_commit(bar(B_KEMPTY + ((j + 1) & 1)));   // ... and both score products of the next stage
       if (j == 0) tc::mma_commit(bar(B_KEMPTY));            // stage 0 scores were issued before the loop
     }
+    }
   } else if (warp >= 2) {
     // ---- softmax warp groups: group w owns query tile qt[w], one query row per thread --------------
     const int w = (warp - 2) / 4;
@@ -239,7 +295,7 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
     const int i0 = (w ? qt1 : qt0) * BQ;
     const int gi = i0 + r;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-    const uint32_t s_addr = lane_addr + w * 128, o_addr = lane_addr + O_COL + w * HD;
+    const uint32_t o_addr = lane_addr + O_COL + w * HD;
     const float c = P.scale * LOG2E;
     const float tau = RESCALE_LOG2 / c;              // the same threshold in raw score units
     pdl_wait();                                      // before this role writes anything
@@ -248,11 +304,18 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
     for (int j = 0; j < n_kvw && ok; ++j) {
       const int j0 = j * BKV;
       { const int it = j; if (r == 0) TR(8 + 8 * w); }
-      if (!tc::mbar_wait(bar(B_SFULL + w), j & 1, status, 208)) { ok = false; break; }
+      // score buffer and barrier phase of this (tile, key tile): see the MMA issuer
+      const int n_item = ROT ? (w ? 2 * j + 1 : j + min(j, n_kv1)) : j;
+      const int sbuf = ROT ? n_item % 3 : w;
+      const uint32_t sph = ROT ? (uint32_t)(n_item / 3) & 1u : (uint32_t)j & 1u;
+      const uint32_t s_addr = lane_addr + (uint32_t)sbuf * 128;
+      if (!tc::mbar_wait(bar(B_SFULL + sbuf), sph, status, 208)) { ok = false; break; }
       { const int it = j; if (r == 0) TR(9 + 8 * w); }
       tc::tc_fence_after();
       const bool need_mask = (j0 + BKV > P.seq) || (P.causal && j0 + BKV - 1 > i0);
-      float mx, sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f, alpha, mc;
+      float mx, alpha, mc;
+      float2 sum01 = make_float2(0.f, 0.f), sum23 = sum01;
+      const float2 c2 = make_float2(c, c);
       bool moved;
       if constexpr (TILES == 2) {
         // The row's 128 scores come into registers with one wait (one block per SM: a thread may hold them all):
@@ -272,8 +335,9 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
         }
         float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
   #pragma unroll
-        for (int k = 0; k < 128; k += 4) {
-          mx0 = fmaxf(mx0, sv[k]); mx1 = fmaxf(mx1, sv[k + 1]); mx2 = fmaxf(mx2, sv[k + 2]); mx3 = fmaxf(mx3, sv[k + 3]);
+        for (int k = 0; k < 128; k += 8) {               // three-input maxima: one instruction per two scores
+          mx0 = tc::fmax3(mx0, sv[k], sv[k + 1]); mx1 = tc::fmax3(mx1, sv[k + 2], sv[k + 3]);
+          mx2 = tc::fmax3(mx2, sv[k + 4], sv[k + 5]); mx3 = tc::fmax3(mx3, sv[k + 6], sv[k + 7]);
         }
         mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
         { const int it = j; if (r == 0) TR(10 + 8 * w); }
@@ -294,17 +358,22 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
             tc::tmem_ld32(o_addr + cc * 32, o);
             tc::tmem_ld_wait();
   #pragma unroll
-            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * a);
+            for (int k = 0; k < 32; k += 2) {
+              const float2 v = __fmul2_rn(make_float2(__uint_as_float(o[k]), __uint_as_float(o[k + 1])), make_float2(a, a));
+              o[k] = __float_as_uint(v.x); o[k + 1] = __float_as_uint(v.y);
+            }
             tc::tmem_st32(o_addr + cc * 32, o);
           }
         }
         { const int it = j; if (r == 0) TR(11 + 8 * w); }
         // P = exp2(S c - m c), its row sum, and P packed to bf16 (128 scores become 64 packed columns)
+        const float2 nmc2 = make_float2(-mc, -mc);
   #pragma unroll
         for (int k = 0; k < 128; k += 4) {
-          const float p0 = tc::fast_exp2(fmaf(sv[k], c, -mc)), p1 = tc::fast_exp2(fmaf(sv[k + 1], c, -mc));
-          const float p2 = tc::fast_exp2(fmaf(sv[k + 2], c, -mc)), p3 = tc::fast_exp2(fmaf(sv[k + 3], c, -mc));
-          sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+          const float2 x01 = __ffma2_rn(make_float2(sv[k], sv[k + 1]), c2, nmc2);       // two-wide fp32 operations
+          const float2 x23 = __ffma2_rn(make_float2(sv[k + 2], sv[k + 3]), c2, nmc2);
+          const float p0 = tc::fast_exp2(x01.x), p1 = tc::fast_exp2(x01.y), p2 = tc::fast_exp2(x23.x), p3 = tc::fast_exp2(x23.y);
+          sum01 = __fadd2_rn(sum01, make_float2(p0, p1)); sum23 = __fadd2_rn(sum23, make_float2(p2, p3));
           sr[k / 2] = tc::pack_bf16(p0, p1);
           sr[k / 2 + 1] = tc::pack_bf16(p2, p3);
         }
@@ -329,8 +398,9 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
           float* sc = reinterpret_cast<float*>(sr);
           if (need_mask) mask_chunk(sc, cc);
 #pragma unroll
-          for (int k = 0; k < 32; k += 4) {
-            mx0 = fmaxf(mx0, sc[k]); mx1 = fmaxf(mx1, sc[k + 1]); mx2 = fmaxf(mx2, sc[k + 2]); mx3 = fmaxf(mx3, sc[k + 3]);
+          for (int k = 0; k < 32; k += 8) {
+            mx0 = tc::fmax3(mx0, sc[k], sc[k + 1]); mx1 = tc::fmax3(mx1, sc[k + 2], sc[k + 3]);
+            mx2 = tc::fmax3(mx2, sc[k + 4], sc[k + 5]); mx3 = tc::fmax3(mx3, sc[k + 6], sc[k + 7]);
           }
         }
         mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
@@ -349,10 +419,14 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
             tc::tmem_ld32(o_addr + cc * 32, o);
             tc::tmem_ld_wait();
 #pragma unroll
-            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * a);
+            for (int k = 0; k < 32; k += 2) {
+              const float2 v = __fmul2_rn(make_float2(__uint_as_float(o[k]), __uint_as_float(o[k + 1])), make_float2(a, a));
+              o[k] = __float_as_uint(v.x); o[k + 1] = __float_as_uint(v.y);
+            }
             tc::tmem_st32(o_addr + cc * 32, o);
           }
         }
+        const float2 nmc2 = make_float2(-mc, -mc);
         // pass 2: P packed to bf16 over the score columns already consumed (32 scores become 16 packed columns;
         // the thread owns the lane, so nobody else's data is overwritten)
 #pragma unroll 1
@@ -365,9 +439,10 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
           uint32_t pk[16];
 #pragma unroll
           for (int k = 0; k < 32; k += 4) {
-            const float p0 = tc::fast_exp2(fmaf(sc[k], c, -mc)), p1 = tc::fast_exp2(fmaf(sc[k + 1], c, -mc));
-            const float p2 = tc::fast_exp2(fmaf(sc[k + 2], c, -mc)), p3 = tc::fast_exp2(fmaf(sc[k + 3], c, -mc));
-            sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+            const float2 x01 = __ffma2_rn(make_float2(sc[k], sc[k + 1]), c2, nmc2);
+            const float2 x23 = __ffma2_rn(make_float2(sc[k + 2], sc[k + 3]), c2, nmc2);
+            const float p0 = tc::fast_exp2(x01.x), p1 = tc::fast_exp2(x01.y), p2 = tc::fast_exp2(x23.x), p3 = tc::fast_exp2(x23.y);
+            sum01 = __fadd2_rn(sum01, make_float2(p0, p1)); sum23 = __fadd2_rn(sum23, make_float2(p2, p3));
             pk[k / 2] = tc::pack_bf16(p0, p1);
             pk[k / 2 + 1] = tc::pack_bf16(p2, p3);
           }
@@ -375,10 +450,10 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
         }
       }
       if (moved) l *= alpha;
-      l += (sum0 + sum1) + (sum2 + sum3);
+      l += (sum01.x + sum01.y) + (sum23.x + sum23.y);
       tc::tmem_st_wait();
       tc::tc_fence_before();
-      tc::mbar_arrive(bar(B_PFULL + w));
+      tc::mbar_arrive(bar(B_PFULL + sbuf));
       { const int it = j; if (r == 0) TR(12 + 8 * w); }
     }
     if (ok && n_kvw > 0) ok = tc::mbar_wait(bar(B_PVDONE + w), (n_kvw - 1) & 1, status, 210);
@@ -818,7 +893,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       // barrier only after finishing the previous iteration, including its reads of the dQ staging tile.
       float* s_lse = s_stage + (it & 1) * 256;
       float* s_d = s_lse + 128;
-      if (t < 256) s_lse[t] = t < 128 ? (stat_oob ? INFINITY : stat_next * LOG2E) : (stat_oob ? 0.f : stat_next);   // s_d follows s_lse
+      // stored negated (-LSE log2e, -D): both enter the arithmetic below as addends of two-wide operations
+      if (t < 256) s_lse[t] = t < 128 ? (stat_oob ? -INFINITY : -(stat_next * LOG2E)) : (stat_oob ? 0.f : -stat_next);   // s_d follows s_lse
       stat_next = fetch_stat(it + 1);
       tc::mbar_arrive(bar(BB_LSEREADY));
       if (!tc::mbar_wait(bar(BB_LSEREADY), it & 1, status, 308)) { ok = false; break; }
@@ -839,10 +915,6 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       if (!PIPE) {
         if (!tc::mbar_wait(bar(BB_SREAD), it & 1, status, 311)) { ok = false; break; }
         tc::tc_fence_after();
-      } else if (it > 0) {
-        // P^T has its own columns, single-buffered: the dV product of the previous tile must have read them
-        if (!tc::mbar_wait(bar(BB_DVDONE), (it - 1) & 1, status, 312)) { ok = false; break; }
-        tc::tc_fence_after();
       }
       // One 16-column chunk: P^T = exp2(S^T c - LSE) to tensor memory, dS^T = P^T (dP^T - D) to the swizzled
       // shared-memory operand tile, both rounded to bf16.  MASKED is the rare path (diagonal / ragged tiles).
@@ -857,24 +929,33 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         for (int k = 0; k < 16; k += 4) {
           const float4 l4 = *reinterpret_cast<const float4*>(&s_lse[c0 + k]);
           const float4 d4 = *reinterpret_cast<const float4*>(&s_d[c0 + k]);
-          const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dvv[4] = {d4.x, d4.y, d4.z, d4.w};
-          float pv[4], gv[4];
+          // two-wide fp32 operations (one instruction per pair): x = S^T c - LSE, then dS^T = P^T (dP^T - D)
+          const float2 c2 = make_float2(c, c);
+          const float2 x01 = __ffma2_rn(make_float2(__uint_as_float(sv[cc * 16 + k]), __uint_as_float(sv[cc * 16 + k + 1])), c2, make_float2(l4.x, l4.y));
+          const float2 x23 = __ffma2_rn(make_float2(__uint_as_float(sv[cc * 16 + k + 2]), __uint_as_float(sv[cc * 16 + k + 3])), c2, make_float2(l4.z, l4.w));
+          float pv[4] = {tc::fast_exp2(x01.x), tc::fast_exp2(x01.y), tc::fast_exp2(x23.x), tc::fast_exp2(x23.y)};
+          if (MASKED) {
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            float p = tc::fast_exp2(fmaf(__uint_as_float(sv[cc * 16 + k + u]), c, -lv[u]));
-            if (MASKED) {
+            for (int u = 0; u < 4; ++u) {
               const int gi = i0 + c0 + k + u;
-              if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) p = 0.f;
+              if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) pv[u] = 0.f;
             }
-            pv[u] = p;
-            gv[u] = p * (__uint_as_float(dpv[k + u]) - dvv[u]);
           }
+          const float2 g01 = __fmul2_rn(make_float2(pv[0], pv[1]), __fadd2_rn(make_float2(__uint_as_float(dpv[k]), __uint_as_float(dpv[k + 1])), make_float2(d4.x, d4.y)));
+          const float2 g23 = __fmul2_rn(make_float2(pv[2], pv[3]), __fadd2_rn(make_float2(__uint_as_float(dpv[k + 2]), __uint_as_float(dpv[k + 3])), make_float2(d4.z, d4.w)));
+          const float gv[4] = {g01.x, g01.y, g23.x, g23.y};
           pp[k / 2] = tc::pack_bf16(pv[0], pv[1]);
           pp[k / 2 + 1] = tc::pack_bf16(pv[2], pv[3]);
           dd[k / 2] = tc::pack_bf16(gv[0], gv[1]);
           dd[k / 2 + 1] = tc::pack_bf16(gv[2], gv[3]);
         }
         if (t == 0) TR(16 + cc);
+        if (PIPE && cc == 0 && it > 0) {
+          // P^T has its own columns, single-buffered: the dV product of the previous tile must have read them.
+          // The wait sits here, behind the first chunk's arithmetic, which needs only S^T and dP^T.
+          if (!tc::mbar_wait(bar(BB_DVDONE), (it - 1) & 1, status, 312)) { ok = false; return; }
+          tc::tc_fence_after();
+        }
         tc::tmem_st8(lane_addr + P_COL + c0 / 2, pp);
         // 16 query columns = 2 swizzled 16-byte chunks of this key row inside its 64-query panel
 #pragma unroll
@@ -886,11 +967,12 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       };
       if (need_mask) {
         chunk(0, std::true_type{});
-        chunk(1, std::true_type{});
+        if (ok) chunk(1, std::true_type{});
       } else {
         chunk(0, std::false_type{});
-        chunk(1, std::false_type{});
+        if (ok) chunk(1, std::false_type{});
       }
+      if (!ok) break;
       tc::tmem_st_wait();
       if (t == 0) TR(15);
       tc::fence_proxy_async();
