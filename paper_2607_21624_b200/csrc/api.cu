@@ -126,7 +126,7 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   p->sv_k = o;     o += mat(p->dkv);
   p->sv_v = o;     o += mat(p->dkv);
   p->sv_a = o;     o += mat(p->dq);
-  p->sv_lse = o;   o += fbl_align_up(rows_bh * sizeof(float), FBL_ALIGN);
+  p->sv_lse = o;   o += fbl_align_up(rows_bh * sizeof(float) + 512, FBL_ALIGN);   // + one 128-float copy window past the last row
   p->saved_bytes = o;
 
   // partial-sum area: column-sum slabs or split-K slices, whichever is larger

@@ -557,19 +557,22 @@ struct alignas(64) AttnBwdParams {
 template <int HD>
 struct BwdSmem {
   static constexpr bool PIPE = HD == 64;
-  static constexpr uint32_t NQ = PIPE ? 2 : 1, NP = PIPE ? 2 : 1;      // stages of Q/dO and of dS^T / staging
+  // stages: Q (needed first, for the next S^T, and freed last, by dK) three deep, dO and dS^T two deep, one dQ
+  // staging tile; everything single at HD = 128
+  static constexpr uint32_t NQQ = PIPE ? 3 : 1, NDO = PIPE ? 2 : 1, NP = PIPE ? 2 : 1, NS = 1;
   static constexpr uint32_t PANELS = HD / 64;
   static constexpr uint32_t TILE = PANELS * 16384;
   static constexpr uint32_t STAGE_BYTES = 128 * HD * 4;               // one fp32 dQ tile
-  static constexpr uint32_t K_OFF = 0, V_OFF = TILE, Q_OFF = 2 * TILE, DO_OFF = Q_OFF + NQ * TILE;
-  static constexpr uint32_t DS_OFF = DO_OFF + NQ * TILE, STAGE_OFF = DS_OFF + NP * 32768;
-  static constexpr uint32_t LSE_OFF = STAGE_OFF + NP * STAGE_BYTES;    // 2 buffers x (128 floats LSE*log2e, 128 floats D)
-  static constexpr uint32_t BAR_OFF = LSE_OFF + 2048;
-  static constexpr uint32_t N_BARS = 16;
+  static constexpr uint32_t K_OFF = 0, V_OFF = TILE, Q_OFF = 2 * TILE, DO_OFF = Q_OFF + NQQ * TILE;
+  static constexpr uint32_t DS_OFF = DO_OFF + NDO * TILE, STAGE_OFF = DS_OFF + NP * 32768;
+  static constexpr uint32_t LSE_OFF = STAGE_OFF + NS * STAGE_BYTES;    // 128 floats of LSE per Q stage, then 128 of D per dO stage
+  static constexpr uint32_t D_OFF = LSE_OFF + NQQ * 512;
+  static constexpr uint32_t BAR_OFF = D_OFF + NDO * 512;
+  static constexpr uint32_t N_BARS = 20;
   static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16;
 };
 
-enum { BB_KVFULL = 0, BB_QDOFULL = 1, BB_QDOEMPTY = 3, BB_SFULL = 5, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_LSEREADY, BB_DQSTAGED, BB_STAGEFREE = BB_DQSTAGED + 2, BB_SREAD = BB_STAGEFREE + 2, BB_DVDONE };
+enum { BB_KVFULL = 0, BB_QFULL = 1, BB_QEMPTY = 4, BB_DOFULL = 7, BB_DOEMPTY = 9, BB_SFULL = 11, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_DQSTAGED, BB_STAGEFREE = BB_DQSTAGED + 2, BB_SREAD = BB_STAGEFREE + 2, BB_DVDONE };
 
 constexpr int BWD_THREADS = 608;     // warp 0 TMA loads, warp 1 MMA, warps 2-17 softmax (four per TMEM lane quarter), warp 18 dQ reductions
 constexpr int BWD_SM_THREADS = 512;
@@ -578,7 +581,7 @@ template <int HD>
 __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __grid_constant__ AttnBwdParams P) {
   using SM = BwdSmem<HD>;
   constexpr bool PIPE = SM::PIPE;
-  constexpr uint32_t PANELS = SM::PANELS, NQ = SM::NQ, NP = SM::NP;
+  constexpr uint32_t PANELS = SM::PANELS, NQQ = SM::NQQ, NDO = SM::NDO, NP = SM::NP, NS = SM::NS;
   constexpr uint32_t S_COL = 0, DP_COL = 128, DV_COL = 256, DK_COL = 256 + HD;
   constexpr uint32_t DQ_COL = PIPE ? 384 : DP_COL;   // HD = 128: dQ reuses the dP^T columns
   constexpr uint32_t P_COL = PIPE ? 448 : S_COL;     // HD = 64: own columns; HD = 128: P^T overwrites S^T in place
@@ -607,15 +610,18 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
 
   if (threadIdx.x == 0) {
     tc::mbar_init(bar(BB_KVFULL), 1);
+    for (int s = 0; s < 3; ++s) {
+      tc::mbar_init(bar(BB_QFULL + s), 1);
+      tc::mbar_init(bar(BB_QEMPTY + s), 1);
+    }
     for (int s = 0; s < 2; ++s) {
-      tc::mbar_init(bar(BB_QDOFULL + s), 1);
-      tc::mbar_init(bar(BB_QDOEMPTY + s), 1);
+      tc::mbar_init(bar(BB_DOFULL + s), 1);
+      tc::mbar_init(bar(BB_DOEMPTY + s), 1);
     }
     tc::mbar_init(bar(BB_SFULL), 1);
     tc::mbar_init(bar(BB_PDSFULL), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_DQFULL), 1);
     tc::mbar_init(bar(BB_DQDRAINED), BWD_SM_THREADS);
-    tc::mbar_init(bar(BB_LSEREADY), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_DQSTAGED), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_DQSTAGED + 1), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_STAGEFREE), 1);
@@ -631,8 +637,10 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     tc::tma_load_3d(base + SM::K_OFF, &P.tk, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
     tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
     if (n_it > 0) {
-      tc::mbar_expect_tx(bar(BB_QDOFULL), PIPE ? 2 * SM::TILE : SM::TILE);
-      tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(BB_QDOFULL), 0, row0 + qt_begin * BQ, g * P.group * (int)PANELS);
+      // LSE travels with Q and D with dO: 128 floats each, into the iteration's staging buffer
+      tc::mbar_expect_tx(bar(BB_QFULL), SM::TILE + 512);
+      tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(BB_QFULL), 0, row0 + qt_begin * BQ, g * P.group * (int)PANELS);
+      tc::bulk_load(base + SM::LSE_OFF, P.lse + ((long long)b * P.hq + g * P.group) * P.t_pad + qt_begin * BQ, 512, bar(BB_QFULL));
     }
   }
   if (warp == 1) {
@@ -645,6 +653,14 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
   uint32_t tmem_base;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
   pdl_launch_dependents();
+  // Where a block's dQ tiles are staged for the bulk reduction: one staging tile; with the pipelined variant the
+  // last tile goes to the dS^T buffer that the last iteration does not use (its readers, the dK and dQ products of
+  // the tile before, are complete by then), so the block's final drain does not wait for the previous reduction.
+  auto stage_is_alt = [&](int dit) { return PIPE && dit == n_it - 1 && n_it >= 2; };
+  auto stage_addr = [&](int dit) -> uint32_t {
+    return stage_is_alt(dit) ? base + SM::DS_OFF + (uint32_t)(n_it % (int)NP) * 32768u
+                             : base + SM::STAGE_OFF + (uint32_t)(dit % (int)NS) * SM::STAGE_BYTES;
+  };
   // Of this kernel's inputs only dO (and D) come from the kernel before it (the dA GEMM); K, V, Q and LSE are the
   // forward pass's.  Each role therefore waits for that kernel where it first needs it: the producer has K, V
   // and the first Q tile on their way before it does.
@@ -654,29 +670,22 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     bool waited = false;
     for (int it = 0; it < n_it; ++it) {
       const int h = g * P.group + it / per_head, qt = qt_begin + it % per_head;
-      if (PIPE) {
-        const uint32_t s = it % NQ, ph = (it / NQ) & 1;
-        if (it > 0) {
-          if (!tc::mbar_wait(bar(BB_QDOEMPTY + s), ph ^ 1, status, 301)) break;
-          tc::mbar_expect_tx(bar(BB_QDOFULL + s), 2 * SM::TILE);
-          tc::tma_load_3d(base + SM::Q_OFF + s * SM::TILE, &P.tq, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
-        }
-        if (!waited) { pdl_wait(); waited = true; }
-        tc::tma_load_3d(base + SM::DO_OFF + s * SM::TILE, &P.tdo, bar(BB_QDOFULL + s), 0, row0 + qt * BQ, h * (int)PANELS);
-      } else {
-        // single buffers: Q and dO have a barrier pair each (slot 0: Q, slot 1: dO), since Q is free after the dK
-        // product and dO only after the dV product, and the next score tile needs Q alone
-        const uint32_t ph = it & 1;
-        if (it > 0) {
-          if (!tc::mbar_wait(bar(BB_QDOEMPTY), ph ^ 1, status, 301)) break;
-          tc::mbar_expect_tx(bar(BB_QDOFULL), SM::TILE);
-          tc::tma_load_3d(base + SM::Q_OFF, &P.tq, bar(BB_QDOFULL), 0, row0 + qt * BQ, h * (int)PANELS);
-        }
-        if (!tc::mbar_wait(bar(BB_QDOEMPTY + 1), ph ^ 1, status, 313)) break;
-        if (!waited) { pdl_wait(); waited = true; }
-        tc::mbar_expect_tx(bar(BB_QDOFULL + 1), SM::TILE);
-        tc::tma_load_3d(base + SM::DO_OFF, &P.tdo, bar(BB_QDOFULL + 1), 0, row0 + qt * BQ, h * (int)PANELS);
+      // LSE travels with Q and D with dO, 128 floats each.  A stage's previous readers (the products, and for
+      // LSE / D the softmax warps, which finish a tile before its dK and dV products are issued) are behind the
+      // barrier that frees it.  Rows past the sequence end may hold anything: the softmax warps mask them.
+      const long long stat_off = ((long long)b * P.hq + h) * P.t_pad + qt * BQ;
+      const uint32_t sq = it % NQQ, sd = it % NDO;
+      if (it > 0) {
+        if (!tc::mbar_wait(bar(BB_QEMPTY + sq), ((it / NQQ) & 1) ^ 1, status, 301)) break;
+        tc::mbar_expect_tx(bar(BB_QFULL + sq), SM::TILE + 512);
+        tc::tma_load_3d(base + SM::Q_OFF + sq * SM::TILE, &P.tq, bar(BB_QFULL + sq), 0, row0 + qt * BQ, h * (int)PANELS);
+        tc::bulk_load(base + SM::LSE_OFF + sq * 512, P.lse + stat_off, 512, bar(BB_QFULL + sq));
       }
+      if (!tc::mbar_wait(bar(BB_DOEMPTY + sd), ((it / NDO) & 1) ^ 1, status, 313)) break;
+      if (!waited) { pdl_wait(); waited = true; }
+      tc::mbar_expect_tx(bar(BB_DOFULL + sd), SM::TILE + 512);
+      tc::tma_load_3d(base + SM::DO_OFF + sd * SM::TILE, &P.tdo, bar(BB_DOFULL + sd), 0, row0 + qt * BQ, h * (int)PANELS);
+      tc::bulk_load(base + SM::D_OFF + sd * 512, P.dvec + stat_off, 512, bar(BB_DOFULL + sd));
     }
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer --------------------------------------------------------------------------
@@ -692,7 +701,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     const uint32_t do_km = tc::smem_desc_lo(base + SM::DO_OFF, 16), do_mn = tc::smem_desc_lo(base + SM::DO_OFF, 16384);
     const uint32_t ds_km = tc::smem_desc_lo(base + SM::DS_OFF, 16), ds_mn = tc::smem_desc_lo(base + SM::DS_OFF, 16384);
     auto issue_s = [&](int it) {              // S^T = K Q^T of tile `it`
-      const uint32_t qs = q_km + (it % NQ) * (SM::TILE >> 4);
+      const uint32_t qs = q_km + (it % NQQ) * (SM::TILE >> 4);
 #pragma unroll
       for (uint32_t kk = 0; kk < HD / 16; ++kk) {
         const uint32_t o = (kk / 4) * 1024 + (kk % 4) * 2;
@@ -700,7 +709,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       }
     };
     auto issue_dp = [&](int it) {             // dP^T = V dO^T of tile `it`; then both score tiles are announced
-      const uint32_t dos = do_km + (it % NQ) * (SM::TILE >> 4);
+      const uint32_t dos = do_km + (it % NDO) * (SM::TILE >> 4);
 #pragma unroll
       for (uint32_t kk = 0; kk < HD / 16; ++kk) {
         const uint32_t o = (kk / 4) * 1024 + (kk % 4) * 2;
@@ -709,14 +718,14 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       tc::mma_commit(bar(BB_SFULL));
     };
     auto issue_dv = [&](int it) {             // dV += P^T dO, P^T read from tensor memory
-      const uint32_t dos = do_mn + (it % NQ) * (SM::TILE >> 4);
+      const uint32_t dos = do_mn + (it % NDO) * (SM::TILE >> 4);
 #pragma unroll
       for (uint32_t kk = 0; kk < BQ / 16; ++kk)                      // dO: MN-major, 16 query rows per step;
         tc::mma_bf16_ts_w(tmem_base + DV_COL, tmem_base + P_COL + kk * 8,   // 16 queries = 8 packed columns
                           dos + kk * 128, hi, idesc_kv, (it > 0 || kk > 0) ? 1u : 0u);
     };
     auto issue_dk = [&](int it) {             // dK += dS^T Q
-      const uint32_t qs = q_mn + (it % NQ) * (SM::TILE >> 4);
+      const uint32_t qs = q_mn + (it % NQQ) * (SM::TILE >> 4);
       const uint32_t dss = ds_km + (it % NP) * 2048;
 #pragma unroll
       for (uint32_t kk = 0; kk < BQ / 16; ++kk) {
@@ -734,8 +743,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     };
     bool ok = tc::mbar_wait(bar(BB_KVFULL), 0, status, 302);
     if (ok && n_it > 0) {
-      ok = tc::mbar_wait(bar(BB_QDOFULL), 0, status, 303);
-      if (ok && !PIPE) ok = tc::mbar_wait(bar(BB_QDOFULL + 1), 0, status, 314);
+      ok = tc::mbar_wait(bar(BB_QFULL), 0, status, 303) && tc::mbar_wait(bar(BB_DOFULL), 0, status, 314);
       if (ok) { tc::tc_fence_after(); issue_s(0); issue_dp(0); }
     }
     if (PIPE) {
@@ -747,7 +755,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
           // S^T(it+1) as soon as every softmax warp has copied S^T(it) to registers: it is computed while
           // they work on tile it
           if (!tc::mbar_wait(bar(BB_SREAD), it & 1, status, 311)) { ok = false; break; }
-          if (!tc::mbar_wait(bar(BB_QDOFULL + ((it + 1) % NQ)), ((it + 1) / NQ) & 1, status, 303)) { ok = false; break; }
+          if (!tc::mbar_wait(bar(BB_QFULL + ((it + 1) % NQQ)), ((it + 1) / NQQ) & 1, status, 303)) { ok = false; break; }
           TR(1);
           tc::tc_fence_after();
           issue_s(it + 1);
@@ -755,16 +763,20 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
         TR(2);
         tc::tc_fence_after();
-        if (it + 1 < n_it) issue_dp(it + 1);            // dP^T(it) has been read as well: announce tile it + 1
+        if (it + 1 < n_it) {
+          if (!tc::mbar_wait(bar(BB_DOFULL + ((it + 1) % NDO)), ((it + 1) / NDO) & 1, status, 314)) { ok = false; break; }
+          issue_dp(it + 1);                             // dP^T(it) has been read as well: announce tile it + 1
+        }
         TR(3);
         issue_dv(it);
         tc::mma_commit(bar(BB_DVDONE));                 // P^T(it) has been read: P^T(it+1) may be stored
+        tc::mma_commit(bar(BB_DOEMPTY + (it % NDO)));   // ... and dO of this tile is not read again
         TR(4);
+        issue_dk(it);
+        tc::mma_commit(bar(BB_QEMPTY + (it % NQQ)));    // nor is Q
         if (it > 0 && !tc::mbar_wait(bar(BB_DQDRAINED), (it - 1) & 1, status, 304)) { ok = false; break; }
         TR(5);
         tc::tc_fence_after();
-        issue_dk(it);
-        tc::mma_commit(bar(BB_QDOEMPTY + (it % NQ)));   // Q / dO of this tile are not read again
         issue_dq(it);
         TR(6);
       }
@@ -778,17 +790,17 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         // the dV and dK products
         issue_dq(it);
         issue_dk(it);
-        tc::mma_commit(bar(BB_QDOEMPTY));               // Q of this tile is not read again: the next one is fetched
+        tc::mma_commit(bar(BB_QEMPTY));                 // Q of this tile is not read again: the next one is fetched
         issue_dv(it);                                   // while dV runs
-        tc::mma_commit(bar(BB_QDOEMPTY + 1));           // ... and dO
+        tc::mma_commit(bar(BB_DOEMPTY));                // ... and dO
         TR(2);
         if (it + 1 < n_it) {
-          if (!tc::mbar_wait(bar(BB_QDOFULL), (it + 1) & 1, status, 303)) { ok = false; break; }
+          if (!tc::mbar_wait(bar(BB_QFULL), (it + 1) & 1, status, 303)) { ok = false; break; }
           TR(3);
           tc::tc_fence_after();
           issue_s(it + 1);                   // the S^T columns (P^T by now) were last read by dV above
           if (!tc::mbar_wait(bar(BB_DQDRAINED), it & 1, status, 304)) { ok = false; break; }
-          if (!tc::mbar_wait(bar(BB_QDOFULL + 1), (it + 1) & 1, status, 314)) { ok = false; break; }
+          if (!tc::mbar_wait(bar(BB_DOFULL), (it + 1) & 1, status, 314)) { ok = false; break; }
           TR(4);
           tc::tc_fence_after();
           issue_dp(it + 1);                  // the dP^T columns held dQ until it was drained
@@ -805,14 +817,14 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       pdl_wait();                                    // the accumulator's zero-fill precedes the kernel before this one
       for (int dit = 0; dit < n_it; ++dit) {
         const int h = g * P.group + dit / per_head, i0 = (qt_begin + dit % per_head) * BQ;
-        if (!tc::mbar_wait(bar(BB_DQSTAGED + (dit % NP)), (dit / (int)NP) & 1, status, 309)) break;   // one per buffer, like STAGEFREE
-        const uint32_t stage = base + SM::STAGE_OFF + (dit % NP) * SM::STAGE_BYTES;
+        if (!tc::mbar_wait(bar(BB_DQSTAGED + (dit % NS)), (dit / (int)NS) & 1, status, 309)) break;   // one per buffer, like STAGEFREE
+        const uint32_t stage = stage_addr(dit);
 #pragma unroll
         for (int pn = 0; pn < (int)PANELS; ++pn)
           tc::tma_reduce_add_4d(&P.tdq, stage + pn * 32768, 0, 0, row0 + i0, h * (int)PANELS + pn);
         tc::bulk_commit_group();
         tc::bulk_wait_group_read0();                 // the staging tile has been read: it may be overwritten
-        tc::mbar_arrive(bar(BB_STAGEFREE + (dit % NP)));     // one barrier per staging buffer: a waiter is never
+        tc::mbar_arrive(bar(BB_STAGEFREE + (dit % NS)));     // one barrier per staging buffer: a waiter is never
                                                              // more than one phase behind
       }
       tc::bulk_wait_group0();
@@ -834,10 +846,10 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     // staging tile in shared memory in the 128-byte-swizzled box layout of the accumulator's tensor map; the
     // reduction warp then adds the whole tile to global memory asynchronously, off the critical path.
     auto drain_dq = [&](int dit) -> bool {
-      const uint32_t stage = base + SM::STAGE_OFF + (dit % NP) * SM::STAGE_BYTES;
+      const uint32_t stage = stage_addr(dit);
       if (!tc::mbar_wait(bar(BB_DQFULL), dit & 1, status, 307)) return false;
       // the staging buffer's previous tile must have been read by its bulk reduction
-      if (dit >= (int)NP && !tc::mbar_wait(bar(BB_STAGEFREE + (dit % NP)), (dit / (int)NP - 1) & 1, status, 310)) return false;
+      if (dit >= (int)NS && !stage_is_alt(dit) && !tc::mbar_wait(bar(BB_STAGEFREE + (dit % NS)), (dit / (int)NS - 1) & 1, status, 310)) return false;
       { const int it = dit; if (t == 0) TR(8); }
       tc::tc_fence_after();
 #pragma unroll 1
@@ -861,43 +873,18 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       { const int it = dit; if (t == 0) TR(7); }
       tc::mbar_arrive(bar(BB_DQDRAINED));            // TMEM side done: the tensor pipe may reuse the columns
       tc::fence_proxy_async();
-      tc::mbar_arrive(bar(BB_DQSTAGED + (dit % NP)));     // staging side done: the reduction warp takes over
+      tc::mbar_arrive(bar(BB_DQSTAGED + (dit % NS)));     // staging side done: the reduction warp takes over
       return true;
     };
-
-    // LSE / D of a query tile: thread t < 128 fetches LSE[t], thread 128 <= t < 256 fetches D[t - 128].  The
-    // value for the next iteration is requested one iteration ahead so its latency is off the critical path.
-    // (head, query tile) of the tile being fetched and of the tile being processed advance by counting: an
-    // integer division per thread and iteration is a noticeable share of this loop's instructions
-    int f_h = 0, f_q = 0;                           // fetch position: head within the group, query tile within the head
-    // The value is used (scaled, stored to shared memory) only at the top of the next iteration: nothing here may
-    // depend on the load, or the thread would wait out its L2 latency before reaching the barrier below.
-    bool stat_oob = false;
-    auto fetch_stat = [&](int fit) -> float {
-      const int h = g * P.group + f_h, i0 = (qt_begin + f_q) * BQ;
-      if (++f_q == per_head) { f_q = 0; ++f_h; }
-      const int gi = i0 + (t & 127);
-      stat_oob = t >= 256 || fit >= n_it || gi >= P.seq;
-      if (stat_oob) return 0.f;
-      const long long o = ((long long)b * P.hq + h) * P.t_pad + gi;
-      return __ldg((t < 128 ? P.lse : P.dvec) + o);
-    };
-    float stat_next = fetch_stat(0);
 
     int c_q = 0;                                    // query tile within the head of the tile being processed
     for (int it = 0; it < n_it && ok; ++it) {
       const int i0 = (qt_begin + c_q) * BQ;
       if (++c_q == per_head) c_q = 0;
-      // LSE and D of this query tile, staged in shared memory (two buffers by iteration parity: every
-      // reader of a buffer's previous use arrived at PDSFULL two iterations ago).  All threads pass this
-      // barrier only after finishing the previous iteration, including its reads of the dQ staging tile.
-      float* s_lse = s_stage + (it & 1) * 256;
-      float* s_d = s_lse + 128;
-      // stored negated (-LSE log2e, -D): both enter the arithmetic below as addends of two-wide operations
-      if (t < 256) s_lse[t] = t < 128 ? (stat_oob ? -INFINITY : -(stat_next * LOG2E)) : (stat_oob ? 0.f : -stat_next);   // s_d follows s_lse
-      stat_next = fetch_stat(it + 1);
-      tc::mbar_arrive(bar(BB_LSEREADY));
-      if (!tc::mbar_wait(bar(BB_LSEREADY), it & 1, status, 308)) { ok = false; break; }
+      // LSE and D of this query tile were copied to shared memory by the producer (a buffer per Q / dO stage)
+      // and arrived before the score products awaited below were issued
+      const float* s_lse = s_stage + (it % NQQ) * 128;
+      const float* s_d = s_stage + NQQ * 128 + (it % NDO) * 128;
       if (t == 0) TR(9);
       if (!tc::mbar_wait(bar(BB_SFULL), it & 1, status, 306)) { ok = false; break; }
       if (t == 0) TR(10);
@@ -929,10 +916,11 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         for (int k = 0; k < 16; k += 4) {
           const float4 l4 = *reinterpret_cast<const float4*>(&s_lse[c0 + k]);
           const float4 d4 = *reinterpret_cast<const float4*>(&s_d[c0 + k]);
-          // two-wide fp32 operations (one instruction per pair): x = S^T c - LSE, then dS^T = P^T (dP^T - D)
+          // two-wide fp32 operations (one instruction per pair): x = S^T c - LSE log2e, then dS^T = P^T (dP^T - D)
           const float2 c2 = make_float2(c, c);
-          const float2 x01 = __ffma2_rn(make_float2(__uint_as_float(sv[cc * 16 + k]), __uint_as_float(sv[cc * 16 + k + 1])), c2, make_float2(l4.x, l4.y));
-          const float2 x23 = __ffma2_rn(make_float2(__uint_as_float(sv[cc * 16 + k + 2]), __uint_as_float(sv[cc * 16 + k + 3])), c2, make_float2(l4.z, l4.w));
+          const float2 nl2e = make_float2(-LOG2E, -LOG2E), neg1 = make_float2(-1.f, -1.f);
+          const float2 x01 = __ffma2_rn(make_float2(__uint_as_float(sv[cc * 16 + k]), __uint_as_float(sv[cc * 16 + k + 1])), c2, __fmul2_rn(make_float2(l4.x, l4.y), nl2e));
+          const float2 x23 = __ffma2_rn(make_float2(__uint_as_float(sv[cc * 16 + k + 2]), __uint_as_float(sv[cc * 16 + k + 3])), c2, __fmul2_rn(make_float2(l4.z, l4.w), nl2e));
           float pv[4] = {tc::fast_exp2(x01.x), tc::fast_exp2(x01.y), tc::fast_exp2(x23.x), tc::fast_exp2(x23.y)};
           if (MASKED) {
 #pragma unroll
@@ -941,9 +929,16 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
               if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) pv[u] = 0.f;
             }
           }
-          const float2 g01 = __fmul2_rn(make_float2(pv[0], pv[1]), __fadd2_rn(make_float2(__uint_as_float(dpv[k]), __uint_as_float(dpv[k + 1])), make_float2(d4.x, d4.y)));
-          const float2 g23 = __fmul2_rn(make_float2(pv[2], pv[3]), __fadd2_rn(make_float2(__uint_as_float(dpv[k + 2]), __uint_as_float(dpv[k + 3])), make_float2(d4.z, d4.w)));
-          const float gv[4] = {g01.x, g01.y, g23.x, g23.y};
+          const float2 g01 = __fmul2_rn(make_float2(pv[0], pv[1]), __ffma2_rn(make_float2(d4.x, d4.y), neg1, make_float2(__uint_as_float(dpv[k]), __uint_as_float(dpv[k + 1]))));
+          const float2 g23 = __fmul2_rn(make_float2(pv[2], pv[3]), __ffma2_rn(make_float2(d4.z, d4.w), neg1, make_float2(__uint_as_float(dpv[k + 2]), __uint_as_float(dpv[k + 3]))));
+          float gv[4] = {g01.x, g01.y, g23.x, g23.y};
+          if (MASKED) {                              // LSE / D of rows past the sequence end are not defined
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int gi = i0 + c0 + k + u;
+              if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) gv[u] = 0.f;
+            }
+          }
           pp[k / 2] = tc::pack_bf16(pv[0], pv[1]);
           pp[k / 2 + 1] = tc::pack_bf16(pv[2], pv[3]);
           dd[k / 2] = tc::pack_bf16(gv[0], gv[1]);
