@@ -408,7 +408,21 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
   // of sliced weight-gradient GEMMs and the dQ accumulator.  No fill then separates later kernels of the step,
   // so each can start (programmatic dependent launch) while its predecessor drains.
   const bool split_o = p->use_tc && p->ksplit_o > 1, split_qkv = p->use_tc && p->ksplit_qkv > 1;
-  FBL_CUDA(cudaMemsetAsync(status, 0, p->zero_bytes, st));
+  // Without sliced GEMMs on the tensor-core path (only the dQ accumulator and the status word to clear) the first
+  // GEMM launch does it instead: its idle epilogue warps zero the accumulator while its first tiles are computed.
+  // The fill node was also the barrier between the forward and the backward kernels, which the attention backward
+  // relies on when it requests forward-pass data (K, V, Q, LSE) before waiting for the kernel in front of it: that
+  // GEMM is therefore launched without programmatic overlap, i.e. only once the forward pass has completed.
+  bool first_gemm_fills = false;
+  // (Measured: 2 % on workload 2; for accumulators of tens of MB the stores delay the launch's own first tiles by
+  // more than the fill node costs, so large plans keep the node.)
+  if (p->use_tc && p->acc_bytes == 0 && attn_bwd_tc_supported(p) && p->zero_bytes - p->sb_dqacc <= ((size_t)16 << 20)) {
+    GemmArgs gw = GemmArgs{}, ga = GemmArgs{};
+    gw.m = p->dq; gw.n = D; gw.n_terms = 1; gw.t[0] = {A, p->n_pad, 1, dY, p->n_pad, 0, n}; gw.c = dWo; gw.c_rpad = p->dq;
+    ga.m = n; ga.n = p->dq; ga.n_terms = 1; ga.t[0] = {dY, p->n_pad, 0, Wo, p->dq, 1, D}; ga.c = dA; ga.c_rpad = p->n_pad;
+    first_gemm_fills = gemm_tc_supported(p, gw) && gemm_tc_supported(p, ga);
+  }
+  if (!first_gemm_fills) FBL_CUDA(cudaMemsetAsync(status, 0, p->zero_bytes, st));
   FBL_PROF_BEGIN();
   bool dvec_ready = false;
   {
@@ -429,6 +443,10 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
       ga.dot_with = A; ga.dot_out = dvec; ga.dot_hd = p->d.head_dim; ga.dot_hq = p->d.n_q_heads;
       dvec_ready = true;
       if (split_o) { gw.ksplit = p->ksplit_o; gw.acc = (float*)(sc + p->sb_acc_o); }
+      if (first_gemm_fills) {
+        gs[0].zero_ptr = dqacc; gs[0].zero_bytes = p->zero_bytes - p->sb_dqacc;
+        gs[0].reset_status = 1; gs[0].serial = 1;
+      }
       FBL_STEP("dWo+dA", 1, launch_gemm_tc_group(p, gs, 2, status, st));
       if (split_o) {
         ConvertGroup cg = {};

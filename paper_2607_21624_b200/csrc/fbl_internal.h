@@ -81,6 +81,10 @@ struct GemmArgs {
   // reduction loop cut into ksplit slices whose fp32 partial tiles are added into `acc` (zeroed by the caller, same
   // element order as C with 4-byte elements); C itself is then produced from acc by launch_convert_f32_group
   int ksplit; float* acc;
+  // of a group's first problem: chores of the launch (zero-fill zero_bytes, a multiple of 16, at zero_ptr for a
+  // later kernel of the pass; reset the pass's status word), and `serial`: the launch may not start before
+  // everything ahead of it on the stream has completed
+  void* zero_ptr; size_t zero_bytes; int reset_status, serial;
 };
 
 cudaError_t launch_gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);

@@ -44,7 +44,22 @@ struct alignas(64) TcGroup {
   int count;
   int32_t* status;
   int trace_slot;
+  // Optional chores for the epilogue warps while the first tile's main loop runs: zero-fill a buffer that a later
+  // kernel of the pass adds into (16-byte units, dealt evenly to the blocks), and reset the pass's status word.
+  uint4* zero_ptr;
+  long long zero_vec;
+  int reset_status;
 };
+
+__device__ __forceinline__ void group_chores(const TcGroup& G, int tid, int n_threads) {
+  if (G.reset_status && blockIdx.x == 0 && tid == 0) *G.status = 0;
+  if (G.zero_vec > 0) {
+    const long long per = (G.zero_vec + gridDim.x - 1) / gridDim.x;
+    const long long lo = (long long)blockIdx.x * per, hi = min(G.zero_vec, lo + per);
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    for (long long i = lo + tid; i < hi; i += n_threads) G.zero_ptr[i] = z;
+  }
+}
 
 #ifdef FBL_TRACE_GEMM
 int g_trace_launch = 0;
@@ -240,6 +255,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
     // its TMEM lane quarter and two 32 x 64 staging tiles, and issues its own stores: no block-wide hand-off per
     // panel, and the store of one panel overlaps the conversion of the next. ---------------------------------
     pdl_wait();                                       // the previous kernel may still be reading what we overwrite
+    group_chores(G, threadIdx.x - 64, 128);
     const int q = warp % 4;                           // the TMEM lane quarter this warp may access
     const int r = q * 32 + lane;                      // row of the tile owned by this thread
     const bool tracer = threadIdx.x == 64;
@@ -537,6 +553,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1) gemm_tc_pair
   } else if (warp >= 2) {
     // ---- epilogue (both CTAs): this CTA's 128 accumulator rows, as in the single-CTA kernel -------------
     pdl_wait();
+    group_chores(G, threadIdx.x - 64, 128);
     const int q = warp % 4;
     const int r = q * 32 + lane;
     int ti = 0, pc = 0;
@@ -740,6 +757,7 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
   memset(&G, 0, sizeof(G));
   G.count = count;
   G.status = status;
+  G.zero_ptr = (uint4*)gs[0].zero_ptr; G.zero_vec = (long long)(gs[0].zero_bytes / 16); G.reset_status = gs[0].reset_status;
 #ifdef FBL_TRACE_GEMM
   G.trace_slot = (g_trace_launch++) & 1;      // two GEMM launches per pass
 #endif
@@ -782,7 +800,8 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
   cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
   if (attr_err != cudaSuccess) return attr_err;
   const int grid = tiles < p->sm_count ? tiles : p->sm_count;
-  return launch_pdl(k, dim3(grid), dim3(192), SP::TOTAL, st, G);
+  return gs[0].serial ? launch_serial(k, dim3(grid), dim3(192), SP::TOTAL, st, G)
+                      : launch_pdl(k, dim3(grid), dim3(192), SP::TOTAL, st, G);
 }
 
 cudaError_t launch_group_pair(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
@@ -790,6 +809,7 @@ cudaError_t launch_group_pair(const fbl_plan* p, const GemmArgs* gs, int count, 
   memset(&G, 0, sizeof(G));
   G.count = count;
   G.status = status;
+  G.zero_ptr = (uint4*)gs[0].zero_ptr; G.zero_vec = (long long)(gs[0].zero_bytes / 16); G.reset_status = gs[0].reset_status;
 #ifdef FBL_TRACE_GEMM
   G.trace_slot = (g_trace_launch++) & 1;      // two GEMM launches per pass
 #endif
@@ -832,7 +852,8 @@ cudaError_t launch_group_pair(const fbl_plan* p, const GemmArgs* gs, int count, 
   cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
   if (attr_err != cudaSuccess) return attr_err;
   const int pairs = tiles < p->sm_count / 2 ? tiles : p->sm_count / 2;
-  return launch_pdl(k, dim3(2 * pairs), dim3(192), SP::TOTAL, st, G);
+  return gs[0].serial ? launch_serial(k, dim3(2 * pairs), dim3(192), SP::TOTAL, st, G)
+                      : launch_pdl(k, dim3(2 * pairs), dim3(192), SP::TOTAL, st, G);
 }
 
 cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
