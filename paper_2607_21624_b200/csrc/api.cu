@@ -508,7 +508,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
   float* O4[4] = {dbo, dbq, dbk, dbv};
   const int C4[4] = {D, p->dq, p->dkv, p->dkv};
   if (bias && norm_bwd_takes_colsums(p)) {
-    FBL_STEP("db+norm_bwd", 3, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, (float*)part, st, 4, M4, C4, O4));
+    FBL_STEP("db+norm_bwd", 2, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, (float*)part, st, 4, M4, C4, O4));
     return FBL_OK;
   }
   if (bias) FBL_STEP("db", 2, launch_colsum_group(p->d.dtype, 4, M4, p->n_pad, C4, O4, (float*)part, st));

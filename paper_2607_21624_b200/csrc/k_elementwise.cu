@@ -337,6 +337,50 @@ __global__ void __launch_bounds__(256, 2) norm_fwd_rows_kernel(const __nv_bfloat
   }
 }
 
+constexpr int COLSUM_SLAB = 256;
+
+struct ColsumGroup {
+  const void* m[4];
+  float* out[4];
+  int cols[4];
+  int64_t part_off[4];      // float offset of each matrix's partials inside the scratch area
+  int count;
+};
+
+// First stage of a token-axis column sum: the block's (64-column panel p, slab of 256 rows) of matrix `which`,
+// 32 storage tiles, reduced to one row of partials.  `red` is 32 x (tile width + 1) floats of shared memory.
+template <typename T>
+__device__ __forceinline__ void colsum_slab(const ColsumGroup& G, int64_t rows, float* __restrict__ part_base, int p,
+                                            int slab, int which, float (*red)[tile_w_of<T>::value + 1]) {
+  constexpr int TW = tile_w_of<T>::value;
+  constexpr int V = Vec16<T>::N;
+  const int cols = G.cols[which];
+  if (p * TW >= cols) return;
+  const T* M = (const T*)G.m[which];
+  float* part = part_base + G.part_off[which];
+  const int rr = threadIdx.x / 8, l8 = threadIdx.x % 8;
+  float acc[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) acc[i] = 0.f;
+  const int64_t r_end = min((int64_t)(slab + 1) * COLSUM_SLAB, rows);
+#pragma unroll 8                              // a slab is eight 32-row steps: all their loads in flight together
+  for (int64_t r = (int64_t)slab * COLSUM_SLAB + rr; r < r_end; r += 32) {
+    float v[V];
+    load16(M + ((int64_t)p * rows + r) * TW + l8 * V, v);
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] += v[i];
+  }
+#pragma unroll
+  for (int i = 0; i < V; ++i) red[rr][l8 * V + i] = acc[i];
+  __syncthreads();
+  if (threadIdx.x < TW) {
+    float s = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < 32; ++k) s += red[k][threadIdx.x];
+    part[(int64_t)slab * cols + p * TW + threadIdx.x] = s;
+  }
+}
+
 template <int NV, int WPR>
 __global__ void __launch_bounds__(256, 2) norm_bwd_rows_kernel(const __nv_bfloat16* __restrict__ dXn,
                                                             const __nv_bfloat16* __restrict__ X,
@@ -344,12 +388,23 @@ __global__ void __launch_bounds__(256, 2) norm_bwd_rows_kernel(const __nv_bfloat
                                                             const float* __restrict__ stats,
                                                             const float* __restrict__ gamma,
                                                             __nv_bfloat16* __restrict__ dX, float* __restrict__ partials,
-                                                            int64_t n_pad, int rms) {
+                                                            int64_t n_pad, int rms, int n_norm, ColsumGroup CG,
+                                                            float* __restrict__ cs_part, int cs_panels, int cs_slabs) {
   constexpr int D = NV * 256 * WPR;
   constexpr int RPB = 8 / WPR;
   __shared__ float s_dg[D];
   __shared__ float s_db[D];
   __shared__ float s_part[32];
+  // Blocks behind the first n_norm ones do the first stage of the bias gradients' column sums (one launch less):
+  // block n_norm + (which * slabs + slab) * panels + p
+  if ((int)blockIdx.x >= n_norm) {
+    __shared__ float cs_red[32][65];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int idx = (int)blockIdx.x - n_norm;
+    colsum_slab<__nv_bfloat16>(CG, n_pad, cs_part, idx % cs_panels, (idx / cs_panels) % cs_slabs, idx / (cs_panels * cs_slabs), cs_red);
+    return;
+  }
   int buf = 0;
   for (int i = threadIdx.x; i < D; i += 256) { s_dg[i] = 0.f; s_db[i] = 0.f; }
   __syncthreads();
@@ -372,7 +427,7 @@ __global__ void __launch_bounds__(256, 2) norm_bwd_rows_kernel(const __nv_bfloat
 #pragma unroll
     for (int i = 0; i < 8; ++i) { ag[j][i] = 0.f; ab[j][i] = 0.f; }
   // each block owns a contiguous range of rows (neighbouring 128-byte pieces in every panel)
-  const int64_t per_block = ((n_pad + gridDim.x - 1) / gridDim.x + RPB - 1) / RPB * RPB;
+  const int64_t per_block = ((n_pad + n_norm - 1) / n_norm + RPB - 1) / RPB * RPB;
   const int64_t r_end = min(n_pad, ((int64_t)blockIdx.x + 1) * per_block);
   for (int64_t r = (int64_t)blockIdx.x * per_block + slot; r < r_end; r += RPB) {
     const float mean = stats[2 * r], rstd = stats[2 * r + 1];
@@ -440,15 +495,6 @@ __global__ void __launch_bounds__(256, 2) norm_bwd_rows_kernel(const __nv_bfloat
   }
 }
 
-constexpr int COLSUM_SLAB = 256;
-
-struct ColsumGroup {
-  const void* m[4];
-  float* out[4];
-  int cols[4];
-  int64_t part_off[4];      // float offset of each matrix's partials inside the scratch area
-  int count;
-};
 
 // dgamma[c] (y = 0) or dbeta[c] (y = 1) = sum over the first kernel's blocks of their partial rows.  Blocks with
 // y >= ny_norm finish the bias column sums instead (matrix y - ny_norm: the tree over its slab partials), so that
@@ -509,8 +555,12 @@ void norm_bwd_rows_launch(const fbl_plan* p, const void* dXn, const void* X, con
                           const float* gamma, void* dX, float* dgamma, float* dbeta, float* part, int rms,
                           const ColsumGroup& cg, const float* cpart, int n_slabs, cudaStream_t st) {
   const int blocks = (int)min((int64_t)p->sm_count * 2, p->n_pad / (8 / WPR));
-  launch_pdl(norm_bwd_rows_kernel<NV, WPR>, dim3(blocks), dim3(256), 0, st, (const __nv_bfloat16*)dXn,
-             (const __nv_bfloat16*)X, (const __nv_bfloat16*)dY, stats, gamma, (__nv_bfloat16*)dX, part, p->n_pad, rms);
+  int cs_panels = 0;
+  for (int i = 0; i < cg.count; ++i) cs_panels = cg.cols[i] / 64 > cs_panels ? cg.cols[i] / 64 : cs_panels;
+  const int cs_blocks = cs_panels * n_slabs * cg.count;
+  launch_pdl(norm_bwd_rows_kernel<NV, WPR>, dim3(blocks + cs_blocks), dim3(256), 0, st, (const __nv_bfloat16*)dXn,
+             (const __nv_bfloat16*)X, (const __nv_bfloat16*)dY, stats, gamma, (__nv_bfloat16*)dX, part, p->n_pad, rms,
+             blocks, cg, const_cast<float*>(cpart), cs_panels, n_slabs);
   const int ny = rms ? 1 : 2;
   launch_pdl(norm_bwd_reduce_kernel, dim3((p->d.d_model + 31) / 32, ny + cg.count), dim3(256), 0, st, (const float*)part,
              blocks, p->d.d_model, dgamma, dbeta, ny, cg, cpart, n_slabs);
@@ -552,38 +602,10 @@ bool norm_rows_shape(int d, int* nv, int* wpr) {
 // ------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256) colsum_stage1(ColsumGroup G, int64_t rows, float* __restrict__ part_base) {
-  constexpr int TW = tile_w_of<T>::value;
-  constexpr int V = Vec16<T>::N;
-  __shared__ float red[32][TW + 1];
+  __shared__ float red[32][tile_w_of<T>::value + 1];
   pdl_launch_dependents();
   pdl_wait();
-  const int which = blockIdx.z;
-  const int cols = G.cols[which];
-  const int p = blockIdx.x, slab = blockIdx.y;
-  if (p * TW >= cols) return;
-  const T* M = (const T*)G.m[which];
-  float* part = part_base + G.part_off[which];
-  const int rr = threadIdx.x / 8, l8 = threadIdx.x % 8;
-  float acc[V];
-#pragma unroll
-  for (int i = 0; i < V; ++i) acc[i] = 0.f;
-  const int64_t r_end = min((int64_t)(slab + 1) * COLSUM_SLAB, rows);
-#pragma unroll 8                              // a slab is eight 32-row steps: all their loads in flight together
-  for (int64_t r = (int64_t)slab * COLSUM_SLAB + rr; r < r_end; r += 32) {
-    float v[V];
-    load16(M + ((int64_t)p * rows + r) * TW + l8 * V, v);
-#pragma unroll
-    for (int i = 0; i < V; ++i) acc[i] += v[i];
-  }
-#pragma unroll
-  for (int i = 0; i < V; ++i) red[rr][l8 * V + i] = acc[i];
-  __syncthreads();
-  if (threadIdx.x < TW) {
-    float s = 0.f;
-#pragma unroll 8
-    for (int k = 0; k < 32; ++k) s += red[k][threadIdx.x];
-    part[(int64_t)slab * cols + p * TW + threadIdx.x] = s;
-  }
+  colsum_slab<T>(G, rows, part_base, blockIdx.x, blockIdx.y, blockIdx.z, red);
 }
 
 __global__ void colsum_stage2(ColsumGroup G, const float* __restrict__ part_base, int n_slabs) {
@@ -645,7 +667,8 @@ cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma
 }
 
 // Norm backward, and with it (bias_count > 0, register-resident bf16 path only) the bias column sums of up to four
-// matrices: their first stage runs before the norm kernel, their second stage inside the norm's own second kernel.
+// matrices: their first stage runs as extra blocks of the norm's rows kernel, their second stage inside the norm's
+// own second kernel.
 // `part` holds the column-sum slab partials first and the norm's per-block partial rows behind them.
 bool norm_bwd_takes_colsums(const fbl_plan* p) {
   int nv, wpr;
@@ -675,10 +698,8 @@ cudaError_t launch_norm_bwd(const fbl_plan* p, const void* dXn, const void* X, c
         off += (int64_t)n_slabs * bias_cols[i];
         max_cols = bias_cols[i] > max_cols ? bias_cols[i] : max_cols;
       }
-      cg.count = bias_count;
-      cudaError_t e = launch_pdl(colsum_stage1<__nv_bfloat16>, dim3((unsigned)(max_cols / 64), n_slabs, bias_count), dim3(256), 0,
-                                 st, cg, p->n_pad, part);
-      if (e != cudaSuccess) return e;
+      cg.count = bias_count;                // their first stage rides in the rows kernel's launch, as extra blocks
+      (void)max_cols;
       npart = part + (off + 255) / 256 * 256;
     }
     // token-axis sums in two steps over `npart` (no atomics: the result does not depend on block order)
