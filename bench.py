@@ -260,10 +260,18 @@ def main():
         run.step()                      # first call sets kernel attributes; keep it outside any capture
         stream.synchronize()
         assert run.status() == 0
+        g_fwd = g_bwd = None
         if not args.no_graph:
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph, stream=stream):
                 run.step()
+            # the two halves on their own, for the end-to-end leg (host copies overlap the other half)
+            g_fwd = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_fwd, stream=stream):
+                run.forward()
+            g_bwd = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_bwd, stream=stream):
+                run.backward()
 
     def one_step():
         if graph is not None:
@@ -316,17 +324,33 @@ def main():
     oY_rm = torch.empty(shape, dtype=tdt, device="cuda")
     odX_rm = torch.empty(shape, dtype=tdt, device="cuda")
 
+    # A second stream carries what the other half of the step does not wait for: dY comes in while the forward runs,
+    # Y goes out while the backward runs.  The timed region (events on the main stream) ends after both have joined.
+    side = torch.cuda.Stream()
+    ev_start, ev_dy, ev_fwd, ev_y = (torch.cuda.Event() for _ in range(4))
+
     def e2e_step():
         s = stream.cuda_stream
+        ev_start.record(stream)
         dX_rm.copy_(hX, non_blocking=True)
-        dY_rm.copy_(hdY, non_blocking=True)
+        with torch.cuda.stream(side):
+            side.wait_event(ev_start)
+            dY_rm.copy_(hdY, non_blocking=True)
+            ev_dy.record(side)
         run.plan.pack(TENSOR["X"], dX_rm.data_ptr(), run.buf["X"].data_ptr(), s)
+        g_fwd.replay() if g_fwd is not None else run.forward()
+        ev_fwd.record(stream)
+        with torch.cuda.stream(side):
+            side.wait_event(ev_fwd)
+            run.plan.unpack(TENSOR["Y"], run.buf["Y"].data_ptr(), oY_rm.data_ptr(), side.cuda_stream)
+            hY.copy_(oY_rm, non_blocking=True)
+            ev_y.record(side)
+        stream.wait_event(ev_dy)
         run.plan.pack(TENSOR["DY"], dY_rm.data_ptr(), run.buf["dY"].data_ptr(), s)
-        one_step()
-        run.plan.unpack(TENSOR["Y"], run.buf["Y"].data_ptr(), oY_rm.data_ptr(), s)
+        g_bwd.replay() if g_bwd is not None else run.backward()
         run.plan.unpack(TENSOR["DX"], run.buf["dX"].data_ptr(), odX_rm.data_ptr(), s)
-        hY.copy_(oY_rm, non_blocking=True)
         hdX.copy_(odX_rm, non_blocking=True)
+        stream.wait_event(ev_y)
 
     ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     with torch.cuda.stream(stream):
@@ -342,6 +366,8 @@ def main():
             b.record(stream)
     barrier()
     ms_e2e = sum(a.elapsed_time(b) for a, b in ev2) / len(ev2)
+    assert run.status() == 0
+    assert torch.equal(hY, oY_rm.cpu()) and torch.equal(hdX, odX_rm.cpu())     # both streams had joined
     io_bytes = 2 * cfg.n_tokens * cfg.d_model * (2 if cfg.dtype == "bf16" else 4)
 
     # ---- per-step event timing (separate pass, direct launches) for the roofline of the dominant step ----
