@@ -277,3 +277,21 @@ def test_norm_backward_invariants():
     inp_r = big_inputs(cfg_r)
     _, _, gr = orc.layer_fwd_bwd(scaled_config(cfg_r, eps=0.0), inp_r)
     assert np.abs((gr["dX"] * inp_r["X"]).sum(-1)).max() < 1e-11   # scale invariance (eps = 0)
+
+
+def test_oracle_matches_its_committed_fixture():
+    # Drift guard (not a pin to the paper): the oracle's values on two tiny seeded layers are stored under
+    # tests/golden/ by a script that calls only oracle/; a change of the oracle's arithmetic changes them.
+    import importlib.util
+    import os
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_oracle_golden", os.path.join(here, "make_oracle_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    stored = [ln.split() for ln in open(os.path.join(here, "oracle_layer_tiny.txt")) if not ln.startswith("#")]
+    fresh = [ln.split() for ln in mod.lines()]
+    assert len(stored) == len(fresh) == 14
+    for s, f in zip(stored, fresh):
+        assert s[:3] == f[:3]
+        a, b = np.array(s[3:], dtype=np.float64), np.array(f[3:], dtype=np.float64)
+        assert np.allclose(a, b, rtol=1e-12, atol=1e-14), (s[0], s[1])
