@@ -221,6 +221,7 @@ def main():
     ap.add_argument("--path", type=int, default=0, help="0 default kernels, 1 FFMA kernels only")
     ap.add_argument("--no-graph", action="store_true", help="enqueue kernels directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flush-write-only", action="store_true", help="flush L2 by the 256 MiB write alone (its write-back then overlaps the step)")
     ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling captures)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures)")
     args = ap.parse_args()
@@ -254,6 +255,16 @@ def main():
     run.load_inputs(inp)
     stream = torch.cuda.Stream()
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # 256 MiB > 126 MB L2
+    flush_rd = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device="cuda")  # 256 MiB, only ever read
+    flush_sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def flush_l2():
+        # Write a buffer larger than L2, then read another one: the write evicts the step's data, the read evicts
+        # the write's dirty lines, whose write-back would otherwise run inside the timed step and take DRAM bandwidth
+        # from it (an artefact of the flush, not of the workload).
+        flush.zero_()
+        if not args.flush_write_only:
+            torch.sum(flush_rd, dim=0, keepdim=True, dtype=torch.int32, out=flush_sink)
 
     graph = None
     with torch.cuda.stream(stream):
@@ -294,14 +305,14 @@ def main():
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
-            flush.zero_()
+            flush_l2()
             one_step()
     barrier()
     sampler = ClockSampler(local_rank)
     t_wall0 = time.perf_counter()
     with torch.cuda.stream(stream):
         for a, b in ev:
-            flush.zero_()
+            flush_l2()
             a.record(stream)
             one_step()
             b.record(stream)
@@ -355,12 +366,12 @@ def main():
     ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
-            flush.zero_()
+            flush_l2()
             e2e_step()
     barrier()
     with torch.cuda.stream(stream):
         for a, b in ev2:
-            flush.zero_()
+            flush_l2()
             a.record(stream)
             e2e_step()
             b.record(stream)
@@ -376,7 +387,7 @@ def main():
     reps = max(3, min(args.steps, 10))
     with torch.cuda.stream(stream):
         for _ in range(reps):
-            flush.zero_()
+            flush_l2()
             run.forward()
             stream.synchronize()
             for name, t in run.plan.profile_read():
@@ -434,7 +445,7 @@ def main():
         "metric": "fwd+bwd layer TFLOP/s", "value": tfl, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": workload_name(cfg), "l2": "256 MiB flush write before every timed step",
+        "config": {"workload": workload_name(cfg), "l2": "256 MiB written" + ("" if args.flush_write_only else ", then 256 MiB read (so that the write-back of the flush is over)") + " before every timed step",
                    "launch": "cuda graph replay" if graph is not None else "direct launches",
                    "kernel_path": "default" if args.path == 0 else "ffma", "parallelism": "replicas only"},
         "tokens_per_s": rep.whole_job_rate(cfg.n_tokens, ms),
