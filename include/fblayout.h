@@ -99,10 +99,11 @@ typedef struct fbl_plan fbl_plan; /* opaque: padded sizes, index-map constants, 
  * The plan also fixes, from the shapes alone, into how many slices the token-axis reductions of the weight
  * gradients are cut (1 for all but layers with few weight tiles and many tokens).  Environment variables
  * read here, for tuning and tests only: FBL_KSPLIT_O and FBL_KSPLIT_QKV override those slice counts,
- * FBL_VERBOSE prints the ones chosen to stderr.  Two more are read when a step is enqueued, again for tuning
+ * FBL_VERBOSE prints the ones chosen to stderr.  Three more are read when a step is enqueued, again for tuning
  * and tests only: FBL_GEMM_PAIR (0: never use the CTA-pair GEMM kernel, 1: use it wherever its tile shape is
- * legal; unset: large launches only) and FBL_FWD_TILES (1 or 2 query tiles per forward-attention block at
- * head_dim 64; unset: by sequence length). */
+ * legal; unset: large launches only), FBL_GEMM_ESETS (1 or 2 sets of epilogue warps in the single-CTA GEMM kernel;
+ * unset: 2 where every block of the launch has one tile) and FBL_FWD_TILES (1 or 2 query tiles per
+ * forward-attention block at head_dim 64; unset: by sequence length). */
 int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out);
 void fbl_plan_destroy(fbl_plan* plan);
 

@@ -120,8 +120,8 @@ __device__ __forceinline__ bool tile_at(const TcGroup& G, int w, TileCoord* tc_o
 // shared-memory ring by TMA, warp 1 issues the MMAs into one of two TMEM accumulators, warps 2-5 drain the
 // other accumulator (bias, residual, padding-row mask, bf16 rows in R-Tile order), so the epilogue of
 // one tile overlaps the main loop of the next.
-template <int BN, int STAGES>
-__global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__ TcGroup G) {
+template <int BN, int STAGES, int ESETS>
+__global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __grid_constant__ TcGroup G) {
   using SP = SmemPlan<BN, STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -143,7 +143,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
     }
     for (int a = 0; a < 2; ++a) {
       tc::mbar_init(acc_full(a), 1);
-      tc::mbar_init(acc_empty(a), 128);
+      tc::mbar_init(acc_empty(a), 128 * ESETS);
     }
     tc::fence_barrier_init();
   }
@@ -255,8 +255,13 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
     // its TMEM lane quarter and two 32 x 64 staging tiles, and issues its own stores: no block-wide hand-off per
     // panel, and the store of one panel overlaps the conversion of the next. ---------------------------------
     pdl_wait();                                       // the previous kernel may still be reading what we overwrite
-    group_chores(G, threadIdx.x - 64, 128);
+    group_chores(G, threadIdx.x - 64, 128 * ESETS);
     const int q = warp % 4;                           // the TMEM lane quarter this warp may access
+    // ESETS = 2 (launches in which every block has a single tile, so that nothing overlaps its epilogue): two sets
+    // of four warps share the tile's 64-column panels, first and second half, and the epilogue takes half as long.
+    // Each warp then has one staging tile instead of two (the staging area is the same size).
+    const int set = (warp - 2) / 4;
+    constexpr int PPS = BN / 64 / ESETS;              // panels per set
     const int r = q * 32 + lane;                      // row of the tile owned by this thread
     const bool tracer = threadIdx.x == 64;
     int ti = 0, pc = 0;                               // tiles and panels done by this warp
@@ -268,9 +273,14 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
       const int row = tcd.m0 + r;
       const bool pad = P.t_pad > 0 && (row % P.t_pad) >= P.seq;
       const bool has_res = P.residual && row < P.m;
+      // a head of the fused row reduction must stay within one warp: where it spans more panels than a set has, the
+      // first set takes the whole tile
+      const bool whole = ESETS == 2 && P.dot_with && P.dot_hd > 64 * PPS;
+      const int pn_begin = set == 0 ? 0 : (whole ? BN / 64 : PPS);
+      const int pn_end = ESETS == 1 ? BN / 64 : (set == 0 ? (whole ? BN / 64 : PPS) : BN / 64);
       uint4 rv[8];                                    // residual values of the next panel, requested a panel ahead
-      if (has_res) {
-        const __nv_bfloat16* rp = P.residual + ((long long)(tcd.n0 / 64) * P.c_rpad + row) * 64;
+      if (has_res && pn_begin < pn_end && tcd.n0 + pn_begin * 64 < P.n) {
+        const __nv_bfloat16* rp = P.residual + ((long long)(tcd.n0 / 64 + pn_begin) * P.c_rpad + row) * 64;
 #pragma unroll
         for (int j = 0; j < 8; ++j) rv[j] = *reinterpret_cast<const uint4*>(rp + 8 * j);
       }
@@ -288,7 +298,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
       if (tracer && ti == 0) GTR(5);
       float dot_acc = 0.f;
 #pragma unroll 1
-      for (int pn = 0; pn < BN / 64; ++pn) {
+      for (int pn = pn_begin; pn < pn_end; ++pn) {
         const int n = tcd.n0 + pn * 64;
         if (n >= P.n) break;                           // uniform: N is whole 64-column panels
         uint32_t v[64];
@@ -301,7 +311,8 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
           // buffer by bulk tensor reductions (same staging tiles and swizzle as the bf16 rows below)
 #pragma unroll 1
           for (int hf = 0; hf < 2; ++hf) {
-            const uint32_t stg = base + SP::STG_OFF + (uint32_t)(q * 2 + (pc & 1)) * 4096u;
+            const uint32_t stg = base + SP::STG_OFF + (ESETS == 2 ? (uint32_t)(warp - 2) : (uint32_t)(q * 2 + (pc & 1))) * 4096u;
+            if (ESETS == 2 && lane == 0) tc::bulk_wait_group_read0();     // the single staging tile's previous contents have been read
             __syncwarp();
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -313,7 +324,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
             if (lane == 0) {
               tc::tma_reduce_add_4d(&P.tacc, stg, 0, hf, tcd.m0 + q * 32, n / 64);
               tc::bulk_commit_group();
-              tc::bulk_wait_group_read1();
+              if (ESETS == 1) tc::bulk_wait_group_read1();
             }
             ++pc;
           }
@@ -332,7 +343,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
 #pragma unroll
             for (int k = 0; k < 8; ++k) v[8 * j + k] = __float_as_uint(__uint_as_float(v[8 * j + k]) + __bfloat162float(rb[k]));
           }
-          if (pn + 1 < BN / 64 && n + 64 < P.n) {
+          if (pn + 1 < pn_end && n + 64 < P.n) {
             const __nv_bfloat16* rp = P.residual + ((long long)(n / 64 + 1) * P.c_rpad + row) * 64;
 #pragma unroll
             for (int j = 0; j < 8; ++j) rv[j] = *reinterpret_cast<const uint4*>(rp + 8 * j);
@@ -378,8 +389,9 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
         }
         // Staging tile (pc & 1) of this warp: its previous store (two panels ago) has been read, since lane 0
         // waited for that after committing the store of the panel before this one.
-        const uint32_t stg = base + SP::STG_OFF + (uint32_t)(q * 2 + (pc & 1)) * 4096u;
+        const uint32_t stg = base + SP::STG_OFF + (ESETS == 2 ? (uint32_t)(warp - 2) : (uint32_t)(q * 2 + (pc & 1))) * 4096u;
         if (tracer && ti == 0 && pn == 1) GTR(13);
+        if (ESETS == 2 && lane == 0) tc::bulk_wait_group_read0();    // one staging tile: the store before has read it
         __syncwarp();
         if (tracer && ti == 0 && pn == 1) GTR(14);
 #pragma unroll
@@ -394,7 +406,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
         if (lane == 0) {
           tc::tma_store_3d(&P.tc, stg, 0, tcd.m0 + q * 32, n / 64);
           tc::bulk_commit_group();
-          tc::bulk_wait_group_read1();                 // the store before this one has read its staging tile
+          if (ESETS == 1) tc::bulk_wait_group_read1();  // the store before this one has read its staging tile
         }
         if (tracer && ti == 0 && pn < 1) GTR(11 + 2 * pn);
         ++pc;
@@ -796,10 +808,21 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
     tiles += ((g.m + BM - 1) / BM) * ((g.n + BN - 1) / BN) * P.ksplit;
   }
   using SP = SmemPlan<BN, STAGES>;
-  auto k = gemm_tc_kernel<BN, STAGES>;
+  const int grid = tiles < p->sm_count ? tiles : p->sm_count;
+  // one tile per block at most: the epilogue is exposed, and the variant with two sets of epilogue warps halves it
+  // (with several tiles per block the epilogues overlap the next main loops and the extra warps only cost)
+  const int esets_knob = getenv("FBL_GEMM_ESETS") ? atoi(getenv("FBL_GEMM_ESETS")) : 0;      // tuning knob: 1 or 2
+  const bool two_sets = esets_knob ? esets_knob == 2 : tiles <= p->sm_count;
+  if (two_sets) {
+    auto k = gemm_tc_kernel<BN, STAGES, 2>;
+    cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
+    if (attr_err != cudaSuccess) return attr_err;
+    return gs[0].serial ? launch_serial(k, dim3(grid), dim3(320), SP::TOTAL, st, G)
+                        : launch_pdl(k, dim3(grid), dim3(320), SP::TOTAL, st, G);
+  }
+  auto k = gemm_tc_kernel<BN, STAGES, 1>;
   cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
   if (attr_err != cudaSuccess) return attr_err;
-  const int grid = tiles < p->sm_count ? tiles : p->sm_count;
   return gs[0].serial ? launch_serial(k, dim3(grid), dim3(192), SP::TOTAL, st, G)
                       : launch_pdl(k, dim3(grid), dim3(192), SP::TOTAL, st, G);
 }

@@ -107,6 +107,19 @@ def test_cta_pair_gemm_forced(cfg, monkeypatch):
     run_and_compare(cfg, affine_noise=True)
 
 
+@pytest.mark.parametrize("sets", ["1", "2"])
+def test_gemm_epilogue_sets_forced(sets, monkeypatch):
+    # The single-CTA GEMM kernel drains a tile with one set of four warps, or, in launches where every block has one
+    # tile, with two sets that share the tile's panels.  Small shapes get the second by default, large ones the
+    # first; the knob forces each on shapes with bias, residual, padding rows, sliced reductions and the fused row
+    # reduction at head_dim 64 and 128 (where a head spans both sets' panels and the first set takes the tile).
+    monkeypatch.setenv("FBL_GEMM_ESETS", sets)
+    for cfg in (LayerConfig("g1", 3, 333, 512, 8, 4, 64, "bf16", "layernorm", True, True, True, 1e-5, 51, 0.02),
+                LayerConfig("g2", 2, 200, 256, 2, 1, 128, "bf16", "rmsnorm", False, False, True, 1e-5, 52, 0.02),
+                LayerConfig("g3", 6, 197, 256, 4, 2, 64, "bf16", "layernorm", True, True, False, 1e-5, 53, 0.02)):
+        run_and_compare(cfg, affine_noise=True)
+
+
 def test_forward_tile_variants_forced(monkeypatch):
     # head_dim 64 forward: one-tile blocks (two per SM) are the default for short sequences, two-tile blocks for long
     # ones; force each on a shape the other would get
