@@ -852,26 +852,31 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       if (dit >= (int)NS && !stage_is_alt(dit) && !tc::mbar_wait(bar(BB_STAGEFREE + (dit % NS)), (dit / (int)NS - 1) & 1, status, 310)) return false;
       { const int it = dit; if (t == 0) TR(8); }
       tc::tc_fence_after();
-#pragma unroll 1
-      for (int cc = 0; cc < HD / 64; ++cc) {
-        const int c0 = part * (HD / 4) + cc * 16;    // first of this thread's 16 columns
-        uint32_t o[16];
-        tc::tmem_ld16(lane_addr + DQ_COL + c0, o);
-        tc::tmem_ld_wait();
-        const uint32_t unit = (uint32_t)(r * 2 + (c0 % 64) / 32);                 // 128-byte unit of the box
-        const uint32_t rowaddr = stage + (c0 / 64) * 32768 + unit * 128;
+      // this thread's HD / 4 accumulator columns in one go; the tensor pipe gets the columns back (at HD = 128 the
+      // next tile's dP^T waits for them) as soon as they are in registers, before the stores to the staging tile
+      constexpr int NC = HD / 4;                     // 16 or 32 columns
+      const int c0 = part * NC;
+      uint32_t o[NC];
+      if constexpr (NC == 32) tc::tmem_ld32(lane_addr + DQ_COL + c0, o);
+      else tc::tmem_ld16(lane_addr + DQ_COL + c0, o);
+      tc::tmem_ld_wait();
+      tc::tc_fence_before();
+      tc::mbar_arrive(bar(BB_DQDRAINED));            // TMEM side done: the tensor pipe may reuse the columns
+      { const int it = dit; if (t == 0) TR(7); }
+#pragma unroll
+      for (int u = 0; u < NC / 16; ++u) {            // 16 columns = half of a 128-byte unit of the box
+        const int cu = c0 + u * 16;
+        const uint32_t unit = (uint32_t)(r * 2 + (cu % 64) / 32);
+        const uint32_t rowaddr = stage + (cu / 64) * 32768 + unit * 128;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          const uint32_t chk = (uint32_t)((c0 % 32) / 4 + k);
+          const uint32_t chk = (uint32_t)((cu % 32) / 4 + k);
           const uint32_t addr = rowaddr + ((chk ^ (unit & 7)) * 16);
-          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(__uint_as_float(o[4 * k]) * P.scale),
-                       "f"(__uint_as_float(o[4 * k + 1]) * P.scale), "f"(__uint_as_float(o[4 * k + 2]) * P.scale),
-                       "f"(__uint_as_float(o[4 * k + 3]) * P.scale) : "memory");
+          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(__uint_as_float(o[u * 16 + 4 * k]) * P.scale),
+                       "f"(__uint_as_float(o[u * 16 + 4 * k + 1]) * P.scale), "f"(__uint_as_float(o[u * 16 + 4 * k + 2]) * P.scale),
+                       "f"(__uint_as_float(o[u * 16 + 4 * k + 3]) * P.scale) : "memory");
         }
       }
-      tc::tc_fence_before();
-      { const int it = dit; if (t == 0) TR(7); }
-      tc::mbar_arrive(bar(BB_DQDRAINED));            // TMEM side done: the tensor pipe may reuse the columns
       tc::fence_proxy_async();
       tc::mbar_arrive(bar(BB_DQSTAGED + (dit % NS)));     // staging side done: the reduction warp takes over
       return true;
