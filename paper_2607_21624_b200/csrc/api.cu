@@ -424,7 +424,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
   }
   if (!first_gemm_fills) FBL_CUDA(cudaMemsetAsync(status, 0, p->zero_bytes, st));
   FBL_PROF_BEGIN();
-  bool dvec_ready = false;
+  bool dvec_ready = false, dwo_round = false;
   {
     GemmArgs gs[2];
     GemmArgs& gw = gs[0];   // dWo = A^T dY : token-axis reduction (longest reduction loop: first in the work list)
@@ -448,11 +448,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
         gs[0].reset_status = 1; gs[0].serial = 1;
       }
       FBL_STEP("dWo+dA", 1, launch_gemm_tc_group(p, gs, 2, status, st));
-      if (split_o) {
-        ConvertGroup cg = {};
-        cg.src[0] = gw.acc; cg.dst[0] = dWo; cg.n[0] = up8(p->dq) * (int64_t)D; cg.count = 1;
-        FBL_STEP("dWo round", 1, launch_convert_f32_group(cg, st));
-      }
+      dwo_round = split_o;        // nothing in the step reads dWo: its rounding joins that of dWq, dWk, dWv below
     } else {
       FBL_STEP("dA", 1, run_gemm(p, ga, part, p->part_bytes, status, st));
       FBL_STEP("dWo", 1, run_gemm(p, gw, part, p->part_bytes, status, st));
@@ -494,13 +490,23 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
         }
         cg.count = 3;
       }
+      if (dwo_round) {
+        cg.src[cg.count] = (const float*)(sc + p->sb_acc_o); cg.dst[cg.count] = dWo; cg.n[cg.count] = up8(p->dq) * (int64_t)D;
+        cg.count++;
+        dwo_round = false;
+      }
       FBL_STEP("dWqkv+dXn", 1, launch_gemm_tc_group(p, gs, 4, status, st));
-      if (split_qkv) FBL_STEP("dWqkv round", 1, launch_convert_f32_group(cg, st));
+      if (cg.count > 0) FBL_STEP("dW round", 1, launch_convert_f32_group(cg, st));     // one rounding launch for all sliced GEMMs
     } else {
       FBL_STEP("dXn", 1, run_gemm(p, gx, part, p->part_bytes, status, st));
       for (int i = 0; i < 3; ++i)
         FBL_STEP(i == 0 ? "dWq" : i == 1 ? "dWk" : "dWv", 1, run_gemm(p, gs[i], part, p->part_bytes, status, st));
     }
+  }
+  if (dwo_round) {
+    ConvertGroup cg = {};
+    cg.src[0] = (const float*)(sc + p->sb_acc_o); cg.dst[0] = dWo; cg.n[0] = up8(p->dq) * (int64_t)D; cg.count = 1;
+    FBL_STEP("dW round", 1, launch_convert_f32_group(cg, st));
   }
   // every bias gradient is a token-axis column sum: the four of them share their launches, and the second stage
   // shares the norm backward's second kernel where that kernel exists
