@@ -106,3 +106,31 @@ def test_step_does_not_depend_on_previous_buffer_contents(cfg):
             assert np.array_equal(ref[n], got[n]), (n, hex(fill))
         for n in ("dX", "dWq"):                       # downstream of the dQ accumulation, whose order is free
             assert np.abs(ref[n] - got[n]).max() <= 2e-2 * np.abs(ref[n]).max() + 1e-6, (n, hex(fill))
+
+
+@pytest.mark.parametrize("cfg", [
+    LayerConfig("e10", 2, 300, 256, 4, 2, 64, "bf16", "layernorm", True, True, True, 1e-5, 56, 0.02),
+    LayerConfig("e11", 4, 512, 768, 12, 12, 64, "bf16", "layernorm", True, True, False, 1e-5, 57, 0.02),
+    LayerConfig("e12", 1, 640, 512, 4, 4, 128, "bf16", "rmsnorm", True, False, True, 1e-5, 58, 0.02),
+], ids=lambda c: c.name)
+def test_many_back_to_back_steps_are_identical(cfg):
+    # Forty forward + backward passes enqueued without any host synchronisation in between: every kernel is launched
+    # so that it may start while its predecessor drains, across the boundary between steps too.  Whatever one step
+    # leaves behind (accumulators, staging areas, barriers' worth of in-flight copies) must not reach the next: the
+    # order-free outputs of the last step equal those of a lone first step bit for bit.
+    import torch
+    from paper_2607_21624_b200 import LayerRunner
+    run = LayerRunner(cfg)
+    run.load_inputs(make_inputs(cfg, affine_noise=True))
+    names = ("Y", "dWo", "dWk", "dWv")
+    run.step()
+    torch.cuda.synchronize()
+    first = {n: run.fetch(n) for n in names + ("dX", "dWq")}
+    for _ in range(40):
+        run.step()
+    torch.cuda.synchronize()
+    assert run.status() == 0
+    for n in names:
+        assert np.array_equal(first[n], run.fetch(n)), n
+    for n in ("dX", "dWq"):
+        assert np.abs(first[n] - run.fetch(n)).max() <= 2e-2 * np.abs(first[n]).max() + 1e-6, n
