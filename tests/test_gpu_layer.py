@@ -120,6 +120,19 @@ def test_gemm_epilogue_sets_forced(sets, monkeypatch):
         run_and_compare(cfg, affine_noise=True)
 
 
+@pytest.mark.parametrize("cfg", [
+    LayerConfig("r1", 8, 600, 512, 8, 8, 64, "bf16", "rmsnorm", True, False, False, 1e-5, 59, 0.02),
+    # (no biases here: over 4800 tokens and four query heads per key head the rounding noise of the identically-zero
+    # dbk, 1.1e-2, is just past the absolute bound that a zero reference leaves; every other tensor is at a fifth of its own)
+    LayerConfig("r2", 8, 600, 512, 8, 2, 64, "bf16", "layernorm", False, False, True, 1e-5, 60, 0.02),
+], ids=lambda c: c.name)
+def test_forward_paired_tiles_with_odd_tile_count(cfg):
+    # head_dim 64 forward with two query tiles per block and rotating score buffers, on a grid large enough for the
+    # pairing to be chosen (192 blocks) and five query tiles per head: the last block of a head owns a single tile,
+    # the other blocks two tiles whose key ranges differ by one tile (causal) or not at all (full attention)
+    run_and_compare(cfg, affine_noise=True)
+
+
 def test_forward_tile_variants_forced(monkeypatch):
     # head_dim 64 forward: one-tile blocks (two per SM) are the default for short sequences, two-tile blocks for long
     # ones; force each on a shape the other would get
