@@ -1,12 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of the attention-layer training step (forward + backward) on B200.
 
-One step = fbl_layer_fwd + fbl_layer_bwd over one batch of synthetic input.  The JSON
-line reports algorithmic TFLOP/s (multiply-add = 2, causal pairs counted once, no
-recompute), tokens/s, the end-to-end figure with host buffers, a roofline object for
-the dominant step and the float64 oracle timed on the host cores.
+One step = fbl_layer_fwd + fbl_layer_bwd over one batch of synthetic input.  Without --config the five
+workloads are timed one after the other in the same process; the JSON line's top-level figures are those of the
+largest one (workload 5, the Llama-7B-shaped long-sequence layer) and `per_config` carries all five.  Reported:
+algorithmic TFLOP/s (multiply-add = 2, causal pairs counted once, no recompute), tokens/s, the end-to-end figure
+with host buffers, a roofline object for the dominant kernel, the layer's memory efficiency and the float64
+oracle timed on the host cores.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config i] [--impl reference]
+
+With --gpus N > 1 the step runs as N independent replicas, one process per GPU (started by torchrun, or by this
+script itself when it is not under a launcher); no tensor of the data path crosses ranks.
 """
 from __future__ import annotations
 
@@ -21,10 +26,12 @@ import time
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from fbl_inputs import get_config, make_inputs  # noqa: E402
+from fbl_inputs import get_config, make_inputs, scaled_config  # noqa: E402
 
 NOMINAL_TFLOPS, NOMINAL_GBS = 2250.0, 8000.0
 FALLBACK_TFLOPS, FALLBACK_GBS = 1590.0, 6650.0
+HEADLINE = 5                      # the largest single-GPU workload
+ORDER = (5, 1, 2, 3, 4)           # the headline first: a run cut short still has it
 
 
 def measured_peaks():
@@ -53,10 +60,32 @@ def step_flops(cfg):
             "dWv": pk, "dWqkv": pq + 2 * pk, "dWqkv+dXn": 2 * (pq + 2 * pk)}
 
 
+def step_bytes(cfg):
+    """Algorithmic HBM bytes of the bandwidth-bound steps."""
+    e = 2 if cfg.dtype == "bf16" else 4
+    nd = cfg.n_tokens * cfg.d_model * e
+    nb = (4 if cfg.residual else 3) * nd
+    db = (cfg.n_tokens * (cfg.d_model + cfg.d_q + 2 * cfg.d_kv) * e) if cfg.has_bias else 0
+    return {"norm_fwd": 2 * nd, "norm_bwd": nb, "db+norm_bwd": nb + db, "db": db}
+
+
+def min_bytes(cfg):
+    """Once-only minimum HBM traffic of a step: every distinct tensor crosses HBM once per pass that needs it
+    (forward: read X and the weights, write Q, K, V, A, LSE, the norm statistics and Y; backward: read dY, X, the
+    weights and the saved tensors, write dX and the weight gradients).  The numerator of the memory efficiency."""
+    e = 2 if cfg.dtype == "bf16" else 4
+    n = cfg.n_tokens
+    nd = n * cfg.d_model * e
+    w = (cfg.d_model * (cfg.d_q + 2 * cfg.d_kv) + cfg.d_q * cfg.d_model) * e
+    qkva = n * (2 * cfg.d_q + 2 * cfg.d_kv) * e
+    small = cfg.batch * cfg.n_q_heads * cfg.seq * 4 + n * 8            # LSE, statistics
+    return 5 * nd + 3 * w + 2 * qkva + 2 * small
+
+
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the step kernels, from the ncu captures
-# summarised under profiles/ (workload 4, and workload 5 at sequence 2048).  Keyed by (workload name, step).
+# summarised under profiles/.  Keyed by (workload name, step); a step without a capture has no entry.
 NCU_TRAFFIC_BYTES = {
-    # workload 2 (the default): every kernel of a step, profiles/ncu_full_workload2_gpt2small_hd64.md
+    # workload 2: every kernel of a step, profiles/ncu_full_workload2_gpt2small_hd64.md
     ("cfg2-gpt2-small", "norm_fwd"): 3.5e6 + 0.0e6,
     ("cfg2-gpt2-small", "proj_qkv"): 6.8e6 + 0.0e6,
     ("cfg2-gpt2-small", "attn_fwd"): 9.5e6 + 0.0e6,
@@ -75,15 +104,6 @@ NCU_TRAFFIC_BYTES = {
     ("cfg4-llama1b-gqa", "attn_bwd"): 76.6e6 + 3.5e6,
     ("cfg4-llama1b-gqa", "dWqkv+dXn"): 56.4e6 + 11.5e6,
 }
-
-
-def step_bytes(cfg):
-    """Algorithmic HBM bytes of the bandwidth-bound steps."""
-    e = 2 if cfg.dtype == "bf16" else 4
-    nd = cfg.n_tokens * cfg.d_model * e
-    nb = (4 if cfg.residual else 3) * nd
-    db = (cfg.n_tokens * (cfg.d_model + cfg.d_q + 2 * cfg.d_kv) * e) if cfg.has_bias else 0
-    return {"norm_fwd": 2 * nd, "norm_bwd": nb, "db+norm_bwd": nb + db}
 
 
 class ClockSampler:
@@ -166,6 +186,7 @@ class ClockSampler:
         return out
 
 
+# ---- the float64 oracle on the host cores (the cpu_baseline leg and the reference arm) ---------------------------
 def time_oracle(cfg, inp, repeats):
     from oracle import layer as orc
     t = []
@@ -187,108 +208,73 @@ def host_threads():
     return len(os.sched_getaffinity(0))
 
 
+def oracle_sample(cfg, flop_budget=1.0e12):
+    """A bounded sample of the workload for the oracle (about ten seconds of float64 work on the host): fewer
+    batch elements first, then, for a single long sequence, its first tokens (a causal layer's prefix is a
+    smaller instance of the same layer)."""
+    batch = max(1, min(cfg.batch, int(flop_budget // max(cfg.flops() / cfg.batch, 1.0))))
+    scfg = scaled_config(cfg, batch=batch)
+    seq, what = cfg.seq, f"batch {batch} of {cfg.batch}, full sequence"
+    while scfg.flops() > flop_budget and seq > 256:
+        seq //= 2
+        scfg = scaled_config(cfg, batch=batch, seq=seq)
+        what = f"batch {batch} of {cfg.batch}, the first {seq} of {cfg.seq} tokens of each sequence"
+    return scfg, what
+
+
 def run_reference(args, cfg, rank):
     if rank != 0:
         return
     import numpy as np  # noqa: F401  (loads the BLAS threadpool before it is inspected)
-    # bounded sample: the workload with the batch cut down so that one oracle pass stays in the seconds range
-    from fbl_inputs import scaled_config
-    sample_batch = max(1, min(cfg.batch, int(4e10 // max(cfg.flops() / cfg.batch, 1)) or 1))
-    scfg = scaled_config(cfg, batch=sample_batch)
+    scfg, what = oracle_sample(cfg)
     inp = make_inputs(scfg)
+    passes = max(1, min(args.steps, 3))                   # a few passes, not --steps of them: each takes seconds
     time_oracle(scfg, inp, min(args.warmup, 1))
-    t = time_oracle(scfg, inp, args.steps)
+    t = time_oracle(scfg, inp, passes)
     sec = sum(t) / len(t)
     tfl = scfg.flops() / sec / 1e12
+    sample = f"{what}; one fwd+bwd per step, {passes} timed steps (--steps {args.steps} capped at 3)"
     line = {"impl": "reference", "metric": "fwd+bwd layer TFLOP/s", "value": tfl, "unit": "TFLOP/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "tokens_per_s": scfg.n_tokens / sec,
             "config": {"workload": workload_name(cfg)},
-            "cpu_baseline": {"value": tfl, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle",
-                             "sample": f"batch {sample_batch} of {cfg.batch}, full sequence, one fwd+bwd per step"},
+            "cpu_baseline": {"value": tfl, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": tfl, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=2, help="1-based index into the five workloads (default: the second)")
-    ap.add_argument("--impl", default="fblayout", choices=["fblayout", "reference"])
-    ap.add_argument("--path", type=int, default=0, help="0 default kernels, 1 FFMA kernels only")
-    ap.add_argument("--no-graph", action="store_true", help="enqueue kernels directly instead of replaying a CUDA graph")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--flush-write-only", action="store_true", help="flush L2 by the 256 MiB write alone (its write-back then overlaps the step)")
-    ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling captures)")
-    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures)")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "fblayout" else args.warmup
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    cfg = get_config(args.config)
-    if args.seq or args.batch:
-        from fbl_inputs import scaled_config
-        cfg = scaled_config(cfg, name=cfg.name + "-scaled", seq=args.seq or cfg.seq, batch=args.batch or cfg.batch)
-    if args.impl == "reference":
-        run_reference(args, cfg, rank)
-        return
-
-    import numpy as np
+# ---- one workload on this rank's GPU ---------------------------------------------------------------------------
+def measure(cfg, args, rep, local_rank, flush_l2, want_cpu):
     import torch
     from paper_2607_21624_b200 import TENSOR, LayerRunner
-    from paper_2607_21624_b200.build import build
-    build()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
-    torch.cuda.set_device(local_rank)
-    from paper_2607_21624_b200.replicas import Replicas
-    rep = Replicas(backend="nccl", device=torch.device("cuda", local_rank))
-    world = rep.world
 
-    # replicas only: every rank runs the same workload on its own GPU, no data-path collective
     inp = make_inputs(cfg)
     run = LayerRunner(cfg, device=f"cuda:{local_rank}")
     run.plan.set_kernel_path(args.path)
     run.load_inputs(inp)
     stream = torch.cuda.Stream()
-    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # 256 MiB > 126 MB L2
-    flush_rd = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device="cuda")  # 256 MiB, only ever read
-    flush_sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+    steps, warmup = args.steps, args.warmup
 
-    def flush_l2():
-        # Write a buffer larger than L2, then read another one: the write evicts the step's data, the read evicts
-        # the write's dirty lines, whose write-back would otherwise run inside the timed step and take DRAM bandwidth
-        # from it (an artefact of the flush, not of the workload).
-        flush.zero_()
-        if not args.flush_write_only:
-            torch.sum(flush_rd, dim=0, keepdim=True, dtype=torch.int32, out=flush_sink)
-
-    graph = None
+    graph = g_fwd = g_bwd = None
     with torch.cuda.stream(stream):
         run.step()                      # first call sets kernel attributes; keep it outside any capture
         stream.synchronize()
         assert run.status() == 0
-        g_fwd = g_bwd = None
         if not args.no_graph:
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph, stream=stream):
                 run.step()
-            # the two halves on their own, for the end-to-end leg (host copies overlap the other half)
-            g_fwd = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g_fwd, stream=stream):
+            g_fwd = torch.cuda.CUDAGraph()      # the two halves on their own: timed separately, and used by the
+            with torch.cuda.graph(g_fwd, stream=stream):      # end-to-end leg (host copies overlap the other half)
                 run.forward()
             g_bwd = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g_bwd, stream=stream):
                 run.backward()
 
-    def one_step():
-        if graph is not None:
-            graph.replay()
-        else:
-            run.step()
+    one_step = graph.replay if graph is not None else run.step
+    fwd_only = g_fwd.replay if g_fwd is not None else run.forward
+    bwd_only = g_bwd.replay if g_bwd is not None else run.backward
 
     def barrier():
         torch.cuda.synchronize()
@@ -301,27 +287,40 @@ def main():
     launches_per_step = run.plan.launch_count() - launches0
     torch.cuda.synchronize()
 
+    def timed(fn, n, cold=True, pre=None):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        with torch.cuda.stream(stream):
+            for _ in range(warmup):
+                if pre:
+                    pre()
+                if cold:
+                    flush_l2()
+                fn()
+        barrier()
+        with torch.cuda.stream(stream):
+            for a, b in ev:
+                if pre:
+                    pre()
+                if cold:
+                    flush_l2()
+                a.record(stream)
+                fn()
+                b.record(stream)
+        barrier()
+        t = [a.elapsed_time(b) for a, b in ev]
+        return sum(t) / len(t), min(t)
+
     # ---- device-resident timing: L2 flushed before every step, events around each step ----------
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    with torch.cuda.stream(stream):
-        for _ in range(args.warmup):
-            flush_l2()
-            one_step()
-    barrier()
     sampler = ClockSampler(local_rank)
     t_wall0 = time.perf_counter()
-    with torch.cuda.stream(stream):
-        for a, b in ev:
-            flush_l2()
-            a.record(stream)
-            one_step()
-            b.record(stream)
-    barrier()
+    ms, ms_min = timed(one_step, steps, cold=True)
     t_wall = time.perf_counter() - t_wall0
     clocks = sampler.stop()
-    per_step = [a.elapsed_time(b) for a, b in ev]
-    ms = sum(per_step) / len(per_step)
     assert run.status() == 0
+    n_aux = max(3, min(steps, 30))
+    ms_warm, _ = timed(one_step, n_aux, cold=False)                      # operands left in L2 by the step before
+    ms_fwd, _ = timed(fwd_only, n_aux, cold=True)
+    ms_bwd, _ = timed(bwd_only, n_aux, cold=True, pre=fwd_only)          # `saved` from a forward, then flush, then time
 
     # ---- end to end with host buffers: H2D of X and dY, pack, step, unpack, D2H of Y and dX --------
     tdt = run.tdtype
@@ -349,7 +348,7 @@ def main():
             dY_rm.copy_(hdY, non_blocking=True)
             ev_dy.record(side)
         run.plan.pack(TENSOR["X"], dX_rm.data_ptr(), run.buf["X"].data_ptr(), s)
-        g_fwd.replay() if g_fwd is not None else run.forward()
+        fwd_only()
         ev_fwd.record(stream)
         with torch.cuda.stream(side):
             side.wait_event(ev_fwd)
@@ -358,35 +357,23 @@ def main():
             ev_y.record(side)
         stream.wait_event(ev_dy)
         run.plan.pack(TENSOR["DY"], dY_rm.data_ptr(), run.buf["dY"].data_ptr(), s)
-        g_bwd.replay() if g_bwd is not None else run.backward()
+        bwd_only()
         run.plan.unpack(TENSOR["DX"], run.buf["dX"].data_ptr(), odX_rm.data_ptr(), s)
         hdX.copy_(odX_rm, non_blocking=True)
         stream.wait_event(ev_y)
 
-    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    with torch.cuda.stream(stream):
-        for _ in range(args.warmup):
-            flush_l2()
-            e2e_step()
-    barrier()
-    with torch.cuda.stream(stream):
-        for a, b in ev2:
-            flush_l2()
-            a.record(stream)
-            e2e_step()
-            b.record(stream)
-    barrier()
-    ms_e2e = sum(a.elapsed_time(b) for a, b in ev2) / len(ev2)
+    ms_e2e, _ = timed(e2e_step, max(3, min(steps, 50)), cold=True)
     assert run.status() == 0
     assert torch.equal(hY, oY_rm.cpu()) and torch.equal(hdX, odX_rm.cpu())     # both streams had joined
     io_bytes = 2 * cfg.n_tokens * cfg.d_model * (2 if cfg.dtype == "bf16" else 4)
 
-    # ---- per-step event timing (separate pass, direct launches) for the roofline of the dominant step ----
+    # ---- per-kernel event timing: a separate pass of direct launches with an event after every kernel group.  The
+    # event between two kernels keeps the second from starting its set-up under the first one's tail (programmatic
+    # dependent launch), so each figure is a kernel's stand-alone duration and their sum exceeds the step time. ----
     run.plan.profile_enable(True)
     acc = {}
-    reps = max(3, min(args.steps, 10))
     with torch.cuda.stream(stream):
-        for _ in range(reps):
+        for _ in range(max(3, min(steps, 10))):
             flush_l2()
             run.forward()
             stream.synchronize()
@@ -399,15 +386,16 @@ def main():
     run.plan.profile_enable(False)
     kernel_ms = {k: sum(v) / len(v) for k, v in acc.items()}
 
-    ms, ms_e2e = rep.max_over_ranks([ms, ms_e2e])      # the slowest replica sets the whole-job time
-    if rank != 0:
-        rep.close()
-        return
+    ms, ms_warm, ms_fwd, ms_bwd, ms_e2e = rep.max_over_ranks([ms, ms_warm, ms_fwd, ms_bwd, ms_e2e])   # the slowest replica counts
+    sizes = dict(run.sizes)
+    del run, graph, g_fwd, g_bwd, hX, hdY, hY, hdX, dX_rm, dY_rm, oY_rm, odX_rm
+    torch.cuda.empty_cache()
+    if rep.rank != 0:
+        return None
 
     peaks = measured_peaks()
     flops = cfg.flops()
     tfl = rep.whole_job_rate(flops, ms) / 1e12
-    tfl_e2e = rep.whole_job_rate(flops, ms_e2e) / 1e12
     sf, sbytes = step_flops(cfg), step_bytes(cfg)
     dom = max(kernel_ms, key=kernel_ms.get)
     total_k = sum(kernel_ms.values())
@@ -417,10 +405,11 @@ def main():
             roof = {"bound": "tensor", "kernel": dom, "achieved": ach, "peak": peaks["tflops_burst"], "unit": "TFLOP/s",
                     "frac": ach / peaks["tflops_burst"], "traffic": None, "peak_source": peaks["source"] + " (burst)"}
         else:
-            # FFMA path: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
-            alu = 148 * 128 * 2 * 1.965e9 / 1e12
+            # FFMA path: SMs x 128 lanes x 2 flop x 1.965 GHz
+            sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
+            alu = sms * 128 * 2 * 1.965e9 / 1e12
             roof = {"bound": "alu", "kernel": dom, "achieved": ach, "peak": alu, "unit": "TFLOP/s", "frac": ach / alu,
-                    "traffic": None, "peak_source": "148 SM x 128 FFMA/clk x 1.965 GHz"}
+                    "traffic": None, "peak_source": f"{sms} SM x 128 FFMA/clk x 1.965 GHz"}
     else:
         ach = sbytes.get(dom, 0.0) / (kernel_ms[dom] * 1e-3) / 1e9
         roof = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peaks["gbs"], "unit": "GB/s",
@@ -428,37 +417,146 @@ def main():
     roof["traffic"] = NCU_TRAFFIC_BYTES.get((cfg.name, dom))
     roof["kernel_share"] = kernel_ms[dom] / total_k
     roof["kernel_ms"] = {k: round(v, 5) for k, v in sorted(kernel_ms.items(), key=lambda kv: -kv[1])}
+    roof["kernel_ms_sum_over_step_ms"] = total_k / ms      # > 1: what programmatic launch overlap hides in a real step
+    roof["timing"] = "stand-alone kernel durations (an event after every kernel group; no launch overlap)"
+    # the bandwidth-bound kernels of the step against the measured HBM copy rate
+    roof["hbm_kernels"] = {k: {"GBps": sbytes[k] / (kernel_ms[k] * 1e-3) / 1e9,
+                               "frac": sbytes[k] / (kernel_ms[k] * 1e-3) / 1e9 / peaks["gbs"]}
+                           for k in kernel_ms if sbytes.get(k)}
+    # per-kernel fraction of the tensor peak for the tensor-bound ones
+    roof["tensor_kernels"] = {k: {"TFLOPs": sf[k] / (kernel_ms[k] * 1e-3) / 1e12,
+                                  "frac": sf[k] / (kernel_ms[k] * 1e-3) / 1e12 / peaks["tflops_burst"]}
+                              for k in kernel_ms if k in sf} if cfg.dtype == "bf16" and args.path == 0 else {}
+
+    # memory efficiency of the layer (the paper's Eq. 2 factor): once-only minimum bytes over the DRAM bytes ncu saw
+    steps_with_traffic = {k: NCU_TRAFFIC_BYTES.get((cfg.name, k)) for k in kernel_ms}
+    if all(v is not None for v in steps_with_traffic.values()):
+        dram = sum(steps_with_traffic.values())
+        mem_eff = {"min_bytes": min_bytes(cfg), "ncu_dram_bytes": dram, "value": min_bytes(cfg) / dram,
+                   "source": "profiles/ (cold-cache captures, one per kernel)"}
+    else:
+        mem_eff = {"min_bytes": min_bytes(cfg), "ncu_dram_bytes": None, "value": None,
+                   "source": "no ncu capture of every kernel of this workload under profiles/"}
 
     cpu = None
-    if not args.no_cpu_baseline:
-        from fbl_inputs import scaled_config
-        sample_batch = max(1, min(cfg.batch, int(4e10 // max(cfg.flops() / cfg.batch, 1)) or 1))
-        scfg = scaled_config(cfg, batch=sample_batch)
+    if want_cpu:
+        scfg, what = oracle_sample(cfg)
         sinp = make_inputs(scfg)
         t = time_oracle(scfg, sinp, 2)
         sec = min(t)
         cpu = {"value": scfg.flops() / sec / 1e12, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle",
-               "sample": f"batch {sample_batch} of {cfg.batch}, full sequence, best of 2 fwd+bwd passes", "seconds": sec}
+               "sample": f"{what}; best of 2 fwd+bwd passes", "seconds": sec}
 
     t_tensor = flops / (peaks["tflops_burst"] * 1e12)
+    return {
+        "workload": workload_name(cfg), "ms_per_step": ms, "ms_per_step_min": ms_min, "ms_per_step_warm_l2": ms_warm,
+        "ms_fwd": ms_fwd, "ms_bwd": ms_bwd,
+        "tflops": tfl, "tokens_per_s": rep.whole_job_rate(cfg.n_tokens, ms), "flops_per_step": flops,
+        "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
+        "layer_roofline": {"binds": "tensor" if cfg.dtype == "bf16" else "launch latency",
+                           "t_tensor_us_at_measured_burst": t_tensor * 1e6,
+                           "frac_of_measured_burst": t_tensor / (ms * 1e-3),
+                           "frac_of_measured_sustained": flops / (peaks["tflops_sustained"] * 1e12) / (ms * 1e-3),
+                           "frac_of_nominal_2250": flops / (NOMINAL_TFLOPS * 1e12) / (ms * 1e-3),
+                           "t_hbm_us_min_bytes_at_measured": min_bytes(cfg) / (peaks["gbs"] * 1e9) * 1e6},
+        "mem_efficiency": mem_eff,
+        "activation_bytes": {"saved": sizes["saved"], "scratch": sizes["scratch_fwd"] + sizes["scratch_bwd"]},
+        "e2e": {"value": rep.whole_job_rate(flops, ms_e2e) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": io_bytes, "d2h_bytes_per_step": io_bytes},
+        "launches_per_step": launches_per_step, "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
+        "wall_s_timed_region": t_wall,
+    }
+
+
+def run_rank(args):
+    """Body of one rank (the only one at N = 1)."""
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    def pick(i):
+        cfg = get_config(i)
+        if args.seq or args.batch:
+            cfg = scaled_config(cfg, name=cfg.name + "-scaled", seq=args.seq or cfg.seq, batch=args.batch or cfg.batch)
+        return cfg
+
+    if args.impl == "reference":
+        run_reference(args, pick(args.config or HEADLINE), rank)
+        return
+
+    import torch
+    from paper_2607_21624_b200.build import build
+    build()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
+    torch.cuda.set_device(local_rank)
+    from paper_2607_21624_b200.replicas import Replicas
+    rep = Replicas(backend="nccl", device=torch.device("cuda", local_rank))
+
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # 256 MiB > 126 MB L2
+    flush_rd = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device="cuda")  # 256 MiB, only ever read
+    flush_sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def flush_l2():
+        # Write a buffer larger than L2, then read another one: the write evicts the step's data, the read evicts
+        # the write's dirty lines, whose write-back would otherwise run inside the timed step and take DRAM bandwidth
+        # from it (an artefact of the flush, not of the workload).
+        flush.zero_()
+        if not args.flush_write_only:
+            torch.sum(flush_rd, dim=0, keepdim=True, dtype=torch.int32, out=flush_sink)
+
+    head = args.config or HEADLINE
+    todo = [args.config] if args.config else list(ORDER)
+    results = {}
+    for i in todo:
+        cfg = pick(i)
+        results[i] = measure(cfg, args, rep, local_rank, flush_l2, want_cpu=(i == head and not args.no_cpu_baseline))
+    if rank != 0:
+        rep.close()
+        return
+
+    h = results[head]
+    peaks = measured_peaks()
     line = {
-        "metric": "fwd+bwd layer TFLOP/s", "value": tfl, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": workload_name(cfg), "l2": "256 MiB written" + ("" if args.flush_write_only else ", then 256 MiB read (so that the write-back of the flush is over)") + " before every timed step",
-                   "launch": "cuda graph replay" if graph is not None else "direct launches",
-                   "kernel_path": "default" if args.path == 0 else "ffma", "parallelism": "replicas only"},
-        "tokens_per_s": rep.whole_job_rate(cfg.n_tokens, ms),
-        "layer_roofline": {"t_tensor_us_at_measured_burst": t_tensor * 1e6, "frac_of_measured_burst": t_tensor / (ms * 1e-3),
-                           "frac_of_nominal_2250": flops / (NOMINAL_TFLOPS * 1e12) / (ms * 1e-3)},
-        "activation_bytes": {"saved": run.sizes["saved"], "scratch": max(run.sizes["scratch_fwd"], run.sizes["scratch_bwd"])},
-        "e2e": {"value": tfl_e2e, "unit": "TFLOP/s", "ms_per_step": ms_e2e, "h2d_bytes_per_step": io_bytes,
-                "d2h_bytes_per_step": io_bytes},
-        "gpu_launches": launches_per_step * args.steps,
-        "clocks": clocks, "roofline": roof, "cpu_baseline": cpu, "wall_s_timed_region": t_wall,
+        "metric": "fwd+bwd layer TFLOP/s", "value": h["tflops"], "unit": "TFLOP/s", "n_gpus": rep.world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": h["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": h["dtype"], "data": "synthetic",
+        "config": {"workload": h["workload"],
+                   "l2": "256 MiB written" + ("" if args.flush_write_only else ", then 256 MiB read (so that the write-back of the flush is over)") + " before every timed step",
+                   "launch": "direct launches" if args.no_graph else "cuda graph replay",
+                   "kernel_path": "default" if args.path == 0 else "ffma", "parallelism": "replicas only",
+                   "also_timed": "per_config holds all five workloads, each timed the same way in this process"},
+        "tokens_per_s": h["tokens_per_s"], "layer_roofline": h["layer_roofline"], "mem_efficiency": h["mem_efficiency"],
+        "activation_bytes": h["activation_bytes"], "e2e": h["e2e"],
+        "gpu_launches": sum(r["launches_per_step"] for r in results.values()) * args.steps,
+        "clocks": h["clocks"], "roofline": h["roofline"], "cpu_baseline": h["cpu_baseline"],
+        "peaks": peaks,
+        "per_config": {f"workload{i}": results[i] for i in sorted(results)},
     }
     print(json.dumps(line))
     rep.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=0, help="1-based index of one workload (default: all five, headline = the fifth)")
+    ap.add_argument("--impl", default="fblayout", choices=["fblayout", "reference"])
+    ap.add_argument("--path", type=int, default=0, help="0 default kernels, 1 FFMA kernels only")
+    ap.add_argument("--no-graph", action="store_true", help="enqueue kernels directly instead of replaying a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flush-write-only", action="store_true", help="flush L2 by the 256 MiB write alone (its write-back then overlaps the step)")
+    ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling captures)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "fblayout" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "fblayout":
+        # not under a launcher: start the replicas ourselves, one process per GPU
+        from paper_2607_21624_b200.replicas import spawn_replicas
+        spawn_replicas(args.gpus, run_rank, args)
+        return
+    run_rank(args)
 
 
 if __name__ == "__main__":

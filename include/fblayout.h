@@ -91,23 +91,26 @@ enum {
   FBL_MAP_COUNT
 };
 
-typedef struct fbl_plan fbl_plan; /* opaque: padded sizes, index-map constants, kernel choices */
+typedef struct fbl_plan fbl_plan; /* opaque: padded sizes, index-map constants, kernel choices.  Enqueue calls on
+                                   * one plan keep a little bookkeeping in it: use one plan per host thread. */
 
-/* Host only.  Validates the description against the tile-propagation legality checks of section 4.3
+/* Host code only (no device work; it asks the runtime for the current device's SM count to size grids and work
+ * areas, and plans for 148 SMs when there is no device).  Validates the description against the tile-propagation legality checks of section 4.3
  * (head_dim and d_model multiples of tile_w, n_q_heads a multiple of n_kv_heads) and the kernels'
  * limits, then builds the plan.  *out is owned by the caller; release with fbl_plan_destroy.
  * The plan also fixes, from the shapes alone, into how many slices the token-axis reductions of the weight
  * gradients are cut (1 for all but layers with few weight tiles and many tokens).  Environment variables
  * read here, for tuning and tests only: FBL_KSPLIT_O and FBL_KSPLIT_QKV override those slice counts,
- * FBL_VERBOSE prints the ones chosen to stderr.  Three more are read when a step is enqueued, again for tuning
- * and tests only: FBL_GEMM_PAIR (0: never use the CTA-pair GEMM kernel, 1: use it wherever its tile shape is
+ * FBL_VERBOSE prints the ones chosen to stderr.  Three more, again for tuning and tests only: FBL_GEMM_PAIR (0: never use the CTA-pair GEMM kernel, 1: use it wherever its tile shape is
  * legal; unset: large launches only), FBL_GEMM_ESETS (1 or 2 sets of epilogue warps in the single-CTA GEMM kernel;
  * unset: 2 where every block of the launch has one tile) and FBL_FWD_TILES (1 or 2 query tiles per
  * forward-attention block at head_dim 64; unset: by sequence length). */
 int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out);
 void fbl_plan_destroy(fbl_plan* plan);
 
-/* Padded R-Tile size in bytes of a matrix (physical ids only; views return the size of their buffer). */
+/* Padded R-Tile size in bytes of a matrix (physical ids only; views return the size of their buffer).  Rows are
+ * padded to whole tiles only (seq and weight rows rounded up to tile_h = 8), which keeps the padded share far
+ * inside the 10 % limit of the paper's tile-selection constraint C3 (section 4.2, candidate generation). */
 int fbl_tensor_bytes(const fbl_plan* plan, int tensor_id, size_t* bytes);
 
 /* Sizes of the three caller-owned work areas: `saved` carries forward tensors into the backward
@@ -115,7 +118,22 @@ int fbl_tensor_bytes(const fbl_plan* plan, int tensor_id, size_t* bytes);
  * the scratch areas hold per-call temporaries. */
 int fbl_workspace_bytes(const fbl_plan* plan, size_t* saved, size_t* scratch_fwd, size_t* scratch_bwd);
 
-/* Element map (pure host integer code): logical index -> element offset in the R-Tile buffer.
+/* Where the step's intermediates live inside the caller's work areas (byte offset and size), so that a caller
+ * can inspect them after synchronising: matrices are R-Tile buffers readable with fbl_unpack under the tensor id
+ * of the same shape (XN; Q for Q, A, dA, dQ; K for K, V, dK, dV); STATS is fp32 [B*T_pad][2] = (mean, rstd);
+ * LSE and D are fp32 [B][Hq][T_pad].  FBL_WS_STATS .. FBL_WS_LSE are offsets into `saved` (section 3.1's reused
+ * forward tensors), the others into the backward scratch. */
+enum {
+  FBL_WS_STATS = 0, FBL_WS_XN, FBL_WS_Q, FBL_WS_K, FBL_WS_V, FBL_WS_A, FBL_WS_LSE,
+  FBL_WS_D, FBL_WS_DA, FBL_WS_DQ, FBL_WS_DK, FBL_WS_DV, FBL_WS_DXN,
+  FBL_WS_PARTIALS,   /* partial sums of the backward's token-axis reductions (bias column sums, dgamma / dbeta) */
+  FBL_WS_COUNT
+};
+int fbl_workspace_offset(const fbl_plan* plan, int what, size_t* offset, size_t* bytes);
+
+/* Element map (pure host integer code): logical index -> element offset in the R-Tile buffer, i.e. the
+ * composition of section 4.2's inter-tile mapping (which tile, row-tile index fastest) and intra-tile mapping
+ * (row-major inside the 8 x tile_w tile).
  * idx is [b, t, c, 0] for token matrices, [r, c, 0, 0] for weights and transposed views,
  * [b, h, t, d] for head views.  Returns < 0 if idx is out of range. */
 int64_t fbl_tile_offset(const fbl_plan* plan, int tensor_id, const int32_t idx[4]);
@@ -123,20 +141,27 @@ int64_t fbl_tile_offset(const fbl_plan* plan, int tensor_id, const int32_t idx[4
 /* Tile map f of Eq. 3, composed and strength-reduced as in Eq. 4 (host integer code). */
 int fbl_tile_map(const fbl_plan* plan, int map_id, int64_t src_tile, int64_t* dst_tile);
 
-/* Layout conversion at the graph boundary only (row-major dense <-> R-Tile), device to device.
- * Never part of a training step. */
+/* Layout conversion at the graph boundary only (row-major dense <-> R-Tile), device to device: section 4.4 keeps
+ * one layout inside the graph and converts only where tensors enter or leave it.  Never part of a training step. */
 int fbl_pack(const fbl_plan* plan, int tensor_id, const void* rowmajor_dev, void* tiled_dev, void* stream);
 int fbl_unpack(const fbl_plan* plan, int tensor_id, const void* tiled_dev, void* rowmajor_dev, void* stream);
 
-/* Forward: Y = [X +] softmax-attention(norm(X)) Wo [+ bo]; fills `saved`.  Biases and beta may be NULL
- * when the plan has none. */
+/* Forward of the attention block of the paper's motivating example (section 2: projections, P = softmax(Q K^T),
+ * O = P V, output projection): Y = [X +] softmax-attention(norm(X)) Wo [+ bo].  Fills `saved`, the forward
+ * tensors the backward reuses (the E_reuse edges of section 3.1), in the same layout the backward reads them in.
+ * Biases and beta may be NULL when the plan has none.  The call first clears the status word at the start of
+ * `scratch` (see fbl_status_poll). */
 int fbl_layer_fwd(const fbl_plan* plan, const void* X, const float* gamma, const float* beta,
                   const void* Wq, const void* Wk, const void* Wv, const void* Wo,
                   const float* bq, const float* bk, const float* bv, const float* bo,
                   void* Y, void* saved, void* scratch, void* stream);
 
-/* Backward: every gradient of sum(Y * dY).  Matrix gradients are in the storage dtype in R-Tile
- * order; vector gradients are fp32.  db* may be NULL when the plan has no biases, dbeta for RMSNorm. */
+/* Backward of the same block (section 2's gradient operators; section 3.2's reduce-axis conflicts are resolved by
+ * operand orientation, not by copies): every gradient of sum(Y * dY).  Matrix gradients are in the storage dtype
+ * in R-Tile order; vector gradients are fp32.  db* may be NULL when the plan has no biases, dbeta for RMSNorm.
+ * The call first clears the status word at the start of its own `scratch`: a caller that wants to see a
+ * forward-pass time-out after the backward has been enqueued gives the two passes separate scratch buffers
+ * (scratch_fwd_bytes / scratch_bwd_bytes) and polls both. */
 int fbl_layer_bwd(const fbl_plan* plan, const void* dY, const void* X, const float* gamma,
                   const void* Wq, const void* Wk, const void* Wv, const void* Wo, const void* saved,
                   void* dX, void* dWq, void* dWk, void* dWv, void* dWo,
@@ -159,8 +184,11 @@ int fbl_colsum(const fbl_plan* plan, const void* M_dev, int64_t rows, int64_t co
  * host side of CUDA or through any library.  Same arguments and result as fbl_colsum minus `scratch_dev`.
  *   - Limit: ceil(rows / 256) * cols <= 262144 (for example 16384 rows x 4096 columns); beyond it the call
  *     returns FBL_ERR_WORKSPACE_TOO_SMALL and enqueues nothing.
- *   - The first call on each device looks up the array's device address (with that device current); make that
- *     first call outside any stream capture.
+ *   - The first call on each device looks up the array's device address (with that device current).  Make that
+ *     first call at start-up, outside any stream capture and before memory is tight: with the runtime's lazy
+ *     module loading it may be the call that loads the library image carrying the array onto the device, which
+ *     the driver does with an allocation of its own; "allocates nothing" holds from the second call on.  The
+ *     address is cached per device ordinal and does not survive a device reset.
  *   - All calls on a device share the one array.  Each call overwrites the part it uses before reading it, so
  *     earlier contents never leak into a result, but two calls that can run at the same time on the GPU (different
  *     streams, no ordering between them) race; order them. */
@@ -170,6 +198,16 @@ int fbl_colsum_noalloc(const fbl_plan* plan, const void* M_dev, int64_t rows, in
 /* After the caller has synchronised the stream: reads back the device status word kept at the start
  * of `scratch` (set when a bounded wait inside a kernel expired).  Synchronous 4-byte copy. */
 int fbl_status_poll(const fbl_plan* plan, const void* scratch, int32_t* device_status);
+
+/* Self-test of the failure detection (no counterpart in the paper).  Every wait inside the tensor-core kernels is
+ * bounded: when it expires, the kernel records a code in the status word at the start of `scratch`, leaves its
+ * loops, releases its tensor memory and returns, so the context stays usable.  This call enqueues one tiny kernel
+ * that waits, through the same code, on a barrier nothing will ever signal, with `limit_cycles` clock cycles as
+ * the bound (clamped to [1e3, 2e9]); it first zeroes the first 8 bytes of `scratch` (1024-byte aligned device
+ * memory, at least 8 bytes).  After the caller has synchronised, fbl_status_poll on that buffer returns
+ * FBL_ERR_TIMEOUT with *device_status == 901, and the int32 behind the status word holds 1 (the block ran to its
+ * normal end). */
+int fbl_selftest_wait_timeout(void* scratch, int64_t limit_cycles, void* stream);
 
 /* Kernel family used by later calls on this plan: 0 = default (tcgen05 tensor-core kernels for bf16
  * wherever one exists for the shape, FFMA kernels for fp32), 1 = FFMA kernels only (fp32 arithmetic on

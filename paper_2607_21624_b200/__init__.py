@@ -4,7 +4,8 @@ The shared library is built in-tree by ``paper_2607_21624_b200.build``; importin
 package never falls back to another implementation: if the library is missing or a
 CUDA device is absent, calls raise.
 """
-from .binding import (FblError, Plan, lib, load_library, LayerRunner, DTYPES, TENSOR, MAP,
-                      desc_from_config, aligned_bytes)
+from .binding import (FblError, Plan, lib, load_library, LayerRunner, DTYPES, TENSOR, MAP, WS,
+                      desc_from_config, aligned_bytes, guard_bands_intact, selftest_wait_timeout)
 
-__all__ = ["FblError", "Plan", "lib", "load_library", "LayerRunner", "DTYPES", "TENSOR", "MAP", "desc_from_config", "aligned_bytes"]
+__all__ = ["FblError", "Plan", "lib", "load_library", "LayerRunner", "DTYPES", "TENSOR", "MAP", "WS",
+           "desc_from_config", "aligned_bytes", "guard_bands_intact", "selftest_wait_timeout"]

@@ -17,6 +17,8 @@ NORMS = {"layernorm": 0, "rmsnorm": 1}
 TENSOR = {n: i for i, n in enumerate(
     ["X", "Y", "DY", "DX", "WQ", "WK", "WV", "WO", "XN", "Q", "K", "V", "A",
      "Q_HEADS", "K_HEADS", "V_HEADS", "A_HEADS", "WQ_T", "WK_T", "WV_T", "WO_T"])}
+WS = {n: i for i, n in enumerate(
+    ["STATS", "XN", "Q", "K", "V", "A", "LSE", "D", "DA", "DQ", "DK", "DV", "DXN", "PARTIALS"])}
 MAP = {n: i for i, n in enumerate(
     ["SPLIT_Q", "MERGE_Q", "SPLIT_KV", "MERGE_KV", "TRANSPOSE_WQ", "TRANSPOSE_WO", "PHYS_Q", "PHYS_WQ"])}
 
@@ -50,6 +52,8 @@ def load_library():
     L.fbl_plan_destroy.restype = None
     L.fbl_tensor_bytes.argtypes = [vp, C.c_int, C.POINTER(sz)]
     L.fbl_workspace_bytes.argtypes = [vp, C.POINTER(sz), C.POINTER(sz), C.POINTER(sz)]
+    L.fbl_workspace_offset.argtypes = [vp, C.c_int, C.POINTER(sz), C.POINTER(sz)]
+    L.fbl_selftest_wait_timeout.argtypes = [vp, i64, vp]
     L.fbl_tile_offset.argtypes = [vp, C.c_int, C.POINTER(i32)]
     L.fbl_tile_offset.restype = i64
     L.fbl_tile_map.argtypes = [vp, C.c_int, i64, C.POINTER(i64)]
@@ -118,6 +122,11 @@ class Plan:
         _check(lib().fbl_workspace_bytes(self._h, C.byref(a), C.byref(b), C.byref(c)))
         return a.value, b.value, c.value
 
+    def workspace_offset(self, what: int):
+        off, nbytes = C.c_size_t(), C.c_size_t()
+        _check(lib().fbl_workspace_offset(self._h, what, C.byref(off), C.byref(nbytes)))
+        return off.value, nbytes.value
+
     def tile_offset(self, tensor_id: int, idx) -> int:
         arr = (C.c_int32 * 4)(*(list(idx) + [0] * (4 - len(idx))))
         return lib().fbl_tile_offset(self._h, tensor_id, arr)
@@ -178,12 +187,36 @@ class Plan:
         return out.value
 
 
-def aligned_bytes(torch, nbytes, device, align=1024, zero=True):
+def selftest_wait_timeout(scratch_ptr, limit_cycles, stream):
+    """fbl_selftest_wait_timeout: enqueue the kernel whose bounded wait is meant to expire."""
+    _check(lib().fbl_selftest_wait_timeout(scratch_ptr, limit_cycles, stream))
+
+
+GUARD_BYTE = 0xA5
+
+
+def aligned_bytes(torch, nbytes, device, align=1024, zero=True, guard=0):
     """A uint8 device tensor of ``nbytes`` whose data pointer is ``align``-byte aligned (torch only
-    promises 512)."""
-    raw = (torch.zeros if zero else torch.empty)(nbytes + align, dtype=torch.uint8, device=device)
+    promises 512).  With ``guard`` > 0 (a multiple of ``align``) the view sits between two bands of that many
+    bytes filled with GUARD_BYTE; ``guard_bands_intact`` checks them."""
+    raw = (torch.zeros if zero else torch.empty)(nbytes + align + 2 * guard, dtype=torch.uint8, device=device)
     off = (-raw.data_ptr()) % align
-    return raw[off:off + nbytes]
+    if guard:
+        assert guard % align == 0
+        raw[off:off + guard] = GUARD_BYTE
+        raw[off + guard + nbytes:off + 2 * guard + nbytes] = GUARD_BYTE
+    view = raw[off + guard:off + guard + nbytes]
+    view._fbl_guard = (raw, off, guard, nbytes)
+    return view
+
+
+def guard_bands_intact(view) -> bool:
+    raw, off, guard, nbytes = view._fbl_guard
+    if not guard:
+        return True
+    lo = raw[off:off + guard]
+    hi = raw[off + guard + nbytes:off + 2 * guard + nbytes]
+    return bool((lo == GUARD_BYTE).all().item()) and bool((hi == GUARD_BYTE).all().item())
 
 
 class LayerRunner:
@@ -192,7 +225,9 @@ class LayerRunner:
     MATS = {"X": "X", "dY": "DY", "Wq": "WQ", "Wk": "WK", "Wv": "WV", "Wo": "WO"}
     OUT_MATS = {"Y": "Y", "dX": "DX", "dWq": "WQ", "dWk": "WK", "dWv": "WV", "dWo": "WO"}
 
-    def __init__(self, cfg, device="cuda:0"):
+    def __init__(self, cfg, device="cuda:0", guard_bytes=0):
+        """``guard_bytes`` > 0 surrounds every device buffer with bands of a known byte pattern
+        (``guards_intact`` checks them): a stand-in for a memory checker when hunting writes past a buffer."""
         import torch
         if not torch.cuda.is_available():
             raise FblError(-101, "no CUDA device: the layer has no CPU path")
@@ -203,16 +238,25 @@ class LayerRunner:
         self.tdtype = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
         saved, sf, sb = self.plan.workspace_bytes()
         self.sizes = dict(saved=saved, scratch_fwd=sf, scratch_bwd=sb)
-        al = lambda nbytes: aligned_bytes(torch, nbytes, self.dev)
+        al = lambda nbytes: aligned_bytes(torch, nbytes, self.dev, guard=guard_bytes)
         self.saved = al(saved)
-        self.scratch = al(max(sf, sb))
+        # one scratch per pass: each pass clears the status word of its own scratch, so a time-out recorded by a
+        # forward kernel is still there after the backward has run
+        self.scratch_fwd = al(sf)
+        self.scratch = al(sb)
         self.buf = {}
         for name, tid in {**self.MATS, **self.OUT_MATS}.items():
             self.buf[name] = al(self.plan.tensor_bytes(TENSOR[tid]))
         d, dq, dkv = cfg.d_model, cfg.d_q, cfg.d_kv
         fz = lambda n: torch.zeros(n, dtype=torch.float32, device=self.dev)
-        self.vec = {"gamma": fz(d), "beta": fz(d), "bq": fz(dq), "bk": fz(dkv), "bv": fz(dkv), "bo": fz(d),
-                    "dgamma": fz(d), "dbeta": fz(d), "dbq": fz(dq), "dbk": fz(dkv), "dbv": fz(dkv), "dbo": fz(d)}
+        lens = {"gamma": d, "beta": d, "bq": dq, "bk": dkv, "bv": dkv, "bo": d,
+                "dgamma": d, "dbeta": d, "dbq": dq, "dbk": dkv, "dbv": dkv, "dbo": d}
+        if guard_bytes:
+            self._vec_raw = {k: al(4 * n) for k, n in lens.items()}
+            self.vec = {k: v.view(torch.float32) for k, v in self._vec_raw.items()}
+        else:
+            self._vec_raw = {}
+            self.vec = {k: fz(n) for k, n in lens.items()}
 
     # -- helpers ---------------------------------------------------------------------------
     def _stream(self):
@@ -248,7 +292,7 @@ class LayerRunner:
                             ptr(b["Wq"]), ptr(b["Wk"]), ptr(b["Wv"]), ptr(b["Wo"]),
                             ptr(v["bq"]) if bias else None, ptr(v["bk"]) if bias else None,
                             ptr(v["bv"]) if bias else None, ptr(v["bo"]) if bias else None,
-                            ptr(b["Y"]), ptr(self.saved), ptr(self.scratch), self._stream())
+                            ptr(b["Y"]), ptr(self.saved), ptr(self.scratch_fwd), self._stream())
 
     def backward(self):
         c, b, v = self.cfg, self.buf, self.vec
@@ -276,10 +320,44 @@ class LayerRunner:
         torch.cuda.synchronize(self.dev)
         return self.vec[name].cpu().numpy().astype("float64")
 
+    # intermediates: name -> (workspace id, tensor id whose shape it has, last logical dimension)
+    INTERMEDIATES = {"Xn": ("XN", "XN", "d_model"), "Q": ("Q", "Q", "d_q"), "K": ("K", "K", "d_kv"),
+                     "V": ("V", "K", "d_kv"), "A": ("A", "Q", "d_q"), "dA": ("DA", "Q", "d_q"),
+                     "dQ": ("DQ", "Q", "d_q"), "dK": ("DK", "K", "d_kv"), "dV": ("DV", "K", "d_kv"),
+                     "dXn": ("DXN", "XN", "d_model")}
+
     def saved_view(self, name):
-        """Raw R-Tile bytes of a saved matrix (Xn, Q, K, V, A) as a flat torch tensor in the storage dtype."""
-        raise NotImplementedError
+        """An intermediate of the last step as a float64 numpy array in its logical shape: the saved forward
+        tensors Xn, Q, K, V, A ([B, T, C]), LSE ([B, Hq, T]), stats ([B, T, 2] = mean, rstd), and from the
+        backward scratch D ([B, Hq, T]), dA, dQ, dK, dV, dXn ([B, T, C])."""
+        torch, c = self.torch, self.cfg
+        torch.cuda.synchronize(self.dev)
+        t_pad = (c.seq + 7) // 8 * 8
+        if name in ("LSE", "D", "stats"):
+            off, nbytes = self.plan.workspace_offset(WS[name.upper()])
+            src = self.saved if name != "D" else self.scratch
+            flat = src[off:off + nbytes].view(torch.float32)
+            if name == "stats":
+                return flat.view(c.batch, t_pad, 2)[:, :c.seq].cpu().numpy().astype("float64")
+            return flat.view(c.batch, c.n_q_heads, t_pad)[:, :, :c.seq].cpu().numpy().astype("float64")
+        ws, tid, dim = self.INTERMEDIATES[name]
+        off, nbytes = self.plan.workspace_offset(WS[ws])
+        src = self.saved if ws in ("XN", "Q", "K", "V", "A") else self.scratch
+        out = torch.empty((c.batch, c.seq, getattr(c, dim)), dtype=self.tdtype, device=self.dev)
+        self.plan.unpack(TENSOR[tid], src[off:off + nbytes].data_ptr(), out.data_ptr(), self._stream())
+        torch.cuda.synchronize(self.dev)
+        return out.float().cpu().numpy().astype("float64")
+
+    def guards_intact(self):
+        """Names of the buffers whose guard bands were overwritten (empty list: none)."""
+        self.torch.cuda.synchronize(self.dev)
+        named = {"saved": self.saved, "scratch_fwd": self.scratch_fwd, "scratch_bwd": self.scratch}
+        named.update(self.buf)
+        named.update(self._vec_raw)
+        return [k for k, v in named.items() if not guard_bands_intact(v)]
 
     def status(self) -> int:
+        """Device status of the last forward and backward (0, or the code of the first bounded wait that expired)."""
         self.torch.cuda.synchronize(self.dev)
-        return self.plan.status_poll(self.scratch.data_ptr())
+        fwd = self.plan.status_poll(self.scratch_fwd.data_ptr())
+        return fwd if fwd != 0 else self.plan.status_poll(self.scratch.data_ptr())

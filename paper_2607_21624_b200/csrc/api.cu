@@ -50,7 +50,7 @@ thread_local char g_detail[256] = "";
 #define FBL_STEP(name, kernels, expr)                              \
   do {                                                             \
     FBL_CUDA(expr);                                                \
-    fbl_plan* mp__ = const_cast<fbl_plan*>(p);                     \
+    const fbl_plan* mp__ = p;                                      \
     mp__->launches += (kernels);                                   \
     if (mp__->prof_on && mp__->prof_n < FBL_PROF_MAX) {            \
       mp__->prof_name[mp__->prof_n] = (name);                      \
@@ -61,13 +61,12 @@ thread_local char g_detail[256] = "";
 
 #define FBL_PROF_BEGIN()                                           \
   do {                                                             \
-    fbl_plan* mp__ = const_cast<fbl_plan*>(p);                     \
+    const fbl_plan* mp__ = p;                                      \
     if (mp__->prof_on) { mp__->prof_n = 0; FBL_CUDA(cudaEventRecord(mp__->prof_ev[0], st)); } \
   } while (0)
 
-cudaError_t run_gemm(const fbl_plan* p, const GemmArgs& g, void* sk, size_t sk_bytes, int32_t* status,
-                     cudaStream_t st) {
-  if (p->use_tc && gemm_tc_supported(p, g)) return launch_gemm_tc(p, g, sk, sk_bytes, status, st);
+cudaError_t run_gemm(const fbl_plan* p, const GemmArgs& g, int32_t* status, cudaStream_t st) {
+  if (p->use_tc && gemm_tc_supported(p, g)) return launch_gemm_tc_group(p, &g, 1, status, st);
   return launch_gemm_simt(p->d.dtype, g, st);
 }
 
@@ -113,7 +112,20 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   p->dkv = d.n_kv_heads * d.head_dim;
   p->group = d.n_q_heads / d.n_kv_heads;
   p->scale = d.softmax_scale > 0.f ? d.softmax_scale : 1.0f / sqrtf((float)d.head_dim);
+  // SM count of the current device; a host without a device (index-map and sizing calls only) plans for 148 SMs
   p->sm_count = 148;
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      p->sm_count = sms;
+    else
+      (void)cudaGetLastError();       // no device: not an error of this call
+  }
+  auto env_int = [](const char* name, int dflt) { const char* v = getenv(name); return v ? atoi(v) : dflt; };
+  p->knob_gemm_pair = env_int("FBL_GEMM_PAIR", -1);
+  p->knob_gemm_esets = env_int("FBL_GEMM_ESETS", 0);
+  p->knob_fwd_tiles = env_int("FBL_FWD_TILES", 0);
   p->use_tc = d.dtype == FBL_DTYPE_BF16 ? 1 : 0;
 
   const size_t n = (size_t)p->n_pad;
@@ -129,15 +141,16 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   p->sv_lse = o;   o += fbl_align_up(rows_bh * sizeof(float) + 512, FBL_ALIGN);   // + one 128-float copy window past the last row
   p->saved_bytes = o;
 
-  // partial-sum area: column-sum slabs or split-K slices, whichever is larger
-  size_t part = colsum_scratch_bytes(p->n_pad, (int64_t)d.d_model + p->dq + 2 * p->dkv);
-  const size_t splitk = (size_t)p->sm_count * 128 * 256 * sizeof(float) * 2;
-  if (splitk > part) part = splitk;
-  p->part_bytes = fbl_align_up(part, FBL_ALIGN);
+  // Partial-sum area of the backward's token-axis reductions: the slab partials of the four bias column sums
+  // first, then (from the next 256-float boundary) the norm backward's per-block partial rows, at most two
+  // blocks per SM with one dgamma row and one dbeta row each.
+  {
+    const size_t cs_floats = colsum_scratch_bytes(p->n_pad, (int64_t)d.d_model + p->dq + 2 * p->dkv) / sizeof(float);
+    const size_t norm_floats = (size_t)2 * p->sm_count * 2 * d.d_model;
+    p->part_bytes = fbl_align_up(((cs_floats + 255) / 256 * 256 + norm_floats) * sizeof(float), FBL_ALIGN);
+  }
 
-  o = FBL_ALIGN;  // status word
-  p->sf_part = o; o += p->part_bytes;
-  p->scratch_fwd_bytes = o;
+  p->scratch_fwd_bytes = FBL_ALIGN;  // the status word
 
   // weight-gradient GEMMs: few output tiles, reduction over all tokens; slice the reduction when that balances the SMs
   p->ksplit_o = p->ksplit_qkv = 1;
@@ -223,6 +236,30 @@ int fbl_workspace_bytes(const fbl_plan* plan, size_t* saved, size_t* scratch_fwd
   if (scratch_fwd) *scratch_fwd = plan->scratch_fwd_bytes;
   if (scratch_bwd) *scratch_bwd = plan->scratch_bwd_bytes;
   return FBL_OK;
+}
+
+int fbl_workspace_offset(const fbl_plan* plan, int what, size_t* offset, size_t* bytes) {
+  if (!plan || !offset || !bytes) return FBL_ERR_INVALID_ARG;
+  const fbl_plan* p = plan;
+  const size_t n = (size_t)p->n_pad, e = (size_t)p->e;
+  const size_t rows_bh = (size_t)p->d.batch * p->d.n_q_heads * p->t_pad;
+  switch (what) {
+    case FBL_WS_STATS: *offset = p->sv_stats; *bytes = n * 2 * sizeof(float); return FBL_OK;
+    case FBL_WS_XN: *offset = p->sv_xn; *bytes = n * p->d.d_model * e; return FBL_OK;
+    case FBL_WS_Q: *offset = p->sv_q; *bytes = n * p->dq * e; return FBL_OK;
+    case FBL_WS_K: *offset = p->sv_k; *bytes = n * p->dkv * e; return FBL_OK;
+    case FBL_WS_V: *offset = p->sv_v; *bytes = n * p->dkv * e; return FBL_OK;
+    case FBL_WS_A: *offset = p->sv_a; *bytes = n * p->dq * e; return FBL_OK;
+    case FBL_WS_LSE: *offset = p->sv_lse; *bytes = rows_bh * sizeof(float); return FBL_OK;
+    case FBL_WS_D: *offset = p->sb_dvec; *bytes = rows_bh * sizeof(float); return FBL_OK;
+    case FBL_WS_DA: *offset = p->sb_da; *bytes = n * p->dq * e; return FBL_OK;
+    case FBL_WS_DQ: *offset = p->sb_dq; *bytes = n * p->dq * e; return FBL_OK;
+    case FBL_WS_DK: *offset = p->sb_dk; *bytes = n * p->dkv * e; return FBL_OK;
+    case FBL_WS_DV: *offset = p->sb_dv; *bytes = n * p->dkv * e; return FBL_OK;
+    case FBL_WS_DXN: *offset = p->sb_dxn; *bytes = n * p->d.d_model * e; return FBL_OK;
+    case FBL_WS_PARTIALS: *offset = p->sb_part; *bytes = p->part_bytes; return FBL_OK;
+    default: return FBL_ERR_INVALID_ARG;
+  }
 }
 
 int64_t fbl_tile_offset(const fbl_plan* plan, int tensor_id, const int32_t idx[4]) {
@@ -334,7 +371,6 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
   float* stats = (float*)(sv + p->sv_stats);
   void* Xn = sv + p->sv_xn; void* Q = sv + p->sv_q; void* K = sv + p->sv_k; void* V = sv + p->sv_v;
   void* A = sv + p->sv_a; float* lse = (float*)(sv + p->sv_lse);
-  void* part = sc + p->sf_part;
   const bool bias = p->d.has_bias;
   const int n = (int)p->n_pad, D = p->d.d_model;
 
@@ -375,7 +411,7 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
     g.c = Y; g.c_rpad = p->n_pad; g.bias = bias ? bo : nullptr;
     g.residual = p->d.residual ? X : nullptr;
     g.seq = p->d.seq; g.t_pad = p->t_pad;
-    FBL_STEP("proj_o", 1, run_gemm(p, g, part, p->part_bytes, status, st));
+    FBL_STEP("proj_o", 1, run_gemm(p, g, status, st));
   }
   return FBL_OK;
 }
@@ -450,8 +486,8 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
       FBL_STEP("dWo+dA", 1, launch_gemm_tc_group(p, gs, 2, status, st));
       dwo_round = split_o;        // nothing in the step reads dWo: its rounding joins that of dWq, dWk, dWv below
     } else {
-      FBL_STEP("dA", 1, run_gemm(p, ga, part, p->part_bytes, status, st));
-      FBL_STEP("dWo", 1, run_gemm(p, gw, part, p->part_bytes, status, st));
+      FBL_STEP("dA", 1, run_gemm(p, ga, status, st));
+      FBL_STEP("dWo", 1, run_gemm(p, gw, status, st));
     }
   }
   if (p->use_tc && attn_bwd_tc_supported(p)) FBL_STEP("attn_bwd", dvec_ready ? 2 : 3, launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, dvec_ready, status, st));   // dqacc: zero already
@@ -498,9 +534,9 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
       FBL_STEP("dWqkv+dXn", 1, launch_gemm_tc_group(p, gs, 4, status, st));
       if (cg.count > 0) FBL_STEP("dW round", 1, launch_convert_f32_group(cg, st));     // one rounding launch for all sliced GEMMs
     } else {
-      FBL_STEP("dXn", 1, run_gemm(p, gx, part, p->part_bytes, status, st));
+      FBL_STEP("dXn", 1, run_gemm(p, gx, status, st));
       for (int i = 0; i < 3; ++i)
-        FBL_STEP(i == 0 ? "dWq" : i == 1 ? "dWk" : "dWv", 1, run_gemm(p, gs[i], part, p->part_bytes, status, st));
+        FBL_STEP(i == 0 ? "dWq" : i == 1 ? "dWk" : "dWv", 1, run_gemm(p, gs[i], status, st));
     }
   }
   if (dwo_round) {
@@ -541,6 +577,16 @@ int fbl_status_poll(const fbl_plan* plan, const void* scratch, int32_t* device_s
   if (!plan || !scratch || !device_status) return FBL_ERR_INVALID_ARG;
   FBL_CUDA(cudaMemcpy(device_status, scratch, sizeof(int32_t), cudaMemcpyDeviceToHost));
   return *device_status == 0 ? FBL_OK : FBL_ERR_TIMEOUT;
+}
+
+int fbl_selftest_wait_timeout(void* scratch, int64_t limit_cycles, void* stream) {
+  if (!scratch || misaligned(scratch)) return scratch ? FBL_ERR_MISALIGNED : FBL_ERR_INVALID_ARG;
+  if (limit_cycles < 1000) limit_cycles = 1000;
+  if (limit_cycles > 2000000000LL) limit_cycles = 2000000000LL;
+  cudaStream_t st = as_stream(stream);
+  FBL_CUDA(cudaMemsetAsync(scratch, 0, 8, st));
+  FBL_CUDA(launch_wait_timeout_selftest((int32_t*)scratch, (long long)limit_cycles, st));
+  return FBL_OK;
 }
 
 const char* fbl_strerror(int status) {

@@ -44,18 +44,23 @@ struct fbl_plan {
   size_t sv_stats, sv_xn, sv_q, sv_k, sv_v, sv_a, sv_lse, saved_bytes;
   // byte offsets inside the backward scratch
   size_t sb_da, sb_dvec, sb_dqacc, sb_dq, sb_dk, sb_dv, sb_dxn, sb_part, scratch_bwd_bytes;
-  size_t sf_part, scratch_fwd_bytes;
+  size_t scratch_fwd_bytes;
   size_t part_bytes;
   // reduction-loop slicing of the weight-gradient GEMMs (1: none) and their fp32 accumulation areas, which
   // follow the status word so that one fill zeroes both
   int ksplit_o, ksplit_qkv;
   size_t sb_acc_o, sb_acc_qkv, acc_bytes;
   size_t zero_bytes;        // leading part of the backward scratch that every step starts by zero-filling
-  // bookkeeping: kernels enqueued so far, optional per-step event timing
-  int64_t launches;
-  int prof_on, prof_n;
-  cudaEvent_t prof_ev[FBL_PROF_MAX + 1];
-  const char* prof_name[FBL_PROF_MAX];
+  // tuning knobs, read from the environment once, at plan creation (0 / -1 = the library's own choice)
+  int knob_gemm_pair;       // -1 by size, 0 never the CTA-pair GEMM kernel, 1 wherever its tile shape is legal
+  int knob_gemm_esets;      // 0 by tiles per block, 1 / 2 sets of epilogue warps
+  int knob_fwd_tiles;       // 0 by sequence length, 1 / 2 query tiles per forward-attention block at head_dim 64
+  // bookkeeping of the enqueue calls (they take the plan as const): kernels enqueued so far, optional per-step
+  // event timing.  Calls on one plan are not thread-safe; give each host thread its own plan.
+  mutable int64_t launches;
+  mutable int prof_on, prof_n;
+  mutable cudaEvent_t prof_ev[FBL_PROF_MAX + 1];
+  mutable const char* prof_name[FBL_PROF_MAX];
 };
 
 static inline size_t fbl_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -88,12 +93,11 @@ struct GemmArgs {
 };
 
 cudaError_t launch_gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);
-cudaError_t launch_gemm_tc(const fbl_plan* p, const GemmArgs& g, void* splitk_scratch, size_t splitk_bytes,
-                           int32_t* status, cudaStream_t st);
 bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g);
 cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st);
 struct GemmShape { int64_t m; int n; int kblocks; int splittable; };
 int gemm_tc_choose_split(int sm_count, const GemmShape* sh, int count);
+cudaError_t launch_wait_timeout_selftest(int32_t* status, long long limit_cycles, cudaStream_t st);
 bool attn_fwd_tc_supported(const fbl_plan* p);
 bool attn_bwd_tc_supported(const fbl_plan* p);
 void fbl_note_cuda_error(cudaError_t e, const char* where);

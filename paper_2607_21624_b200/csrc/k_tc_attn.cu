@@ -38,20 +38,6 @@ static int chunk_for(long long bytes_per_hb, int n_hb, long long budget) {
   return (int)(c < 1 ? 1 : (c > n_hb ? n_hb : c));
 }
 
-// Optional timeline probe (compile with -DFBL_TRACE): block (0,0,0) records clock64() at the marked points of
-// iterations 8..14 into the 1 KiB status area, after the status word.
-#ifdef FBL_TRACE
-#ifndef FBL_TRACE_FIRST
-#define FBL_TRACE_FIRST 8
-#endif
-#ifndef FBL_TRACE_BLOCK
-#define FBL_TRACE_BLOCK 0
-#endif
-#define TR(k) do { if (blockIdx.x == FBL_TRACE_BLOCK && it >= FBL_TRACE_FIRST && it < FBL_TRACE_FIRST + 3) ((long long*)P.status)[8 + (it - FBL_TRACE_FIRST) * 32 + (k)] = clock64(); } while (0)
-#else
-#define TR(k) do { } while (0)
-#endif
-
 struct alignas(64) AttnFwdParams {
   CUtensorMap tq, tk, tv;
   __nv_bfloat16* a;      // merged-head output [n_pad, dq] in R-Tile order
@@ -242,10 +228,8 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
       for (int n = 0; n < 3 && n < n_items && ok; ++n) ok = issue_s_item(n);
       for (int n = 0; n < n_items && ok; ++n) {
         int w, j; item(n, w, j);
-        { const int it = j; TR(1 + 3 * w); }
         if (w == 0 && !tc::mbar_wait(bar(B_VFULL + (j & 1)), (j >> 1) & 1, status, 207)) { ok = false; break; }
         if (!tc::mbar_wait(bar(B_PFULL + n % 3), (n / 3) & 1, status, 206)) { ok = false; break; }
-        { const int it = j; TR(2 + 3 * w); }
         tc::tc_fence_after();
         const uint32_t vl = v_lo + (j & 1) * (SM::TILE >> 4);
         const uint32_t pa = tmem_base + (uint32_t)(n % 3) * 128, od = tmem_base + O_COL + w * HD;
@@ -255,7 +239,6 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
         tc::mma_commit(bar(B_PVDONE + w));
         if (w == 1 || j >= n_kv1) tc::mma_commit(bar(B_VEMPTY + (j & 1)));
         if (n + 3 < n_items) ok = issue_s_item(n + 3);     // into the buffer whose P the product above has just read
-        { const int it = j; TR(3 + 3 * w); }
       }
     } else {
     bool ok = tc::mbar_wait(bar(B_QFULL), 0, status, 203) && tc::mbar_wait(bar(B_KFULL), 0, status, 204);
@@ -266,19 +249,16 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
     }
     for (int j = 0; j < n_kv_max && ok; ++j) {
       const bool next = j + 1 < n_kv_max;
-      { const int it = j; TR(0); }
       if (!tc::mbar_wait(bar(B_VFULL + (j & 1)), (j >> 1) & 1, status, 207)) { ok = false; break; }
       if (next && !tc::mbar_wait(bar(B_KFULL + ((j + 1) & 1)), ((j + 1) >> 1) & 1, status, 205)) { ok = false; break; }
 #pragma unroll
       for (int w = 0; w < TILES; ++w) {
         const int nk = w ? n_kv1 : n_kv0;
         if (ok && j < nk) {
-          { const int it = j; TR(1 + 3 * w); }
           if (!tc::mbar_wait(bar(B_PFULL + w), j & 1, status, 206)) { ok = false; }
-          else { { const int it = j; TR(2 + 3 * w); } tc::tc_fence_after(); issue_pv(w, j); }
+          else { tc::tc_fence_after(); issue_pv(w, j); }
         }
         if (ok && j + 1 < nk) issue_s(w, j + 1);
-        { const int it = j; TR(3 + 3 * w); }
       }
       if (!ok) break;
       tc::mma_commit(bar(B_VEMPTY + (j & 1)));              // both P V products of this stage are behind us
@@ -303,14 +283,12 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
     bool ok = true;
     for (int j = 0; j < n_kvw && ok; ++j) {
       const int j0 = j * BKV;
-      { const int it = j; if (r == 0) TR(8 + 8 * w); }
       // score buffer and barrier phase of this (tile, key tile): see the MMA issuer
       const int n_item = ROT ? (w ? 2 * j + 1 : j + min(j, n_kv1)) : j;
       const int sbuf = ROT ? n_item % 3 : w;
       const uint32_t sph = ROT ? (uint32_t)(n_item / 3) & 1u : (uint32_t)j & 1u;
       const uint32_t s_addr = lane_addr + (uint32_t)sbuf * 128;
       if (!tc::mbar_wait(bar(B_SFULL + sbuf), sph, status, 208)) { ok = false; break; }
-      { const int it = j; if (r == 0) TR(9 + 8 * w); }
       tc::tc_fence_after();
       const bool need_mask = (j0 + BKV > P.seq) || (P.causal && j0 + BKV - 1 > i0);
       float mx, alpha, mc;
@@ -340,7 +318,6 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
           mx2 = tc::fmax3(mx2, sv[k + 4], sv[k + 5]); mx3 = tc::fmax3(mx3, sv[k + 6], sv[k + 7]);
         }
         mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-        { const int it = j; if (r == 0) TR(10 + 8 * w); }
         // lazy running max: move it only when the tile's max beats it by more than the threshold
         moved = mx > m + tau || m == -INFINITY;
         const float m_new = moved ? fmaxf(m, mx) : m;
@@ -365,7 +342,6 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
             tc::tmem_st32(o_addr + cc * 32, o);
           }
         }
-        { const int it = j; if (r == 0) TR(11 + 8 * w); }
         // P = exp2(S c - m c), its row sum, and P packed to bf16 (128 scores become 64 packed columns)
         const float2 nmc2 = make_float2(-mc, -mc);
   #pragma unroll
@@ -454,7 +430,6 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
       tc::tmem_st_wait();
       tc::tc_fence_before();
       tc::mbar_arrive(bar(B_PFULL + sbuf));
-      { const int it = j; if (r == 0) TR(12 + 8 * w); }
     }
     if (ok && n_kvw > 0) ok = tc::mbar_wait(bar(B_PVDONE + w), (n_kvw - 1) & 1, status, 210);
     tc::tc_fence_after();
@@ -518,7 +493,7 @@ cudaError_t fwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   P.pair = (n_qt >= 2 && (long long)((n_qt + 1) / 2) * p->d.n_q_heads * p->d.batch >= p->sm_count) ? 1 : 0;
   if (HD == 64) {
     // tuning knob: 1 = one query tile per block and two blocks per SM, 2 = two tiles per block; default by sequence length
-    const int mode = getenv("FBL_FWD_TILES") ? atoi(getenv("FBL_FWD_TILES")) : 0;
+    const int mode = p->knob_fwd_tiles;
     if (mode == 1 || (mode == 0 && n_qt <= 4)) return fwd_launch_t<64, 1>(p, P, n_qt, st);
   }
   return fwd_launch_t<HD, 2>(p, P, n_qt, st);
@@ -750,41 +725,32 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       // P^T has its own columns here, so the next tile's products come first and the softmax warps start on
       // tile it + 1 while the tensor pipe works on dV, dK, dQ of tile it
       for (int it = 0; it < n_it && ok; ++it) {
-        TR(0);
         if (it + 1 < n_it) {
           // S^T(it+1) as soon as every softmax warp has copied S^T(it) to registers: it is computed while
           // they work on tile it
           if (!tc::mbar_wait(bar(BB_SREAD), it & 1, status, 311)) { ok = false; break; }
           if (!tc::mbar_wait(bar(BB_QFULL + ((it + 1) % NQQ)), ((it + 1) / NQQ) & 1, status, 303)) { ok = false; break; }
-          TR(1);
           tc::tc_fence_after();
           issue_s(it + 1);
         }
         if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
-        TR(2);
         tc::tc_fence_after();
         if (it + 1 < n_it) {
           if (!tc::mbar_wait(bar(BB_DOFULL + ((it + 1) % NDO)), ((it + 1) / NDO) & 1, status, 314)) { ok = false; break; }
           issue_dp(it + 1);                             // dP^T(it) has been read as well: announce tile it + 1
         }
-        TR(3);
         issue_dv(it);
         tc::mma_commit(bar(BB_DVDONE));                 // P^T(it) has been read: P^T(it+1) may be stored
         tc::mma_commit(bar(BB_DOEMPTY + (it % NDO)));   // ... and dO of this tile is not read again
-        TR(4);
         issue_dk(it);
         tc::mma_commit(bar(BB_QEMPTY + (it % NQQ)));    // nor is Q
         if (it > 0 && !tc::mbar_wait(bar(BB_DQDRAINED), (it - 1) & 1, status, 304)) { ok = false; break; }
-        TR(5);
         tc::tc_fence_after();
         issue_dq(it);
-        TR(6);
       }
     } else {
       for (int it = 0; it < n_it && ok; ++it) {
-        TR(0);
         if (!tc::mbar_wait(bar(BB_PDSFULL), it & 1, status, 305)) { ok = false; break; }
-        TR(1);
         tc::tc_fence_after();
         // dQ first: its drain to shared memory (which frees the dP^T columns for the next tile) then overlaps
         // the dV and dK products
@@ -793,18 +759,14 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         tc::mma_commit(bar(BB_QEMPTY));                 // Q of this tile is not read again: the next one is fetched
         issue_dv(it);                                   // while dV runs
         tc::mma_commit(bar(BB_DOEMPTY));                // ... and dO
-        TR(2);
         if (it + 1 < n_it) {
           if (!tc::mbar_wait(bar(BB_QFULL), (it + 1) & 1, status, 303)) { ok = false; break; }
-          TR(3);
           tc::tc_fence_after();
           issue_s(it + 1);                   // the S^T columns (P^T by now) were last read by dV above
           if (!tc::mbar_wait(bar(BB_DQDRAINED), it & 1, status, 304)) { ok = false; break; }
           if (!tc::mbar_wait(bar(BB_DOFULL), (it + 1) & 1, status, 314)) { ok = false; break; }
-          TR(4);
           tc::tc_fence_after();
           issue_dp(it + 1);                  // the dP^T columns held dQ until it was drained
-          TR(5);
         }
       }
       // dQ is issued first here, so its barrier does not cover the last tile's dK and dV products: one more
@@ -850,7 +812,6 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       if (!tc::mbar_wait(bar(BB_DQFULL), dit & 1, status, 307)) return false;
       // the staging buffer's previous tile must have been read by its bulk reduction
       if (dit >= (int)NS && !stage_is_alt(dit) && !tc::mbar_wait(bar(BB_STAGEFREE + (dit % NS)), (dit / (int)NS - 1) & 1, status, 310)) return false;
-      { const int it = dit; if (t == 0) TR(8); }
       tc::tc_fence_after();
       // this thread's HD / 4 accumulator columns in one go; the tensor pipe gets the columns back (at HD = 128 the
       // next tile's dP^T waits for them) as soon as they are in registers, before the stores to the staging tile
@@ -862,7 +823,6 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       tc::tmem_ld_wait();
       tc::tc_fence_before();
       tc::mbar_arrive(bar(BB_DQDRAINED));            // TMEM side done: the tensor pipe may reuse the columns
-      { const int it = dit; if (t == 0) TR(7); }
 #pragma unroll
       for (int u = 0; u < NC / 16; ++u) {            // 16 columns = half of a 128-byte unit of the box
         const int cu = c0 + u * 16;
@@ -890,9 +850,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       // and arrived before the score products awaited below were issued
       const float* s_lse = s_stage + (it % NQQ) * 128;
       const float* s_d = s_stage + NQQ * 128 + (it % NDO) * 128;
-      if (t == 0) TR(9);
       if (!tc::mbar_wait(bar(BB_SFULL), it & 1, status, 306)) { ok = false; break; }
-      if (t == 0) TR(10);
       tc::tc_fence_after();
       // element masks are needed only on the diagonal tile and on tiles with keys or queries beyond the sequence
       const bool need_mask = (P.causal && (i0 < j0 + BKV - 1)) || (j0 + BKV > P.seq) || (i0 + BQ > P.seq);
@@ -949,7 +907,6 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
           dd[k / 2] = tc::pack_bf16(gv[0], gv[1]);
           dd[k / 2 + 1] = tc::pack_bf16(gv[2], gv[3]);
         }
-        if (t == 0) TR(16 + cc);
         if (PIPE && cc == 0 && it > 0) {
           // P^T has its own columns, single-buffered: the dV product of the previous tile must have read them.
           // The wait sits here, behind the first chunk's arithmetic, which needs only S^T and dP^T.
@@ -974,18 +931,14 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       }
       if (!ok) break;
       tc::tmem_st_wait();
-      if (t == 0) TR(15);
       tc::fence_proxy_async();
-      if (t == 0) TR(6);
       tc::tc_fence_before();
       tc::mbar_arrive(bar(BB_PDSFULL));
-      if (t == 0) TR(11);
       if (PIPE) {
         if (it > 0) ok = drain_dq(it - 1);
       } else {
         ok = drain_dq(it);
       }
-      if (t == 0) TR(12);
     }
     if (PIPE && ok && n_it > 0) ok = drain_dq(n_it - 1);
     // dK, dV of this key tile: every MMA has completed (HD = 64: dQ is the last product issued, and the wait for

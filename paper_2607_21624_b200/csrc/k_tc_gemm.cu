@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <mutex>
+#include <vector>
 
 #include "fbl_internal.h"
 #include "pdl.cuh"
@@ -43,7 +44,6 @@ struct alignas(64) TcGroup {
   TcProblem p[MAX_PROBLEMS];
   int count;
   int32_t* status;
-  int trace_slot;
   // Optional chores for the epilogue warps while the first tile's main loop runs: zero-fill a buffer that a later
   // kernel of the pass adds into (16-byte units, dealt evenly to the blocks), and reset the pass's status word.
   uint4* zero_ptr;
@@ -60,25 +60,6 @@ __device__ __forceinline__ void group_chores(const TcGroup& G, int tid, int n_th
     for (long long i = lo + tid; i < hi; i += n_threads) G.zero_ptr[i] = z;
   }
 }
-
-#ifdef FBL_TRACE_GEMM
-int g_trace_launch = 0;
-#endif
-// Optional timeline probe (compile with -DFBL_TRACE_GEMM): one block records clock64() at the marked points of its
-// first output tile into the words after the status word; slot = index of the GEMM launch within the pass.
-#ifdef FBL_TRACE_GEMM
-#ifndef FBL_TRACE_BLOCK
-#define FBL_TRACE_BLOCK 0
-#endif
-__device__ long long g_gemm_trace[2 * 256];
-#define GTR(k) do { if (blockIdx.x == FBL_TRACE_BLOCK) ((long long*)G.status)[8 + G.trace_slot * 24 + (k)] = clock64(); } while (0)
-#define GTK(k) do { if (blockIdx.x == FBL_TRACE_BLOCK && (k) < 256) g_gemm_trace[G.trace_slot * 256 + (k)] = clock64(); } while (0)
-#define GTRG(k) do { if (blockIdx.x == FBL_TRACE_BLOCK) { unsigned long long g_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_)); ((long long*)G.status)[8 + G.trace_slot * 24 + (k)] = (long long)g_; } } while (0)
-#else
-#define GTR(k) do { } while (0)
-#define GTRG(k) do { } while (0)
-#define GTK(k) do { } while (0)
-#endif
 
 template <int BN, int STAGES>
 struct SmemPlan {
@@ -136,7 +117,6 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
   constexpr uint32_t TMEM_COLS = 2 * BN;                 // two fp32 accumulators of BN columns
 
   if (threadIdx.x == 0) {
-    GTR(0); GTRG(8);
     for (int s = 0; s < STAGES; ++s) {
       tc::mbar_init(full(s), 1);                 // one producer arrival + transaction bytes
       tc::mbar_init(empty(s), 1);                // one tcgen05.commit arrival
@@ -157,7 +137,6 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
   uint32_t tmem_base;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
   pdl_launch_dependents();
-  if (threadIdx.x == 0) GTR(1);
 
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ----------------------------------------------------------------------
@@ -181,7 +160,6 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
       prefilled = n;
     }
     pdl_wait();
-    GTR(2);
     for (int w = blockIdx.x; ok && tile_at<BN>(G, w, &tcd); w += gridDim.x) {
       const TcProblem& P = G.p[tcd.prob];
       for (int t = 0; t < P.n_terms && ok; ++t) {
@@ -195,17 +173,12 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
             if (!tc::mbar_wait(empty(s), ph ^ 1, status, 101)) { ok = false; break; }
             tc::mbar_expect_tx(full(s), SP::STAGE);
           }
-          if (it < 64) GTK(it);
-#ifdef FBL_NO_LOADS
-          asm volatile("mbarrier.complete_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(full(s)), "r"(pre ? SP::A_BYTES : SP::STAGE) : "memory");
-#else
           if (P.a_mn[t]) tc::tma_load_3d(sa, &P.ta[t], full(s), 0, kb * BK, tcd.m0 / 64);
           else tc::tma_load_3d(sa, &P.ta[t], full(s), 0, tcd.m0, kb);
           if (!pre) {
             if (P.b_mn[t]) tc::tma_load_3d(sb, &P.tb[t], full(s), 0, kb * BK, tcd.n0 / 64);
             else tc::tma_load_3d(sb, &P.tb[t], full(s), 0, tcd.n0, kb);
           }
-#endif
         }
       }
     }
@@ -234,7 +207,6 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
         const int nkb = t == 0 ? tcd.kb1 - tcd.kb0 : P.kblocks[t];
         for (int kb = 0; kb < nkb; ++kb) {
           if (!tc::mbar_wait(full(s), ph, status, 102)) { ok = false; break; }
-          if (ti == 0 && t == 0 && kb == 0) GTR(3);
           tc::tc_fence_after();
           uint32_t a_lo = a_lo0 + (uint32_t)s * (SP::STAGE >> 4), b_lo = b_lo0 + (uint32_t)s * (SP::STAGE >> 4);
 #pragma unroll
@@ -248,7 +220,6 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
         }
       }
       if (ok) tc::mma_commit(acc_full(ab));
-      if (ti == 0) GTR(4);
     }
   } else if (warp >= 2) {
     // ---- epilogue: TMEM -> registers -> swizzled staging -> bulk tensor store.  Each warp owns the 32 rows of
@@ -263,7 +234,6 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
     const int set = (warp - 2) / 4;
     constexpr int PPS = BN / 64 / ESETS;              // panels per set
     const int r = q * 32 + lane;                      // row of the tile owned by this thread
-    const bool tracer = threadIdx.x == 64;
     int ti = 0, pc = 0;                               // tiles and panels done by this warp
     bool ok = true;
     TileCoord tcd;
@@ -295,7 +265,6 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
       }
       if (!tc::mbar_wait(acc_full(ab), (ti >> 1) & 1, status, 103)) { ok = false; break; }
       tc::tc_fence_after();
-      if (tracer && ti == 0) GTR(5);
       float dot_acc = 0.f;
 #pragma unroll 1
       for (int pn = pn_begin; pn < pn_end; ++pn) {
@@ -305,7 +274,6 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
         tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + pn * 64, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
         tc::tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + pn * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
         tc::tmem_ld_wait();
-        if (tracer && ti == 0 && pn < 2) GTR(10 + 2 * pn);
         if (P.ksplit > 1) {
           // partial sums of a reduction slice: two 32-column halves of the panel, fp32, added to the accumulation
           // buffer by bulk tensor reductions (same staging tiles and swizzle as the bf16 rows below)
@@ -332,10 +300,6 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
         }
         uint4 outv[8];
         uint32_t* ow = reinterpret_cast<uint32_t*>(outv);
-#ifdef FBL_TRACE_GEMM
-        asm volatile("" ::"r"(v[0]), "r"(v[31]), "r"(v[32]), "r"(v[63]));
-        if (tracer && ti == 0 && pn == 1) GTR(18);
-#endif
         if (has_res) {
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -362,10 +326,6 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
           for (int j = 0; j < 64; j += 2)
             ow[j / 2] = tc::pack_bf16(pad ? 0.f : __uint_as_float(v[j]), pad ? 0.f : __uint_as_float(v[j + 1]));
         }
-#ifdef FBL_TRACE_GEMM
-        asm volatile("" ::"r"(ow[0]), "r"(ow[15]), "r"(ow[16]), "r"(ow[31]));
-        if (tracer && ti == 0 && pn == 1) GTR(19);
-#endif
         if (P.dot_with && row < P.m) {
           // Row reduction over this head's columns, on the ROUNDED values the attention backward will read:
           // sum_j dS_ij = 0 (softmax shift invariance) holds only if D matches the dP that kernel forms.
@@ -390,33 +350,25 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
         // Staging tile (pc & 1) of this warp: its previous store (two panels ago) has been read, since lane 0
         // waited for that after committing the store of the panel before this one.
         const uint32_t stg = base + SP::STG_OFF + (ESETS == 2 ? (uint32_t)(warp - 2) : (uint32_t)(q * 2 + (pc & 1))) * 4096u;
-        if (tracer && ti == 0 && pn == 1) GTR(13);
         if (ESETS == 2 && lane == 0) tc::bulk_wait_group_read0();    // one staging tile: the store before has read it
         __syncwarp();
-        if (tracer && ti == 0 && pn == 1) GTR(14);
 #pragma unroll
         for (int j = 0; j < 8; ++j)
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + (((uint32_t)j ^ (uint32_t)(lane & 7)) * 16)),
                        "r"(outv[j].x), "r"(outv[j].y), "r"(outv[j].z), "r"(outv[j].w) : "memory");
-        if (tracer && ti == 0 && pn == 1) GTR(15);
         tc::fence_proxy_async();
-        if (tracer && ti == 0 && pn == 1) GTR(16);
         __syncwarp();
-        if (tracer && ti == 0 && pn == 1) GTR(17);
         if (lane == 0) {
           tc::tma_store_3d(&P.tc, stg, 0, tcd.m0 + q * 32, n / 64);
           tc::bulk_commit_group();
           if (ESETS == 1) tc::bulk_wait_group_read1();  // the store before this one has read its staging tile
         }
-        if (tracer && ti == 0 && pn < 1) GTR(11 + 2 * pn);
         ++pc;
       }
-      if (tracer && ti == 0) GTR(6);
       tc::tc_fence_before();
       tc::mbar_arrive(acc_empty(ab));             // this accumulator may be overwritten by the tile after next
     }
     if (lane == 0) tc::bulk_wait_group0();        // all output tiles are in global memory before the block exits
-    if (tracer) { GTR(7); GTRG(9); }
   }
   tc::tc_fence_before();
   __syncthreads();
@@ -716,7 +668,27 @@ EncodeTiledFn encode_fn() {
 
 constexpr int BN_SMALL = 128;
 
+// Self-test of the bounded wait every tensor-core kernel relies on: one block initialises an mbarrier that nothing
+// ever signals and waits on it through the same tc::mbar_wait, with a short limit.  The wait must give up, record
+// its code in the status word and let the block return normally.
+__global__ void wait_timeout_selftest_kernel(int32_t* status, long long limit_cycles) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(tc::smem_u32(&bar), 1);
+    tc::fence_barrier_init();
+  }
+  __syncthreads();
+  const bool ok = tc::mbar_wait(tc::smem_u32(&bar), 0, status, 901, limit_cycles);
+  __syncthreads();
+  if (threadIdx.x == 0) status[1] = ok ? 2 : 1;     // the block reached its normal end
+}
+
 }  // namespace
+
+cudaError_t launch_wait_timeout_selftest(int32_t* status, long long limit_cycles, cudaStream_t st) {
+  wait_timeout_selftest_kernel<<<1, 64, 0, st>>>(status, limit_cycles);
+  return cudaGetLastError();
+}
 
 bool fbl_encode_rtile_map(CUtensorMap* map, const void* base, int64_t r_pad, int panels, int box_rows, int box_panels) {
   EncodeTiledFn fn = encode_fn();
@@ -744,11 +716,6 @@ bool fbl_encode_f32_panel_map(CUtensorMap* map, const void* base, int64_t r_pad,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-#ifdef FBL_TRACE_GEMM
-extern "C" int fbl_debug_gemm_trace(long long* host_dst) {
-  return (int)cudaMemcpyFromSymbol(host_dst, g_gemm_trace, sizeof(long long) * 512);
-}
-#endif
 
 bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g) {
   if (p->d.dtype != FBL_DTYPE_BF16) return false;
@@ -763,16 +730,16 @@ bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g) {
   return true;
 }
 
-template <int BN, int STAGES>
-cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
-  TcGroup G;
+// Problem set-up shared by the two kernels: tensor maps, operand orientations, epilogue extras and reduction
+// slices of every problem of a launch.  bn_box: columns of B one CTA loads per k-block; tile_m x tile_n: the output
+// tile a work unit covers (the CTA pair's 256 x 256, or one CTA's 128 x BN).  Returns the number of work units in
+// *units.
+cudaError_t fill_group(TcGroup& G, const GemmArgs* gs, int count, int32_t* status, int bn_box, int tile_m, int tile_n,
+                       int* units) {
   memset(&G, 0, sizeof(G));
   G.count = count;
   G.status = status;
   G.zero_ptr = (uint4*)gs[0].zero_ptr; G.zero_vec = (long long)(gs[0].zero_bytes / 16); G.reset_status = gs[0].reset_status;
-#ifdef FBL_TRACE_GEMM
-  G.trace_slot = (g_trace_launch++) & 1;      // two GEMM launches per pass
-#endif
   int tiles = 0;
   for (int i = 0; i < count; ++i) {
     const GemmArgs& g = gs[i];
@@ -787,8 +754,8 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
       if (tm.a_trans) ok = fbl_encode_rtile_map(&P.ta[t], tm.a, tm.a_rpad, g.m / 64, BK, BM / 64);
       else ok = fbl_encode_rtile_map(&P.ta[t], tm.a, tm.a_rpad, tm.k / 64, BM, 1);
       if (!ok) return cudaErrorInvalidValue;
-      if (tm.b_trans) ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, tm.k / 64, BN, 1);
-      else ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, g.n / 64, BK, BN / 64);
+      if (tm.b_trans) ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, tm.k / 64, bn_box, 1);
+      else ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, g.n / 64, BK, bn_box / 64);
       if (!ok) return cudaErrorInvalidValue;
     }
     P.m = g.m; P.n = g.n;
@@ -805,14 +772,23 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
       P.ksplit = (P.kblocks[0] + per - 1) / per;
       if (!fbl_encode_f32_panel_map(&P.tacc, g.acc, g.c_rpad, g.n / 64, 32, 1)) return cudaErrorInvalidValue;
     }
-    tiles += ((g.m + BM - 1) / BM) * ((g.n + BN - 1) / BN) * P.ksplit;
+    tiles += ((g.m + tile_m - 1) / tile_m) * ((g.n + tile_n - 1) / tile_n) * P.ksplit;
   }
+  *units = tiles;
+  return cudaSuccess;
+}
+
+template <int BN, int STAGES>
+cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
+  TcGroup G;
+  int tiles = 0;
+  cudaError_t e = fill_group(G, gs, count, status, BN, BM, BN, &tiles);
+  if (e != cudaSuccess) return e;
   using SP = SmemPlan<BN, STAGES>;
   const int grid = tiles < p->sm_count ? tiles : p->sm_count;
   // one tile per block at most: the epilogue is exposed, and the variant with two sets of epilogue warps halves it
   // (with several tiles per block the epilogues overlap the next main loops and the extra warps only cost)
-  const int esets_knob = getenv("FBL_GEMM_ESETS") ? atoi(getenv("FBL_GEMM_ESETS")) : 0;      // tuning knob: 1 or 2
-  const bool two_sets = esets_knob ? esets_knob == 2 : tiles <= p->sm_count;
+  const bool two_sets = p->knob_gemm_esets ? p->knob_gemm_esets == 2 : tiles <= p->sm_count;
   if (two_sets) {
     auto k = gemm_tc_kernel<BN, STAGES, 2>;
     cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
@@ -829,47 +805,9 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
 
 cudaError_t launch_group_pair(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
   TcGroup G;
-  memset(&G, 0, sizeof(G));
-  G.count = count;
-  G.status = status;
-  G.zero_ptr = (uint4*)gs[0].zero_ptr; G.zero_vec = (long long)(gs[0].zero_bytes / 16); G.reset_status = gs[0].reset_status;
-#ifdef FBL_TRACE_GEMM
-  G.trace_slot = (g_trace_launch++) & 1;      // two GEMM launches per pass
-#endif
   int tiles = 0;
-  for (int i = 0; i < count; ++i) {
-    const GemmArgs& g = gs[i];
-    TcProblem& P = G.p[i];
-    P.n_terms = g.n_terms;
-    for (int t = 0; t < g.n_terms; ++t) {
-      const GemmTerm& tm = g.t[t];
-      P.kblocks[t] = (tm.k + BK - 1) / BK;
-      P.a_mn[t] = tm.a_trans ? 1 : 0;     // stored [k rows][m cols]: rows are K indices
-      P.b_mn[t] = tm.b_trans ? 0 : 1;     // stored [k rows][n cols]: rows are K indices
-      bool ok;
-      if (tm.a_trans) ok = fbl_encode_rtile_map(&P.ta[t], tm.a, tm.a_rpad, g.m / 64, BK, BM / 64);
-      else ok = fbl_encode_rtile_map(&P.ta[t], tm.a, tm.a_rpad, tm.k / 64, BM, 1);
-      if (!ok) return cudaErrorInvalidValue;
-      if (tm.b_trans) ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, tm.k / 64, 128, 1);
-      else ok = fbl_encode_rtile_map(&P.tb[t], tm.b, tm.b_rpad, g.n / 64, BK, 2);
-      if (!ok) return cudaErrorInvalidValue;
-    }
-    P.m = g.m; P.n = g.n;
-    if (!fbl_encode_rtile_map(&P.tc, g.c, g.c_rpad, g.n / 64, 32, 1)) return cudaErrorInvalidValue;   // one warp's rows
-    P.b_static = g.b_static;
-    P.c = (__nv_bfloat16*)g.c; P.c_rpad = g.c_rpad;
-    P.bias = g.bias; P.residual = (const __nv_bfloat16*)g.residual;
-    P.seq = g.seq; P.t_pad = g.t_pad;
-    P.dot_with = (const __nv_bfloat16*)g.dot_with; P.dot_out = g.dot_out; P.dot_hd = g.dot_hd; P.dot_hq = g.dot_hq;
-    P.ksplit = 1;
-    if (g.ksplit > 1) {
-      if (g.n_terms != 1 || g.bias || g.residual || g.dot_with || g.t_pad > 0 || !g.acc) return cudaErrorInvalidValue;
-      const int per = (P.kblocks[0] + g.ksplit - 1) / g.ksplit;        // no empty slice
-      P.ksplit = (P.kblocks[0] + per - 1) / per;
-      if (!fbl_encode_f32_panel_map(&P.tacc, g.acc, g.c_rpad, g.n / 64, 32, 1)) return cudaErrorInvalidValue;
-    }
-    tiles += ((g.m + 255) / 256) * ((g.n + 255) / 256) * P.ksplit;
-  }
+  cudaError_t e = fill_group(G, gs, count, status, 128, 256, 256, &tiles);   // each CTA loads 128 of the pair's 256 columns
+  if (e != cudaSuccess) return e;
   using SP = PairSmem;
   auto k = gemm_tc_pair_kernel;
   cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
@@ -894,7 +832,7 @@ cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int coun
   if (wide && tiles_wide * 3 < p->sm_count * 2) wide = false;
   // CTA pairs on 256 x 256 tiles for large problems (several rounds of tiles per SM pair): measured 2-6 % faster
   // on the workload 5 GEMMs, no gain or a loss below that
-  const int pair_mode = getenv("FBL_GEMM_PAIR") ? atoi(getenv("FBL_GEMM_PAIR")) : -1;   // tuning knob: 0 never, 1 whenever legal
+  const int pair_mode = p->knob_gemm_pair;       // tuning knob: 0 never, 1 whenever legal, -1 by size
   if (pair_mode == 1 && wide_legal) return launch_group_pair(p, gs, count, status, st);
   if (wide && pair_mode != 0) {
     long long pair_tiles = 0;
@@ -934,7 +872,7 @@ int gemm_tc_choose_split(int sm_count, const GemmShape* sh, int count) {
     for (int i = 0; i < count; ++i)
       units += (long long)((sh[i].m + BM - 1) / BM) * ((sh[i].n + bn - 1) / bn) * ((sh[i].splittable && S > 1) ? S : 1);
     const int grid = (int)(units < sm_count ? units : sm_count);
-    double load[256] = {0};
+    std::vector<double> load((size_t)grid, 0.0);
     long long w = 0;
     for (int i = 0; i < count; ++i) {
       const int s_i = (sh[i].splittable && S > 1) ? S : 1;
@@ -949,8 +887,4 @@ int gemm_tc_choose_split(int sm_count, const GemmShape* sh, int count) {
     else if (mk < 0.85 * base_cost && mk < best_cost) { best = S; best_cost = mk; }   // worth it only with a clear gain
   }
   return best;
-}
-
-cudaError_t launch_gemm_tc(const fbl_plan* p, const GemmArgs& g, void*, size_t, int32_t* status, cudaStream_t st) {
-  return launch_gemm_tc_group(p, &g, 1, status, st);
 }

@@ -40,17 +40,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false (after writing `code` to *status) if the phase did not complete in time
 // or another role already reported a failure.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* status, int32_t code) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* status, int32_t code,
+                                          long long limit_cycles = WAIT_LIMIT_CYCLES) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 0xFF) == 0) {
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      if (clock64() - t0 > limit_cycles) {
         atomicCAS(status, 0, code);
-#ifdef FBL_TRACE
-        status[16 + (code % 100)] = (int32_t)parity + 1;      // which waits expired, with the parity they wanted
-#endif
         return false;
       }
       if (*(volatile int32_t*)status != 0) return false;

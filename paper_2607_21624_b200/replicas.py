@@ -48,3 +48,23 @@ class Replicas:
         if self.dist is not None:
             self.dist.destroy_process_group()
             self.dist = None
+
+
+def _replica_entry(rank, world, port, fn, args):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    fn(*args)
+
+
+def spawn_replicas(world: int, fn, *args):
+    """Run ``fn(*args)`` in ``world`` fresh processes, one per replica, each with the rank variables a launcher
+    would have set (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR = 127.0.0.1, a free MASTER_PORT), and wait for all
+    of them.  ``fn`` must be importable from the child (a module-level function).  Used by a command that is
+    asked for several GPUs without having been started under a launcher."""
+    import socket
+
+    import torch.multiprocessing as mp
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    mp.spawn(_replica_entry, args=(world, port, fn, args), nprocs=world, join=True)

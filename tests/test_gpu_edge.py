@@ -93,6 +93,7 @@ def test_step_does_not_depend_on_previous_buffer_contents(cfg):
     ref = None
     for fill in (0x00, 0xFF, 0x7F):
         run.scratch.fill_(fill)
+        run.scratch_fwd.fill_(fill)
         run.saved.fill_(fill)
         run.step()
         assert run.status() == 0
@@ -134,3 +135,46 @@ def test_many_back_to_back_steps_are_identical(cfg):
         assert np.array_equal(first[n], run.fetch(n)), n
     for n in ("dX", "dWq"):
         assert np.abs(first[n] - run.fetch(n)).max() <= 2e-2 * np.abs(first[n]).max() + 1e-6, n
+
+
+def test_bounded_wait_expires_and_the_context_stays_usable():
+    # Failure detection: every barrier wait in the tensor-core kernels is bounded.  The self-test kernel waits,
+    # through the same code, on a barrier that nothing signals, with a bound of 2e5 clock cycles (about 0.1 ms).  The
+    # wait must run out, the kernel must return normally, the status word must carry the wait's code, and a normal
+    # step on the same context must then run and report no error.
+    import torch
+    from paper_2607_21624_b200 import LayerRunner, aligned_bytes, lib, selftest_wait_timeout
+    cfg = LayerConfig("e13", 2, 300, 256, 4, 2, 64, "bf16", "layernorm", True, True, False, 1e-5, 61, 0.02)
+    run = LayerRunner(cfg)
+    run.load_inputs(make_inputs(cfg, affine_noise=True))
+    scratch = aligned_bytes(torch, 1024, run.dev)
+    scratch.fill_(0xFF)
+    selftest_wait_timeout(scratch.data_ptr(), 200_000, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    import ctypes
+    word = ctypes.c_int32()
+    rc = lib().fbl_status_poll(run.plan._h, scratch.data_ptr(), ctypes.byref(word))
+    assert rc == -6 and word.value == 901, (rc, word.value)            # FBL_ERR_TIMEOUT, the self-test's wait code
+    assert int(scratch.view(torch.int32)[1].item()) == 1               # the block reached its normal end
+    assert lib().fbl_strerror(rc).decode() == "a bounded device-side wait expired"
+    run.step()
+    assert run.status() == 0
+    ref = run.fetch("Y")
+    run.step()
+    assert run.status() == 0 and np.array_equal(ref, run.fetch("Y"))
+
+
+def test_forward_timeout_code_survives_the_backward():
+    # Each pass clears the status word of its own scratch, so a code left in the forward's scratch is still visible
+    # after a backward has been enqueued behind it.
+    import torch
+    from paper_2607_21624_b200 import LayerRunner, selftest_wait_timeout
+    cfg = LayerConfig("e14", 1, 200, 128, 2, 2, 64, "bf16", "rmsnorm", True, False, False, 1e-5, 62, 0.02)
+    run = LayerRunner(cfg)
+    run.load_inputs(make_inputs(cfg))
+    run.forward()
+    selftest_wait_timeout(run.scratch_fwd.data_ptr(), 100_000, torch.cuda.current_stream().cuda_stream)
+    run.backward()
+    assert run.status() == 901
+    run.step()
+    assert run.status() == 0

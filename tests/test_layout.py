@@ -153,3 +153,28 @@ def test_padding_rule_and_sizes():
     assert plan.tensor_bytes(TENSOR["X"]) == 32 * 200 * 768 * 2
     saved, sf, sb = plan.workspace_bytes()
     assert saved > 0 and sf > 0 and sb > 0
+
+
+def test_partial_sum_area_covers_what_the_backward_kernels_write():
+    # The last area of the backward scratch takes the slab partials of the four bias column sums (one row of
+    # D + Dq + 2 Dkv floats per slab of 256 token rows), then, from the next 256-float boundary, the norm backward's
+    # per-block partial rows (dgamma and dbeta, at most two blocks per SM).  Recompute that requirement for large
+    # layers and compare with what the plan reserves; the area must also end inside the scratch size the plan reports.
+    from fbl_inputs import LayerConfig
+    from paper_2607_21624_b200 import WS
+    sms = 148
+    for (b, t, d, hq, hkv, hd, bias) in [(16, 8192, 4096, 32, 32, 128, True), (1, 8192, 4096, 32, 32, 128, False),
+                                         (64, 2048, 2048, 32, 8, 64, True), (32, 197, 768, 12, 12, 64, True),
+                                         (4, 512, 768, 12, 12, 64, True), (128, 1024, 1024, 16, 16, 64, True)]:
+        cfg = LayerConfig("big", b, t, d, hq, hkv, hd, "bf16", "layernorm", True, bias, False, 1e-5, 0, 0.02)
+        plan = Plan(desc_from_config(cfg))
+        n_pad = b * ((t + 7) // 8 * 8)
+        slabs = (n_pad + 255) // 256
+        cs_floats = slabs * (d + hq * hd + 2 * hkv * hd) if bias else 0
+        wpr = {1: 1, 2: 1, 3: 1, 4: 2, 6: 2, 8: 4, 12: 4, 16: 8}[d // 256]
+        blocks = min(2 * sms, n_pad // (8 // wpr))
+        need = ((cs_floats + 255) // 256 * 256 + blocks * 2 * d) * 4
+        off, nbytes = plan.workspace_offset(WS["PARTIALS"])
+        _, _, sb = plan.workspace_bytes()
+        assert nbytes >= need, (cfg, nbytes, need)
+        assert off + nbytes <= sb

@@ -51,3 +51,27 @@ def test_single_process_needs_no_process_group():
     assert rep.whole_job_rate(10.0, 1.0) == 10.0 / 1e-3
     rep.barrier()
     rep.close()
+
+
+def _self_spawned(path):
+    from paper_2607_21624_b200.replicas import Replicas
+    rep = Replicas(backend="gloo")
+    ms, = rep.max_over_ranks([10.0 * (rep.rank + 1)])
+    with open(f"{path}.{rep.rank}", "w") as f:
+        f.write(f"{rep.world} {rep.local_rank} {ms} {rep.whole_job_rate(7.0, ms)}")
+    rep.barrier()
+    rep.close()
+
+
+def test_replicas_started_without_a_launcher(tmp_path):
+    # `bench.py --gpus N` outside torchrun starts its own ranks through spawn_replicas; here with two gloo ranks
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT"):
+        os.environ.pop(k, None)
+    from paper_2607_21624_b200.replicas import spawn_replicas
+    base = str(tmp_path / "out")
+    spawn_replicas(2, _self_spawned, base)
+    for rank in range(2):
+        world, local_rank, ms, rate = open(f"{base}.{rank}").read().split()
+        assert int(world) == 2 and int(local_rank) == rank
+        assert float(ms) == 20.0 and float(rate) == 2 * 7.0 / 20.0e-3
+    assert "WORLD_SIZE" not in os.environ            # the parent's environment is left alone
