@@ -810,8 +810,6 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     auto drain_dq = [&](int dit) -> bool {
       const uint32_t stage = stage_addr(dit);
       if (!tc::mbar_wait(bar(BB_DQFULL), dit & 1, status, 307)) return false;
-      // the staging buffer's previous tile must have been read by its bulk reduction
-      if (dit >= (int)NS && !stage_is_alt(dit) && !tc::mbar_wait(bar(BB_STAGEFREE + (dit % NS)), (dit / (int)NS - 1) & 1, status, 310)) return false;
       tc::tc_fence_after();
       // this thread's HD / 4 accumulator columns in one go; the tensor pipe gets the columns back (at HD = 128 the
       // next tile's dP^T waits for them) as soon as they are in registers, before the stores to the staging tile
@@ -823,6 +821,9 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       tc::tmem_ld_wait();
       tc::tc_fence_before();
       tc::mbar_arrive(bar(BB_DQDRAINED));            // TMEM side done: the tensor pipe may reuse the columns
+      // Only now wait for the staging buffer (its previous tile must have been read by its bulk reduction, which
+      // takes a few thousand cycles): the values sit in registers meanwhile and the columns are already free.
+      if (dit >= (int)NS && !stage_is_alt(dit) && !tc::mbar_wait(bar(BB_STAGEFREE + (dit % NS)), (dit / (int)NS - 1) & 1, status, 310)) return false;
 #pragma unroll
       for (int u = 0; u < NC / 16; ++u) {            // 16 columns = half of a 128-byte unit of the box
         const int cu = c0 + u * 16;
