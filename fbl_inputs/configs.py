@@ -81,3 +81,47 @@ def get_config(i: int) -> LayerConfig:
 def scaled_config(cfg: LayerConfig, **kw) -> LayerConfig:
     """A copy of ``cfg`` with some fields replaced (smaller batch, other flags...)."""
     return replace(cfg, **kw)
+
+
+@dataclass(frozen=True)
+class MlpConfig:
+    """The feed-forward half of a transformer block on the same layout: pre-norm, up projection (with a gate
+    projection for the gated variant), activation, down projection, optional residual."""
+    name: str
+    batch: int
+    seq: int
+    d_model: int
+    d_ff: int
+    dtype: str          # "fp32" or "bf16"
+    norm: str           # "layernorm" or "rmsnorm"
+    act: str            # "gelu" (tanh form, one up projection) or "swiglu" (silu(gate) * up)
+    has_bias: bool
+    residual: bool
+    eps: float
+    seed: int
+    w_std: float
+
+    @property
+    def n_tokens(self) -> int:
+        return self.batch * self.seq
+
+    @property
+    def gated(self) -> bool:
+        return self.act == "swiglu"
+
+    def flops(self) -> float:
+        """Algorithmic forward+backward flops: each projection costs one product forward and two backward."""
+        n_proj = 3 if self.gated else 2
+        return 3.0 * n_proj * 2.0 * self.n_tokens * self.d_model * self.d_ff
+
+
+MLP_CONFIGS = {
+    # the paper's single-MatMul benchmark shapes (R-Tile ablation figure): forward (M=512, K=2048, N=8192) and the
+    # backward product dA = dO B^T (M=512, K=8192, N=2048) are the up projection of this block and its input gradient
+    "matmul-512x2048x8192": MlpConfig("mlp-matmul-512x2048x8192", 1, 512, 2048, 8192, "bf16", "layernorm", "gelu",
+                                      True, True, 1e-5, 11, 0.02),
+    # Llama-3.2-1B-shaped gated block (d_ff = 8192) behind the attention layer of workload 4
+    "llama1b": MlpConfig("mlp-llama1b-swiglu", 2, 2048, 2048, 8192, "bf16", "rmsnorm", "swiglu", False, True, 1e-5, 12, 0.02),
+    # GPT-2-small-shaped block (d_ff = 3072) behind the attention layer of workload 2
+    "gpt2": MlpConfig("mlp-gpt2-small-gelu", 4, 512, 768, 3072, "bf16", "layernorm", "gelu", True, True, 1e-5, 13, 0.02),
+}

@@ -14,6 +14,7 @@ from .configs import LayerConfig
 TENSOR_IDS = {
     "X": 0, "Wq": 1, "Wk": 2, "Wv": 3, "Wo": 4,
     "bq": 5, "bk": 6, "bv": 7, "bo": 8, "gamma": 9, "beta": 10, "dY": 11,
+    "W1": 12, "Wg": 13, "W2": 14, "b1": 15, "bg": 16, "b2": 17,
 }
 
 _M64 = np.uint64(0xFFFFFFFFFFFFFFFF)
@@ -99,4 +100,32 @@ def make_inputs(cfg: LayerConfig, *, affine_noise: bool = False) -> dict:
         out["bo"] = vec("bo", d, cfg.w_std)
     else:
         out["bq"] = out["bk"] = out["bv"] = out["bo"] = None
+    return out
+
+
+def make_mlp_inputs(cfg, *, affine_noise: bool = False) -> dict:
+    """All inputs of the feed-forward block ``cfg`` (an ``MlpConfig``) as float64 arrays of storage-rounded values:
+    X, dY ~ N(0, 1); W1, Wg [d_model, d_ff] and W2 [d_ff, d_model] ~ N(0, w_std^2); vectors are fp32."""
+    s = cfg.seed
+    d, f = cfg.d_model, cfg.d_ff
+
+    def mat(name, shape, std):
+        cnt = int(np.prod(shape))
+        return round_to_storage(normal_f64(s, TENSOR_IDS[name], 0, cnt).reshape(shape) * std, cfg.dtype)
+
+    def vec(name, length, std, mean=0.0):
+        return (normal_f64(s, TENSOR_IDS[name], 0, length) * std + mean).astype(np.float32).astype(np.float64)
+
+    out = {"X": mat("X", (cfg.batch, cfg.seq, d), 1.0), "dY": mat("dY", (cfg.batch, cfg.seq, d), 1.0),
+           "W1": mat("W1", (d, f), cfg.w_std), "W2": mat("W2", (f, d), cfg.w_std),
+           "Wg": mat("Wg", (d, f), cfg.w_std) if cfg.gated else None}
+    if affine_noise:
+        out["gamma"] = vec("gamma", d, 0.1, 1.0)
+        out["beta"] = vec("beta", d, 0.1) if cfg.norm == "layernorm" else None
+    else:
+        out["gamma"] = np.ones(d)
+        out["beta"] = np.zeros(d) if cfg.norm == "layernorm" else None
+    out["b1"] = vec("b1", f, cfg.w_std) if cfg.has_bias else None
+    out["bg"] = vec("bg", f, cfg.w_std) if cfg.has_bias and cfg.gated else None
+    out["b2"] = vec("b2", d, cfg.w_std) if cfg.has_bias else None
     return out
