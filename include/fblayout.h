@@ -168,6 +168,56 @@ int fbl_layer_bwd(const fbl_plan* plan, const void* dY, const void* X, const flo
                   float* dbq, float* dbk, float* dbv, float* dbo, float* dgamma, float* dbeta,
                   void* scratch, void* stream);
 
+/* ---------------------------------------------------------------------------------------------------------------
+ * The feed-forward half of the block on the same layout: pre-norm, up projection (plus a gate projection for the
+ * gated variant), activation, down projection, optional residual.  Its matmuls are the paper's reduce-axis-conflict
+ * operator (section 4.1: Y = X W reduces over d_in, dW = X^T dY over the tokens, dX = dY W^T over d_out) at the
+ * shapes of its single-MatMul benchmark (section 5.2, R-Tile ablation: forward (512, 2048, 8192), backward
+ * (512, 8192, 2048)); as in the attention layer every operand stays in R-Tile order in both passes and W^T, Xn^T,
+ * H^T are operand-orientation flags, never copies.
+ *   forward   Xn = norm(X); U = Xn W1 + b1; [G = Xn Wg + bg;]  H = gelu(U) | silu(G) * U;  Y = H W2 + b2 [+ X]
+ *   backward  dW2 = H^T dY, db2; dH = dY W2^T; dU = dH gelu'(U) | dU = dH silu(G), dG = dH U silu'(G);
+ *             dW1 = Xn^T dU, db1 [, dWg = Xn^T dG, dbg]; dXn = dU W1^T [+ dG Wg^T]; norm backward -> dX, dgamma, dbeta
+ * gelu is the tanh form u/2 (1 + tanh(sqrt(2/pi) (u + 0.044715 u^3))).  Conventions (pointers, alignment, padding,
+ * status word, return codes) are those of the attention layer's calls.  W1, Wg: [d_model, d_ff]; W2: [d_ff, d_model];
+ * b1, bg: [d_ff]; b2: [d_model].  Wg, bg, dWg, dbg are NULL for FBL_ACT_GELU; biases and their gradients NULL without
+ * has_bias; beta, dbeta NULL for RMSNorm. */
+enum { FBL_ACT_GELU = 0, FBL_ACT_SWIGLU = 1 };
+typedef struct {
+  int32_t batch, seq, d_model, d_ff;
+  int32_t dtype;        /* FBL_DTYPE_*  */
+  int32_t norm;         /* FBL_NORM_*   */
+  int32_t act;          /* FBL_ACT_*    */
+  int32_t has_bias;     /* 0 / 1 */
+  int32_t residual;     /* 0 / 1: Y = X + mlp(norm(X)) */
+  float eps;
+} fbl_mlp_desc;
+typedef struct fbl_mlp_plan fbl_mlp_plan;
+/* Matrix ids for fbl_mlp_tensor_bytes, fbl_mlp_pack and fbl_mlp_unpack. */
+enum { FBL_MT_X = 0 /* [B, T, d_model]: X, Y, dY, dX, Xn, dXn */, FBL_MT_H /* [B, T, d_ff]: U, G, H, dU, dG */,
+       FBL_MT_W1 /* [d_model, d_ff]: W1, Wg and gradients */, FBL_MT_W2 /* [d_ff, d_model] */, FBL_MT_COUNT };
+/* Offsets of the block's intermediates: STATS .. H inside `saved`, the others inside the backward scratch. */
+enum { FBL_MWS_STATS = 0, FBL_MWS_XN, FBL_MWS_U, FBL_MWS_G, FBL_MWS_H, FBL_MWS_DU, FBL_MWS_DG, FBL_MWS_DXN, FBL_MWS_COUNT };
+
+int fbl_mlp_plan_create(const fbl_mlp_desc* desc, fbl_mlp_plan** out);   /* d_model, d_ff multiples of tile_w */
+void fbl_mlp_plan_destroy(fbl_mlp_plan* plan);
+int fbl_mlp_tensor_bytes(const fbl_mlp_plan* plan, int matrix_id, size_t* bytes);
+int fbl_mlp_workspace_bytes(const fbl_mlp_plan* plan, size_t* saved, size_t* scratch_fwd, size_t* scratch_bwd);
+int fbl_mlp_workspace_offset(const fbl_mlp_plan* plan, int what, size_t* offset, size_t* bytes);
+int fbl_mlp_pack(const fbl_mlp_plan* plan, int matrix_id, const void* rowmajor_dev, void* tiled_dev, void* stream);
+int fbl_mlp_unpack(const fbl_mlp_plan* plan, int matrix_id, const void* tiled_dev, void* rowmajor_dev, void* stream);
+int fbl_mlp_fwd(const fbl_mlp_plan* plan, const void* X, const float* gamma, const float* beta,
+                const void* W1, const void* Wg, const void* W2, const float* b1, const float* bg, const float* b2,
+                void* Y, void* saved, void* scratch, void* stream);
+int fbl_mlp_bwd(const fbl_mlp_plan* plan, const void* dY, const void* X, const float* gamma,
+                const void* W1, const void* Wg, const void* W2, const void* saved,
+                void* dX, void* dW1, void* dWg, void* dW2, float* db1, float* dbg, float* db2,
+                float* dgamma, float* dbeta, void* scratch, void* stream);
+int fbl_mlp_status_poll(const fbl_mlp_plan* plan, const void* scratch, int32_t* device_status);
+/* 0 = default kernels (tcgen05 for bf16), 1 = FFMA kernels only, as fbl_plan_set_kernel_path. */
+int fbl_mlp_set_kernel_path(fbl_mlp_plan* plan, int path);
+int64_t fbl_mlp_launch_count(const fbl_mlp_plan* plan);
+
 /* Token-axis column reduction used for every bias gradient (db = sum over tokens, the matmul
  * backward's M-axis reduction of section 4.1): out[c] = sum_r M[r, c] for an R-Tile matrix of
  * `rows` x `cols` (rows a multiple of 8, cols of tile_w) in the plan's dtype.  Two stages over tiles:

@@ -7,5 +7,8 @@ CUDA device is absent, calls raise.
 from .binding import (FblError, Plan, lib, load_library, LayerRunner, DTYPES, TENSOR, MAP, WS,
                       desc_from_config, aligned_bytes, guard_bands_intact, selftest_wait_timeout)
 
-__all__ = ["FblError", "Plan", "lib", "load_library", "LayerRunner", "DTYPES", "TENSOR", "MAP", "WS",
+from .mlp import MlpPlan, MlpRunner, mlp_desc_from_config, MLP_TENSOR, MLP_WS
+
+__all__ = ["MlpPlan", "MlpRunner", "mlp_desc_from_config", "MLP_TENSOR", "MLP_WS",
+           "FblError", "Plan", "lib", "load_library", "LayerRunner", "DTYPES", "TENSOR", "MAP", "WS",
            "desc_from_config", "aligned_bytes", "guard_bands_intact", "selftest_wait_timeout"]

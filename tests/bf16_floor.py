@@ -111,3 +111,61 @@ def floor_figures(cfg, inp, ref=None):
                          viol=float((e > BF16_ATOL + BF16_RTOL * np.abs(r)).mean()),
                          numel=int(r.size))
     return fig
+
+
+def emulate_mlp(cfg, inp):
+    """The feed-forward block (oracle/mlp.py) with bf16-rounded intermediates (Xn, U, G, H, Y, dH-derived dU and
+    dG, dXn, dX, weight gradients) and exact sums."""
+    from oracle import mlp as om
+    X, dY = inp["X"], inp["dY"]
+    z = lambda b: b if b is not None else 0.0
+    B, T, D = X.shape
+    flat = lambda t: t.reshape(B * T, -1)
+    Xn_exact, xhat, rstd, mu = orc.norm_fwd(X, inp["gamma"], inp["beta"], cfg.eps, cfg.norm)
+    Xn = r16(Xn_exact)
+    U = r16(Xn @ inp["W1"] + z(inp["b1"]))
+    if cfg.gated:
+        G = r16(Xn @ inp["Wg"] + z(inp["bg"]))
+        H = r16(om.silu(G) * U)
+    else:
+        G = None
+        H = r16(om.gelu(U))
+    Y = H @ inp["W2"] + z(inp["b2"])
+    if cfg.residual:
+        Y = Y + X
+    out = {"Y": r16(Y), "dW2": r16(flat(H).T @ flat(dY)), "db2": flat(dY).sum(axis=0)}
+    dH = r16(dY @ inp["W2"].T)
+    if cfg.gated:
+        dU, dG = r16(dH * om.silu(G)), r16(dH * U * om.silu_grad(G))
+        out["dWg"], out["dbg"] = r16(flat(Xn).T @ flat(dG)), flat(dG).sum(axis=0)
+        dXn = r16(dU @ inp["W1"].T + dG @ inp["Wg"].T)
+    else:
+        dU = r16(dH * om.gelu_grad(U))
+        dXn = r16(dU @ inp["W1"].T)
+    out["dW1"], out["db1"] = r16(flat(Xn).T @ flat(dU)), flat(dU).sum(axis=0)
+    out["dgamma"] = flat(dXn * xhat).sum(axis=0)
+    if cfg.norm == "layernorm":
+        out["dbeta"] = flat(dXn).sum(axis=0)
+    gg = dXn * inp["gamma"]
+    c2 = (gg * xhat).mean(axis=-1, keepdims=True)
+    dX = rstd * (gg - (gg.mean(axis=-1, keepdims=True) if cfg.norm == "layernorm" else 0.0) - xhat * c2)
+    if cfg.residual:
+        dX = dX + dY
+    out["dX"] = r16(dX)
+    return out
+
+
+def floor_figures_mlp(cfg, inp, ref):
+    """As floor_figures, for the feed-forward block; ``ref``: the oracle's outputs by name."""
+    fig = {}
+    for name, got in emulate_mlp(cfg, inp).items():
+        if not cfg.has_bias and name in ("db1", "dbg", "db2"):
+            continue
+        r = ref[name]
+        e = np.abs(got - r)
+        fig[name] = dict(max_abs=float(e.max()),
+                         worst_over_bound=float(e.max() / (BF16_ATOL + BF16_RTOL * np.abs(r).max())),
+                         fro=float(np.linalg.norm(got - r) / (np.linalg.norm(r) + 1e-300)),
+                         viol=float((e > BF16_ATOL + BF16_RTOL * np.abs(r)).mean()),
+                         numel=int(r.size))
+    return fig
