@@ -468,6 +468,69 @@ def measure(cfg, args, rep, local_rank, flush_l2, want_cpu):
     }
 
 
+def measure_mlp(key, args, rep, local_rank, flush_l2):
+    """The feed-forward block `key` of fbl_inputs.MLP_CONFIGS on this rank's GPU: forward + backward, cold L2, graph replay."""
+    import torch
+    from fbl_inputs import MLP_CONFIGS, make_mlp_inputs
+    from paper_2607_21624_b200 import MlpRunner
+    cfg = MLP_CONFIGS[key]
+    run = MlpRunner(cfg, device=f"cuda:{local_rank}")
+    run.plan.set_kernel_path(args.path)
+    run.load_inputs(make_mlp_inputs(cfg))
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        run.step()
+        stream.synchronize()
+        assert run.status() == 0
+        l0 = run.plan.launch_count()
+        run.step()
+        launches = run.plan.launch_count() - l0
+        graph = g_fwd = None
+        if not args.no_graph:
+            graph, g_fwd = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                run.step()
+            with torch.cuda.graph(g_fwd, stream=stream):
+                run.forward()
+    step = graph.replay if graph is not None else run.step
+    fwd = g_fwd.replay if g_fwd is not None else run.forward
+
+    def timed(fn, n):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        with torch.cuda.stream(stream):
+            for _ in range(args.warmup):
+                flush_l2()
+                fn()
+            for a, b in ev:
+                flush_l2()
+                a.record(stream)
+                fn()
+                b.record(stream)
+        torch.cuda.synchronize()
+        rep.barrier()
+        t = [a.elapsed_time(b) for a, b in ev]
+        return sum(t) / len(t)
+
+    ms = timed(step, args.steps)
+    ms_fwd = timed(fwd, max(3, min(args.steps, 30)))
+    assert run.status() == 0
+    ms, ms_fwd = rep.max_over_ranks([ms, ms_fwd])
+    sizes = dict(run.sizes)
+    del run, graph, g_fwd
+    torch.cuda.empty_cache()
+    if rep.rank != 0:
+        return None
+    peaks = measured_peaks()
+    flops = cfg.flops()
+    return {"workload": (f"{cfg.name}: B={cfg.batch} T={cfg.seq} D={cfg.d_model} F={cfg.d_ff} {cfg.act} {cfg.norm} {cfg.dtype}"),
+            "ms_per_step": ms, "ms_fwd": ms_fwd, "tflops": rep.whole_job_rate(flops, ms) / 1e12,
+            "tokens_per_s": rep.whole_job_rate(cfg.n_tokens, ms), "flops_per_step": flops, "dtype": "bf16",
+            "layer_roofline": {"binds": "tensor", "frac_of_measured_burst": flops / (peaks["tflops_burst"] * 1e12) / (ms * 1e-3),
+                               "frac_of_nominal_2250": flops / (NOMINAL_TFLOPS * 1e12) / (ms * 1e-3)},
+            "activation_bytes": {"saved": sizes["saved"], "scratch": sizes["scratch_fwd"] + sizes["scratch_bwd"]},
+            "launches_per_step": launches}
+
+
 def run_rank(args):
     """Body of one rank (the only one at N = 1)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -510,6 +573,10 @@ def run_rank(args):
     for i in todo:
         cfg = pick(i)
         results[i] = measure(cfg, args, rep, local_rank, flush_l2, want_cpu=(i == head and not args.no_cpu_baseline))
+    mlp = {}
+    if not args.config and not args.no_mlp:          # the feed-forward blocks behind these attention layers
+        for key in ("matmul-512x2048x8192", "gpt2", "llama1b"):
+            mlp[key] = measure_mlp(key, args, rep, local_rank, flush_l2)
     if rank != 0:
         rep.close()
         return
@@ -527,10 +594,11 @@ def run_rank(args):
                    "also_timed": "per_config holds all five workloads, each timed the same way in this process"},
         "tokens_per_s": h["tokens_per_s"], "layer_roofline": h["layer_roofline"], "mem_efficiency": h["mem_efficiency"],
         "activation_bytes": h["activation_bytes"], "e2e": h["e2e"],
-        "gpu_launches": sum(r["launches_per_step"] for r in results.values()) * args.steps,
+        "gpu_launches": (sum(r["launches_per_step"] for r in results.values())
+                         + sum(r["launches_per_step"] for r in mlp.values())) * args.steps,
         "clocks": h["clocks"], "roofline": h["roofline"], "cpu_baseline": h["cpu_baseline"],
         "peaks": peaks,
-        "per_config": {f"workload{i}": results[i] for i in sorted(results)},
+        "per_config": {**{f"workload{i}": results[i] for i in sorted(results)}, **{f"mlp_{k}": v for k, v in mlp.items()}},
     }
     print(json.dumps(line))
     rep.close()
@@ -546,6 +614,7 @@ def main():
     ap.add_argument("--path", type=int, default=0, help="0 default kernels, 1 FFMA kernels only")
     ap.add_argument("--no-graph", action="store_true", help="enqueue kernels directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-mlp", action="store_true", help="skip the feed-forward blocks' entries of per_config")
     ap.add_argument("--flush-write-only", action="store_true", help="flush L2 by the 256 MiB write alone (its write-back then overlaps the step)")
     ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling captures)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures)")
