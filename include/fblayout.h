@@ -259,6 +259,33 @@ int fbl_status_poll(const fbl_plan* plan, const void* scratch, int32_t* device_s
  * normal end). */
 int fbl_selftest_wait_timeout(void* scratch, int64_t limit_cycles, void* stream);
 
+/* ---------------------------------------------------------------------------------------------------------------
+ * Offline tile selection (section 4.2, step 1 and Eq. 1, Eq. 2; Supplement Algorithm 1), restated for this GPU.
+ *
+ * fbl_rtile_candidates: storage-tile shape candidates for a set of matrices.  The initial pool is every
+ * (tile_h, tile_w) with tile_h in {1, 2, 4, 8, 16, 32, 64, 128} rows and tile_w * elem_bytes in {32, 64, 128, 256,
+ * 512} bytes; it is filtered by the three constraints in the paper's order and each survivor gets its N_cache of
+ * Eq. 1 (with the 1 x 128-byte line of this memory system as the cache tile) and its worst padding ratio:
+ *   C1 computation: a tile row must be exactly the 128-byte span of the tensor cores' swizzled shared-memory operand
+ *      rows, and tile_h a multiple of the 8-row swizzle atom that still divides the 128-row compute tile (so that
+ *      any run of tiles is a legal K-major or MN-major operand: the tile-invariance property);
+ *   C2 memory: a tile is at most one 4 KiB bulk-copy box row group and starts on a 128-byte line (whole lines);
+ *   C3 shape: the padded size of every matrix exceeds its size by at most `max_pad_ratio` (the paper uses 0.10).
+ * `shapes` holds n_shapes pairs (rows, cols).  Survivors are written to `out` (at most max_out), ordered by
+ * ascending N_cache, then ascending padding; the return value is their count (or a negative fbl_status).
+ * reject_counts[0..2], if not NULL, receive how many pool entries C1, C2 and C3 removed. */
+typedef struct { int32_t tile_h, tile_w, n_cache; float pad_ratio; } fbl_rtile_cand;
+int fbl_rtile_candidates(const int64_t* shapes, int n_shapes, int elem_bytes, float max_pad_ratio,
+                         fbl_rtile_cand* out, int max_out, int32_t reject_counts[3]);
+
+/* The compute-tile configuration of one GEMM launch of the step, as chosen offline (the profiling step of
+ * section 4.2 / 6 and the argmax of Eq. 2 live in the Python module rtile.py, which times the candidates through
+ * these calls): output-tile width 128 or 256 (0: built-in heuristic), CTA-pair kernel 0 / 1 (-1: heuristic),
+ * epilogue warp sets 1 / 2 (0: heuristic).  A choice whose tile shape is not legal for the launch's shapes falls
+ * back to the heuristic.  Takes effect for later fbl_layer_fwd / fbl_layer_bwd calls on this plan. */
+enum { FBL_GEMM_PROJ_QKV = 0, FBL_GEMM_PROJ_O, FBL_GEMM_DWO_DA, FBL_GEMM_DWQKV_DXN, FBL_GEMM_LAUNCH_COUNT };
+int fbl_plan_set_gemm_choice(fbl_plan* plan, int launch_id, int tile_n, int cta_pair, int epilogue_sets);
+
 /* Kernel family used by later calls on this plan: 0 = default (tcgen05 tensor-core kernels for bf16
  * wherever one exists for the shape, FFMA kernels for fp32), 1 = FFMA kernels only (fp32 arithmetic on
  * the same layout; lets a caller cross-check the tensor-core path on the device). */

@@ -225,8 +225,11 @@ class LayerRunner:
     MATS = {"X": "X", "dY": "DY", "Wq": "WQ", "Wk": "WK", "Wv": "WV", "Wo": "WO"}
     OUT_MATS = {"Y": "Y", "dX": "DX", "dWq": "WQ", "dWk": "WK", "dWv": "WV", "dWo": "WO"}
 
-    def __init__(self, cfg, device="cuda:0", guard_bytes=0):
-        """``guard_bytes`` > 0 surrounds every device buffer with bands of a known byte pattern
+    def __init__(self, cfg, device="cuda:0", guard_bytes=0, tile_choices=None):
+        """``tile_choices``: the GEMM launches' compute-tile configurations ({launch name: [tile_n, cta_pair,
+        epilogue_sets]}, see rtile.py); None takes the layer's entry of the offline table shipped with the package,
+        if it has one, {} leaves every launch to the built-in heuristics.
+        ``guard_bytes`` > 0 surrounds every device buffer with bands of a known byte pattern
         (``guards_intact`` checks them): a stand-in for a memory checker when hunting writes past a buffer."""
         import torch
         if not torch.cuda.is_available():
@@ -235,6 +238,12 @@ class LayerRunner:
         self.cfg = cfg
         self.dev = torch.device(device)
         self.plan = Plan(desc_from_config(cfg))
+        from . import rtile
+        if tile_choices is None:
+            tile_choices = rtile.load_table().get(rtile.shape_key(cfg), {}).get("choices", {})
+        self.tile_choices = tile_choices
+        if tile_choices:
+            rtile.apply(self.plan, tile_choices)
         self.tdtype = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
         saved, sf, sb = self.plan.workspace_bytes()
         self.sizes = dict(saved=saved, scratch_fwd=sf, scratch_bwd=sb)

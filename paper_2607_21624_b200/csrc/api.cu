@@ -65,8 +65,8 @@ thread_local char g_detail[256] = "";
     if (mp__->prof_on) { mp__->prof_n = 0; FBL_CUDA(cudaEventRecord(mp__->prof_ev[0], st)); } \
   } while (0)
 
-cudaError_t run_gemm(const fbl_plan* p, const GemmArgs& g, int32_t* status, cudaStream_t st) {
-  if (p->use_tc && gemm_tc_supported(p, g)) return launch_gemm_tc_group(p, &g, 1, status, st);
+cudaError_t run_gemm(const fbl_plan* p, const GemmArgs& g, int32_t* status, cudaStream_t st, int launch_id = -1) {
+  if (p->use_tc && gemm_tc_supported(p, g)) return launch_gemm_tc_group(p, &g, 1, status, st, launch_id);
   return launch_gemm_simt(p->d.dtype, g, st);
 }
 
@@ -126,6 +126,7 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   p->knob_gemm_pair = env_int("FBL_GEMM_PAIR", -1);
   p->knob_gemm_esets = env_int("FBL_GEMM_ESETS", 0);
   p->knob_fwd_tiles = env_int("FBL_FWD_TILES", 0);
+  for (int i = 0; i < FBL_GEMM_LAUNCH_COUNT; ++i) p->choice[i] = {0, -1, 0};
   p->use_tc = d.dtype == FBL_DTYPE_BF16 ? 1 : 0;
 
   const size_t n = (size_t)p->n_pad;
@@ -216,6 +217,14 @@ int fbl_profile_read(const fbl_plan* plan, int max_steps, const char** names, fl
 }
 
 int64_t fbl_launch_count(const fbl_plan* plan) { return plan ? plan->launches : -1; }
+
+int fbl_plan_set_gemm_choice(fbl_plan* plan, int launch_id, int tile_n, int cta_pair, int epilogue_sets) {
+  if (!plan || launch_id < 0 || launch_id >= FBL_GEMM_LAUNCH_COUNT) return FBL_ERR_INVALID_ARG;
+  if ((tile_n != 0 && tile_n != 128 && tile_n != 256) || cta_pair < -1 || cta_pair > 1 || epilogue_sets < 0 || epilogue_sets > 2)
+    return FBL_ERR_INVALID_ARG;
+  plan->choice[launch_id] = {tile_n, cta_pair, epilogue_sets};
+  return FBL_OK;
+}
 
 int fbl_plan_set_kernel_path(fbl_plan* plan, int path) {
   if (!plan || (path != 0 && path != 1)) return FBL_ERR_INVALID_ARG;
@@ -395,7 +404,7 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
       tc = tc && gemm_tc_supported(p, g);
     }
     if (tc) {
-      FBL_STEP("proj_qkv", 1, launch_gemm_tc_group(p, gs, 3, status, st));   // one launch, blockIdx.z picks Q, K or V
+      FBL_STEP("proj_qkv", 1, launch_gemm_tc_group(p, gs, 3, status, st, FBL_GEMM_PROJ_QKV));   // one launch, blockIdx.z picks Q, K or V
     } else {
       for (int i = 0; i < 3; ++i)
         FBL_STEP(i == 0 ? "proj_q" : i == 1 ? "proj_k" : "proj_v", 1, launch_gemm_simt(p->d.dtype, gs[i], st));
@@ -411,7 +420,7 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
     g.c = Y; g.c_rpad = p->n_pad; g.bias = bias ? bo : nullptr;
     g.residual = p->d.residual ? X : nullptr;
     g.seq = p->d.seq; g.t_pad = p->t_pad;
-    FBL_STEP("proj_o", 1, run_gemm(p, g, status, st));
+    FBL_STEP("proj_o", 1, run_gemm(p, g, status, st, FBL_GEMM_PROJ_O));
   }
   return FBL_OK;
 }
@@ -483,7 +492,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
         gs[0].zero_ptr = dqacc; gs[0].zero_bytes = p->zero_bytes - p->sb_dqacc;
         gs[0].reset_status = 1; gs[0].serial = 1;
       }
-      FBL_STEP("dWo+dA", 1, launch_gemm_tc_group(p, gs, 2, status, st));
+      FBL_STEP("dWo+dA", 1, launch_gemm_tc_group(p, gs, 2, status, st, FBL_GEMM_DWO_DA));
       dwo_round = split_o;        // nothing in the step reads dWo: its rounding joins that of dWq, dWk, dWv below
     } else {
       FBL_STEP("dA", 1, run_gemm(p, ga, status, st));
@@ -531,7 +540,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
         cg.count++;
         dwo_round = false;
       }
-      FBL_STEP("dWqkv+dXn", 1, launch_gemm_tc_group(p, gs, 4, status, st));
+      FBL_STEP("dWqkv+dXn", 1, launch_gemm_tc_group(p, gs, 4, status, st, FBL_GEMM_DWQKV_DXN));
       if (cg.count > 0) FBL_STEP("dW round", 1, launch_convert_f32_group(cg, st));     // one rounding launch for all sliced GEMMs
     } else {
       FBL_STEP("dXn", 1, run_gemm(p, gx, status, st));

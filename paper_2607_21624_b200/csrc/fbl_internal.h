@@ -55,6 +55,9 @@ struct fbl_plan {
   int knob_gemm_pair;       // -1 by size, 0 never the CTA-pair GEMM kernel, 1 wherever its tile shape is legal
   int knob_gemm_esets;      // 0 by tiles per block, 1 / 2 sets of epilogue warps
   int knob_fwd_tiles;       // 0 by sequence length, 1 / 2 query tiles per forward-attention block at head_dim 64
+  // Compute-tile configuration of each GEMM launch of a step, fixed offline by the tile chooser (0 / -1: the
+  // built-in heuristics decide): output-tile width, CTA-pair kernel, sets of epilogue warps.
+  struct GemmChoice { int bn, pair, esets; } choice[FBL_GEMM_LAUNCH_COUNT];
   // bookkeeping of the enqueue calls (they take the plan as const): kernels enqueued so far, optional per-step
   // event timing.  Calls on one plan are not thread-safe; give each host thread its own plan.
   mutable int64_t launches;
@@ -94,7 +97,8 @@ struct GemmArgs {
 
 cudaError_t launch_gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);
 bool gemm_tc_supported(const fbl_plan* p, const GemmArgs& g);
-cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st);
+cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st,
+                                 int launch_id = -1);
 struct GemmShape { int64_t m; int n; int kblocks; int splittable; };
 int gemm_tc_choose_split(int sm_count, const GemmShape* sh, int count);
 cudaError_t launch_wait_timeout_selftest(int32_t* status, long long limit_cycles, cudaStream_t st);

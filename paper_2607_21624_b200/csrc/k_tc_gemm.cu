@@ -779,7 +779,7 @@ cudaError_t fill_group(TcGroup& G, const GemmArgs* gs, int count, int32_t* statu
 }
 
 template <int BN, int STAGES>
-cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
+cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st, int esets_choice) {
   TcGroup G;
   int tiles = 0;
   cudaError_t e = fill_group(G, gs, count, status, BN, BM, BN, &tiles);
@@ -788,7 +788,8 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
   const int grid = tiles < p->sm_count ? tiles : p->sm_count;
   // one tile per block at most: the epilogue is exposed, and the variant with two sets of epilogue warps halves it
   // (with several tiles per block the epilogues overlap the next main loops and the extra warps only cost)
-  const bool two_sets = p->knob_gemm_esets ? p->knob_gemm_esets == 2 : tiles <= p->sm_count;
+  const int esets_knob = esets_choice ? esets_choice : p->knob_gemm_esets;
+  const bool two_sets = esets_knob ? esets_knob == 2 : tiles <= p->sm_count;
   if (two_sets) {
     auto k = gemm_tc_kernel<BN, STAGES, 2>;
     cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
@@ -817,8 +818,11 @@ cudaError_t launch_group_pair(const fbl_plan* p, const GemmArgs* gs, int count, 
                       : launch_pdl(k, dim3(2 * pairs), dim3(192), SP::TOTAL, st, G);
 }
 
-cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st) {
+cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int count, int32_t* status, cudaStream_t st,
+                                 int launch_id) {
   if (count < 1 || count > MAX_PROBLEMS) return cudaErrorInvalidValue;
+  fbl_plan::GemmChoice ch = {0, -1, 0};
+  if (launch_id >= 0 && launch_id < FBL_GEMM_LAUNCH_COUNT) ch = p->choice[launch_id];
   bool wide = true;                       // 128 x 256 tiles when every problem's N is whole 256-column blocks
   int tiles_wide = 0;
   for (int i = 0; i < count; ++i) {
@@ -832,7 +836,10 @@ cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int coun
   if (wide && tiles_wide * 3 < p->sm_count * 2) wide = false;
   // CTA pairs on 256 x 256 tiles for large problems (several rounds of tiles per SM pair): measured 2-6 % faster
   // on the workload 5 GEMMs, no gain or a loss below that
-  const int pair_mode = p->knob_gemm_pair;       // tuning knob: 0 never, 1 whenever legal, -1 by size
+  // an offline choice for this launch overrides the heuristics below wherever its tile shape is legal
+  if (ch.bn == 128) wide = false;
+  else if (ch.bn == 256 && wide_legal) wide = true;
+  const int pair_mode = ch.pair >= 0 ? ch.pair : p->knob_gemm_pair;       // 0 never, 1 whenever legal, -1 by size
   if (pair_mode == 1 && wide_legal) return launch_group_pair(p, gs, count, status, st);
   if (wide && pair_mode != 0) {
     long long pair_tiles = 0;
@@ -840,8 +847,8 @@ cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int coun
       pair_tiles += (long long)((gs[i].m + 255) / 256) * (gs[i].n / 256) * (gs[i].ksplit > 1 ? gs[i].ksplit : 1);
     if (pair_tiles >= 4 * (p->sm_count / 2)) return launch_group_pair(p, gs, count, status, st);
   }
-  if (wide) return launch_group_bn<256, 4>(p, gs, count, status, st);
-  return launch_group_bn<128, 6>(p, gs, count, status, st);
+  if (wide) return launch_group_bn<256, 4>(p, gs, count, status, st, ch.esets);
+  return launch_group_bn<128, 6>(p, gs, count, status, st, ch.esets);
 }
 
 // How many slices to cut the reduction loops of the splittable problems of a group into (the same number for all

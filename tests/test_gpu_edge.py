@@ -178,3 +178,28 @@ def test_forward_timeout_code_survives_the_backward():
     assert run.status() == 901
     run.step()
     assert run.status() == 0
+
+
+def test_offline_tile_choices_sweep_and_apply():
+    # The profiling step of the tile chooser on a small layer: every GEMM launch is timed under every configuration
+    # (tile width 128 / 256, CTA pair, one or two sets of epilogue warps), Eq. 2 picks one per launch, and a step
+    # under the picked table, and under each forced configuration, still matches the oracle.
+    from paper_2607_21624_b200 import rtile
+    cfg = LayerConfig("t1", 3, 333, 512, 8, 4, 64, "bf16", "layernorm", True, True, True, 1e-5, 63, 0.02)
+    res = rtile.sweep(cfg, reps=2)[(0, 0)]
+    picked, detail = rtile.choose(cfg, res)
+    assert set(picked) == set(rtile.LAUNCHES)
+    for name in rtile.LAUNCHES:
+        assert len(res[name]) == len(rtile.legal_choices(cfg)) and all(ms > 0 for ms in res[name].values())
+    import paper_2607_21624_b200.binding as binding
+    for table in [picked] + [{n: list(c) for n in rtile.LAUNCHES} for c in rtile.legal_choices(cfg)]:
+        orig = binding.LayerRunner.__init__
+
+        def patched(self, cfg_, device="cuda:0", guard_bytes=0, tile_choices=None, _t=table):
+            orig(self, cfg_, device=device, guard_bytes=guard_bytes, tile_choices=_t)
+        binding.LayerRunner.__init__ = patched
+        try:
+            run = run_and_compare(cfg, affine_noise=True, intermediates=False)
+            assert run.tile_choices == table
+        finally:
+            binding.LayerRunner.__init__ = orig
