@@ -286,6 +286,43 @@ int fbl_rtile_candidates(const int64_t* shapes, int n_shapes, int elem_bytes, fl
 enum { FBL_GEMM_PROJ_QKV = 0, FBL_GEMM_PROJ_O, FBL_GEMM_DWO_DA, FBL_GEMM_DWQKV_DXN, FBL_GEMM_LAUNCH_COUNT };
 int fbl_plan_set_gemm_choice(fbl_plan* plan, int launch_id, int tile_n, int cta_pair, int epilogue_sets);
 
+/* ---------------------------------------------------------------------------------------------------------------
+ * Tile propagation and index-transformation elimination for an arbitrary chain of reshape / permute operators
+ * (section 4.3: the three dependency checks, Eq. 3 T_dst[i] = f(T_src[j]), Eq. 4 f = f_n o ... o f_1 and the strength
+ * reduction of the composed index function).  Pure host integer code.
+ *
+ * A tensor of logical shape `shape` (rank <= 8, row-major) is stored as the R-Tile matrix [prod(shape[:-1]), shape[-1]]
+ * with tile_h x tile_w tiles.  After the chain the result, of whatever rank, is stored the same way with the same
+ * tile shape.  If the chain only moves whole tiles, fbl_tile_chain_create builds the composed tile map f (source tile
+ * number -> destination tile number, both row-major over their tile grids) as a short list of terms
+ *     f(j) = sum_k ((j / div_k) % mod_k) * mul_k           (mod_k = 0: no modulo, the outermost digit)
+ * in which digits that stay adjacent have been merged (the rule (i mod Ca) mod Cb = i mod Cb for Cb | Ca applied to
+ * the whole chain), and returns FBL_OK.  Otherwise it returns FBL_ERR_UNSUPPORTED_SHAPE and reports the first
+ * operator that breaks the tile structure and which check it fails:
+ *   FBL_TP_DIMENSION   the axes a tile spans do not end up as the destination's tile axes (the chain moves the tile's
+ *                      row or column axis elsewhere, e.g. a transpose of the last two axes, or changes the element
+ *                      count: an expand / repeat, where the paper too falls back);
+ *   FBL_TP_BOUNDARY    a reshape cuts inside a tile: the split (or merged) extent is not a whole number of tiles
+ *                      (hidden 768 -> 16 x 48 with tile_w 64), or the innermost row extent is not a multiple of tile_h;
+ *   FBL_TP_CONTINUITY  the elements of a tile row (or the rows of a tile) lose their stride-1 order.
+ * Sizes must already include padding (a 197-token sequence is passed as 200 for tile_h = 8). */
+enum { FBL_VIEW_RESHAPE = 0, FBL_VIEW_PERMUTE = 1, FBL_VIEW_EXPAND = 2 };
+enum { FBL_TP_OK = 0, FBL_TP_DIMENSION = 1, FBL_TP_BOUNDARY = 2, FBL_TP_CONTINUITY = 3 };
+typedef struct {
+  int32_t kind;        /* FBL_VIEW_*                                                              */
+  int32_t rank;        /* rank of the result                                                      */
+  int64_t shape[8];    /* RESHAPE / EXPAND: the new shape                                          */
+  int32_t perm[8];     /* PERMUTE: result axis k is input axis perm[k]                            */
+} fbl_view_op;
+typedef struct { int64_t div, mod, mul; } fbl_tile_term;
+typedef struct fbl_tile_chain fbl_tile_chain;
+int fbl_tile_chain_create(const int64_t* shape, int rank, int tile_h, int tile_w, const fbl_view_op* ops, int n_ops,
+                          fbl_tile_chain** out, int32_t* failed_op, int32_t* failed_check);
+void fbl_tile_chain_destroy(fbl_tile_chain* chain);
+int64_t fbl_tile_chain_tiles(const fbl_tile_chain* chain);                       /* tiles of the tensor */
+int fbl_tile_chain_terms(const fbl_tile_chain* chain, fbl_tile_term* terms, int max_terms);   /* returns the count */
+int fbl_tile_chain_map(const fbl_tile_chain* chain, int64_t src_tile, int64_t* dst_tile);     /* evaluates f */
+
 /* Kernel family used by later calls on this plan: 0 = default (tcgen05 tensor-core kernels for bf16
  * wherever one exists for the shape, FFMA kernels for fp32), 1 = FFMA kernels only (fp32 arithmetic on
  * the same layout; lets a caller cross-check the tensor-core path on the device). */
