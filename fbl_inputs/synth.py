@@ -15,6 +15,7 @@ TENSOR_IDS = {
     "X": 0, "Wq": 1, "Wk": 2, "Wv": 3, "Wo": 4,
     "bq": 5, "bk": 6, "bv": 7, "bo": 8, "gamma": 9, "beta": 10, "dY": 11,
     "W1": 12, "Wg": 13, "W2": 14, "b1": 15, "bg": 16, "b2": 17,
+    "Aq": 18, "Ak": 19, "Av": 20, "Bq": 21, "Bk": 22, "Bv": 23,
 }
 
 _M64 = np.uint64(0xFFFFFFFFFFFFFFFF)
@@ -128,4 +129,17 @@ def make_mlp_inputs(cfg, *, affine_noise: bool = False) -> dict:
     out["b1"] = vec("b1", f, cfg.w_std) if cfg.has_bias else None
     out["bg"] = vec("bg", f, cfg.w_std) if cfg.has_bias and cfg.gated else None
     out["b2"] = vec("b2", d, cfg.w_std) if cfg.has_bias else None
+    return out
+
+
+def make_lora_inputs(cfg: LayerConfig, rank: int, *, affine_noise: bool = False, a_std: float = 0.05, b_std: float = 0.05) -> dict:
+    """The layer's inputs plus rank-``rank`` adapters Aq, Ak, Av ~ N(0, a_std^2) [d_model, rank] and Bq, Bk, Bv ~
+    N(0, b_std^2) [rank, d_q | d_kv], rounded to the storage dtype.  (Fine-tuning starts from B = 0; a non-zero B
+    is drawn so that every gradient path carries signal.)"""
+    out = make_inputs(cfg, affine_noise=affine_noise)
+    for k, cols in (("q", cfg.d_q), ("k", cfg.d_kv), ("v", cfg.d_kv)):
+        a = normal_f64(cfg.seed, TENSOR_IDS["A" + k], 0, cfg.d_model * rank).reshape(cfg.d_model, rank) * a_std
+        b = normal_f64(cfg.seed, TENSOR_IDS["B" + k], 0, rank * cols).reshape(rank, cols) * b_std
+        out["A" + k] = round_to_storage(a, cfg.dtype)
+        out["B" + k] = round_to_storage(b, cfg.dtype)
     return out
