@@ -218,6 +218,39 @@ int fbl_mlp_status_poll(const fbl_mlp_plan* plan, const void* scratch, int32_t* 
 int fbl_mlp_set_kernel_path(fbl_mlp_plan* plan, int path);
 int64_t fbl_mlp_launch_count(const fbl_mlp_plan* plan);
 
+/* ---------------------------------------------------------------------------------------------------------------
+ * Low-rank adapters on the Q, K and V projections with the base weights frozen: the paper's fine-tuning setting
+ * (section 2, motivating example X A_LoRA B_LoRA; section 5.1).  Q = Xn Wq + bq + (Xn Aq) Bq, likewise K and V; only
+ * the adapters and the layer input receive gradients, so the weight-gradient products of the frozen projections
+ * (and their token-axis reductions) are skipped, and the adapters add thin products whose reduction axes are the
+ * rank (forward, dT B^T) and the tokens (dA = Xn^T dT, dB = T^T d*).  A scale alpha / r is folded into B by the
+ * caller.
+ *
+ * Storage.  The three adapters live in two R-Tile matrices with each adapter's rank padded to one 64-wide block
+ * (FBL_LORA_BLOCK) of zeros, so that every product is whole tiles:
+ *   A_all [d_model, 192]              column block i (i = 0 q, 1 k, 2 v) holds A_i in its first `rank` columns;
+ *   B_all [192, d_q + 2 d_kv]         block-diagonal: rows 64 i .. 64 i + rank of column block i hold B_i, the rest 0.
+ * fbl_lora_pack / fbl_lora_unpack convert one adapter matrix (row-major [d_model, rank] or [rank, d_out]) to and from
+ * its block; the caller zero-fills A_all and B_all once before packing.  dA_all and dB_all come back in the same
+ * shapes; off-diagonal blocks of dB_all are not gradients of anything and must be ignored (fbl_lora_unpack does).
+ *
+ * fbl_plan_enable_lora must precede fbl_workspace_bytes (the work areas grow by T = Xn A_all and dT).  rank 1..64.
+ * Biases, if the plan has them, are applied but frozen; dgamma / dbeta may be NULL (frozen norm). */
+enum { FBL_LORA_BLOCK = 64 };
+enum { FBL_LORA_AQ = 0, FBL_LORA_AK, FBL_LORA_AV, FBL_LORA_BQ, FBL_LORA_BK, FBL_LORA_BV };
+int fbl_plan_enable_lora(fbl_plan* plan, int rank);
+int fbl_lora_bytes(const fbl_plan* plan, size_t* a_all_bytes, size_t* b_all_bytes);
+int fbl_lora_pack(const fbl_plan* plan, int which, const void* rowmajor_dev, void* all_dev, void* stream);
+int fbl_lora_unpack(const fbl_plan* plan, int which, const void* all_dev, void* rowmajor_dev, void* stream);
+int fbl_layer_fwd_lora(const fbl_plan* plan, const void* X, const float* gamma, const float* beta,
+                       const void* Wq, const void* Wk, const void* Wv, const void* Wo,
+                       const float* bq, const float* bk, const float* bv, const float* bo,
+                       const void* A_all, const void* B_all, void* Y, void* saved, void* scratch, void* stream);
+int fbl_layer_bwd_lora(const fbl_plan* plan, const void* dY, const void* X, const float* gamma,
+                       const void* Wq, const void* Wk, const void* Wv, const void* Wo,
+                       const void* A_all, const void* B_all, const void* saved,
+                       void* dX, void* dA_all, void* dB_all, float* dgamma, float* dbeta, void* scratch, void* stream);
+
 /* Token-axis column reduction used for every bias gradient (db = sum over tokens, the matmul
  * backward's M-axis reduction of section 4.1): out[c] = sum_r M[r, c] for an R-Tile matrix of
  * `rows` x `cols` (rows a multiple of 8, cols of tile_w) in the plan's dtype.  Two stages over tiles:

@@ -7,8 +7,9 @@ CUDA device is absent, calls raise.
 from .binding import (FblError, Plan, lib, load_library, LayerRunner, DTYPES, TENSOR, MAP, WS,
                       desc_from_config, aligned_bytes, guard_bands_intact, selftest_wait_timeout)
 
+from .lora import LoraRunner
 from .mlp import MlpPlan, MlpRunner, mlp_desc_from_config, MLP_TENSOR, MLP_WS
 
-__all__ = ["MlpPlan", "MlpRunner", "mlp_desc_from_config", "MLP_TENSOR", "MLP_WS",
+__all__ = ["LoraRunner", "MlpPlan", "MlpRunner", "mlp_desc_from_config", "MLP_TENSOR", "MLP_WS",
            "FblError", "Plan", "lib", "load_library", "LayerRunner", "DTYPES", "TENSOR", "MAP", "WS",
            "desc_from_config", "aligned_bytes", "guard_bands_intact", "selftest_wait_timeout"]

@@ -225,7 +225,7 @@ class LayerRunner:
     MATS = {"X": "X", "dY": "DY", "Wq": "WQ", "Wk": "WK", "Wv": "WV", "Wo": "WO"}
     OUT_MATS = {"Y": "Y", "dX": "DX", "dWq": "WQ", "dWk": "WK", "dWv": "WV", "dWo": "WO"}
 
-    def __init__(self, cfg, device="cuda:0", guard_bytes=0, tile_choices=None):
+    def __init__(self, cfg, device="cuda:0", guard_bytes=0, tile_choices=None, _before_sizes=None):
         """``tile_choices``: the GEMM launches' compute-tile configurations ({launch name: [tile_n, cta_pair,
         epilogue_sets]}, see rtile.py); None takes the layer's entry of the offline table shipped with the package,
         if it has one, {} leaves every launch to the built-in heuristics.
@@ -245,6 +245,8 @@ class LayerRunner:
         if tile_choices:
             rtile.apply(self.plan, tile_choices)
         self.tdtype = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
+        if _before_sizes is not None:
+            _before_sizes(self.plan)          # a subclass's plan options that change the work areas
         saved, sf, sb = self.plan.workspace_bytes()
         self.sizes = dict(saved=saved, scratch_fwd=sf, scratch_bwd=sb)
         al = lambda nbytes: aligned_bytes(torch, nbytes, self.dev, guard=guard_bytes)

@@ -55,6 +55,10 @@ struct fbl_plan {
   int knob_gemm_pair;       // -1 by size, 0 never the CTA-pair GEMM kernel, 1 wherever its tile shape is legal
   int knob_gemm_esets;      // 0 by tiles per block, 1 / 2 sets of epilogue warps
   int knob_fwd_tiles;       // 0 by sequence length, 1 / 2 query tiles per forward-attention block at head_dim 64
+  // low-rank adapters on Q, K, V (fbl_plan_enable_lora): rank, and the offsets of T = Xn [Aq|Ak|Av] inside `saved`,
+  // of dT and of the unused norm-parameter gradients inside the backward scratch
+  int lora_rank;
+  size_t sv_t, sb_dt, sb_frozen;
   // Compute-tile configuration of each GEMM launch of a step, fixed offline by the tile chooser (0 / -1: the
   // built-in heuristics decide): output-tile width, CTA-pair kernel, sets of epilogue warps.
   struct GemmChoice { int bn, pair, esets; } choice[FBL_GEMM_LAUNCH_COUNT];
@@ -78,7 +82,7 @@ struct GemmTerm {
 };
 struct GemmArgs {
   int m, n, n_terms;
-  GemmTerm t[3];
+  GemmTerm t[4];
   void* c; int64_t c_rpad;        // C[m,n] stored [m rows][n cols]
   const float* bias;              // per output column, or nullptr
   const void* residual;           // same layout as C, or nullptr
