@@ -245,12 +245,25 @@ def run_reference(args, cfg, rank):
 
 
 # ---- one workload on this rank's GPU ---------------------------------------------------------------------------
-def measure(cfg, args, rep, local_rank, flush_l2, want_cpu):
-    import torch
-    from paper_2607_21624_b200 import TENSOR, LayerRunner
+def lora_flops(cfg, r):
+    """Algorithmic flops of a step with rank-r adapters on Q, K, V and frozen base weights: the base step without its
+    four weight-gradient products, plus the adapters' six thin products (and their term in dXn)."""
+    n, d, dqkv = cfg.n_tokens, cfg.d_model, cfg.d_q + 2 * cfg.d_kv
+    frozen = 2.0 * n * d * dqkv + 2.0 * n * cfg.d_q * d
+    return cfg.flops() - frozen + 3 * 2.0 * n * d * 3 * r + 3 * 2.0 * n * r * dqkv
 
-    inp = make_inputs(cfg)
-    run = LayerRunner(cfg, device=f"cuda:{local_rank}")
+
+def measure(cfg, args, rep, local_rank, flush_l2, want_cpu, lora_rank=0):
+    import torch
+    from paper_2607_21624_b200 import TENSOR, LayerRunner, LoraRunner
+
+    if lora_rank:
+        from fbl_inputs import make_lora_inputs
+        inp = make_lora_inputs(cfg, lora_rank)
+        run = LoraRunner(cfg, lora_rank, device=f"cuda:{local_rank}")
+    else:
+        inp = make_inputs(cfg)
+        run = LayerRunner(cfg, device=f"cuda:{local_rank}")
     run.plan.set_kernel_path(args.path)
     run.load_inputs(inp)
     stream = torch.cuda.Stream()
@@ -394,9 +407,14 @@ def measure(cfg, args, rep, local_rank, flush_l2, want_cpu):
         return None
 
     peaks = measured_peaks()
-    flops = cfg.flops()
+    flops = lora_flops(cfg, lora_rank) if lora_rank else cfg.flops()
     tfl = rep.whole_job_rate(flops, ms) / 1e12
     sf, sbytes = step_flops(cfg), step_bytes(cfg)
+    if lora_rank:
+        thin = 2.0 * cfg.n_tokens * lora_rank
+        sf.update({"lora_T": thin * 3 * cfg.d_model, "lora_dA": thin * 3 * cfg.d_model, "lora_dT": thin * (cfg.d_q + 2 * cfg.d_kv),
+                   "proj_qkv": sf["proj_qkv"] + thin * (cfg.d_q + 2 * cfg.d_kv),
+                   "dB+dXn": sf["dXn"] + thin * (cfg.d_q + 2 * cfg.d_kv) + thin * 3 * cfg.d_model})
     dom = max(kernel_ms, key=kernel_ms.get)
     total_k = sum(kernel_ms.values())
     if dom in sf:
@@ -449,7 +467,8 @@ def measure(cfg, args, rep, local_rank, flush_l2, want_cpu):
 
     t_tensor = flops / (peaks["tflops_burst"] * 1e12)
     return {
-        "workload": workload_name(cfg), "ms_per_step": ms, "ms_per_step_min": ms_min, "ms_per_step_warm_l2": ms_warm,
+        "workload": workload_name(cfg) + (f" + rank-{lora_rank} adapters on Q, K, V, base weights frozen" if lora_rank else ""),
+        "ms_per_step": ms, "ms_per_step_min": ms_min, "ms_per_step_warm_l2": ms_warm,
         "ms_fwd": ms_fwd, "ms_bwd": ms_bwd,
         "tflops": tfl, "tokens_per_s": rep.whole_job_rate(cfg.n_tokens, ms), "flops_per_step": flops,
         "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
@@ -577,6 +596,10 @@ def run_rank(args):
     if not args.config and not args.no_mlp:          # the feed-forward blocks behind these attention layers
         for key in ("matmul-512x2048x8192", "gpt2", "llama1b"):
             mlp[key] = measure_mlp(key, args, rep, local_rank, flush_l2)
+    lora = {}
+    if not args.config and not args.no_mlp:          # the paper's fine-tuning setting on two of the workloads
+        for i in (2, 4):
+            lora[i] = measure(pick(i), args, rep, local_rank, flush_l2, want_cpu=False, lora_rank=16)
     if rank != 0:
         rep.close()
         return
@@ -595,10 +618,12 @@ def run_rank(args):
         "tokens_per_s": h["tokens_per_s"], "layer_roofline": h["layer_roofline"], "mem_efficiency": h["mem_efficiency"],
         "activation_bytes": h["activation_bytes"], "e2e": h["e2e"],
         "gpu_launches": (sum(r["launches_per_step"] for r in results.values())
-                         + sum(r["launches_per_step"] for r in mlp.values())) * args.steps,
+                         + sum(r["launches_per_step"] for r in mlp.values())
+                         + sum(r["launches_per_step"] for r in lora.values())) * args.steps,
         "clocks": h["clocks"], "roofline": h["roofline"], "cpu_baseline": h["cpu_baseline"],
         "peaks": peaks,
-        "per_config": {**{f"workload{i}": results[i] for i in sorted(results)}, **{f"mlp_{k}": v for k, v in mlp.items()}},
+        "per_config": {**{f"workload{i}": results[i] for i in sorted(results)}, **{f"mlp_{k}": v for k, v in mlp.items()},
+                       **{f"lora16_workload{i}": v for i, v in lora.items()}},
     }
     print(json.dumps(line))
     rep.close()
@@ -614,7 +639,7 @@ def main():
     ap.add_argument("--path", type=int, default=0, help="0 default kernels, 1 FFMA kernels only")
     ap.add_argument("--no-graph", action="store_true", help="enqueue kernels directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-mlp", action="store_true", help="skip the feed-forward blocks' entries of per_config")
+    ap.add_argument("--no-mlp", action="store_true", help="skip the feed-forward and adapter entries of per_config")
     ap.add_argument("--flush-write-only", action="store_true", help="flush L2 by the 256 MiB write alone (its write-back then overlaps the step)")
     ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling captures)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures)")
