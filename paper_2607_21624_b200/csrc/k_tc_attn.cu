@@ -11,6 +11,7 @@
 
 #include <type_traits>
 
+#include "attn_common.cuh"
 #include "fbl_internal.h"
 #include "pdl.cuh"
 #include "tc_common.cuh"
@@ -19,24 +20,6 @@ namespace {
 
 constexpr int BQ = 128, BKV = 128;
 constexpr float LOG2E = 1.4426950408889634f;
-
-// Block numbering shared by both kernels.  (head, batch) pairs are taken in chunks small enough for their
-// operands to stay in L2 together; inside a chunk the causal-work index ("slot": query-tile slot forward, key
-// tile backward) varies slowest, heaviest first, so the block scheduler, which dispatches in block-id order,
-// hands out the long blocks of a chunk before its short ones.
-__device__ __forceinline__ void decode_block(int lin, int n_slots, int n_hb, int chunk, int* slot, int* hb) {
-  const int per_chunk = n_slots * chunk;
-  const int full = (n_hb / chunk) * per_chunk;
-  int c0, csize, rem;
-  if (lin < full) { c0 = (lin / per_chunk) * chunk; csize = chunk; rem = lin % per_chunk; }
-  else { c0 = (n_hb / chunk) * chunk; csize = n_hb - c0; rem = lin - full; }
-  *slot = rem / csize;
-  *hb = c0 + rem % csize;
-}
-static int chunk_for(long long bytes_per_hb, int n_hb, long long budget) {
-  long long c = budget / (bytes_per_hb > 0 ? bytes_per_hb : 1);
-  return (int)(c < 1 ? 1 : (c > n_hb ? n_hb : c));
-}
 
 struct alignas(64) AttnFwdParams {
   CUtensorMap tq, tk, tv;
@@ -543,11 +526,11 @@ struct BwdSmem {
   static constexpr uint32_t LSE_OFF = STAGE_OFF + NS * STAGE_BYTES;    // 128 floats of LSE per Q stage, then 128 of D per dO stage
   static constexpr uint32_t D_OFF = LSE_OFF + NQQ * 512;
   static constexpr uint32_t BAR_OFF = D_OFF + NDO * 512;
-  static constexpr uint32_t N_BARS = 20;
+  static constexpr uint32_t N_BARS = 24;          // BB_* below: 22 in use
   static constexpr uint32_t TOTAL = BAR_OFF + 8 * N_BARS + 16;
 };
 
-enum { BB_KVFULL = 0, BB_QFULL = 1, BB_QEMPTY = 4, BB_DOFULL = 7, BB_DOEMPTY = 9, BB_SFULL = 11, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_DQSTAGED, BB_STAGEFREE = BB_DQSTAGED + 2, BB_SREAD = BB_STAGEFREE + 2, BB_DVDONE };
+enum { BB_KVFULL = 0, BB_QFULL = 1, BB_QEMPTY = 4, BB_DOFULL = 7, BB_DOEMPTY = 9, BB_SFULL = 11, BB_PDSFULL, BB_DQFULL, BB_DQDRAINED, BB_DQSTAGED, BB_STAGEFREE = BB_DQSTAGED + 2, BB_SREAD = BB_STAGEFREE + 2, BB_DVDONE, BB_DPFULL };
 
 constexpr int BWD_THREADS = 608;     // warp 0 TMA loads, warp 1 MMA, warps 2-17 softmax (four per TMEM lane quarter), warp 18 dQ reductions
 constexpr int BWD_SM_THREADS = 512;
@@ -603,6 +586,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     tc::mbar_init(bar(BB_STAGEFREE + 1), 1);
     tc::mbar_init(bar(BB_SREAD), BWD_SM_THREADS);
     tc::mbar_init(bar(BB_DVDONE), 1);
+    tc::mbar_init(bar(BB_DPFULL), 1);
     tc::fence_barrier_init();
     // This thread is the TMA producer: K, V and the first Q tile (forward-pass data) are requested right here, so
     // that their latency overlaps the tensor-memory allocation and the block-wide barrier below.
@@ -682,15 +666,16 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         const uint32_t o = (kk / 4) * 1024 + (kk % 4) * 2;
         tc::mma_bf16_ss_w(tmem_base + S_COL, k_km + o, hi, qs + o, hi, idesc_s, kk > 0);
       }
-    };
-    auto issue_dp = [&](int it) {             // dP^T = V dO^T of tile `it`; then both score tiles are announced
+      if (!PIPE) tc::mma_commit(bar(BB_SFULL));     // HD = 128: the softmax warps start on the scores while dP^T is
+    };                                              // still to come (it waits for the previous tile's dQ drain)
+    auto issue_dp = [&](int it) {             // dP^T = V dO^T of tile `it`, announced on its own barrier
       const uint32_t dos = do_km + (it % NDO) * (SM::TILE >> 4);
 #pragma unroll
       for (uint32_t kk = 0; kk < HD / 16; ++kk) {
         const uint32_t o = (kk / 4) * 1024 + (kk % 4) * 2;
         tc::mma_bf16_ss_w(tmem_base + DP_COL, v_km + o, hi, dos + o, hi, idesc_s, kk > 0);
       }
-      tc::mma_commit(bar(BB_SFULL));
+      tc::mma_commit(bar(PIPE ? BB_SFULL : BB_DPFULL));      // HD = 64: one announcement for both score tiles
     };
     auto issue_dv = [&](int it) {             // dV += P^T dO, P^T read from tensor memory
       const uint32_t dos = do_mn + (it % NDO) * (SM::TILE >> 4);
@@ -867,6 +852,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
         if (!tc::mbar_wait(bar(BB_SREAD), it & 1, status, 311)) { ok = false; break; }
         tc::tc_fence_after();
       }
+      if constexpr (PIPE) {
       // One 16-column chunk: P^T = exp2(S^T c - LSE) to tensor memory, dS^T = P^T (dP^T - D) to the swizzled
       // shared-memory operand tile, both rounded to bf16.  MASKED is the rare path (diagonal / ragged tiles).
       auto chunk = [&](int cc, auto masked_tag) {
@@ -929,6 +915,82 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       } else {
         chunk(0, std::false_type{});
         if (ok) chunk(1, std::false_type{});
+      }
+      } else {
+      // Phase A needs only S^T: P^T = exp2(S^T c - LSE) for this thread's 32 query columns, kept in the score
+      // registers as fp32 and stored to tensor memory as bf16.  It runs while the tensor pipe is still busy with
+      // dP^T of this tile (which at HD = 128 also waits for the previous tile's dQ to be drained).
+      auto phase_a = [&](auto masked_tag) {
+        constexpr bool MASKED = decltype(masked_tag)::value;
+        const float2 c2 = make_float2(c, c), nl2e = make_float2(-LOG2E, -LOG2E);
+#pragma unroll
+        for (int k = 0; k < 32; k += 4) {
+          const float4 l4 = *reinterpret_cast<const float4*>(&s_lse[part * 32 + k]);
+          const float2 x01 = __ffma2_rn(make_float2(__uint_as_float(sv[k]), __uint_as_float(sv[k + 1])), c2, __fmul2_rn(make_float2(l4.x, l4.y), nl2e));
+          const float2 x23 = __ffma2_rn(make_float2(__uint_as_float(sv[k + 2]), __uint_as_float(sv[k + 3])), c2, __fmul2_rn(make_float2(l4.z, l4.w), nl2e));
+          float pv[4] = {tc::fast_exp2(x01.x), tc::fast_exp2(x01.y), tc::fast_exp2(x23.x), tc::fast_exp2(x23.y)};
+          if (MASKED) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int gi = i0 + part * 32 + k + u;
+              if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) pv[u] = 0.f;
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) sv[k + u] = __float_as_uint(pv[u]);
+        }
+      };
+      if (need_mask) phase_a(std::true_type{}); else phase_a(std::false_type{});
+      {
+        uint32_t pp[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) pp[k] = tc::pack_bf16(__uint_as_float(sv[2 * k]), __uint_as_float(sv[2 * k + 1]));
+        if (PIPE && it > 0) {
+          // P^T has its own columns, single-buffered: the dV product of the previous tile must have read them
+          if (!tc::mbar_wait(bar(BB_DVDONE), (it - 1) & 1, status, 312)) { ok = false; break; }
+          tc::tc_fence_after();
+        }
+        tc::tmem_st16(lane_addr + P_COL + part * 16, pp);
+      }
+      // Phase B: dS^T = P^T (dP^T - D), rounded to bf16, to the swizzled shared-memory operand tile, in two
+      // 16-column chunks.  MASKED is the rare path (diagonal / ragged tiles).
+      if (!tc::mbar_wait(bar(BB_DPFULL), it & 1, status, 316)) { ok = false; break; }
+      tc::tc_fence_after();
+      auto phase_b = [&](int cc, auto masked_tag) {
+        constexpr bool MASKED = decltype(masked_tag)::value;
+        const int c0 = part * 32 + cc * 16;
+        uint32_t dpv[16];
+        tc::tmem_ld16(lane_addr + DP_COL + c0, dpv);
+        tc::tmem_ld_wait();
+        uint32_t dd[8];
+        const float2 neg1 = make_float2(-1.f, -1.f);
+#pragma unroll
+        for (int k = 0; k < 16; k += 4) {
+          const float4 d4 = *reinterpret_cast<const float4*>(&s_d[c0 + k]);
+          const float* pv = reinterpret_cast<const float*>(&sv[cc * 16 + k]);
+          const float2 g01 = __fmul2_rn(make_float2(pv[0], pv[1]), __ffma2_rn(make_float2(d4.x, d4.y), neg1, make_float2(__uint_as_float(dpv[k]), __uint_as_float(dpv[k + 1]))));
+          const float2 g23 = __fmul2_rn(make_float2(pv[2], pv[3]), __ffma2_rn(make_float2(d4.z, d4.w), neg1, make_float2(__uint_as_float(dpv[k + 2]), __uint_as_float(dpv[k + 3]))));
+          float gv[4] = {g01.x, g01.y, g23.x, g23.y};
+          if (MASKED) {                              // LSE / D of rows past the sequence end are not defined
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int gi = i0 + c0 + k + u;
+              if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) gv[u] = 0.f;
+            }
+          }
+          dd[k / 2] = tc::pack_bf16(gv[0], gv[1]);
+          dd[k / 2 + 1] = tc::pack_bf16(gv[2], gv[3]);
+        }
+        // 16 query columns = 2 swizzled 16-byte chunks of this key row inside its 64-query panel
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch) {
+          const uint32_t chk = (uint32_t)((part % 2) * 4 + cc * 2 + ch);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dsrow + ((chk ^ (uint32_t)(r & 7)) * 16)),
+                       "r"(dd[ch * 4]), "r"(dd[ch * 4 + 1]), "r"(dd[ch * 4 + 2]), "r"(dd[ch * 4 + 3]) : "memory");
+        }
+      };
+      if (need_mask) { phase_b(0, std::true_type{}); phase_b(1, std::true_type{}); }
+      else { phase_b(0, std::false_type{}); phase_b(1, std::false_type{}); }
       }
       if (!ok) break;
       tc::tmem_st_wait();
