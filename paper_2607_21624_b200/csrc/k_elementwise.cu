@@ -381,6 +381,20 @@ __device__ __forceinline__ void colsum_slab(const ColsumGroup& G, int64_t rows, 
   }
 }
 
+// Shared memory of the kernel below: per warp its private token-axis sums (dgamma and dbeta parts of its columns,
+// as float4 slots [which][2 NV][32 lanes]: consecutive lanes, consecutive slots, conflict-free), then gamma.
+template <int NV, int WPR>
+struct NormBwdSmem {
+  static constexpr int D = NV * 256 * WPR;
+  static constexpr int ACC_F4_PER_WARP = 2 * 2 * NV * 32;
+  static constexpr size_t ACC_BYTES = (size_t)8 * ACC_F4_PER_WARP * 16;
+  static constexpr size_t BYTES = ACC_BYTES + (size_t)D * 4;
+};
+
+// A warp (or WPR warps) owns a row; the row's X and dXn stay in registers as raw bf16 vectors, and the next row's
+// are requested before the current row's two reductions, so X and dXn cross HBM exactly once with a row in flight
+// per warp at all times.  The token-axis sums (dgamma, dbeta) of a warp's rows accumulate in its private
+// shared-memory slots (registers are better spent on the row in flight).
 template <int NV, int WPR>
 __global__ void __launch_bounds__(256, 2) norm_bwd_rows_kernel(const __nv_bfloat16* __restrict__ dXn,
                                                             const __nv_bfloat16* __restrict__ X,
@@ -390,10 +404,10 @@ __global__ void __launch_bounds__(256, 2) norm_bwd_rows_kernel(const __nv_bfloat
                                                             __nv_bfloat16* __restrict__ dX, float* __restrict__ partials,
                                                             int64_t n_pad, int rms, int n_norm, ColsumGroup CG,
                                                             float* __restrict__ cs_part, int cs_panels, int cs_slabs) {
-  constexpr int D = NV * 256 * WPR;
+  using SMEM = NormBwdSmem<NV, WPR>;
+  constexpr int D = SMEM::D;
   constexpr int RPB = 8 / WPR;
-  __shared__ float s_dg[D];
-  __shared__ float s_db[D];
+  extern __shared__ __align__(16) uint8_t norm_smem[];
   __shared__ float s_part[32];
   // Blocks behind the first n_norm ones do the first stage of the bias gradients' column sums (one launch less):
   // block n_norm + (which * slabs + slab) * panels + p
@@ -405,57 +419,78 @@ __global__ void __launch_bounds__(256, 2) norm_bwd_rows_kernel(const __nv_bfloat
     colsum_slab<__nv_bfloat16>(CG, n_pad, cs_part, idx % cs_panels, (idx / cs_panels) % cs_slabs, idx / (cs_panels * cs_slabs), cs_red);
     return;
   }
-  int buf = 0;
-  for (int i = threadIdx.x; i < D; i += 256) { s_dg[i] = 0.f; s_db[i] = 0.f; }
-  __syncthreads();
-  pdl_launch_dependents();
+  float4* s_acc = reinterpret_cast<float4*>(norm_smem);
+  float* s_gamma = reinterpret_cast<float*>(norm_smem + SMEM::ACC_BYTES);
   const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
   const int slot = wib / WPR, part = wib % WPR;
-  float gm[NV][8];                           // gamma is an input of the step: read before waiting for the GEMM
-#pragma unroll
-  for (int j = 0; j < NV; ++j) {
-    const int c0 = ((part * NV + j) * 32 + lane) * 8;
-    const float4 g0 = *reinterpret_cast<const float4*>(gamma + c0), g1 = *reinterpret_cast<const float4*>(gamma + c0 + 4);
-    gm[j][0] = g0.x; gm[j][1] = g0.y; gm[j][2] = g0.z; gm[j][3] = g0.w;
-    gm[j][4] = g1.x; gm[j][5] = g1.y; gm[j][6] = g1.z; gm[j][7] = g1.w;
-  }
+  int buf = 0;
+  // gamma is an input of the step: into shared memory before waiting for the GEMM in front; the sums start at zero
+  for (int i = threadIdx.x; i < D; i += 256) s_gamma[i] = gamma[i];
+  for (int i = threadIdx.x; i < 8 * SMEM::ACC_F4_PER_WARP; i += 256) s_acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  __syncthreads();
+  pdl_launch_dependents();
+  float4* my_acc = s_acc + wib * SMEM::ACC_F4_PER_WARP;       // [which][2 j + h][lane]
+  auto vec_off = [&](int j, int64_t r) {
+    const int v = (part * NV + j) * 32 + lane;
+    return ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8;
+  };
   pdl_wait();
-  // token-axis partial sums of this warp's rows, kept in registers and folded into shared memory at the end
-  float ag[NV][8], ab[NV][8];
-#pragma unroll
-  for (int j = 0; j < NV; ++j)
-#pragma unroll
-    for (int i = 0; i < 8; ++i) { ag[j][i] = 0.f; ab[j][i] = 0.f; }
   // each block owns a contiguous range of rows (neighbouring 128-byte pieces in every panel)
   const int64_t per_block = ((n_pad + n_norm - 1) / n_norm + RPB - 1) / RPB * RPB;
   const int64_t r_end = min(n_pad, ((int64_t)blockIdx.x + 1) * per_block);
-  for (int64_t r = (int64_t)blockIdx.x * per_block + slot; r < r_end; r += RPB) {
-    const float mean = stats[2 * r], rstd = stats[2 * r + 1];
-    float xh[NV][8], g[NV][8];
-    float s1 = 0.f, s2 = 0.f;
-    uint4 yraw[NV];                          // the residual's gradient, requested together with the other two rows
-    if (dY) {
-#pragma unroll
-      for (int j = 0; j < NV; ++j) {
-        const int v = (part * NV + j) * 32 + lane;
-        yraw[j] = *reinterpret_cast<const uint4*>(dY + ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8);
-      }
-    }
+  int64_t r = (int64_t)blockIdx.x * per_block + slot;
+  uint4 xr[NV], gr[NV];
+  float2 st = make_float2(0.f, 0.f);
+  if (r < r_end) {
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      const int v = (part * NV + j) * 32 + lane;
-      const int64_t off = ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8;
-      float gv[8];
-      load16(X + off, xh[j]);
-      load16(dXn + off, gv);
+      xr[j] = *reinterpret_cast<const uint4*>(X + vec_off(j, r));
+      gr[j] = *reinterpret_cast<const uint4*>(dXn + vec_off(j, r));
+    }
+    st = *reinterpret_cast<const float2*>(stats + 2 * r);
+  }
+  while (r < r_end) {
+    const int64_t rn = r + RPB;
+    uint4 xn[NV], gn[NV], yr[NV];
+    float2 stn = make_float2(0.f, 0.f);
+    if (rn < r_end) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        xh[j][i] = (xh[j][i] - mean) * rstd;
-        ag[j][i] = fmaf(gv[i], xh[j][i], ag[j][i]);
-        ab[j][i] += gv[i];
-        g[j][i] = gv[i] * gm[j][i];
-        s1 += g[j][i];
-        s2 = fmaf(g[j][i], xh[j][i], s2);
+      for (int j = 0; j < NV; ++j) {
+        xn[j] = *reinterpret_cast<const uint4*>(X + vec_off(j, rn));
+        gn[j] = *reinterpret_cast<const uint4*>(dXn + vec_off(j, rn));
+      }
+      stn = *reinterpret_cast<const float2*>(stats + 2 * rn);
+    }
+    if (dY) {
+#pragma unroll
+      for (int j = 0; j < NV; ++j) yr[j] = *reinterpret_cast<const uint4*>(dY + vec_off(j, r));
+    }
+    const float mean = st.x, rstd = st.y;
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      const __nv_bfloat16* xe = reinterpret_cast<const __nv_bfloat16*>(&xr[j]);
+      const __nv_bfloat16* ge = reinterpret_cast<const __nv_bfloat16*>(&gr[j]);
+      const int c0 = ((part * NV + j) * 32 + lane) * 8;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const float4 gm = *reinterpret_cast<const float4*>(s_gamma + c0 + 4 * h);
+        const float gmv[4] = {gm.x, gm.y, gm.z, gm.w};
+        float4 ag = my_acc[(2 * j + h) * 32 + lane], ab = my_acc[(2 * NV + 2 * j + h) * 32 + lane];
+        float* agv = reinterpret_cast<float*>(&ag);
+        float* abv = reinterpret_cast<float*>(&ab);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float xh = (__bfloat162float(xe[4 * h + i]) - mean) * rstd;
+          const float gv = __bfloat162float(ge[4 * h + i]);
+          const float g = gv * gmv[i];
+          agv[i] = fmaf(gv, xh, agv[i]);
+          abv[i] += gv;
+          s1 += g;
+          s2 = fmaf(g, xh, s2);
+        }
+        my_acc[(2 * j + h) * 32 + lane] = ag;
+        my_acc[(2 * NV + 2 * j + h) * 32 + lane] = ab;
       }
     }
     row_sum2<WPR>(s1, s2, s_part, slot, part, buf);
@@ -463,35 +498,46 @@ __global__ void __launch_bounds__(256, 2) norm_bwd_rows_kernel(const __nv_bfloat
     s2 *= (1.f / D);
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      const int v = (part * NV + j) * 32 + lane;
-      const int64_t off = ((int64_t)(v / 8) * n_pad + r) * 64 + (v % 8) * 8;
+      const __nv_bfloat16* xe = reinterpret_cast<const __nv_bfloat16*>(&xr[j]);
+      const __nv_bfloat16* ge = reinterpret_cast<const __nv_bfloat16*>(&gr[j]);
+      const __nv_bfloat16* ye = reinterpret_cast<const __nv_bfloat16*>(&yr[j]);
+      const int c0 = ((part * NV + j) * 32 + lane) * 8;
       float o[8];
-      const __nv_bfloat16* ye = reinterpret_cast<const __nv_bfloat16*>(&yraw[j]);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float dx = rstd * (g[j][i] - s1 - xh[j][i] * s2);
-        o[i] = dY ? __bfloat162float(ye[i]) + dx : dx;
+      for (int h = 0; h < 2; ++h) {
+        const float4 gm = *reinterpret_cast<const float4*>(s_gamma + c0 + 4 * h);
+        const float gmv[4] = {gm.x, gm.y, gm.z, gm.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float xh = (__bfloat162float(xe[4 * h + i]) - mean) * rstd;
+          const float g = __bfloat162float(ge[4 * h + i]) * gmv[i];
+          const float dx = rstd * (g - s1 - xh * s2);
+          o[4 * h + i] = dY ? __bfloat162float(ye[4 * h + i]) + dx : dx;
+        }
       }
-      store16(dX + off, o);
+      store16(dX + vec_off(j, r), o);
     }
+#pragma unroll
+    for (int j = 0; j < NV; ++j) { xr[j] = xn[j]; gr[j] = gn[j]; }
+    st = stn;
+    r = rn;
   }
-  // Fold the warps' sums in shared memory.  Slot (k, lane) with k = (part*NV + j)*8 + i holds column
-  // ((part*NV + j)*32 + lane)*8 + i: consecutive lanes hit consecutive banks.
-#pragma unroll
-  for (int j = 0; j < NV; ++j)
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int k = ((part * NV + j) * 8 + i) * 32 + lane;
-      atomicAdd(&s_dg[k], ag[j][i]);
-      if (!rms) atomicAdd(&s_db[k], ab[j][i]);
-    }
   __syncthreads();
-  // this block's token-axis partial sums: row blockIdx.x of partials[blocks][2][D]; a second kernel adds the rows
+  // this block's token-axis partial sums: the RPB warps that share a column range are added, and the row goes to
+  // row blockIdx.x of partials[blocks][2][D]; a second kernel adds the rows
   float* mine = partials + (int64_t)blockIdx.x * 2 * D;
+  const float* accf = reinterpret_cast<const float*>(s_acc);
   for (int c = threadIdx.x; c < D; c += 256) {
-    const int k = ((c / 256) * 8 + c % 8) * 32 + (c / 8) % 32;
-    mine[c] = s_dg[k];
-    if (!rms) mine[D + c] = s_db[k];
+    const int v = c / 8, i = c % 8, ln = v % 32, pj = v / 32, pt = pj / NV, j = pj % NV;
+    float sg = 0.f, sb = 0.f;
+#pragma unroll
+    for (int sl = 0; sl < RPB; ++sl) {
+      const float* w = accf + (size_t)(sl * WPR + pt) * SMEM::ACC_F4_PER_WARP * 4;
+      sg += w[((2 * j + i / 4) * 32 + ln) * 4 + i % 4];
+      sb += w[((2 * NV + 2 * j + i / 4) * 32 + ln) * 4 + i % 4];
+    }
+    mine[c] = sg;
+    if (!rms) mine[D + c] = sb;
   }
 }
 
@@ -558,7 +604,9 @@ void norm_bwd_rows_launch(const fbl_plan* p, const void* dXn, const void* X, con
   int cs_panels = 0;
   for (int i = 0; i < cg.count; ++i) cs_panels = cg.cols[i] / 64 > cs_panels ? cg.cols[i] / 64 : cs_panels;
   const int cs_blocks = cs_panels * n_slabs * cg.count;
-  launch_pdl(norm_bwd_rows_kernel<NV, WPR>, dim3(blocks + cs_blocks), dim3(256), 0, st, (const __nv_bfloat16*)dXn,
+  constexpr size_t smem = NormBwdSmem<NV, WPR>::BYTES;
+  cudaFuncSetAttribute(norm_bwd_rows_kernel<NV, WPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  launch_pdl(norm_bwd_rows_kernel<NV, WPR>, dim3(blocks + cs_blocks), dim3(256), smem, st, (const __nv_bfloat16*)dXn,
              (const __nv_bfloat16*)X, (const __nv_bfloat16*)dY, stats, gamma, (__nv_bfloat16*)dX, part, p->n_pad, rms,
              blocks, cg, const_cast<float*>(cpart), cs_panels, n_slabs);
   const int ny = rms ? 1 : 2;

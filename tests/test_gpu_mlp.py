@@ -89,8 +89,8 @@ def test_mlp_back_to_back_steps_are_identical():
     run.load_inputs(make_mlp_inputs(cfg, affine_noise=True))
     run.step()
     torch.cuda.synchronize()
-    names = ("Y", "dX", "dW1", "dWg", "dW2", "db1")
-    first = {n: run.fetch(n) for n in names + ("dgamma",)}
+    names = ("Y", "dX", "dW1", "dWg", "dW2", "db1", "dgamma")
+    first = {n: run.fetch(n) for n in names}
     for fill in (0xFF, 0x7F):
         run.saved.fill_(fill)
         run.scratch.fill_(fill)
