@@ -82,28 +82,33 @@ def min_bytes(cfg):
     return 5 * nd + 3 * w + 2 * qkva + 2 * small
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the step kernels, from the ncu captures
-# summarised under profiles/.  Keyed by (workload name, step); a step without a capture has no entry.
-NCU_TRAFFIC_BYTES = {
-    # workload 2: every kernel of a step, profiles/ncu_full_workload2_gpt2small_hd64.md
-    ("cfg2-gpt2-small", "norm_fwd"): 3.5e6 + 0.0e6,
-    ("cfg2-gpt2-small", "proj_qkv"): 6.8e6 + 0.0e6,
-    ("cfg2-gpt2-small", "attn_fwd"): 9.5e6 + 0.0e6,
-    ("cfg2-gpt2-small", "proj_o"): 4.4e6 + 0.0e6,
-    ("cfg2-gpt2-small", "dWo+dA"): 7.5e6 + 0.0e6,
-    ("cfg2-gpt2-small", "attn_bwd"): 19.1e6 + 0.5e6 + 6.3e6,      # main kernel + rounding of the fp32 dQ
-    ("cfg2-gpt2-small", "dWqkv+dXn"): 16.2e6 + 1.3e6,
-    # norm backward's rows kernel (with the bias column sums' first stage as extra blocks; its DRAM write figure in the
-    # capture is the flush buffer's write-back and is left out: the kernel's own output is 3.1 MB) and the shared second stage
-    ("cfg2-gpt2-small", "db+norm_bwd"): 18.9e6 + 3.1e6 + 1.7e6,
-    # workload 4, profiles/ncu_full_workload4_llama1b_gqa_hd64.md
-    ("cfg4-llama1b-gqa", "proj_qkv"): 29.4e6 + 0.3e6,
-    ("cfg4-llama1b-gqa", "attn_fwd"): 25.2e6 + 0.0e6,
-    ("cfg4-llama1b-gqa", "proj_o"): 25.2e6 + 0.0e6,
-    ("cfg4-llama1b-gqa", "dWo+dA"): 42.6e6 + 2.8e6,
-    ("cfg4-llama1b-gqa", "attn_bwd"): 76.6e6 + 3.5e6,
-    ("cfg4-llama1b-gqa", "dWqkv+dXn"): 56.4e6 + 11.5e6,
+# DRAM bytes per step kernel (dram__bytes_read.sum + dram__bytes_write.sum, MB in the table, bytes in the dict) from the
+# ncu capture of one step of every workload summarised in profiles/ncu_step_kernels_all_workloads.md.  ncu flushes the
+# caches before each captured launch, so reads are cold; a kernel's own output mostly stays in L2 and is not counted.
+# Workload 5 is captured at sequence 2048 (the full 8192-token step holds 2.5 GB and its kernels run for milliseconds:
+# too large for a multi-pass capture).  For the kernels whose traffic grows with the tokens (attention, norms) the
+# full workload's entries are that capture's figures times 4, the ratio of the token counts; the GEMMs' traffic has
+# a weight share that does not grow, so they get no scaled entry.
+_MB = 1e6
+_NCU_MB = {
+    "cfg1-tiny-fp32": {"norm_fwd": 0.03, "proj_q": 0.10, "proj_k": 0.10, "proj_v": 0.10, "attn_fwd": 0.07, "proj_o": 0.10,
+                       "dA": 0.10, "dWo": 0.11, "attn_bwd": 0.04 + 0.11 + 0.02, "dXn": 0.16, "dWq": 0.11, "dWk": 0.11,
+                       "dWv": 0.11, "norm_bwd": 0.05},
+    "cfg2-gpt2-small": {"norm_fwd": 3.46, "proj_qkv": 6.76, "attn_fwd": 9.47, "proj_o": 4.39, "dWo+dA": 7.53,
+                        "attn_bwd": 19.12 + 6.30, "dWqkv+dXn": 16.18, "db+norm_bwd": 18.92 + 1.69},
+    "cfg3-vit-base": {"norm_fwd": 10.16, "proj_qkv": 13.43, "attn_fwd": 29.53, "proj_o": 11.07, "dWo+dA": 23.26,
+                      "attn_bwd": 59.97 + 19.67, "dWqkv+dXn": 50.12, "dW round": 11.06, "norm_bwd": 19.75 + 1.83},
+    "cfg4-llama1b-gqa": {"norm_fwd": 16.81, "proj_qkv": 29.42, "attn_fwd": 25.22, "proj_o": 25.23, "dWo+dA": 45.53,
+                         "attn_bwd": 77.46 + 33.56, "dWqkv+dXn": 62.33, "norm_bwd": 33.72 + 2.44},
+    "cfg5-llama7b-long-scaled": {"norm_fwd": 16.82, "proj_qkv": 147.11, "attn_fwd": 50.56, "proj_o": 50.49, "dWo+dA": 110.03,
+                                 "attn_bwd": 118.07 + 33.56, "dWqkv+dXn": 383.49, "norm_bwd": 33.91 + 4.87},
 }
+_NCU_MB["cfg5-llama7b-long"] = {k: 4.0 * v for k, v in _NCU_MB["cfg5-llama7b-long-scaled"].items()
+                                if k in ("norm_fwd", "attn_fwd", "attn_bwd", "norm_bwd")}     # the token-proportional kernels
+NCU_TRAFFIC_BYTES = {(w, k): v * _MB for w, steps in _NCU_MB.items() for k, v in steps.items()}
+NCU_TRAFFIC_NOTE = {"cfg5-llama7b-long": "seq-2048 capture x 4 (token ratio)"}
+# the layer's memory efficiency of workload 5 is the one of its captured seq-2048 instance
+MEM_EFF_PROXY = {"cfg5-llama7b-long": ("cfg5-llama7b-long-scaled", dict(seq=2048))}
 
 
 class ClockSampler:
@@ -433,6 +438,8 @@ def measure(cfg, args, rep, local_rank, flush_l2, want_cpu, lora_rank=0):
         roof = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peaks["gbs"], "unit": "GB/s",
                 "frac": ach / peaks["gbs"], "traffic": None, "peak_source": peaks["source"]}
     roof["traffic"] = NCU_TRAFFIC_BYTES.get((cfg.name, dom))
+    if cfg.name in NCU_TRAFFIC_NOTE:
+        roof["traffic_note"] = NCU_TRAFFIC_NOTE[cfg.name]
     roof["kernel_share"] = kernel_ms[dom] / total_k
     roof["kernel_ms"] = {k: round(v, 5) for k, v in sorted(kernel_ms.items(), key=lambda kv: -kv[1])}
     roof["kernel_ms_sum_over_step_ms"] = total_k / ms      # > 1: what programmatic launch overlap hides in a real step
@@ -447,11 +454,16 @@ def measure(cfg, args, rep, local_rank, flush_l2, want_cpu, lora_rank=0):
                               for k in kernel_ms if k in sf} if cfg.dtype == "bf16" and args.path == 0 else {}
 
     # memory efficiency of the layer (the paper's Eq. 2 factor): once-only minimum bytes over the DRAM bytes ncu saw
-    steps_with_traffic = {k: NCU_TRAFFIC_BYTES.get((cfg.name, k)) for k in kernel_ms}
+    proxy_name, proxy_cfg = cfg.name, cfg
+    if cfg.name in MEM_EFF_PROXY:
+        proxy_name = MEM_EFF_PROXY[cfg.name][0]
+        proxy_cfg = scaled_config(cfg, **MEM_EFF_PROXY[cfg.name][1])
+    steps_with_traffic = {k: NCU_TRAFFIC_BYTES.get((proxy_name, k)) for k in kernel_ms}
     if all(v is not None for v in steps_with_traffic.values()):
         dram = sum(steps_with_traffic.values())
-        mem_eff = {"min_bytes": min_bytes(cfg), "ncu_dram_bytes": dram, "value": min_bytes(cfg) / dram,
-                   "source": "profiles/ (cold-cache captures, one per kernel)"}
+        mem_eff = {"min_bytes": min_bytes(proxy_cfg), "ncu_dram_bytes": dram, "value": min_bytes(proxy_cfg) / dram,
+                   "source": "profiles/ncu_step_kernels_all_workloads.md (cold-cache captures, one per kernel)"
+                             + ("; measured on this workload's 2048-token instance" if proxy_name != cfg.name else "")}
     else:
         mem_eff = {"min_bytes": min_bytes(cfg), "ncu_dram_bytes": None, "value": None,
                    "source": "no ncu capture of every kernel of this workload under profiles/"}
