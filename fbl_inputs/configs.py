@@ -28,6 +28,7 @@ class LayerConfig:
     seed: int
     w_std: float
     softmax_scale: float = 0.0   # <= 0 means 1/sqrt(head_dim)
+    rope_base: float = 0.0       # > 0: rotary position embedding on Q and K (half-split pairing) with this base
 
     @property
     def n_tokens(self) -> int:

@@ -15,6 +15,7 @@ forward, per batch element
                 xhat = (X-mu) rstd, Xn = xhat*gamma + beta
      RMSNorm    rstd = (mean_d X^2 + eps)^-1/2, xhat = X rstd, Xn = xhat*gamma
   2. Q = Xn Wq + bq, K = Xn Wk + bk, V = Xn Wv + bv
+  2b. (optional, cfg.rope_base > 0) rotary position embedding on Q and K, see ``rope``
   3. query head h owns columns [h*hd, (h+1)*hd); its KV head is g = h // G
   4. S_ij = scale * sum_d Q[i,h,d] K[j,g,d]; causal keeps only j <= i
      m_i = max_j S_ij, l_i = sum_j exp(S_ij - m_i), P_ij = exp(S_ij - m_i)/l_i,
@@ -61,6 +62,24 @@ def norm_fwd(X, gamma, beta, eps, kind):
     raise ValueError(kind)
 
 
+def rope(x, heads, base, inverse=False, pos_offset=0):
+    """Rotary position embedding on x: [B, T, heads * hd], half-split pairing: inside every head, element i < hd/2
+    is paired with element i + hd/2 and the pair of token t is rotated by the angle (t + pos_offset) * base^(-2i/hd):
+        y_i      = x_i cos - x_{i+hd/2} sin
+        y_{i+hd/2} = x_{i+hd/2} cos + x_i sin
+    ``inverse`` rotates by the opposite angle (the transpose of the rotation: what the backward applies)."""
+    B, T, C = x.shape
+    hd = C // heads
+    half = hd // 2
+    ang = (np.arange(T, dtype=np.float64)[:, None] + pos_offset) * base ** (-2.0 * np.arange(half, dtype=np.float64) / hd)[None, :]
+    cos, sin = np.cos(ang)[None, :, None, :], np.sin(ang)[None, :, None, :]
+    if inverse:
+        sin = -sin
+    xh = x.reshape(B, T, heads, hd)
+    lo, hi = xh[..., :half], xh[..., half:]
+    return np.concatenate([lo * cos - hi * sin, hi * cos + lo * sin], axis=-1).reshape(B, T, C)
+
+
 def attention_head_fwd(q, k, v, scale, causal):
     """Steps 4-5 for one (batch, head).  q: [T, hd], k, v: [T, hd].  Returns O, P, LSE."""
     T = q.shape[0]
@@ -82,6 +101,8 @@ def layer_fwd(cfg, X, gamma, beta, Wq, Wk, Wv, Wo, bq=None, bk=None, bv=None, bo
     Q = Xn @ Wq + (bq if bq is not None else 0.0)
     K = Xn @ Wk + (bk if bk is not None else 0.0)
     V = Xn @ Wv + (bv if bv is not None else 0.0)
+    if getattr(cfg, "rope_base", 0.0) > 0.0:       # optional step 2b: Q and K rotated by position; `saved` holds the rotated ones
+        Q, K = rope(Q, Hq, cfg.rope_base), rope(K, Hkv, cfg.rope_base)
     A = np.zeros((B, T, Hq * hd))
     LSE = np.zeros((B, Hq, T))
     for b in range(B):
@@ -131,6 +152,11 @@ def layer_bwd(cfg, dY, X, gamma, Wq, Wk, Wv, Wo, saved):
             dK[b, :, ks] += cfg.scale * (dS.T @ q)
             Dvec[b, h] = Di
 
+    # optional step 7b: back through the rotation of Q and K (an orthogonal map: its transpose is the inverse rotation)
+    dQ_rot, dK_rot = dQ, dK
+    if getattr(cfg, "rope_base", 0.0) > 0.0:
+        dQ, dK = rope(dQ, Hq, cfg.rope_base, inverse=True), rope(dK, Hkv, cfg.rope_base, inverse=True)
+
     # step 8
     dWq = flat(Xn).T @ flat(dQ)
     dWk = flat(Xn).T @ flat(dK)
@@ -150,7 +176,7 @@ def layer_bwd(cfg, dY, X, gamma, Wq, Wk, Wv, Wo, saved):
     if cfg.residual:
         dX = dX + dY
     out = dict(dX=dX, dWq=dWq, dWk=dWk, dWv=dWv, dWo=dWo, dgamma=dgamma,
-               dA=dA, dQ=dQ, dK=dK, dV=dV, dXn=dXn, D=Dvec)
+               dA=dA, dQ=dQ, dK=dK, dV=dV, dXn=dXn, D=Dvec, dQ_rot=dQ_rot, dK_rot=dK_rot)
     if cfg.norm == "layernorm":
         out["dbeta"] = dbeta
     out.update(dbq=dbq, dbk=dbk, dbv=dbv, dbo=dbo)   # defined with or without biases in the layer

@@ -295,3 +295,52 @@ def test_oracle_matches_its_committed_fixture():
         assert s[:3] == f[:3]
         a, b = np.array(s[3:], dtype=np.float64), np.array(f[3:], dtype=np.float64)
         assert np.allclose(a, b, rtol=1e-12, atol=1e-14), (s[0], s[1])
+
+
+def test_rope_is_a_position_dependent_rotation():
+    # identity at position 0; norm-preserving; inverse undoes it; a textbook 2-D rotation for head_dim 2
+    rng = np.random.default_rng(0)
+    x = rng.normal(size=(2, 5, 12))
+    y = orc.rope(x, 3, 10000.0)
+    assert np.array_equal(y[:, 0], x[:, 0])
+    assert np.abs(np.linalg.norm(y.reshape(2, 5, 3, 4), axis=-1) - np.linalg.norm(x.reshape(2, 5, 3, 4), axis=-1)).max() < 1e-12
+    assert np.abs(orc.rope(y, 3, 10000.0, inverse=True) - x).max() < 1e-12
+    z = orc.rope(np.array([[[1.0, 0.0], [1.0, 0.0], [0.0, 1.0]]]), 1, 10000.0)          # hd = 2: one pair, angle = t
+    assert np.abs(z[0, 1] - [np.cos(1.0), np.sin(1.0)]).max() < 1e-15
+    assert np.abs(z[0, 2] - [-np.sin(2.0), np.cos(2.0)]).max() < 1e-15
+    # frequencies: pair i of an 8-wide head turns by t * base^(-2i/8)
+    e = np.zeros((1, 4, 8)); e[0, :, 1] = 1.0
+    w = orc.rope(e, 1, 100.0)
+    assert np.abs(w[0, 3, 1] - np.cos(3 * 100.0 ** (-2 / 8))) < 1e-15 and np.abs(w[0, 3, 5] - np.sin(3 * 100.0 ** (-2 / 8))) < 1e-15
+
+
+def test_rope_scores_depend_on_relative_position_only():
+    # q_i . k_j after rotation depends on i - j: shifting every position by a constant leaves the scores unchanged
+    rng = np.random.default_rng(1)
+    q, k = rng.normal(size=(1, 6, 8)), rng.normal(size=(1, 6, 8))
+    s0 = orc.rope(q, 2, 50.0).reshape(6, 2, 4).transpose(1, 0, 2) @ orc.rope(k, 2, 50.0).reshape(6, 2, 4).transpose(1, 2, 0)
+    s7 = orc.rope(q, 2, 50.0, pos_offset=7).reshape(6, 2, 4).transpose(1, 0, 2) @ orc.rope(k, 2, 50.0, pos_offset=7).reshape(6, 2, 4).transpose(1, 2, 0)
+    assert np.abs(s0 - s7).max() < 1e-12
+
+
+@pytest.mark.parametrize("kw", [dict(norm="rmsnorm", causal=True, hq=4, hkv=2), dict(norm="layernorm", causal=False, hq=2, hkv=2, residual=True)])
+def test_finite_differences_with_rope(kw):
+    cfg = scaled_config(LayerConfig("tiny-rope", 2, 7, 12, kw["hq"], kw["hkv"], 4, "fp32", kw["norm"], kw["causal"], True,
+                                    kw.get("residual", False), 1e-5, 13, 0.3), d_model=kw["hq"] * 4, rope_base=100.0)
+    inp = big_inputs(cfg)
+    _, _, g = orc.layer_fwd_bwd(cfg, inp)
+    names = {"X": "dX", "Wq": "dWq", "Wk": "dWk", "Wv": "dWv", "Wo": "dWo", "gamma": "dgamma", "bq": "dbq", "bk": "dbk"}
+    h = 1e-6
+    for pname, gname in names.items():
+        flat, got = inp[pname].reshape(-1), g[gname].reshape(-1)
+        scale = np.abs(got).max() + 1e-3
+        for i in range(0, flat.size, 3):
+            keep = flat[i]
+            flat[i] = keep + h
+            lp = loss(cfg, inp)
+            flat[i] = keep - h
+            lm = loss(cfg, inp)
+            flat[i] = keep
+            assert abs((lp - lm) / (2 * h) - got[i]) <= 3e-6 * scale, (pname, i)
+    # with the rotation in place the key bias no longer cancels: dbk is a real gradient now
+    assert np.abs(g["dbk"]).max() > 1e-6
