@@ -356,6 +356,14 @@ int64_t fbl_tile_chain_tiles(const fbl_tile_chain* chain);                      
 int fbl_tile_chain_terms(const fbl_tile_chain* chain, fbl_tile_term* terms, int max_terms);   /* returns the count */
 int fbl_tile_chain_map(const fbl_tile_chain* chain, int64_t src_tile, int64_t* dst_tile);     /* evaluates f */
 
+/* Rotary position embedding on Q and K (an element-wise, position-dependent rotation between the projections and the
+ * scores: in the paper's classification a layout-independent operator, so it runs in place on the R-Tile buffers
+ * without any conversion).  Half-split pairing: inside every head element i < head_dim/2 is paired with element
+ * i + head_dim/2 and the pair of token t turns by t * base^(-2i/head_dim).  `saved` then holds the rotated Q and K;
+ * the backward rotates dQ and dK by the opposite angle before the weight-gradient and input-gradient products.
+ * base > 1 (10000 is customary); head_dim a multiple of 16.  Applies to fbl_layer_fwd / bwd and their _lora forms. */
+int fbl_plan_enable_rope(fbl_plan* plan, float base);
+
 /* Kernel family used by later calls on this plan: 0 = default (tcgen05 tensor-core kernels for bf16
  * wherever one exists for the shape, FFMA kernels for fp32), 1 = FFMA kernels only (fp32 arithmetic on
  * the same layout; lets a caller cross-check the tensor-core path on the device). */

@@ -66,6 +66,7 @@ def load_library():
     L.fbl_colsum_noalloc.argtypes = [vp, vp, i64, i64, vp, vp]
     L.fbl_status_poll.argtypes = [vp, vp, C.POINTER(i32)]
     L.fbl_plan_set_kernel_path.argtypes = [vp, C.c_int]
+    L.fbl_plan_enable_rope.argtypes = [vp, C.c_float]
     L.fbl_profile_enable.argtypes = [vp, C.c_int]
     L.fbl_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_char_p), C.POINTER(C.c_float)]
     L.fbl_launch_count.argtypes = [vp]
@@ -245,6 +246,8 @@ class LayerRunner:
         if tile_choices:
             rtile.apply(self.plan, tile_choices)
         self.tdtype = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
+        if getattr(cfg, "rope_base", 0.0) > 0.0:
+            _check(lib().fbl_plan_enable_rope(self.plan._h, cfg.rope_base))
         if _before_sizes is not None:
             _before_sizes(self.plan)          # a subclass's plan options that change the work areas
         saved, sf, sb = self.plan.workspace_bytes()

@@ -226,6 +226,12 @@ int fbl_plan_set_gemm_choice(fbl_plan* plan, int launch_id, int tile_n, int cta_
   return FBL_OK;
 }
 
+int fbl_plan_enable_rope(fbl_plan* plan, float base) {
+  if (!plan || !(base > 1.f) || plan->d.head_dim % 16 != 0) return FBL_ERR_INVALID_ARG;
+  plan->rope_base = base;
+  return FBL_OK;
+}
+
 int fbl_plan_set_kernel_path(fbl_plan* plan, int path) {
   if (!plan || (path != 0 && path != 1)) return FBL_ERR_INVALID_ARG;
   plan->use_tc = (path == 0 && plan->d.dtype == FBL_DTYPE_BF16) ? 1 : 0;
@@ -410,6 +416,7 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
         FBL_STEP(i == 0 ? "proj_q" : i == 1 ? "proj_k" : "proj_v", 1, launch_gemm_simt(p->d.dtype, gs[i], st));
     }
   }
+  if (p->rope_base > 0.f) FBL_STEP("rope", 1, launch_rope(p, Q, p->d.n_q_heads, K, p->d.n_kv_heads, 0, st));
   if (p->use_tc && attn_fwd_tc_supported(p)) FBL_STEP("attn_fwd", 1, launch_attn_fwd_tc(p, Q, K, V, A, lse, status, st));
   else FBL_STEP("attn_fwd", 1, launch_attn_fwd_simt(p, Q, K, V, A, lse, st));
   {
@@ -501,6 +508,8 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
   }
   if (p->use_tc && attn_bwd_tc_supported(p)) FBL_STEP("attn_bwd", dvec_ready ? 2 : 3, launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, dvec_ready, status, st));   // dqacc: zero already
   else FBL_STEP("attn_bwd", 3, launch_attn_bwd_simt(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, st));
+  // back through the rotation of Q and K: its transpose is the rotation by the opposite angle
+  if (p->rope_base > 0.f) FBL_STEP("rope_bwd", 1, launch_rope(p, dQ, p->d.n_q_heads, dK, p->d.n_kv_heads, 1, st));
   {
     const void* G[3] = {dQ, dK, dV};
     void* DW[3] = {dWq, dWk, dWv};

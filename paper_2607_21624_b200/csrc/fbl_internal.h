@@ -57,6 +57,7 @@ struct fbl_plan {
   int knob_fwd_tiles;       // 0 by sequence length, 1 / 2 query tiles per forward-attention block at head_dim 64
   // low-rank adapters on Q, K, V (fbl_plan_enable_lora): rank, and the offsets of T = Xn [Aq|Ak|Av] inside `saved`,
   // of dT and of the unused norm-parameter gradients inside the backward scratch
+  float rope_base;          // > 0: rotary position embedding on Q and K (fbl_plan_enable_rope)
   int lora_rank;
   size_t sv_t, sb_dt, sb_frozen;
   // Compute-tile configuration of each GEMM launch of a step, fixed offline by the tile chooser (0 / -1: the
@@ -112,6 +113,7 @@ void fbl_note_cuda_error(cudaError_t e, const char* where);
 
 cudaError_t launch_pack(int dtype, int unpack, const void* src, void* dst, int64_t outer, int64_t rows,
                         int64_t rows_pad, int cols, cudaStream_t st);
+cudaError_t launch_rope(const fbl_plan* p, void* A, int heads_a, void* B, int heads_b, int inverse, cudaStream_t st);
 bool norm_fwd_resets_status(const fbl_plan* p);   // the forward norm kernel for this plan zeroes the status word itself
 cudaError_t launch_norm_fwd(const fbl_plan* p, const void* X, const float* gamma, const float* beta, void* Xn,
                             float* stats, int32_t* status, cudaStream_t st);

@@ -2,6 +2,8 @@
 // Thread mapping shared by all of them: 8 consecutive lanes cover one 128-byte tile row with one
 // 16-byte vector each, 4 rows per warp are 512 contiguous bytes, so every warp-level access is a
 // run of whole 128-byte lines.
+#include <math.h>
+
 #include "fbl_internal.h"
 #include "pdl.cuh"
 
@@ -334,6 +336,55 @@ __global__ void __launch_bounds__(256, 2) norm_fwd_rows_kernel(const __nv_bfloat
       }
       r += stride;
     }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Rotary position embedding, in place, on two R-Tile matrices at once (Q and K forward; dQ and dK backward with the
+// opposite angle).  Half-split pairing: inside a head, element i < hd/2 goes with element i + hd/2, and the pair of
+// token t turns by t * base^(-2i/hd).  A thread takes 16 bytes of the low half and the matching 16 bytes of the
+// high half (the same row of the same or of the neighbouring 128-byte panel).
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) rope_kernel(T* __restrict__ A, int heads_a, T* __restrict__ B, int heads_b,
+                                                   int64_t n_pad, int seq, int t_pad, int hd, float neg2_log2_base_over_hd,
+                                                   float sign) {
+  constexpr int TW = tile_w_of<T>::value;
+  constexpr int V = Vec16<T>::N;
+  pdl_launch_dependents();
+  pdl_wait();
+  const int half = hd / 2, vec_per_head = half / V;
+  const int64_t per_a = n_pad * heads_a * vec_per_head, total = per_a + n_pad * heads_b * vec_per_head;
+  for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const bool second = idx >= per_a;
+    T* M = second ? B : A;
+    const int heads = second ? heads_b : heads_a;
+    int64_t rem = second ? idx - per_a : idx;
+    // consecutive threads: consecutive vectors of a row's half-head, then rows (whole 128-byte pieces per warp quarter)
+    const int v = (int)(rem % vec_per_head);
+    rem /= vec_per_head;
+    const int64_t r = rem % n_pad;
+    const int h = (int)(rem / n_pad);
+    const int t = (int)(r % t_pad);
+    if (t >= seq) continue;                                     // padding rows hold zeros and stay zero
+    const int c_lo = h * hd + v * V, c_hi = c_lo + half;
+    T* plo = M + rt_off<TW>(n_pad, r, c_lo);
+    T* phi = M + rt_off<TW>(n_pad, r, c_hi);
+    float lo[V], hi[V];
+    load16(plo, lo);
+    load16(phi, hi);
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      const float inv_freq = exp2f((float)(v * V + i) * neg2_log2_base_over_hd);
+      float sn, cs;
+      sincosf((float)t * inv_freq, &sn, &cs);
+      sn *= sign;
+      const float a = lo[i], b = hi[i];
+      lo[i] = a * cs - b * sn;
+      hi[i] = b * cs + a * sn;
+    }
+    store16(plo, lo);
+    store16(phi, hi);
   }
 }
 
@@ -686,6 +737,19 @@ cudaError_t launch_pack(int dtype, int unpack, const void* src, void* dst, int64
     else pack_kernel<B><<<blocks, 256, 0, st>>>((const B*)src, (B*)dst, outer, rows, rows_pad, cols, total);
   }
   return cudaGetLastError();
+}
+
+cudaError_t launch_rope(const fbl_plan* p, void* A, int heads_a, void* B, int heads_b, int inverse, cudaStream_t st) {
+  const int hd = p->d.head_dim;
+  const float k = -2.f * log2f(p->rope_base) / (float)hd;
+  const int vec = p->d.dtype == FBL_DTYPE_FP32 ? 4 : 8;
+  const int64_t total = p->n_pad * (int64_t)(heads_a + heads_b) * (hd / 2 / vec);
+  const int blocks = (int)min((int64_t)p->sm_count * 16, (total + 255) / 256);
+  if (p->d.dtype == FBL_DTYPE_FP32)
+    return launch_pdl(rope_kernel<float>, dim3(blocks), dim3(256), 0, st, (float*)A, heads_a, (float*)B, heads_b, p->n_pad,
+                      p->d.seq, p->t_pad, hd, k, inverse ? -1.f : 1.f);
+  return launch_pdl(rope_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, (__nv_bfloat16*)A, heads_a,
+                    (__nv_bfloat16*)B, heads_b, p->n_pad, p->d.seq, p->t_pad, hd, k, inverse ? -1.f : 1.f);
 }
 
 bool norm_fwd_resets_status(const fbl_plan* p) {

@@ -176,6 +176,7 @@ int fbl_layer_fwd_lora(const fbl_plan* p, const void* X, const float* gamma, con
     LORA_STEP("proj_qkv", 0, cudaSuccess);
     p->launches += k;
   }
+  if (p->rope_base > 0.f) LORA_STEP("rope", 1, launch_rope(p, Q, p->d.n_q_heads, K, p->d.n_kv_heads, 0, st));
   if (p->use_tc && attn_fwd_tc_supported(p)) LORA_STEP("attn_fwd", 1, launch_attn_fwd_tc(p, Q, K, V, A, lse, status, st));
   else LORA_STEP("attn_fwd", 1, launch_attn_fwd_simt(p, Q, K, V, A, lse, st));
   {
@@ -239,6 +240,7 @@ int fbl_layer_bwd_lora(const fbl_plan* p, const void* dY, const void* X, const f
   }
   if (p->use_tc && attn_bwd_tc_supported(p)) LORA_STEP("attn_bwd", dvec_ready ? 2 : 3, launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, dvec_ready, status, st));
   else LORA_STEP("attn_bwd", 3, launch_attn_bwd_simt(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, st));
+  if (p->rope_base > 0.f) LORA_STEP("rope_bwd", 1, launch_rope(p, dQ, p->d.n_q_heads, dK, p->d.n_kv_heads, 1, st));
   const void* G[3] = {dQ, dK, dV};
   {
     GemmArgs g = {};                       // dT = dQ Bq^T | dK Bk^T | dV Bv^T: B_all's column blocks read with swapped axes;

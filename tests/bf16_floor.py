@@ -36,6 +36,9 @@ def emulate(cfg, inp):
     Xn_exact, xhat, rstd, mu = orc.norm_fwd(X, inp["gamma"], inp["beta"], cfg.eps, cfg.norm)
     Xn = r16(Xn_exact)
     Q, K, V = r16(Xn @ Wq + z(inp["bq"])), r16(Xn @ Wk + z(inp["bk"])), r16(Xn @ Wv + z(inp["bv"]))
+    rope_base = getattr(cfg, "rope_base", 0.0)
+    if rope_base > 0.0:               # rotated in place: read as bf16, written as bf16
+        Q, K = r16(orc.rope(Q, Hq, rope_base)), r16(orc.rope(K, cfg.n_kv_heads, rope_base))
     A = np.zeros((B, T, Hq * hd))
     LSE = np.zeros((B, Hq, T))
     mask = np.tril(np.ones((T, T), dtype=bool)) if cfg.causal else None
@@ -75,6 +78,8 @@ def emulate(cfg, inp):
             dQ[b, :, qs] = cfg.scale * (dS @ k)
             dK[b, :, ks] += cfg.scale * (dS.T @ q)
     dQ, dK, dV = r16(dQ), r16(dK), r16(dV)
+    if rope_base > 0.0:
+        dQ, dK = r16(orc.rope(dQ, Hq, rope_base, inverse=True)), r16(orc.rope(dK, cfg.n_kv_heads, rope_base, inverse=True))
     out["dWq"], out["dWk"], out["dWv"] = r16(flat(Xn).T @ flat(dQ)), r16(flat(Xn).T @ flat(dK)), r16(flat(Xn).T @ flat(dV))
     out["dbq"], out["dbk"], out["dbv"] = flat(dQ).sum(axis=0), flat(dK).sum(axis=0), flat(dV).sum(axis=0)
     dXn = r16(dQ @ Wq.T + dK @ Wk.T + dV @ Wv.T)

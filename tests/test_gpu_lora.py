@@ -52,6 +52,8 @@ CASES = [
     (LayerConfig("l4", 2, 8, 128, 2, 2, 64, "bf16", "layernorm", True, True, False, 1e-5, 94, 0.02), 4),      # FFMA path
     (LayerConfig("l5", 1, 64, 64, 2, 2, 32, "fp32", "layernorm", True, False, False, 1e-5, 95, 0.1), 8),
     (LayerConfig("l6", 2, 77, 128, 2, 1, 64, "fp32", "rmsnorm", False, True, True, 1e-5, 96, 0.1), 5),
+    # with the rotary embedding between the adapted projections and the scores (the Llama fine-tuning arrangement)
+    (LayerConfig("l8", 2, 300, 256, 4, 2, 64, "bf16", "rmsnorm", True, False, True, 1e-5, 98, 0.02, 0.0, 10000.0), 16),
 ]
 
 

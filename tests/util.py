@@ -49,19 +49,20 @@ def bf16_figures(got, ref):
                 numel=int(ref.size))
 
 
-def bf16_ok(name, got, ref, floor=None):
+def bf16_ok(name, got, ref, floor=None, zero_ref_names=ZERO_REF):
     """Apply the criteria above.  ``floor``: this tensor's entry of bf16_floor.floor_figures for the same layer;
-    None (intermediates, which the floor does not list) applies criteria 1 and 2 only.
+    None (intermediates, which the floor does not list) applies criteria 1 and 2 only.  ``zero_ref_names``: tensors
+    whose reference is identically zero (dbk, unless a rotary embedding sits between the key projection and the scores).
     Returns (ok, figures, list of failed criteria)."""
     f = bf16_figures(got, ref)
     failed = []
-    if name not in ZERO_REF and np.abs(ref).max() < 1e-9:
+    if name not in zero_ref_names and np.abs(ref).max() < 1e-9:
         # a reference that vanishes identically (one token per sequence: dS = 0, hence dQ, dK, dWq, dWk, dbq):
         # only the absolute part of the bound means anything
         if f["max_abs"] > BF16_ATOL:
             failed.append("zero-reference bound")
         return not failed, f, failed
-    if name in ZERO_REF:
+    if name in zero_ref_names:
         bound = max(BF16_ATOL, 2.0 * floor["max_abs"]) if floor is not None else BF16_ATOL
         f["worst_over_bound"] = f["max_abs"] / bound
         if f["max_abs"] > bound:
