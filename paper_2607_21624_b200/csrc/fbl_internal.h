@@ -98,6 +98,10 @@ struct GemmArgs {
   // later kernel of the pass; reset the pass's status word), and `serial`: the launch may not start before
   // everything ahead of it on the stream has completed
   void* zero_ptr; size_t zero_bytes; int reset_status, serial;
+  // fused activation of the feed-forward block (tensor-core kernel only): 0 none, 1 GELU forward (c = U, c2 = gelu(U)),
+  // 2 GELU backward (c = value * gelu'(U), U in `residual`), 3 gated forward (c = G, c2 = silu(G) * U, U in `residual`),
+  // 4 gated backward (c = value * silu(G), c2 = value * U * silu'(G); U in `residual`, G in `aux1`)
+  int epi; const void* aux1; void* c2;
 };
 
 cudaError_t launch_gemm_simt(int dtype, const GemmArgs& g, cudaStream_t st);

@@ -39,6 +39,13 @@ struct alignas(64) TcProblem {
   // later kernel rounds the sums to bf16.  Single-term problems without epilogue extras only.
   int ksplit;
   CUtensorMap tacc;
+  // Fused activation of the feed-forward block (kernel variant EPI only; `residual` then points at the first extra
+  // operand U instead of a residual, `aux1` at the second one, G; `tc2` is the second output's map):
+  //   1 GELU forward    C = v (U), C2 = gelu(v)           2 GELU backward    C = v gelu'(U)
+  //   3 gated forward   C = v (G), C2 = silu(v) U          4 gated backward   C = v silu(G), C2 = v U silu'(G)
+  int epi;
+  const __nv_bfloat16* aux1;
+  CUtensorMap tc2;
 };
 struct alignas(64) TcGroup {
   TcProblem p[MAX_PROBLEMS];
@@ -101,7 +108,19 @@ __device__ __forceinline__ bool tile_at(const TcGroup& G, int w, TileCoord* tc_o
 // shared-memory ring by TMA, warp 1 issues the MMAs into one of two TMEM accumulators, warps 2-5 drain the
 // other accumulator (bias, residual, padding-row mask, bf16 rows in R-Tile order), so the epilogue of
 // one tile overlaps the main loop of the next.
-template <int BN, int STAGES, int ESETS>
+__device__ __forceinline__ float tanh_fast(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float gelu_fast(float u) { return 0.5f * u * (1.f + tanh_fast(0.7978845608028654f * (u + 0.044715f * u * u * u))); }
+__device__ __forceinline__ float gelu_grad_fast(float u) {
+  const float t = tanh_fast(0.7978845608028654f * (u + 0.044715f * u * u * u));
+  return 0.5f * (1.f + t) + 0.5f * u * (1.f - t * t) * 0.7978845608028654f * (1.f + 0.134145f * u * u);
+}
+__device__ __forceinline__ float sigmoid_fast(float g) { return __fdividef(1.f, 1.f + __expf(-g)); }
+
+template <int BN, int STAGES, int ESETS, bool EPI = false>
 __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __grid_constant__ TcGroup G) {
   using SP = SmemPlan<BN, STAGES>;
   extern __shared__ uint8_t smem_raw[];
@@ -254,6 +273,14 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
 #pragma unroll
         for (int j = 0; j < 8; ++j) rv[j] = *reinterpret_cast<const uint4*>(rp + 8 * j);
       }
+      uint4 rv2[EPI ? 8 : 1];                         // second extra operand of a fused activation, likewise
+      if constexpr (EPI) {
+        if (P.epi == 4 && row < P.m && pn_begin < pn_end && tcd.n0 + pn_begin * 64 < P.n) {
+          const __nv_bfloat16* rp = P.aux1 + ((long long)(tcd.n0 / 64 + pn_begin) * P.c_rpad + row) * 64;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) rv2[j] = *reinterpret_cast<const uint4*>(rp + 8 * j);
+        }
+      }
       const float* bias = P.bias;
       float bl[BN / 32];                              // this tile's bias: lane l holds columns l*BN/32 ... (requested
       if (bias) {                                     // while the MMAs run, handed out by shuffles below)
@@ -297,6 +324,92 @@ __global__ void __launch_bounds__(64 + 128 * ESETS, 1) gemm_tc_kernel(const __gr
             ++pc;
           }
           continue;
+        }
+        if constexpr (EPI) {
+          if (P.epi != 0) {
+            // ---- fused activation: one or two outputs from this panel ------------------------------------
+            if (bias) {
+#pragma unroll
+              for (int j = 0; j < 64; ++j)
+                v[j] = __float_as_uint(__uint_as_float(v[j]) + __shfl_sync(0xffffffffu, bl[j % (BN / 32)], (pn * 64 + j) / (BN / 32)));
+            }
+            uint4 o1[8], o2[8];
+            uint32_t* w1 = reinterpret_cast<uint32_t*>(o1);
+            uint32_t* w2 = reinterpret_cast<uint32_t*>(o2);
+            const bool live = !pad && row < P.m;
+            const __nv_bfloat16* a0 = reinterpret_cast<const __nv_bfloat16*>(rv);
+            const __nv_bfloat16* a1 = reinterpret_cast<const __nv_bfloat16*>(rv2);
+            const float keep = live ? 1.f : 0.f;            // padding rows and rows past the matrix are written as zero
+            if (P.epi == 1) {
+#pragma unroll
+              for (int j = 0; j < 64; j += 2) {
+                const float x0 = __uint_as_float(v[j]) * keep, x1 = __uint_as_float(v[j + 1]) * keep;
+                w1[j / 2] = tc::pack_bf16(x0, x1);
+                w2[j / 2] = tc::pack_bf16(gelu_fast(x0), gelu_fast(x1));
+              }
+            } else if (P.epi == 2) {
+#pragma unroll
+              for (int j = 0; j < 64; j += 2) {
+                const float x0 = __uint_as_float(v[j]) * keep, x1 = __uint_as_float(v[j + 1]) * keep;
+                w1[j / 2] = tc::pack_bf16(x0 * gelu_grad_fast(__bfloat162float(a0[j])), x1 * gelu_grad_fast(__bfloat162float(a0[j + 1])));
+              }
+            } else if (P.epi == 3) {
+#pragma unroll
+              for (int j = 0; j < 64; j += 2) {
+                const float x0 = __uint_as_float(v[j]) * keep, x1 = __uint_as_float(v[j + 1]) * keep;
+                w1[j / 2] = tc::pack_bf16(x0, x1);
+                w2[j / 2] = tc::pack_bf16(x0 * sigmoid_fast(x0) * __bfloat162float(a0[j]), x1 * sigmoid_fast(x1) * __bfloat162float(a0[j + 1]));
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 64; j += 2) {
+                float y1[2], y2[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                  const float x = __uint_as_float(v[j + u]) * keep;
+                  const float uu = __bfloat162float(a0[j + u]), gg = __bfloat162float(a1[j + u]), sg = sigmoid_fast(gg);
+                  y1[u] = x * gg * sg;
+                  y2[u] = x * uu * sg * (1.f + gg * (1.f - sg));
+                }
+                w1[j / 2] = tc::pack_bf16(y1[0], y1[1]);
+                w2[j / 2] = tc::pack_bf16(y2[0], y2[1]);
+              }
+            }
+            // the next panel's extra operands, requested while this panel's stores are under way
+            if (pn + 1 < pn_end && n + 64 < P.n && row < P.m) {
+              if (P.epi >= 2) {
+                const __nv_bfloat16* rp = P.residual + ((long long)(n / 64 + 1) * P.c_rpad + row) * 64;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) rv[j] = *reinterpret_cast<const uint4*>(rp + 8 * j);
+              }
+              if (P.epi == 4) {
+                const __nv_bfloat16* rp = P.aux1 + ((long long)(n / 64 + 1) * P.c_rpad + row) * 64;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) rv2[j] = *reinterpret_cast<const uint4*>(rp + 8 * j);
+              }
+            }
+            const int n_out = (P.epi == 2) ? 1 : 2;
+#pragma unroll 1
+            for (int oi = 0; oi < n_out; ++oi) {
+              const uint4* ov = oi ? o2 : o1;
+              const uint32_t stg = base + SP::STG_OFF + (ESETS == 2 ? (uint32_t)(warp - 2) : (uint32_t)(q * 2 + (pc & 1))) * 4096u;
+              if (ESETS == 2 && lane == 0) tc::bulk_wait_group_read0();
+              __syncwarp();
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + (((uint32_t)j ^ (uint32_t)(lane & 7)) * 16)),
+                             "r"(ov[j].x), "r"(ov[j].y), "r"(ov[j].z), "r"(ov[j].w) : "memory");
+              tc::fence_proxy_async();
+              __syncwarp();
+              if (lane == 0) {
+                tc::tma_store_3d(oi ? &P.tc2 : &P.tc, stg, 0, tcd.m0 + q * 32, n / 64);
+                tc::bulk_commit_group();
+                if (ESETS == 1) tc::bulk_wait_group_read1();
+              }
+              ++pc;
+            }
+            continue;
+          }
         }
         uint4 outv[8];
         uint32_t* ow = reinterpret_cast<uint32_t*>(outv);
@@ -765,6 +878,13 @@ cudaError_t fill_group(TcGroup& G, const GemmArgs* gs, int count, int32_t* statu
     P.bias = g.bias; P.residual = (const __nv_bfloat16*)g.residual;
     P.seq = g.seq; P.t_pad = g.t_pad;
     P.dot_with = (const __nv_bfloat16*)g.dot_with; P.dot_out = g.dot_out; P.dot_hd = g.dot_hd; P.dot_hq = g.dot_hq;
+    P.epi = g.epi; P.aux1 = (const __nv_bfloat16*)g.aux1;
+    if (g.epi != 0) {
+      if (g.epi < 1 || g.epi > 4 || g.ksplit > 1 || g.dot_with || (g.epi >= 2 && !g.residual) || (g.epi == 4 && !g.aux1) ||
+          (g.epi != 2 && !g.c2))
+        return cudaErrorInvalidValue;
+      if (g.epi != 2 && !fbl_encode_rtile_map(&P.tc2, g.c2, g.c_rpad, g.n / 64, 32, 1)) return cudaErrorInvalidValue;
+    }
     P.ksplit = 1;
     if (g.ksplit > 1) {
       if (g.n_terms != 1 || g.bias || g.residual || g.dot_with || g.t_pad > 0 || !g.acc) return cudaErrorInvalidValue;
@@ -790,6 +910,20 @@ cudaError_t launch_group_bn(const fbl_plan* p, const GemmArgs* gs, int count, in
   // (with several tiles per block the epilogues overlap the next main loops and the extra warps only cost)
   const int esets_knob = esets_choice ? esets_choice : p->knob_gemm_esets;
   const bool two_sets = esets_knob ? esets_knob == 2 : tiles <= p->sm_count;
+  bool epi = false;
+  for (int i = 0; i < count; ++i) epi = epi || gs[i].epi != 0;
+  if (epi) {                       // the variant with the fused activations (feed-forward block only)
+    if (two_sets) {
+      auto k = gemm_tc_kernel<BN, STAGES, 2, true>;
+      cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
+      if (attr_err != cudaSuccess) return attr_err;
+      return launch_pdl(k, dim3(grid), dim3(320), SP::TOTAL, st, G);
+    }
+    auto k = gemm_tc_kernel<BN, STAGES, 1, true>;
+    cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
+    if (attr_err != cudaSuccess) return attr_err;
+    return launch_pdl(k, dim3(grid), dim3(192), SP::TOTAL, st, G);
+  }
   if (two_sets) {
     auto k = gemm_tc_kernel<BN, STAGES, 2>;
     cudaError_t attr_err = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SP::TOTAL);
@@ -836,12 +970,14 @@ cudaError_t launch_gemm_tc_group(const fbl_plan* p, const GemmArgs* gs, int coun
   if (wide && tiles_wide * 3 < p->sm_count * 2) wide = false;
   // CTA pairs on 256 x 256 tiles for large problems (several rounds of tiles per SM pair): measured 2-6 % faster
   // on the workload 5 GEMMs, no gain or a loss below that
+  bool any_epi = false;
+  for (int i = 0; i < count; ++i) any_epi = any_epi || gs[i].epi != 0;
   // an offline choice for this launch overrides the heuristics below wherever its tile shape is legal
   if (ch.bn == 128) wide = false;
   else if (ch.bn == 256 && wide_legal) wide = true;
   const int pair_mode = ch.pair >= 0 ? ch.pair : p->knob_gemm_pair;       // 0 never, 1 whenever legal, -1 by size
-  if (pair_mode == 1 && wide_legal) return launch_group_pair(p, gs, count, status, st);
-  if (wide && pair_mode != 0) {
+  if (pair_mode == 1 && wide_legal && !any_epi) return launch_group_pair(p, gs, count, status, st);
+  if (wide && pair_mode != 0 && !any_epi) {
     long long pair_tiles = 0;
     for (int i = 0; i < count; ++i)
       pair_tiles += (long long)((gs[i].m + 255) / 256) * (gs[i].n / 256) * (gs[i].ksplit > 1 ? gs[i].ksplit : 1);

@@ -320,6 +320,7 @@ int fbl_mlp_fwd(const fbl_mlp_plan* p, const void* X, const float* gamma, const 
     GemmArgs gs[2];
     const void* W[2] = {W1, Wg}; void* O[2] = {U, G}; const float* B[2] = {b1, bg};
     const int cnt = gated ? 2 : 1;
+    bool tc = bp->use_tc != 0;
     for (int i = 0; i < cnt; ++i) {
       GemmArgs& g = gs[i];
       g = GemmArgs{};
@@ -328,12 +329,27 @@ int fbl_mlp_fwd(const fbl_mlp_plan* p, const void* X, const float* gamma, const 
       g.b_static = 1;
       g.c = O[i]; g.c_rpad = p->n_pad; g.bias = bias ? B[i] : nullptr;
       g.seq = p->d.seq; g.t_pad = bp->t_pad;
+      tc = tc && gemm_tc_supported(bp, g);
     }
     int k = 0;
-    MLP_CUDA(run_group(p, gs, cnt, status, st, &k));
-    p->launches += k;
+    if (tc && !gated) {
+      // the activation rides in the up projection's epilogue: U and H = gelu(U) leave the same accumulator tile
+      gs[0].epi = 1; gs[0].c2 = H;
+      MLP_CUDA(run_group(p, gs, 1, status, st, &k));
+      p->launches += k;
+    } else if (tc) {
+      // gated: U first, then the gate projection, whose epilogue reads U's tile and writes G and H = silu(G) * U
+      MLP_CUDA(run_group(p, &gs[0], 1, status, st, &k));
+      p->launches += k;
+      gs[1].epi = 3; gs[1].residual = U; gs[1].c2 = H;
+      MLP_CUDA(run_group(p, &gs[1], 1, status, st, &k));
+      p->launches += k;
+    } else {
+      MLP_CUDA(run_group(p, gs, cnt, status, st, &k));
+      p->launches += k;
+      MLP_STEP(1, act(p, false, nullptr, U, G, H, nullptr, st));
+    }
   }
-  MLP_STEP(1, act(p, false, nullptr, U, G, H, nullptr, st));
   {
     GemmArgs g = {};
     g.m = n; g.n = D; g.n_terms = 1;
@@ -393,10 +409,18 @@ int fbl_mlp_bwd(const fbl_mlp_plan* p, const void* dY, const void* X, const floa
       cg.src[cg.count] = gw.acc; cg.dst[cg.count] = dW2; cg.n[cg.count] = up8(F) * (int64_t)D; cg.count++;
     }
     int k = 0;
-    MLP_CUDA(run_group(p, gs, 2, status, st, &k));
-    p->launches += k;
+    if (both_tc) {
+      // the activation's derivative rides in the dH product's epilogue: dU (and dG) leave the accumulator tile, dH
+      // itself is never stored
+      gh.epi = gated ? 4 : 2; gh.residual = U; gh.aux1 = gated ? G : nullptr; gh.c = dU; gh.c2 = gated ? dG : nullptr;
+      MLP_CUDA(run_group(p, gs, 2, status, st, &k));
+      p->launches += k;
+    } else {
+      MLP_CUDA(run_group(p, gs, 2, status, st, &k));
+      p->launches += k;
+      MLP_STEP(1, act(p, true, dH, U, G, dU, dG, st));
+    }
   }
-  MLP_STEP(1, act(p, true, dH, U, G, dU, dG, st));
   {
     GemmArgs gs[3];
     const void* Gr[2] = {dU, dG}; void* DW[2] = {dW1, dWg};
