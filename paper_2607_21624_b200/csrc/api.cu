@@ -572,7 +572,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
     return FBL_OK;
   }
   if (bias) FBL_STEP("db", 2, launch_colsum_group(p->d.dtype, 4, M4, p->n_pad, C4, O4, (float*)part, st));
-  FBL_STEP("norm_bwd", 2, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, (float*)part, st));
+  FBL_STEP("norm_bwd", norm_bwd_takes_colsums(p) ? 2 : 1, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, (float*)part, st));
   return FBL_OK;
 }
 

@@ -281,7 +281,7 @@ int fbl_layer_bwd_lora(const fbl_plan* p, const void* dY, const void* X, const f
     LORA_STEP("lora_dA", 0, cudaSuccess);
     p->launches += k;
   }
-  LORA_STEP("norm_bwd", 2, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, part, st));
+  LORA_STEP("norm_bwd", norm_bwd_takes_colsums(p) ? 2 : 1, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, part, st));
   return FBL_OK;
 }
 

@@ -465,7 +465,7 @@ int fbl_mlp_bwd(const fbl_mlp_plan* p, const void* dY, const void* X, const floa
     return FBL_OK;
   }
   if (bias) MLP_STEP(2, launch_colsum_group(p->d.dtype, nb, M3, p->n_pad, C3, O3, part, st));
-  MLP_STEP(2, launch_norm_bwd(bp, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, part, st));
+  MLP_STEP(norm_bwd_takes_colsums(bp) ? 2 : 1, launch_norm_bwd(bp, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, part, st));
   return FBL_OK;
 }
 
