@@ -126,3 +126,66 @@ MLP_CONFIGS = {
     # GPT-2-small-shaped block (d_ff = 3072) behind the attention layer of workload 2
     "gpt2": MlpConfig("mlp-gpt2-small-gelu", 4, 512, 768, 3072, "bf16", "layernorm", "gelu", True, True, 1e-5, 13, 0.02),
 }
+
+
+@dataclass(frozen=True)
+class XattnConfig:
+    """A pre-norm cross-attention layer: queries from the normalised hidden states X [batch, seq, d_model], keys
+    and values from a memory M [batch, seq_kv, d_mem] (an encoder's output, used as it is), no mask."""
+    name: str
+    batch: int
+    seq: int            # query tokens per sequence
+    seq_kv: int         # memory tokens per sequence
+    d_model: int
+    d_mem: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    dtype: str
+    norm: str
+    has_bias: bool
+    residual: bool
+    eps: float
+    seed: int
+    w_std: float
+    softmax_scale: float = 0.0
+    causal: bool = False          # a memory position has no order relative to a query: never masked
+    rope_base: float = 0.0
+
+    @property
+    def n_tokens(self) -> int:
+        return self.batch * self.seq
+
+    @property
+    def d_q(self) -> int:
+        return self.n_q_heads * self.head_dim
+
+    @property
+    def d_kv(self) -> int:
+        return self.n_kv_heads * self.head_dim
+
+    @property
+    def group(self) -> int:
+        return self.n_q_heads // self.n_kv_heads
+
+    @property
+    def scale(self) -> float:
+        return self.softmax_scale if self.softmax_scale > 0 else self.head_dim ** -0.5
+
+    def flops(self) -> float:
+        """Algorithmic forward+backward flops: every projection once forward and twice backward, the two attention
+        products once forward and four times backward (dV, dP, dQ, dK)."""
+        nq, nk = self.batch * self.seq, self.batch * self.seq_kv
+        proj = 2.0 * nq * self.d_model * self.d_q * 2 + 2.0 * nk * self.d_mem * self.d_kv * 2
+        one_gemm = 2.0 * self.batch * self.n_q_heads * self.seq * self.seq_kv * self.head_dim
+        return 3.0 * proj + 6.0 * one_gemm
+
+
+XATTN_CONFIGS = {
+    # Whisper-large-shaped decoder cross-attention (the paper's model table: Whisper-Large, batch 2): 20 heads of 64
+    # over d_model 1280; 1500 encoder positions stand for 30 s of audio, 448 is the decoder's token limit
+    "whisper-large": XattnConfig("xattn-whisper-large", 2, 448, 1500, 1280, 1280, 20, 20, 64, "bf16", "layernorm",
+                                 True, True, 1e-5, 21, 0.02),
+    # a small ragged case the oracle finishes in well under a second
+    "tiny": XattnConfig("xattn-tiny-fp32", 2, 37, 75, 64, 96, 2, 1, 32, "fp32", "layernorm", True, True, 1e-5, 22, 0.05),
+}

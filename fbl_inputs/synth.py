@@ -16,6 +16,7 @@ TENSOR_IDS = {
     "bq": 5, "bk": 6, "bv": 7, "bo": 8, "gamma": 9, "beta": 10, "dY": 11,
     "W1": 12, "Wg": 13, "W2": 14, "b1": 15, "bg": 16, "b2": 17,
     "Aq": 18, "Ak": 19, "Av": 20, "Bq": 21, "Bk": 22, "Bv": 23,
+    "M": 24,
 }
 
 _M64 = np.uint64(0xFFFFFFFFFFFFFFFF)
@@ -142,4 +143,33 @@ def make_lora_inputs(cfg: LayerConfig, rank: int, *, affine_noise: bool = False,
         b = normal_f64(cfg.seed, TENSOR_IDS["B" + k], 0, rank * cols).reshape(rank, cols) * b_std
         out["A" + k] = round_to_storage(a, cfg.dtype)
         out["B" + k] = round_to_storage(b, cfg.dtype)
+    return out
+
+
+def make_xattn_inputs(cfg, *, affine_noise: bool = False) -> dict:
+    """All inputs of the cross-attention layer ``cfg`` (an ``XattnConfig``): hidden states X and output gradient dY
+    [batch, seq, d_model], memory M [batch, seq_kv, d_mem] ~ N(0, 1); Wq [d_model, d_q], Wk, Wv [d_mem, d_kv],
+    Wo [d_q, d_model] ~ N(0, w_std^2); vectors fp32.  Storage-rounded float64, as ``make_inputs``."""
+    s = cfg.seed
+    d, dm, dq, dkv = cfg.d_model, cfg.d_mem, cfg.d_q, cfg.d_kv
+
+    def mat(name, shape, std):
+        cnt = int(np.prod(shape))
+        return round_to_storage(normal_f64(s, TENSOR_IDS[name], 0, cnt).reshape(shape) * std, cfg.dtype)
+
+    def vec(name, length, std, mean=0.0):
+        return (normal_f64(s, TENSOR_IDS[name], 0, length) * std + mean).astype(np.float32).astype(np.float64)
+
+    out = {"X": mat("X", (cfg.batch, cfg.seq, d), 1.0), "dY": mat("dY", (cfg.batch, cfg.seq, d), 1.0),
+           "M": mat("M", (cfg.batch, cfg.seq_kv, dm), 1.0),
+           "Wq": mat("Wq", (d, dq), cfg.w_std), "Wk": mat("Wk", (dm, dkv), cfg.w_std),
+           "Wv": mat("Wv", (dm, dkv), cfg.w_std), "Wo": mat("Wo", (dq, d), cfg.w_std)}
+    if affine_noise:
+        out["gamma"] = vec("gamma", d, 0.1, 1.0)
+        out["beta"] = vec("beta", d, 0.1) if cfg.norm == "layernorm" else None
+    else:
+        out["gamma"] = np.ones(d)
+        out["beta"] = np.zeros(d) if cfg.norm == "layernorm" else None
+    for k, n in (("bq", dq), ("bk", dkv), ("bv", dkv), ("bo", d)):
+        out[k] = vec(k, n, cfg.w_std) if cfg.has_bias else None
     return out
