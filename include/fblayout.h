@@ -75,6 +75,7 @@ enum {
   FBL_T_XN, FBL_T_Q, FBL_T_K, FBL_T_V, FBL_T_A,      /* [B, T, D | Dq | Dkv | Dkv | Dq] */
   FBL_T_Q_HEADS, FBL_T_K_HEADS, FBL_T_V_HEADS, FBL_T_A_HEADS, /* [B, H, T, hd] views */
   FBL_T_WQ_T, FBL_T_WK_T, FBL_T_WV_T, FBL_T_WO_T,    /* transposed views [C, R] of the weights */
+  FBL_T_MEM, FBL_T_DMEM,                             /* cross-attention plans only: memory [B, Tkv, Dmem] and its gradient */
   FBL_T_COUNT
 };
 
@@ -363,6 +364,34 @@ int fbl_tile_chain_map(const fbl_tile_chain* chain, int64_t src_tile, int64_t* d
  * the backward rotates dQ and dK by the opposite angle before the weight-gradient and input-gradient products.
  * base > 1 (10000 is customary); head_dim a multiple of 16.  Applies to fbl_layer_fwd / bwd and their _lora forms. */
 int fbl_plan_enable_rope(fbl_plan* plan, float base);
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * Cross-attention (section 2 names it beside MHA and GQA among the attention forms whose partitioning the layout has to
+ * serve; Whisper and Stable Diffusion in the model table contain it).  The layer of fbl_layer_fwd with K and V
+ * projected from a second sequence, the memory M [batch, seq_kv, d_mem], used as it is (no norm on it):
+ *     Xn = norm(X);  Q = Xn Wq + bq;  K = M Wk + bk;  V = M Wv + bv;  A = softmax(scale Q K^T) V per head, no mask;
+ *     Y = A Wo + bo (+ X).
+ * The same kernels run it: the attention kernels take the key side's row count and sequence length separately from
+ * the query side's, the projections of the two sides share one grouped launch, and the backward adds dM = dK Wk^T +
+ * dV Wv^T (one accumulator, two reduction loops).  Nothing is transposed or re-partitioned for the second sequence.
+ *
+ * fbl_xattn_plan_create: desc describes the query side (seq = query tokens per sequence; causal must be 0); seq_kv >= 1
+ * memory tokens per sequence; d_mem a multiple of tile_w.  The plan is an fbl_plan: fbl_tensor_bytes / fbl_pack /
+ * fbl_unpack / fbl_tile_offset (K, V, Wk, Wv take the memory's extents; FBL_T_MEM / FBL_T_DMEM are valid),
+ * fbl_workspace_bytes / _offset, fbl_status_poll, fbl_profile_* and fbl_plan_destroy apply.  fbl_layer_fwd / _bwd
+ * reject it (FBL_ERR_INVALID_ARG) and fbl_xattn_fwd / _bwd reject a self-attention plan; adapters and the rotary
+ * embedding are not available on it.
+ * All pointers are device pointers, 1024-byte aligned, in the R-Tile layout; vectors fp32; ownership stays with the
+ * caller; the calls enqueue on `stream` and return.  Errors as for fbl_layer_fwd / _bwd. */
+int fbl_xattn_plan_create(const fbl_layer_desc* desc, int32_t seq_kv, int32_t d_mem, fbl_plan** out);
+int fbl_xattn_fwd(const fbl_plan* plan, const void* X, const void* M, const float* gamma, const float* beta,
+                  const void* Wq, const void* Wk, const void* Wv, const void* Wo, const float* bq, const float* bk,
+                  const float* bv, const float* bo, void* Y, void* saved, void* scratch, void* stream);
+/* Adds dM [batch, seq_kv, d_mem] to the outputs of fbl_layer_bwd; dWk, dWv are [d_mem, Dkv]. */
+int fbl_xattn_bwd(const fbl_plan* plan, const void* dY, const void* X, const void* M, const float* gamma,
+                  const void* Wq, const void* Wk, const void* Wv, const void* Wo, const void* saved, void* dX, void* dM,
+                  void* dWq, void* dWk, void* dWv, void* dWo, float* dbq, float* dbk, float* dbv, float* dbo,
+                  float* dgamma, float* dbeta, void* scratch, void* stream);
 
 /* Kernel family used by later calls on this plan: 0 = default (tcgen05 tensor-core kernels for bf16
  * wherever one exists for the shape, FFMA kernels for fp32), 1 = FFMA kernels only (fp32 arithmetic on

@@ -8,8 +8,9 @@ from .binding import (FblError, Plan, lib, load_library, LayerRunner, DTYPES, TE
                       desc_from_config, aligned_bytes, guard_bands_intact, selftest_wait_timeout)
 
 from .lora import LoraRunner
+from .xattn import XattnRunner
 from .mlp import MlpPlan, MlpRunner, mlp_desc_from_config, MLP_TENSOR, MLP_WS
 
-__all__ = ["LoraRunner", "MlpPlan", "MlpRunner", "mlp_desc_from_config", "MLP_TENSOR", "MLP_WS",
+__all__ = ["LoraRunner", "XattnRunner", "MlpPlan", "MlpRunner", "mlp_desc_from_config", "MLP_TENSOR", "MLP_WS",
            "FblError", "Plan", "lib", "load_library", "LayerRunner", "DTYPES", "TENSOR", "MAP", "WS",
            "desc_from_config", "aligned_bytes", "guard_bands_intact", "selftest_wait_timeout"]

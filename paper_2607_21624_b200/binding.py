@@ -16,7 +16,7 @@ DTYPES = {"fp32": 0, "bf16": 1}
 NORMS = {"layernorm": 0, "rmsnorm": 1}
 TENSOR = {n: i for i, n in enumerate(
     ["X", "Y", "DY", "DX", "WQ", "WK", "WV", "WO", "XN", "Q", "K", "V", "A",
-     "Q_HEADS", "K_HEADS", "V_HEADS", "A_HEADS", "WQ_T", "WK_T", "WV_T", "WO_T"])}
+     "Q_HEADS", "K_HEADS", "V_HEADS", "A_HEADS", "WQ_T", "WK_T", "WV_T", "WO_T", "MEM", "DMEM"])}
 WS = {n: i for i, n in enumerate(
     ["STATS", "XN", "Q", "K", "V", "A", "LSE", "D", "DA", "DQ", "DK", "DV", "DXN", "PARTIALS"])}
 MAP = {n: i for i, n in enumerate(
@@ -97,10 +97,16 @@ def desc_from_config(cfg) -> FblLayerDesc:
 class Plan:
     """One fbl_plan.  Methods carry the C entry points' names without the ``fbl_`` prefix."""
 
-    def __init__(self, desc: FblLayerDesc):
+    def __init__(self, desc: FblLayerDesc, cross=None):
+        """``cross`` = (seq_kv, d_mem) makes a cross-attention plan (fbl_xattn_plan_create)."""
         self._h = C.c_void_p()
         self.desc = desc
-        _check(lib().fbl_plan_create(C.byref(desc), C.byref(self._h)))
+        if cross is None:
+            _check(lib().fbl_plan_create(C.byref(desc), C.byref(self._h)))
+        else:
+            L = lib()
+            L.fbl_xattn_plan_create.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]
+            _check(L.fbl_xattn_plan_create(C.byref(desc), int(cross[0]), int(cross[1]), C.byref(self._h)))
 
     def close(self):
         if self._h:
@@ -238,7 +244,7 @@ class LayerRunner:
         self.torch = torch
         self.cfg = cfg
         self.dev = torch.device(device)
-        self.plan = Plan(desc_from_config(cfg))
+        self.plan = self._make_plan(cfg)
         from . import rtile
         if tile_choices is None:
             tile_choices = rtile.load_table().get(rtile.shape_key(cfg), {}).get("choices", {})
@@ -273,6 +279,9 @@ class LayerRunner:
             self.vec = {k: fz(n) for k, n in lens.items()}
 
     # -- helpers ---------------------------------------------------------------------------
+    def _make_plan(self, cfg):
+        return Plan(desc_from_config(cfg))
+
     def _stream(self):
         return self.torch.cuda.current_stream(self.dev).cuda_stream
 
@@ -357,7 +366,8 @@ class LayerRunner:
         ws, tid, dim = self.INTERMEDIATES[name]
         off, nbytes = self.plan.workspace_offset(WS[ws])
         src = self.saved if ws in ("XN", "Q", "K", "V", "A") else self.scratch
-        out = torch.empty((c.batch, c.seq, getattr(c, dim)), dtype=self.tdtype, device=self.dev)
+        rows = getattr(c, "seq_kv", c.seq) if tid == "K" else c.seq
+        out = torch.empty((c.batch, rows, getattr(c, dim)), dtype=self.tdtype, device=self.dev)
         self.plan.unpack(TENSOR[tid], src[off:off + nbytes].data_ptr(), out.data_ptr(), self._stream())
         torch.cuda.synchronize(self.dev)
         return out.float().cpu().numpy().astype("float64")

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libfblayout.so")
-SOURCES = ["api.cu", "mlp.cu", "lora.cu", "rtile_select.cu", "tile_propagation.cu", "k_elementwise.cu", "k_simt.cu", "k_tc_gemm.cu", "k_tc_attn.cu"]
+SOURCES = ["api.cu", "mlp.cu", "lora.cu", "xattn.cu", "rtile_select.cu", "tile_propagation.cu", "k_elementwise.cu", "k_simt.cu", "k_tc_gemm.cu", "k_tc_attn.cu"]
 
 
 def _stale() -> bool:

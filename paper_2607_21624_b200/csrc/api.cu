@@ -22,10 +22,13 @@ bool mat_shape(const fbl_plan* p, int id, MatShape* s) {
     case FBL_T_Q: case FBL_T_A: case FBL_T_Q_HEADS: case FBL_T_A_HEADS:
       *s = {d.batch, d.seq, p->t_pad, p->dq}; return true;
     case FBL_T_K: case FBL_T_V: case FBL_T_K_HEADS: case FBL_T_V_HEADS:
-      *s = {d.batch, d.seq, p->t_pad, p->dkv}; return true;
+      *s = {d.batch, p->seq_kv, p->t_pad_kv, p->dkv}; return true;
+    case FBL_T_MEM: case FBL_T_DMEM:
+      if (!p->cross) return false;
+      *s = {d.batch, p->seq_kv, p->t_pad_kv, p->d_mem}; return true;
     case FBL_T_WQ: case FBL_T_WQ_T: *s = {1, d.d_model, up8(d.d_model), p->dq}; return true;
     case FBL_T_WK: case FBL_T_WV: case FBL_T_WK_T: case FBL_T_WV_T:
-      *s = {1, d.d_model, up8(d.d_model), p->dkv}; return true;
+      *s = {1, p->d_mem, up8(p->d_mem), p->dkv}; return true;
     case FBL_T_WO: case FBL_T_WO_T: *s = {1, p->dq, up8(p->dq), d.d_model}; return true;
     default: return false;
   }
@@ -80,10 +83,15 @@ extern "C" {
 
 const char* fbl_last_error_detail(void) { return g_detail; }
 
-int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
+// Shared by the two plan constructors.  cross = 0: self-attention (the key side is the layer's own sequence);
+// cross = 1: K and V are projected from a memory [batch, seq_kv, d_mem].
+static int plan_build(const fbl_layer_desc* desc, int cross, int seq_kv_in, int d_mem_in, fbl_plan** out) {
   if (!desc || !out) return FBL_ERR_INVALID_ARG;
   *out = nullptr;
   const fbl_layer_desc& d = *desc;
+  const int seq_kv = cross ? seq_kv_in : d.seq, d_mem = cross ? d_mem_in : d.d_model;
+  if (cross && (seq_kv <= 0 || d_mem <= 0)) return FBL_ERR_INVALID_ARG;
+  if (cross && d.causal) return FBL_ERR_INVALID_ARG;      // memory positions have no order relative to the queries
   if (d.batch <= 0 || d.seq <= 0 || d.d_model <= 0 || d.n_q_heads <= 0 || d.n_kv_heads <= 0 || d.head_dim <= 0)
     return FBL_ERR_INVALID_ARG;
   if (d.dtype != FBL_DTYPE_FP32 && d.dtype != FBL_DTYPE_BF16) return FBL_ERR_INVALID_ARG;
@@ -94,12 +102,13 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   // Tile-propagation legality (section 4.3): the GQA head map needs whole groups; the head split
   // must fall on tile boundaries (tile_w divides head_dim) and d_model must be whole tiles.
   if (d.n_q_heads % d.n_kv_heads != 0) return FBL_ERR_UNSUPPORTED_SHAPE;
-  if (d.head_dim % tw != 0 || d.d_model % tw != 0) return FBL_ERR_UNSUPPORTED_SHAPE;
+  if (d.head_dim % tw != 0 || d.d_model % tw != 0 || d_mem % tw != 0) return FBL_ERR_UNSUPPORTED_SHAPE;
   if (d.dtype == FBL_DTYPE_FP32 && d.head_dim != 32 && d.head_dim != 64 && d.head_dim != 128)
     return FBL_ERR_UNSUPPORTED_SHAPE;
   if (d.dtype == FBL_DTYPE_BF16 && d.head_dim != 64 && d.head_dim != 128) return FBL_ERR_UNSUPPORTED_SHAPE;
   if ((int64_t)d.batch * up8(d.seq) > (int64_t)1 << 30) return FBL_ERR_UNSUPPORTED_SHAPE;
-  if (d.d_model > 16384 || (int64_t)d.n_q_heads * d.head_dim > 16384) return FBL_ERR_UNSUPPORTED_SHAPE;
+  if ((int64_t)d.batch * up8(seq_kv) > (int64_t)1 << 30) return FBL_ERR_UNSUPPORTED_SHAPE;
+  if (d.d_model > 16384 || d_mem > 16384 || (int64_t)d.n_q_heads * d.head_dim > 16384) return FBL_ERR_UNSUPPORTED_SHAPE;
 
   fbl_plan* p = new (std::nothrow) fbl_plan();
   if (!p) return FBL_ERR_INVALID_ARG;
@@ -108,6 +117,11 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   p->tw = tw;
   p->t_pad = (int)up8(d.seq);
   p->n_pad = (int64_t)d.batch * p->t_pad;
+  p->cross = cross;
+  p->seq_kv = seq_kv;
+  p->d_mem = d_mem;
+  p->t_pad_kv = (int)up8(seq_kv);
+  p->n_pad_kv = (int64_t)d.batch * p->t_pad_kv;
   p->dq = d.n_q_heads * d.head_dim;
   p->dkv = d.n_kv_heads * d.head_dim;
   p->group = d.n_q_heads / d.n_kv_heads;
@@ -129,15 +143,16 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   for (int i = 0; i < FBL_GEMM_LAUNCH_COUNT; ++i) p->choice[i] = {0, -1, 0};
   p->use_tc = d.dtype == FBL_DTYPE_BF16 ? 1 : 0;
 
-  const size_t n = (size_t)p->n_pad;
+  const size_t n = (size_t)p->n_pad, nk = (size_t)p->n_pad_kv;
   auto mat = [&](size_t cols) { return fbl_align_up(n * cols * (size_t)e, FBL_ALIGN); };
+  auto mat_kv = [&](size_t cols) { return fbl_align_up(nk * cols * (size_t)e, FBL_ALIGN); };
   const size_t rows_bh = (size_t)d.batch * d.n_q_heads * p->t_pad;
   size_t o = 0;
   p->sv_stats = o; o += fbl_align_up(n * 2 * sizeof(float), FBL_ALIGN);
   p->sv_xn = o;    o += mat(d.d_model);
   p->sv_q = o;     o += mat(p->dq);
-  p->sv_k = o;     o += mat(p->dkv);
-  p->sv_v = o;     o += mat(p->dkv);
+  p->sv_k = o;     o += mat_kv(p->dkv);
+  p->sv_v = o;     o += mat_kv(p->dkv);
   p->sv_a = o;     o += mat(p->dq);
   p->sv_lse = o;   o += fbl_align_up(rows_bh * sizeof(float) + 512, FBL_ALIGN);   // + one 128-float copy window past the last row
   p->saved_bytes = o;
@@ -146,7 +161,7 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   // first, then (from the next 256-float boundary) the norm backward's per-block partial rows, at most two
   // blocks per SM with one dgamma row and one dbeta row each.
   {
-    const size_t cs_floats = colsum_scratch_bytes(p->n_pad, (int64_t)d.d_model + p->dq + 2 * p->dkv) / sizeof(float);
+    const size_t cs_floats = colsum_scratch_bytes(p->n_pad, (int64_t)d.d_model + p->dq + (cross ? 0 : 2 * p->dkv)) / sizeof(float);
     const size_t norm_floats = (size_t)2 * p->sm_count * 2 * d.d_model;
     p->part_bytes = fbl_align_up(((cs_floats + 255) / 256 * 256 + norm_floats) * sizeof(float), FBL_ALIGN);
   }
@@ -154,8 +169,16 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   p->scratch_fwd_bytes = FBL_ALIGN;  // the status word
 
   // weight-gradient GEMMs: few output tiles, reduction over all tokens; slice the reduction when that balances the SMs
-  p->ksplit_o = p->ksplit_qkv = 1;
-  if (p->use_tc) {
+  p->ksplit_o = p->ksplit_qkv = p->ksplit_kv = 1;
+  if (p->use_tc && cross) {
+    const int kb_q = (int)((p->n_pad + 63) / 64), kb_k = (int)((p->n_pad_kv + 63) / 64);
+    const GemmShape go[2] = {{p->dq, d.d_model, kb_q, 1}, {p->n_pad, p->dq, (d.d_model + 63) / 64, 0}};
+    p->ksplit_o = gemm_tc_choose_split(p->sm_count, go, 2);
+    const GemmShape gq[2] = {{d.d_model, p->dq, kb_q, 1}, {p->n_pad, d.d_model, (p->dq + 63) / 64, 0}};
+    p->ksplit_qkv = gemm_tc_choose_split(p->sm_count, gq, 2);
+    const GemmShape gk[3] = {{d_mem, p->dkv, kb_k, 1}, {d_mem, p->dkv, kb_k, 1}, {p->n_pad_kv, d_mem, (2 * p->dkv + 63) / 64, 0}};
+    p->ksplit_kv = gemm_tc_choose_split(p->sm_count, gk, 3);
+  } else if (p->use_tc) {
     const int kb_tok = (int)((p->n_pad + 63) / 64);
     const GemmShape go[2] = {{p->dq, d.d_model, kb_tok, 1}, {p->n_pad, p->dq, (d.d_model + 63) / 64, 0}};
     p->ksplit_o = gemm_tc_choose_split(p->sm_count, go, 2);
@@ -170,20 +193,30 @@ int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) {
   p->sb_acc_o = o;
   if (p->ksplit_o > 1) o += fbl_align_up((size_t)up8(p->dq) * d.d_model * sizeof(float), FBL_ALIGN);
   p->sb_acc_qkv = o;
-  if (p->ksplit_qkv > 1) o += fbl_align_up((size_t)up8(d.d_model) * (p->dq + 2 * p->dkv) * sizeof(float), FBL_ALIGN);
+  if (p->ksplit_qkv > 1) o += fbl_align_up((size_t)up8(d.d_model) * (p->dq + (cross ? 0 : 2 * p->dkv)) * sizeof(float), FBL_ALIGN);
+  p->sb_acc_kv = o;
+  if (cross && p->ksplit_kv > 1) o += fbl_align_up((size_t)up8(d_mem) * 2 * p->dkv * sizeof(float), FBL_ALIGN);
   p->acc_bytes = o - FBL_ALIGN;
   p->sb_dqacc = o; o += fbl_align_up(n * p->dq * sizeof(float), FBL_ALIGN);   // zero-filled with the areas before it
   p->zero_bytes = o;
   p->sb_da = o;    o += mat(p->dq);
   p->sb_dvec = o;  o += fbl_align_up(rows_bh * sizeof(float), FBL_ALIGN);
   p->sb_dq = o;    o += mat(p->dq);
-  p->sb_dk = o;    o += mat(p->dkv);
-  p->sb_dv = o;    o += mat(p->dkv);
+  p->sb_dk = o;    o += mat_kv(p->dkv);
+  p->sb_dv = o;    o += mat_kv(p->dkv);
   p->sb_dxn = o;   o += mat(d.d_model);
   p->sb_part = o;  o += p->part_bytes;
+  p->sb_part_kv = o;
+  if (cross) o += fbl_align_up(colsum_scratch_bytes(p->n_pad_kv, 2 * (int64_t)p->dkv), FBL_ALIGN);
   p->scratch_bwd_bytes = o;
   *out = p;
   return FBL_OK;
+}
+
+int fbl_plan_create(const fbl_layer_desc* desc, fbl_plan** out) { return plan_build(desc, 0, 0, 0, out); }
+
+int fbl_xattn_plan_create(const fbl_layer_desc* desc, int32_t seq_kv, int32_t d_mem, fbl_plan** out) {
+  return plan_build(desc, 1, seq_kv, d_mem, out);
 }
 
 void fbl_plan_destroy(fbl_plan* plan) {
@@ -227,7 +260,7 @@ int fbl_plan_set_gemm_choice(fbl_plan* plan, int launch_id, int tile_n, int cta_
 }
 
 int fbl_plan_enable_rope(fbl_plan* plan, float base) {
-  if (!plan || !(base > 1.f) || plan->d.head_dim % 16 != 0) return FBL_ERR_INVALID_ARG;
+  if (!plan || plan->cross || !(base > 1.f) || plan->d.head_dim % 16 != 0) return FBL_ERR_INVALID_ARG;
   plan->rope_base = base;
   return FBL_OK;
 }
@@ -256,21 +289,21 @@ int fbl_workspace_bytes(const fbl_plan* plan, size_t* saved, size_t* scratch_fwd
 int fbl_workspace_offset(const fbl_plan* plan, int what, size_t* offset, size_t* bytes) {
   if (!plan || !offset || !bytes) return FBL_ERR_INVALID_ARG;
   const fbl_plan* p = plan;
-  const size_t n = (size_t)p->n_pad, e = (size_t)p->e;
+  const size_t n = (size_t)p->n_pad, nk = (size_t)p->n_pad_kv, e = (size_t)p->e;
   const size_t rows_bh = (size_t)p->d.batch * p->d.n_q_heads * p->t_pad;
   switch (what) {
     case FBL_WS_STATS: *offset = p->sv_stats; *bytes = n * 2 * sizeof(float); return FBL_OK;
     case FBL_WS_XN: *offset = p->sv_xn; *bytes = n * p->d.d_model * e; return FBL_OK;
     case FBL_WS_Q: *offset = p->sv_q; *bytes = n * p->dq * e; return FBL_OK;
-    case FBL_WS_K: *offset = p->sv_k; *bytes = n * p->dkv * e; return FBL_OK;
-    case FBL_WS_V: *offset = p->sv_v; *bytes = n * p->dkv * e; return FBL_OK;
+    case FBL_WS_K: *offset = p->sv_k; *bytes = nk * p->dkv * e; return FBL_OK;
+    case FBL_WS_V: *offset = p->sv_v; *bytes = nk * p->dkv * e; return FBL_OK;
     case FBL_WS_A: *offset = p->sv_a; *bytes = n * p->dq * e; return FBL_OK;
     case FBL_WS_LSE: *offset = p->sv_lse; *bytes = rows_bh * sizeof(float); return FBL_OK;
     case FBL_WS_D: *offset = p->sb_dvec; *bytes = rows_bh * sizeof(float); return FBL_OK;
     case FBL_WS_DA: *offset = p->sb_da; *bytes = n * p->dq * e; return FBL_OK;
     case FBL_WS_DQ: *offset = p->sb_dq; *bytes = n * p->dq * e; return FBL_OK;
-    case FBL_WS_DK: *offset = p->sb_dk; *bytes = n * p->dkv * e; return FBL_OK;
-    case FBL_WS_DV: *offset = p->sb_dv; *bytes = n * p->dkv * e; return FBL_OK;
+    case FBL_WS_DK: *offset = p->sb_dk; *bytes = nk * p->dkv * e; return FBL_OK;
+    case FBL_WS_DV: *offset = p->sb_dv; *bytes = nk * p->dkv * e; return FBL_OK;
     case FBL_WS_DXN: *offset = p->sb_dxn; *bytes = n * p->d.d_model * e; return FBL_OK;
     case FBL_WS_PARTIALS: *offset = p->sb_part; *bytes = p->part_bytes; return FBL_OK;
     default: return FBL_ERR_INVALID_ARG;
@@ -285,9 +318,9 @@ int64_t fbl_tile_offset(const fbl_plan* plan, int tensor_id, const int32_t idx[4
   switch (tensor_id) {
     case FBL_T_Q_HEADS: case FBL_T_A_HEADS: case FBL_T_K_HEADS: case FBL_T_V_HEADS: {
       const int heads = (tensor_id == FBL_T_K_HEADS || tensor_id == FBL_T_V_HEADS) ? d.n_kv_heads : d.n_q_heads;
-      if (idx[0] < 0 || idx[0] >= d.batch || idx[1] < 0 || idx[1] >= heads || idx[2] < 0 || idx[2] >= d.seq ||
+      if (idx[0] < 0 || idx[0] >= d.batch || idx[1] < 0 || idx[1] >= heads || idx[2] < 0 || idx[2] >= s.rows ||
           idx[3] < 0 || idx[3] >= d.head_dim) return -1;
-      r = (int64_t)idx[0] * plan->t_pad + idx[2];
+      r = (int64_t)idx[0] * s.rows_pad + idx[2];
       c = (int64_t)idx[1] * d.head_dim + idx[3];
       break;
     }
@@ -359,7 +392,7 @@ int fbl_tile_map(const fbl_plan* plan, int map_id, int64_t src, int64_t* dst) {
 static int pack_common(const fbl_plan* plan, int tensor_id, const void* src, void* dst, void* stream, int unpack) {
   MatShape s;
   if (!plan || !src || !dst || !mat_shape(plan, tensor_id, &s)) return FBL_ERR_INVALID_ARG;
-  if (tensor_id >= FBL_T_Q_HEADS) return FBL_ERR_INVALID_ARG;   // views are not separate buffers
+  if (tensor_id >= FBL_T_Q_HEADS && tensor_id <= FBL_T_WO_T) return FBL_ERR_INVALID_ARG;   // views are not separate buffers
   if (misaligned(unpack ? src : dst)) return FBL_ERR_MISALIGNED;
   FBL_CUDA(launch_pack(plan->d.dtype, unpack, src, dst, s.outer, s.rows, s.rows_pad, s.cols, as_stream(stream)));
   return FBL_OK;
@@ -375,6 +408,7 @@ int fbl_layer_fwd(const fbl_plan* p, const void* X, const float* gamma, const fl
                   const void* Wk, const void* Wv, const void* Wo, const float* bq, const float* bk, const float* bv,
                   const float* bo, void* Y, void* saved, void* scratch, void* stream) {
   if (!p || !X || !gamma || !Wq || !Wk || !Wv || !Wo || !Y || !saved || !scratch) return FBL_ERR_INVALID_ARG;
+  if (p->cross) return FBL_ERR_INVALID_ARG;              // a cross-attention plan runs through fbl_xattn_fwd / _bwd
   if (p->d.has_bias && (!bq || !bk || !bv || !bo)) return FBL_ERR_INVALID_ARG;
   if (p->d.norm == FBL_NORM_LAYERNORM && !beta) return FBL_ERR_INVALID_ARG;
   const void* ptrs[] = {X, Wq, Wk, Wv, Wo, Y, saved, scratch};
@@ -439,6 +473,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
   if (!p || !dY || !X || !gamma || !Wq || !Wk || !Wv || !Wo || !saved || !dX || !dWq || !dWk || !dWv || !dWo ||
       !dgamma || !scratch)
     return FBL_ERR_INVALID_ARG;
+  if (p->cross) return FBL_ERR_INVALID_ARG;
   if (p->d.has_bias && (!dbq || !dbk || !dbv || !dbo)) return FBL_ERR_INVALID_ARG;
   if (p->d.norm == FBL_NORM_LAYERNORM && !dbeta) return FBL_ERR_INVALID_ARG;
   const void* ptrs[] = {dY, X, Wq, Wk, Wv, Wo, saved, dX, dWq, dWk, dWv, dWo, scratch};

@@ -36,6 +36,10 @@ struct fbl_plan {
   int tw;       // tile_w in elements
   int t_pad;    // seq rounded up to 8
   int64_t n_pad;  // batch * t_pad
+  // Key side of the attention: the same sequence in self-attention; in a cross-attention plan (cross = 1) the memory
+  // sequence [batch, seq_kv, d_mem] that K and V are projected from
+  int cross, seq_kv, t_pad_kv, d_mem;
+  int64_t n_pad_kv;
   int dq, dkv, group;
   float scale;
   int sm_count;
@@ -50,6 +54,10 @@ struct fbl_plan {
   // follow the status word so that one fill zeroes both
   int ksplit_o, ksplit_qkv;
   size_t sb_acc_o, sb_acc_qkv, acc_bytes;
+  // cross-attention only: slices of dWk / dWv, their accumulation area, dM's place is the caller's; partial sums of
+  // the dK / dV column sums
+  int ksplit_kv;
+  size_t sb_acc_kv, sb_part_kv;
   size_t zero_bytes;        // leading part of the backward scratch that every step starts by zero-filling
   // tuning knobs, read from the environment once, at plan creation (0 / -1 = the library's own choice)
   int knob_gemm_pair;       // -1 by size, 0 never the CTA-pair GEMM kernel, 1 wherever its tile shape is legal

@@ -85,6 +85,7 @@ template <typename T, int HD>
 __global__ void __launch_bounds__(256) attn_fwd_simt_kernel(const T* __restrict__ Q, const T* __restrict__ K,
                                                             const T* __restrict__ V, T* __restrict__ A,
                                                             float* __restrict__ lse, int64_t n_pad, int seq, int t_pad,
+                                                            int64_t n_pad_k, int seq_k, int t_pad_k,
                                                             int hq, int group, int causal, float scale) {
   constexpr int TW = tile_w_of<T>::value;
   constexpr int LD = HD + 1;
@@ -98,7 +99,7 @@ __global__ void __launch_bounds__(256) attn_fwd_simt_kernel(const T* __restrict_
   float* s_m = s_alpha + BQ;
   float* s_l = s_m + BQ;
   const int i0 = blockIdx.x * BQ, h = blockIdx.y, b = blockIdx.z, gk = h / group;
-  const int64_t row0 = (int64_t)b * t_pad;
+  const int64_t row0 = (int64_t)b * t_pad, row0k = (int64_t)b * t_pad_k;   // query-side and key-side rows of this sequence
   const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
   for (int e = threadIdx.x; e < BQ * HD; e += 256) {
     const int i = e / HD, d = e % HD;
@@ -106,13 +107,13 @@ __global__ void __launch_bounds__(256) attn_fwd_simt_kernel(const T* __restrict_
   }
   if (threadIdx.x < BQ) { s_m[threadIdx.x] = -INFINITY; s_l[threadIdx.x] = 0.f; }
   float o[4][ND] = {};
-  const int j_end = causal ? min(seq, i0 + BQ) : seq;
+  const int j_end = causal ? min(seq_k, i0 + BQ) : seq_k;
   for (int j0 = 0; j0 < j_end; j0 += BKV) {
     __syncthreads();
     for (int e = threadIdx.x; e < BKV * HD; e += 256) {
       const int j = e / HD, d = e % HD;
-      const bool ok = j0 + j < seq;
-      const int64_t off = rt_off<TW>(n_pad, row0 + j0 + j, gk * HD + d);
+      const bool ok = j0 + j < seq_k;
+      const int64_t off = rt_off<TW>(n_pad_k, row0k + j0 + j, gk * HD + d);
       Ks[j * LD + d] = ok ? to_f(K[off]) : 0.f;
       Vs[j * LD + d] = ok ? to_f(V[off]) : 0.f;
     }
@@ -132,7 +133,7 @@ __global__ void __launch_bounds__(256) attn_fwd_simt_kernel(const T* __restrict_
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int gi = i0 + ty * 4 + i, gj = j0 + tx * 4 + j;
-        const bool masked = gj >= seq || (causal && gj > gi);
+        const bool masked = gj >= seq_k || (causal && gj > gi);
         Ss[(ty * 4 + i) * (BKV + 1) + tx * 4 + j] = masked ? -INFINITY : s[i][j] * scale;
       }
     __syncthreads();
@@ -233,7 +234,7 @@ __global__ void __launch_bounds__(256) attn_bwd_simt_kernel(const T* __restrict_
                                                             const float* __restrict__ lse,
                                                             const float* __restrict__ dvec, float* __restrict__ dqacc,
                                                             T* __restrict__ dK, T* __restrict__ dV, int64_t n_pad,
-                                                            int seq, int t_pad, int hq, int group, int causal,
+                                                            int seq, int t_pad, int64_t n_pad_k, int seq_k, int t_pad_k, int hq, int group, int causal,
                                                             float scale) {
   constexpr int TW = tile_w_of<T>::value;
   constexpr int LD = HD + 1;
@@ -249,12 +250,12 @@ __global__ void __launch_bounds__(256) attn_bwd_simt_kernel(const T* __restrict_
   float* s_lse = Ds + BQ * LS;
   float* s_d = s_lse + BQ;
   const int j0 = blockIdx.x * BKV, gk = blockIdx.y, b = blockIdx.z;
-  const int64_t row0 = (int64_t)b * t_pad;
+  const int64_t row0 = (int64_t)b * t_pad, row0k = (int64_t)b * t_pad_k;
   const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
   for (int e = threadIdx.x; e < BKV * HD; e += 256) {
     const int j = e / HD, d = e % HD;
-    const bool ok = j0 + j < seq;
-    const int64_t off = rt_off<TW>(n_pad, row0 + j0 + j, gk * HD + d);
+    const bool ok = j0 + j < seq_k;
+    const int64_t off = rt_off<TW>(n_pad_k, row0k + j0 + j, gk * HD + d);
     Ks[j * LD + d] = ok ? to_f(K[off]) : 0.f;
     Vs[j * LD + d] = ok ? to_f(V[off]) : 0.f;
   }
@@ -302,7 +303,7 @@ __global__ void __launch_bounds__(256) attn_bwd_simt_kernel(const T* __restrict_
         for (int j = 0; j < 4; ++j) {
           const int li = ty * 4 + i, lj = tx * 4 + j;
           const int gi = i0 + li, gj = j0 + lj;
-          const bool masked = gi >= seq || gj >= seq || (causal && gj > gi);
+          const bool masked = gi >= seq || gj >= seq_k || (causal && gj > gi);
           const float p = masked ? 0.f : expf(s[i][j] * scale - s_lse[li]);
           Ps[li * LS + lj] = p;
           Ds[li * LS + lj] = p * (dp[i][j] - s_d[li]);
@@ -349,11 +350,11 @@ __global__ void __launch_bounds__(256) attn_bwd_simt_kernel(const T* __restrict_
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     const int gj = j0 + ty * 4 + j;
-    if (gj >= t_pad) continue;
-    const bool live = gj < seq;
+    if (gj >= t_pad_k) continue;
+    const bool live = gj < seq_k;
 #pragma unroll
     for (int dd = 0; dd < ND; ++dd) {
-      const int64_t off = rt_off<TW>(n_pad, row0 + gj, gk * HD + tx + 16 * dd);
+      const int64_t off = rt_off<TW>(n_pad_k, row0k + gj, gk * HD + tx + 16 * dd);
       dK[off] = from_f<T>(live ? dk[j][dd] * scale : 0.f);
       dV[off] = from_f<T>(live ? dv[j][dd] : 0.f);
     }
@@ -396,6 +397,7 @@ cudaError_t attn_fwd_launch(const fbl_plan* p, const void* Q, const void* K, con
   if (e != cudaSuccess) return e;
   dim3 grid((p->t_pad + BQ - 1) / BQ, p->d.n_q_heads, p->d.batch);
   k<<<grid, 256, sh, st>>>((const T*)Q, (const T*)K, (const T*)V, (T*)A, lse, p->n_pad, p->d.seq, p->t_pad,
+                           p->n_pad_kv, p->seq_kv, p->t_pad_kv,
                            p->d.n_q_heads, p->group, p->d.causal, p->scale);
   return cudaGetLastError();
 }
@@ -407,9 +409,10 @@ cudaError_t attn_bwd_launch(const fbl_plan* p, const void* Q, const void* K, con
   auto k = attn_bwd_simt_kernel<T, HD>;
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
   if (e != cudaSuccess) return e;
-  dim3 grid((p->t_pad + BKV - 1) / BKV, p->d.n_kv_heads, p->d.batch);
+  dim3 grid((p->t_pad_kv + BKV - 1) / BKV, p->d.n_kv_heads, p->d.batch);
   k<<<grid, 256, sh, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)dA, lse, dvec, dqacc, (T*)dK, (T*)dV,
-                           p->n_pad, p->d.seq, p->t_pad, p->d.n_q_heads, p->group, p->d.causal, p->scale);
+                           p->n_pad, p->d.seq, p->t_pad, p->n_pad_kv, p->seq_kv, p->t_pad_kv, p->d.n_q_heads, p->group,
+                           p->d.causal, p->scale);
   return cudaGetLastError();
 }
 

@@ -27,6 +27,7 @@ struct alignas(64) AttnFwdParams {
   float* lse;            // [B, Hq, t_pad]
   long long n_pad;
   int seq, t_pad, hq, group, causal;
+  int seq_k, t_pad_k;    // key-side sequence length and padded length (those of the query side in self-attention)
   int pair;              // 1: each block owns two adjacent query tiles, one per softmax warp group
   int batch, n_slots, chunk;   // grid = n_slots * hq * batch blocks, see decode_block
   float scale;
@@ -80,7 +81,7 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
   int slot_i, hb;
   decode_block((int)blockIdx.x, P.n_slots, P.hq * P.batch, P.chunk, &slot_i, &hb);
   const int h = hb % P.hq, b = hb / P.hq, g = h / P.group;
-  const int row0 = b * P.t_pad;
+  const int row0 = b * P.t_pad, row0k = b * P.t_pad_k;     // first row of this sequence on the query and key sides
   int32_t* status = P.status;
   // with pairing a block owns two adjacent tiles, whose key ranges differ by one tile, so both warp groups stay
   // busy for the whole loop
@@ -89,7 +90,7 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
   const int qt0 = pair ? min(2 * slot_x + 1, n_qt - 1) : slot_x;
   const int qt1 = (pair && 2 * slot_x + 1 < n_qt) ? 2 * slot_x : -1;   // odd tile count: the last block has one tile
   auto kv_tiles = [&](int t) {
-    const int kv_end = t < 0 ? 0 : (P.causal ? min(P.seq, (t + 1) * BQ) : P.seq);
+    const int kv_end = t < 0 ? 0 : (P.causal ? min(P.seq_k, (t + 1) * BQ) : P.seq_k);
     return (kv_end + BKV - 1) / BKV;
   };
   const int n_kv0 = kv_tiles(qt0), n_kv1 = kv_tiles(qt1);
@@ -125,9 +126,9 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
     if (qt1 >= 0) tc::tma_load_3d(base + SM::Q_OFF + SM::TILE, &P.tq, bar(B_QFULL), 0, row0 + qt1 * BQ, h * (int)PANELS);
     if (n_kv_max > 0) {
       tc::mbar_expect_tx(bar(B_KFULL), SM::TILE);
-      tc::tma_load_3d(base + SM::K_OFF, &P.tk, bar(B_KFULL), 0, row0, g * (int)PANELS);
+      tc::tma_load_3d(base + SM::K_OFF, &P.tk, bar(B_KFULL), 0, row0k, g * (int)PANELS);
       tc::mbar_expect_tx(bar(B_VFULL), SM::TILE);
-      tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(B_VFULL), 0, row0, g * (int)PANELS);
+      tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(B_VFULL), 0, row0k, g * (int)PANELS);
     }
   }
   if (warp == 1) {
@@ -148,10 +149,10 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
       const uint32_t ph = (j >> 1) & 1;
       if (!tc::mbar_wait(bar(B_KEMPTY + s), ph ^ 1, status, 201)) break;
       tc::mbar_expect_tx(bar(B_KFULL + s), SM::TILE);
-      tc::tma_load_3d(base + SM::K_OFF + s * SM::TILE, &P.tk, bar(B_KFULL + s), 0, row0 + j * BKV, g * (int)PANELS);
+      tc::tma_load_3d(base + SM::K_OFF + s * SM::TILE, &P.tk, bar(B_KFULL + s), 0, row0k + j * BKV, g * (int)PANELS);
       if (!tc::mbar_wait(bar(B_VEMPTY + s), ph ^ 1, status, 202)) break;
       tc::mbar_expect_tx(bar(B_VFULL + s), SM::TILE);
-      tc::tma_load_3d(base + SM::V_OFF + s * SM::TILE, &P.tv, bar(B_VFULL + s), 0, row0 + j * BKV, g * (int)PANELS);
+      tc::tma_load_3d(base + SM::V_OFF + s * SM::TILE, &P.tv, bar(B_VFULL + s), 0, row0k + j * BKV, g * (int)PANELS);
     }
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer --------------------------------------------------------------------------
@@ -273,7 +274,7 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
       const uint32_t s_addr = lane_addr + (uint32_t)sbuf * 128;
       if (!tc::mbar_wait(bar(B_SFULL + sbuf), sph, status, 208)) { ok = false; break; }
       tc::tc_fence_after();
-      const bool need_mask = (j0 + BKV > P.seq) || (P.causal && j0 + BKV - 1 > i0);
+      const bool need_mask = (j0 + BKV > P.seq_k) || (P.causal && j0 + BKV - 1 > i0);
       float mx, alpha, mc;
       float2 sum01 = make_float2(0.f, 0.f), sum23 = sum01;
       const float2 c2 = make_float2(c, c);
@@ -291,7 +292,7 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
   #pragma unroll
           for (int k = 0; k < 128; ++k) {
             const int gj = j0 + k;
-            if (gj >= P.seq || (P.causal && gj > gi)) sv[k] = -INFINITY;
+            if (gj >= P.seq_k || (P.causal && gj > gi)) sv[k] = -INFINITY;
           }
         }
         float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
@@ -345,7 +346,7 @@ __global__ void __launch_bounds__(64 + 128 * TILES, TILES == 1 ? 2 : 1) attn_fwd
 #pragma unroll
           for (int k = 0; k < 32; ++k) {
             const int gj = j0 + cc * 32 + k;
-            if (gj >= P.seq || (P.causal && gj > gi)) sc[k] = -INFINITY;
+            if (gj >= P.seq_k || (P.causal && gj > gi)) sc[k] = -INFINITY;
           }
         };
         float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
@@ -454,7 +455,7 @@ cudaError_t fwd_launch_t(const fbl_plan* p, AttnFwdParams& P, int n_qt, cudaStre
   if (TILES == 1) P.pair = 0;
   P.batch = p->d.batch;
   P.n_slots = P.pair ? (n_qt + 1) / 2 : n_qt;
-  P.chunk = chunk_for((long long)p->d.seq * HD * 4, p->d.n_q_heads * p->d.batch, 96ll << 20);   // K and V of one head
+  P.chunk = chunk_for((long long)p->seq_kv * HD * 4, p->d.n_q_heads * p->d.batch, 96ll << 20);   // K and V of one head
   dim3 grid((unsigned)(P.n_slots * p->d.n_q_heads * p->d.batch));
   return launch_pdl(k, grid, dim3(64 + 128 * TILES), FwdSmem<HD, TILES>::TOTAL, st, P);
 }
@@ -466,10 +467,11 @@ cudaError_t fwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   memset(&P, 0, sizeof(P));
   const int panels = HD / 64;
   if (!fbl_encode_rtile_map(&P.tq, Q, p->n_pad, p->dq / 64, BQ, panels)) return cudaErrorInvalidValue;
-  if (!fbl_encode_rtile_map(&P.tk, K, p->n_pad, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
-  if (!fbl_encode_rtile_map(&P.tv, V, p->n_pad, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
+  if (!fbl_encode_rtile_map(&P.tk, K, p->n_pad_kv, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
+  if (!fbl_encode_rtile_map(&P.tv, V, p->n_pad_kv, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
   P.a = (__nv_bfloat16*)A; P.lse = lse; P.n_pad = p->n_pad;
   P.seq = p->d.seq; P.t_pad = p->t_pad; P.hq = p->d.n_q_heads; P.group = p->group; P.causal = p->d.causal;
+  P.seq_k = p->seq_kv; P.t_pad_k = p->t_pad_kv;
   P.scale = p->scale; P.status = status;
   const int n_qt = (p->d.seq + BQ - 1) / BQ;
   // two query tiles per block when that still leaves at least one block per SM
@@ -499,8 +501,9 @@ struct alignas(64) AttnBwdParams {
   float* dqacc;          // fp32 [n_pad, dq] in the bf16 tile order
   __nv_bfloat16* dk;
   __nv_bfloat16* dv;
-  long long n_pad;
+  long long n_pad, n_pad_k;          // rows of the query-side (Q, dO, dQ) and key-side (K, V, dK, dV) buffers
   int seq, t_pad, hq, group, causal, dkv;
+  int seq_k, t_pad_k;                // key-side sequence length and padded length
   int batch, chunk;      // grid = key tiles * KV heads * batch blocks, see decode_block
   float scale;
   int32_t* status;
@@ -553,9 +556,9 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
   // under a causal mask key tile 0 has the most query tiles: it is slot 0
   const int n_kvh = P.hq / P.group;
   int slot_i, gb;
-  decode_block((int)blockIdx.x, (P.t_pad + BKV - 1) / BKV, n_kvh * P.batch, P.chunk, &slot_i, &gb);
+  decode_block((int)blockIdx.x, (P.t_pad_k + BKV - 1) / BKV, n_kvh * P.batch, P.chunk, &slot_i, &gb);
   const int j0 = slot_i * BKV, g = gb % n_kvh, b = gb / n_kvh;
-  const int row0 = b * P.t_pad;
+  const int row0 = b * P.t_pad, row0k = b * P.t_pad_k;
   const int n_qt = (P.seq + BQ - 1) / BQ;
   const int qt_begin = P.causal ? j0 / BQ : 0;
   const int per_head = n_qt - qt_begin;
@@ -593,8 +596,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     tc::tma_prefetch_desc(&P.tk); tc::tma_prefetch_desc(&P.tv); tc::tma_prefetch_desc(&P.tq);
     tc::tma_prefetch_desc(&P.tdo); tc::tma_prefetch_desc(&P.tdq);
     tc::mbar_expect_tx(bar(BB_KVFULL), 2 * SM::TILE);
-    tc::tma_load_3d(base + SM::K_OFF, &P.tk, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
-    tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(BB_KVFULL), 0, row0 + j0, g * (int)PANELS);
+    tc::tma_load_3d(base + SM::K_OFF, &P.tk, bar(BB_KVFULL), 0, row0k + j0, g * (int)PANELS);
+    tc::tma_load_3d(base + SM::V_OFF, &P.tv, bar(BB_KVFULL), 0, row0k + j0, g * (int)PANELS);
     if (n_it > 0) {
       // LSE travels with Q and D with dO: 128 floats each, into the iteration's staging buffer
       tc::mbar_expect_tx(bar(BB_QFULL), SM::TILE + 512);
@@ -839,7 +842,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
       if (!tc::mbar_wait(bar(BB_SFULL), it & 1, status, 306)) { ok = false; break; }
       tc::tc_fence_after();
       // element masks are needed only on the diagonal tile and on tiles with keys or queries beyond the sequence
-      const bool need_mask = (P.causal && (i0 < j0 + BKV - 1)) || (j0 + BKV > P.seq) || (i0 + BQ > P.seq);
+      const bool need_mask = (P.causal && (i0 < j0 + BKV - 1)) || (j0 + BKV > P.seq_k) || (i0 + BQ > P.seq);
       const uint32_t dsrow = base + SM::DS_OFF + (it % NP) * 32768 + (part / 2) * 16384 + r * 128;
       // this thread's 32 score columns first: with HD = 128 the packed P^T overwrites S^T columns that belong to
       // other warps of the same lane quarter, so every warp must have read its scores before any P^T store
@@ -876,7 +879,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
               const int gi = i0 + c0 + k + u;
-              if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) pv[u] = 0.f;
+              if (gj >= P.seq_k || gi >= P.seq || (P.causal && gi < gj)) pv[u] = 0.f;
             }
           }
           const float2 g01 = __fmul2_rn(make_float2(pv[0], pv[1]), __ffma2_rn(make_float2(d4.x, d4.y), neg1, make_float2(__uint_as_float(dpv[k]), __uint_as_float(dpv[k + 1]))));
@@ -886,7 +889,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
               const int gi = i0 + c0 + k + u;
-              if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) gv[u] = 0.f;
+              if (gj >= P.seq_k || gi >= P.seq || (P.causal && gi < gj)) gv[u] = 0.f;
             }
           }
           pp[k / 2] = tc::pack_bf16(pv[0], pv[1]);
@@ -933,7 +936,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
               const int gi = i0 + part * 32 + k + u;
-              if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) pv[u] = 0.f;
+              if (gj >= P.seq_k || gi >= P.seq || (P.causal && gi < gj)) pv[u] = 0.f;
             }
           }
 #pragma unroll
@@ -975,7 +978,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
               const int gi = i0 + c0 + k + u;
-              if (gj >= P.seq || gi >= P.seq || (P.causal && gi < gj)) gv[u] = 0.f;
+              if (gj >= P.seq_k || gi >= P.seq || (P.causal && gi < gj)) gv[u] = 0.f;
             }
           }
           dd[k / 2] = tc::pack_bf16(gv[0], gv[1]);
@@ -1009,7 +1012,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
     if (!PIPE && ok && n_it > 0) ok = tc::mbar_wait(bar(BB_DVDONE), 0, status, 315);
     tc::tc_fence_after();
     if (ok && n_it > 0) {
-      const bool live = gj < P.seq;
+      const bool live = gj < P.seq_k;
 #pragma unroll 1
       for (int which = 0; which < 2; ++which) {
         __nv_bfloat16* out = which ? P.dk : P.dv;
@@ -1020,9 +1023,9 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_tc_kernel(const __gri
           uint32_t o[16];
           tc::tmem_ld16(lane_addr + (which ? DK_COL : DV_COL) + c0, o);   // warp-collective: no lane may skip it
           tc::tmem_ld_wait();
-          if (gj < P.t_pad) {
+          if (gj < P.t_pad_k) {
             const int col = g * HD + c0;
-            __nv_bfloat16* dst = out + ((long long)(col / 64) * P.n_pad + row0 + gj) * 64 + (col % 64);
+            __nv_bfloat16* dst = out + ((long long)(col / 64) * P.n_pad_k + row0k + gj) * 64 + (col % 64);
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
               uint4 v;
@@ -1051,12 +1054,13 @@ cudaError_t bwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   const int panels = HD / 64;
   if (!fbl_encode_rtile_map(&P.tq, Q, p->n_pad, p->dq / 64, BQ, panels)) return cudaErrorInvalidValue;
   if (!fbl_encode_rtile_map(&P.tdo, dA, p->n_pad, p->dq / 64, BQ, panels)) return cudaErrorInvalidValue;
-  if (!fbl_encode_rtile_map(&P.tk, K, p->n_pad, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
-  if (!fbl_encode_rtile_map(&P.tv, V, p->n_pad, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
+  if (!fbl_encode_rtile_map(&P.tk, K, p->n_pad_kv, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
+  if (!fbl_encode_rtile_map(&P.tv, V, p->n_pad_kv, p->dkv / 64, BKV, panels)) return cudaErrorInvalidValue;
   if (!fbl_encode_f32_panel_map(&P.tdq, dqacc, p->n_pad, p->dq / 64, BQ)) return cudaErrorInvalidValue;
   P.lse = lse; P.dvec = dvec; P.dqacc = dqacc; P.dk = (__nv_bfloat16*)dK; P.dv = (__nv_bfloat16*)dV;
   P.n_pad = p->n_pad; P.seq = p->d.seq; P.t_pad = p->t_pad; P.hq = p->d.n_q_heads; P.group = p->group;
   P.causal = p->d.causal; P.dkv = p->dkv; P.scale = p->scale; P.status = status;
+  P.n_pad_k = p->n_pad_kv; P.seq_k = p->seq_kv; P.t_pad_k = p->t_pad_kv;
   auto k = attn_bwd_tc_kernel<HD>;
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdSmem<HD>::TOTAL);
   if (e != cudaSuccess) return e;
@@ -1066,14 +1070,15 @@ cudaError_t bwd_launch(const fbl_plan* p, const void* Q, const void* K, const vo
   // together (small chunks: L2 hits); the pipelined HD = 64 variant hides that latency and prefers balance.
   P.chunk = chunk_for((long long)p->group * p->d.seq * HD * 8, p->d.n_kv_heads * p->d.batch,
                       BwdSmem<HD>::PIPE ? (96ll << 20) : (8ll << 20));
-  dim3 grid((unsigned)(((p->t_pad + BKV - 1) / BKV) * p->d.n_kv_heads * p->d.batch));
+  dim3 grid((unsigned)(((p->t_pad_kv + BKV - 1) / BKV) * p->d.n_kv_heads * p->d.batch));
   return launch_pdl(k, grid, dim3(BWD_THREADS), BwdSmem<HD>::TOTAL, st, P);
 }
 
 }  // namespace
 
 bool attn_fwd_tc_supported(const fbl_plan* p) {
-  return p->d.dtype == FBL_DTYPE_BF16 && (p->d.head_dim == 64 || p->d.head_dim == 128) && p->n_pad >= 128;
+  return p->d.dtype == FBL_DTYPE_BF16 && (p->d.head_dim == 64 || p->d.head_dim == 128) && p->n_pad >= 128 &&
+         p->n_pad_kv >= 128;
 }
 bool attn_bwd_tc_supported(const fbl_plan* p) { return attn_fwd_tc_supported(p); }
 

@@ -98,7 +98,7 @@ cudaError_t run_group(const fbl_plan* p, GemmArgs* gs, int count, int32_t* statu
 extern "C" {
 
 int fbl_plan_enable_lora(fbl_plan* plan, int rank) {
-  if (!plan || rank < 1 || rank > RB) return FBL_ERR_INVALID_ARG;
+  if (!plan || plan->cross || rank < 1 || rank > RB) return FBL_ERR_INVALID_ARG;
   if (plan->lora_rank > 0) return plan->lora_rank == rank ? FBL_OK : FBL_ERR_INVALID_ARG;
   plan->lora_rank = rank;
   const size_t n = (size_t)plan->n_pad;
