@@ -508,6 +508,25 @@ def measure_mlp(key, args, rep, local_rank, flush_l2):
     run = MlpRunner(cfg, device=f"cuda:{local_rank}")
     run.plan.set_kernel_path(args.path)
     run.load_inputs(make_mlp_inputs(cfg))
+    return time_runner(run, cfg, f"{cfg.name}: B={cfg.batch} T={cfg.seq} D={cfg.d_model} F={cfg.d_ff} {cfg.act} {cfg.norm} {cfg.dtype}",
+                       args, rep, flush_l2)
+
+
+def measure_xattn(key, args, rep, local_rank, flush_l2):
+    """The cross-attention layer `key` of fbl_inputs.XATTN_CONFIGS, timed like the feed-forward blocks."""
+    from fbl_inputs import XATTN_CONFIGS, make_xattn_inputs
+    from paper_2607_21624_b200 import XattnRunner
+    cfg = XATTN_CONFIGS[key]
+    run = XattnRunner(cfg, device=f"cuda:{local_rank}")
+    run.plan.set_kernel_path(args.path)
+    run.load_inputs(make_xattn_inputs(cfg))
+    return time_runner(run, cfg, f"{cfg.name}: B={cfg.batch} Tq={cfg.seq} Tkv={cfg.seq_kv} D={cfg.d_model} Dmem={cfg.d_mem} "
+                       f"Hq={cfg.n_q_heads} Hkv={cfg.n_kv_heads} hd={cfg.head_dim} {cfg.norm} {cfg.dtype}", args, rep, flush_l2)
+
+
+def time_runner(run, cfg, workload, args, rep, flush_l2):
+    """Forward + backward of a loaded runner: cold L2 before every step, graph replay, max over ranks."""
+    import torch
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
         run.step()
@@ -553,7 +572,7 @@ def measure_mlp(key, args, rep, local_rank, flush_l2):
         return None
     peaks = measured_peaks()
     flops = cfg.flops()
-    return {"workload": (f"{cfg.name}: B={cfg.batch} T={cfg.seq} D={cfg.d_model} F={cfg.d_ff} {cfg.act} {cfg.norm} {cfg.dtype}"),
+    return {"workload": workload,
             "ms_per_step": ms, "ms_fwd": ms_fwd, "tflops": rep.whole_job_rate(flops, ms) / 1e12,
             "tokens_per_s": rep.whole_job_rate(cfg.n_tokens, ms), "flops_per_step": flops, "dtype": "bf16",
             "layer_roofline": {"binds": "tensor", "frac_of_measured_burst": flops / (peaks["tflops_burst"] * 1e12) / (ms * 1e-3),
@@ -609,9 +628,11 @@ def run_rank(args):
         for key in ("matmul-512x2048x8192", "gpt2", "llama1b"):
             mlp[key] = measure_mlp(key, args, rep, local_rank, flush_l2)
     lora = {}
+    xattn = {}
     if not args.config and not args.no_mlp:          # the paper's fine-tuning setting on two of the workloads
         for i in (2, 4):
             lora[i] = measure(pick(i), args, rep, local_rank, flush_l2, want_cpu=False, lora_rank=16)
+        xattn["whisper-large"] = measure_xattn("whisper-large", args, rep, local_rank, flush_l2)
     if rank != 0:
         rep.close()
         return
@@ -631,11 +652,13 @@ def run_rank(args):
         "activation_bytes": h["activation_bytes"], "e2e": h["e2e"],
         "gpu_launches": (sum(r["launches_per_step"] for r in results.values())
                          + sum(r["launches_per_step"] for r in mlp.values())
-                         + sum(r["launches_per_step"] for r in lora.values())) * args.steps,
+                         + sum(r["launches_per_step"] for r in lora.values())
+                         + sum(r["launches_per_step"] for r in xattn.values())) * args.steps,
         "clocks": h["clocks"], "roofline": h["roofline"], "cpu_baseline": h["cpu_baseline"],
         "peaks": peaks,
         "per_config": {**{f"workload{i}": results[i] for i in sorted(results)}, **{f"mlp_{k}": v for k, v in mlp.items()},
-                       **{f"lora16_workload{i}": v for i, v in lora.items()}},
+                       **{f"lora16_workload{i}": v for i, v in lora.items()},
+                       **{f"xattn_{k}": v for k, v in xattn.items()}},
     }
     print(json.dumps(line))
     rep.close()

@@ -31,11 +31,13 @@ def emulate(cfg, inp):
     z = lambda b: b if b is not None else 0.0
     B, T, D = X.shape
     Hq, hd, G = cfg.n_q_heads, cfg.head_dim, cfg.group
-    flat = lambda t: t.reshape(B * T, -1)
+    flat = lambda t: t.reshape(-1, t.shape[-1])
+    mem = inp.get("M")                 # cross-attention: K and V come from the memory, which is an input (no rounding)
 
     Xn_exact, xhat, rstd, mu = orc.norm_fwd(X, inp["gamma"], inp["beta"], cfg.eps, cfg.norm)
     Xn = r16(Xn_exact)
-    Q, K, V = r16(Xn @ Wq + z(inp["bq"])), r16(Xn @ Wk + z(inp["bk"])), r16(Xn @ Wv + z(inp["bv"]))
+    src_kv = Xn if mem is None else mem
+    Q, K, V = r16(Xn @ Wq + z(inp["bq"])), r16(src_kv @ Wk + z(inp["bk"])), r16(src_kv @ Wv + z(inp["bv"]))
     rope_base = getattr(cfg, "rope_base", 0.0)
     if rope_base > 0.0:               # rotated in place: read as bf16, written as bf16
         Q, K = r16(orc.rope(Q, Hq, rope_base)), r16(orc.rope(K, cfg.n_kv_heads, rope_base))
@@ -80,9 +82,13 @@ def emulate(cfg, inp):
     dQ, dK, dV = r16(dQ), r16(dK), r16(dV)
     if rope_base > 0.0:
         dQ, dK = r16(orc.rope(dQ, Hq, rope_base, inverse=True)), r16(orc.rope(dK, cfg.n_kv_heads, rope_base, inverse=True))
-    out["dWq"], out["dWk"], out["dWv"] = r16(flat(Xn).T @ flat(dQ)), r16(flat(Xn).T @ flat(dK)), r16(flat(Xn).T @ flat(dV))
+    out["dWq"], out["dWk"], out["dWv"] = r16(flat(Xn).T @ flat(dQ)), r16(flat(src_kv).T @ flat(dK)), r16(flat(src_kv).T @ flat(dV))
     out["dbq"], out["dbk"], out["dbv"] = flat(dQ).sum(axis=0), flat(dK).sum(axis=0), flat(dV).sum(axis=0)
-    dXn = r16(dQ @ Wq.T + dK @ Wk.T + dV @ Wv.T)
+    if mem is None:
+        dXn = r16(dQ @ Wq.T + dK @ Wk.T + dV @ Wv.T)
+    else:
+        dXn = r16(dQ @ Wq.T)
+        out["dM"] = r16(dK @ Wk.T + dV @ Wv.T)
     out["dgamma"] = flat(dXn * xhat).sum(axis=0)
     if cfg.norm == "layernorm":
         out["dbeta"] = flat(dXn).sum(axis=0)
@@ -100,7 +106,11 @@ def floor_figures(cfg, inp, ref=None):
     elements outside the element-wise bound |e| <= 1e-2 + 2e-2 |ref|, of the emulation against the oracle
     (``ref``: the oracle's outputs by name, computed here when not given)."""
     if ref is None:
-        Y, _, g = orc.layer_fwd_bwd(cfg, inp)
+        if "M" in inp:
+            from oracle import xattn
+            Y, _, g = xattn.xattn_fwd_bwd(cfg, inp)
+        else:
+            Y, _, g = orc.layer_fwd_bwd(cfg, inp)
         ref = dict(g)
         ref["Y"] = Y
     emu = emulate(cfg, inp)

@@ -63,3 +63,16 @@ def test_zero_bias_gradient_noise_grows_with_tokens_and_group():
     b = np.abs(emulate(large, make_inputs(large, affine_noise=True))["dbk"]).max()
     print(f"max|dbk| floor: {a:.3e} (512 tokens, G=1) -> {b:.3e} (4096 tokens, G=4)")
     assert b > 2.0 * a
+
+
+def test_floor_of_a_cross_attention_layer():
+    # the memory is an input, so K, V and dM see one rounding fewer than their self-attention counterparts; the
+    # floor's figures stay in the same band, and dM (a token tensor) meets the element-wise form everywhere
+    from fbl_inputs import XattnConfig, make_xattn_inputs
+    cfg = XattnConfig("xf", 2, 200, 333, 256, 192, 4, 2, 64, "bf16", "layernorm", True, True, 1e-5, 101, 0.02)
+    fig = floor_figures(cfg, make_xattn_inputs(cfg, affine_noise=True))
+    _show("xattn", fig)
+    assert "dM" in fig and fig["dM"]["viol"] == 0.0 and fig["Y"]["viol"] == 0.0 and fig["dX"]["viol"] == 0.0
+    for name, v in fig.items():
+        if name != "dbk":
+            assert v["fro"] < 6e-3 and v["worst_over_bound"] < 0.3, name

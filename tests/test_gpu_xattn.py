@@ -8,6 +8,7 @@ from oracle import xattn as orc
 from paper_2607_21624_b200 import XattnRunner
 from paper_2607_21624_b200.binding import FblError, LayerRunner
 
+from bf16_floor import floor_figures
 from util import FP32_REL, bf16_ok, fp32_err, record, report
 
 pytestmark = pytest.mark.gpu
@@ -30,6 +31,7 @@ def run_and_compare(cfg, path=0, guard_bytes=0, affine_noise=True):
         names += ["dbq", "dbk", "dbv", "dbo"]
     inter = dict(Xn=saved["Xn"], Q=saved["Q"], K=saved["K"], V=saved["V"], A=saved["A"], LSE=saved["LSE"], D=g["D"],
                  dA=g["dA"], dQ=g["dQ"], dK=g["dK"], dV=g["dV"], dXn=g["dXn"])
+    floors = floor_figures(cfg, inp, ref) if cfg.dtype == "bf16" else {}
     bad, figures = [], {}
     for n in names + list(inter):
         got = run.fetch(n) if n in names else run.saved_view(n)
@@ -45,14 +47,14 @@ def run_and_compare(cfg, path=0, guard_bytes=0, affine_noise=True):
                 ok = err <= FP32_REL
                 print(f"{n:7s} fp32 scale-floored rel err {err:.3e}")
         else:
-            ok, f, failed = bf16_ok(n, got, want)
+            ok, f, failed = bf16_ok(n, got, want, floors.get(n))
             figures[n] = f
-            print(report(n, f), "" if ok else f"FAILED {failed}")
+            print(report(n, f, floors.get(n)), "" if ok else f"FAILED {failed}")
         if not ok:
             bad.append(n)
     if guard_bytes:
         assert run.guards_intact() == [], run.guards_intact()
-    record(cfg.name, figures, {})
+    record(cfg.name, figures, floors)
     assert not bad, bad
     return run
 

@@ -9,7 +9,7 @@ bf16 storage with fp32 accumulation ("2e-2 relative / 1e-2 absolute").  Three cr
     any bf16 implementation, tests/bf16_floor.py, sits at 3e-3 .. 6e-3).
  3. element-wise, |e_i| <= 1e-2 + 2e-2 |ref_i|: the fraction of elements outside it is capped relative to the
     same fraction of the rounding floor, computed for the very layer under test from the oracle alone:
-       Y, dX (token tensors):           at most 10 x the floor's fraction (zero where the floor has none);
+       Y, dX, dM (token tensors):       at most 10 x the floor's fraction (zero where the floor has none);
        dW*, db*, dgamma, dbeta:         at most 2 x the floor's fraction + 1e-3.  These are sums over thousands
                                         of tokens with cancellation, so their small elements carry noise in
                                         proportion to the tensor's scale in any bf16-operand implementation
@@ -29,7 +29,7 @@ import numpy as np
 FP32_REL = 1e-4
 BF16_RTOL, BF16_ATOL = 2e-2, 1e-2
 FRO_MAX = 1e-2
-TOKEN_TENSORS = ("Y", "dX")
+TOKEN_TENSORS = ("Y", "dX", "dM")
 TOKEN_VIOL_OVER_FLOOR = 10.0
 REDUCTION_VIOL_OVER_FLOOR, REDUCTION_VIOL_SLACK = 2.0, 1e-3
 ZERO_REF = ("dbk",)
