@@ -16,7 +16,7 @@
 namespace {
 
 constexpr int BM = 128, BK = 64;
-constexpr int MAX_TERMS = 4, MAX_PROBLEMS = 4;
+constexpr int MAX_TERMS = 4, MAX_PROBLEMS = 5;
 
 struct alignas(64) TcProblem {
   CUtensorMap ta[MAX_TERMS], tb[MAX_TERMS], tc;     // tc: the output, for the epilogue's bulk stores

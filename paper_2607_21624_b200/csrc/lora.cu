@@ -252,7 +252,7 @@ int fbl_layer_bwd_lora(const fbl_plan* p, const void* dY, const void* X, const f
     p->launches += k;
   }
   {
-    GemmArgs gs[4];
+    GemmArgs gs[5];
     for (int i = 0; i < 3; ++i) {          // dB_all[:, block i] = T^T d*: token-axis reduction, T's tiles read MN-major
       GemmArgs& g = gs[i];
       g = GemmArgs{};
@@ -268,17 +268,13 @@ int fbl_layer_bwd_lora(const fbl_plan* p, const void* dY, const void* X, const f
     gx.t[3] = {dT, p->n_pad, 0, A_all, up8(D), 1, RA};
     gx.b_static = 0;
     gx.c = dXn; gx.c_rpad = p->n_pad; gx.seq = p->d.seq; gx.t_pad = p->t_pad;
-    LORA_CUDA(run_group(p, gs, 4, status, st, &k));
-    LORA_STEP("dB+dXn", 0, cudaSuccess);
-    p->launches += k;
-  }
-  {
-    GemmArgs g = {};                       // dA_all = Xn^T dT: token-axis reduction
+    GemmArgs& g = gs[4];                   // dA_all = Xn^T dT: token-axis reduction, in the same launch
+    g = GemmArgs{};
     g.m = D; g.n = RA; g.n_terms = 1;
     g.t[0] = {Xn, p->n_pad, 1, dT, p->n_pad, 0, n};
     g.c = dA_all; g.c_rpad = up8(D);
-    LORA_CUDA(run_group(p, &g, 1, status, st, &k));
-    LORA_STEP("lora_dA", 0, cudaSuccess);
+    LORA_CUDA(run_group(p, gs, 5, status, st, &k));
+    LORA_STEP("dB+dXn+dA", 0, cudaSuccess);
     p->launches += k;
   }
   LORA_STEP("norm_bwd", norm_bwd_takes_colsums(p) ? 2 : 1, launch_norm_bwd(p, dXn, X, p->d.residual ? dY : nullptr, stats, gamma, dX, dgamma, dbeta, part, st));

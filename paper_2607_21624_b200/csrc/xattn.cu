@@ -196,30 +196,37 @@ int fbl_xattn_bwd(const fbl_plan* p, const void* dY, const void* X, const void* 
     bool tc_q = p->use_tc != 0, tc_k = p->use_tc != 0;
     for (int i = 0; i < 2; ++i) tc_q = tc_q && gemm_tc_supported(p, gq[i]);
     for (int i = 0; i < 3; ++i) tc_k = tc_k && gemm_tc_supported(p, gk[i]);
-    if (tc_q) {
-      if (split_q) {
-        gq[0].ksplit = p->ksplit_qkv; gq[0].acc = (float*)(sc + p->sb_acc_qkv);
-        cg.src[cg.count] = gq[0].acc; cg.dst[cg.count] = dWq; cg.n[cg.count] = up8(D) * (int64_t)p->dq; cg.count++;
+    if (tc_q && split_q) {
+      gq[0].ksplit = p->ksplit_qkv; gq[0].acc = (float*)(sc + p->sb_acc_qkv);
+      cg.src[cg.count] = gq[0].acc; cg.dst[cg.count] = dWq; cg.n[cg.count] = up8(D) * (int64_t)p->dq; cg.count++;
+    }
+    if (tc_k && split_kv) {
+      float* acc = (float*)(sc + p->sb_acc_kv);
+      for (int i = 0; i < 2; ++i) {
+        gk[i].ksplit = p->ksplit_kv; gk[i].acc = acc;
+        cg.src[cg.count] = acc; cg.dst[cg.count] = DW[i]; cg.n[cg.count] = up8(Dm) * (int64_t)p->dkv; cg.count++;
+        acc += up8(Dm) * (int64_t)p->dkv;
       }
+    }
+    if (tc_q && tc_k) {
+      // both sides in one launch: the three token-axis reductions first in the work list (longest loops), then the
+      // two input gradients
+      GemmArgs all[5] = {gq[0], gk[0], gk[1], gq[1], gk[2]};
+      XA_STEP("dWqkv+dXn+dM", 1, launch_gemm_tc_group(p, all, 5, status, st));
+    } else {
+    if (tc_q) {
       XA_STEP("dWq+dXn", 1, launch_gemm_tc_group(p, gq, 2, status, st));
     } else {
       XA_STEP("dXn", 1, run_gemm(p, gq[1], status, st));
       XA_STEP("dWq", 1, run_gemm(p, gq[0], status, st));
     }
     if (tc_k) {
-      if (split_kv) {
-        float* acc = (float*)(sc + p->sb_acc_kv);
-        for (int i = 0; i < 2; ++i) {
-          gk[i].ksplit = p->ksplit_kv; gk[i].acc = acc;
-          cg.src[cg.count] = acc; cg.dst[cg.count] = DW[i]; cg.n[cg.count] = up8(Dm) * (int64_t)p->dkv; cg.count++;
-          acc += up8(Dm) * (int64_t)p->dkv;
-        }
-      }
       XA_STEP("dWkv+dM", 1, launch_gemm_tc_group(p, gk, 3, status, st));
     } else {
       XA_STEP("dM", 1, run_gemm(p, gk[2], status, st));
       XA_STEP("dWk", 1, run_gemm(p, gk[0], status, st));
       XA_STEP("dWv", 1, run_gemm(p, gk[1], status, st));
+    }
     }
     if (cg.count > 0) XA_STEP("dW round", 1, launch_convert_f32_group(cg, st));
   }
