@@ -57,7 +57,7 @@ def step_flops(cfg):
     pq, pk, po = 2.0 * n * cfg.d_model * cfg.d_q, 2.0 * n * cfg.d_model * cfg.d_kv, 2.0 * n * cfg.d_q * cfg.d_model
     return {"proj_q": pq, "proj_k": pk, "proj_v": pk, "proj_qkv": pq + 2 * pk, "attn_fwd": 2 * att, "proj_o": po,
             "dA": po, "dWo": po, "dWo+dA": 2 * po, "attn_bwd": 4 * att, "dXn": pq + 2 * pk, "dWq": pq, "dWk": pk,
-            "dWv": pk, "dWqkv": pq + 2 * pk, "dWqkv+dXn": 2 * (pq + 2 * pk), "dW+dXn": 2 * (pq + 2 * pk) + po}
+            "dWv": pk, "dWqkv": pq + 2 * pk, "dWqkv+dXn": 2 * (pq + 2 * pk)}
 
 
 def step_bytes(cfg):

@@ -316,10 +316,8 @@ int fbl_rtile_candidates(const int64_t* shapes, int n_shapes, int elem_bytes, fl
  * section 4.2 / 6 and the argmax of Eq. 2 live in the Python module rtile.py, which times the candidates through
  * these calls): output-tile width 128 or 256 (0: built-in heuristic), CTA-pair kernel 0 / 1 (-1: heuristic),
  * epilogue warp sets 1 / 2 (0: heuristic).  A choice whose tile shape is not legal for the launch's shapes falls
- * back to the heuristic.  Takes effect for later fbl_layer_fwd / fbl_layer_bwd calls on this plan.
- * The four launches: Q, K, V projections (grouped); output projection; dA = dY Wo^T (with D fused), in front of the
- * attention backward; the four weight gradients dWq, dWk, dWv, dWo and dXn (grouped), behind it. */
-enum { FBL_GEMM_PROJ_QKV = 0, FBL_GEMM_PROJ_O, FBL_GEMM_DA, FBL_GEMM_DW_DXN, FBL_GEMM_LAUNCH_COUNT };
+ * back to the heuristic.  Takes effect for later fbl_layer_fwd / fbl_layer_bwd calls on this plan. */
+enum { FBL_GEMM_PROJ_QKV = 0, FBL_GEMM_PROJ_O, FBL_GEMM_DWO_DA, FBL_GEMM_DWQKV_DXN, FBL_GEMM_LAUNCH_COUNT };
 int fbl_plan_set_gemm_choice(fbl_plan* plan, int launch_id, int tile_n, int cta_pair, int epilogue_sets);
 
 /* ---------------------------------------------------------------------------------------------------------------

@@ -184,10 +184,7 @@ static int plan_build(const fbl_layer_desc* desc, int cross, int seq_kv_in, int 
     p->ksplit_o = gemm_tc_choose_split(p->sm_count, go, 2);
     const GemmShape gq[4] = {{d.d_model, p->dq, kb_tok, 1}, {d.d_model, p->dkv, kb_tok, 1}, {d.d_model, p->dkv, kb_tok, 1},
                              {p->n_pad, d.d_model, (p->dq + 2 * p->dkv + 63) / 64, 0}};
-    // dWo is issued with dWq, dWk, dWv and dXn (nothing in the step reads it, and the attention backward then waits
-    // for dA alone): one slice count for the four weight gradients of that launch
-    const GemmShape g5[5] = {gq[0], gq[1], gq[2], go[0], gq[3]};
-    p->ksplit_qkv = p->ksplit_o = gemm_tc_choose_split(p->sm_count, g5, 5);
+    p->ksplit_qkv = gemm_tc_choose_split(p->sm_count, gq, 4);
   }
   if (p->use_tc && getenv("FBL_KSPLIT_O")) p->ksplit_o = atoi(getenv("FBL_KSPLIT_O"));          // tuning knobs
   if (p->use_tc && getenv("FBL_KSPLIT_QKV")) p->ksplit_qkv = atoi(getenv("FBL_KSPLIT_QKV"));
@@ -507,34 +504,41 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
   // (Measured: 2 % on workload 2; for accumulators of tens of MB the stores delay the launch's own first tiles by
   // more than the fill node costs, so large plans keep the node.)
   if (p->use_tc && p->acc_bytes == 0 && attn_bwd_tc_supported(p) && p->zero_bytes - p->sb_dqacc <= ((size_t)16 << 20)) {
-    GemmArgs ga = GemmArgs{};
+    GemmArgs gw = GemmArgs{}, ga = GemmArgs{};
+    gw.m = p->dq; gw.n = D; gw.n_terms = 1; gw.t[0] = {A, p->n_pad, 1, dY, p->n_pad, 0, n}; gw.c = dWo; gw.c_rpad = p->dq;
     ga.m = n; ga.n = p->dq; ga.n_terms = 1; ga.t[0] = {dY, p->n_pad, 0, Wo, p->dq, 1, D}; ga.c = dA; ga.c_rpad = p->n_pad;
-    first_gemm_fills = gemm_tc_supported(p, ga);
+    first_gemm_fills = gemm_tc_supported(p, gw) && gemm_tc_supported(p, ga);
   }
   if (!first_gemm_fills) FBL_CUDA(cudaMemsetAsync(status, 0, p->zero_bytes, st));
   FBL_PROF_BEGIN();
-  bool dvec_ready = false, dwo_pending = true;
-  GemmArgs gw = GemmArgs{};   // dWo = A^T dY : token-axis reduction; nothing in the step reads it, so it is issued with the
-  gw.m = p->dq; gw.n = D; gw.n_terms = 1;         // other weight gradients, behind the attention backward
-  gw.t[0] = {A, p->n_pad, 1, dY, p->n_pad, 0, n};
-  gw.c = dWo; gw.c_rpad = p->dq;
+  bool dvec_ready = false, dwo_round = false;
   {
-    GemmArgs ga = GemmArgs{};   // dA = dY Wo^T : Wo's tiles read with the roles of its two axes swapped
+    GemmArgs gs[2];
+    GemmArgs& gw = gs[0];   // dWo = A^T dY : token-axis reduction (longest reduction loop: first in the work list)
+    gw = GemmArgs{};
+    gw.m = p->dq; gw.n = D; gw.n_terms = 1;
+    gw.t[0] = {A, p->n_pad, 1, dY, p->n_pad, 0, n};
+    gw.c = dWo; gw.c_rpad = p->dq;
+    GemmArgs& ga = gs[1];   // dA = dY Wo^T : Wo's tiles read with the roles of its two axes swapped
+    ga = GemmArgs{};
     ga.m = n; ga.n = p->dq; ga.n_terms = 1;
     ga.t[0] = {dY, p->n_pad, 0, Wo, p->dq, 1, D};
     ga.b_static = 1;
     ga.c = dA; ga.c_rpad = p->n_pad; ga.seq = p->d.seq; ga.t_pad = p->t_pad;
-    if (p->use_tc && gemm_tc_supported(p, ga)) {
+    if (p->use_tc && gemm_tc_supported(p, gw) && gemm_tc_supported(p, ga)) {
       // D = rowsum(dO * O) per head comes out of the dA epilogue, from the fp32 accumulator
       ga.dot_with = A; ga.dot_out = dvec; ga.dot_hd = p->d.head_dim; ga.dot_hq = p->d.n_q_heads;
       dvec_ready = true;
+      if (split_o) { gw.ksplit = p->ksplit_o; gw.acc = (float*)(sc + p->sb_acc_o); }
       if (first_gemm_fills) {
-        ga.zero_ptr = dqacc; ga.zero_bytes = p->zero_bytes - p->sb_dqacc;
-        ga.reset_status = 1; ga.serial = 1;
+        gs[0].zero_ptr = dqacc; gs[0].zero_bytes = p->zero_bytes - p->sb_dqacc;
+        gs[0].reset_status = 1; gs[0].serial = 1;
       }
-      FBL_STEP("dA", 1, launch_gemm_tc_group(p, &ga, 1, status, st, FBL_GEMM_DA));
+      FBL_STEP("dWo+dA", 1, launch_gemm_tc_group(p, gs, 2, status, st, FBL_GEMM_DWO_DA));
+      dwo_round = split_o;        // nothing in the step reads dWo: its rounding joins that of dWq, dWk, dWv below
     } else {
       FBL_STEP("dA", 1, run_gemm(p, ga, status, st));
+      FBL_STEP("dWo", 1, run_gemm(p, gw, status, st));
     }
   }
   if (p->use_tc && attn_bwd_tc_supported(p)) FBL_STEP("attn_bwd", dvec_ready ? 2 : 3, launch_attn_bwd_tc(p, Q, K, V, A, dA, lse, dvec, dqacc, dQ, dK, dV, dvec_ready, status, st));   // dqacc: zero already
@@ -545,7 +549,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
     const void* G[3] = {dQ, dK, dV};
     void* DW[3] = {dWq, dWk, dWv};
     const int cols[3] = {p->dq, p->dkv, p->dkv};
-    GemmArgs gs[5];
+    GemmArgs gs[4];
     bool tc = p->use_tc != 0;
     for (int i = 0; i < 3; ++i) {   // dW* = Xn^T d* : token-axis reductions, Xn's tiles read MN-major
       GemmArgs& g = gs[i];
@@ -555,9 +559,7 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
       g.c = DW[i]; g.c_rpad = D;
       tc = tc && gemm_tc_supported(p, g);
     }
-    gs[3] = gw;
-    tc = tc && gemm_tc_supported(p, gw);
-    GemmArgs& gx = gs[4];           // dXn = dQ Wq^T + dK Wk^T + dV Wv^T : one accumulator, three reduction loops
+    GemmArgs& gx = gs[3];           // dXn = dQ Wq^T + dK Wk^T + dV Wv^T : one accumulator, three reduction loops
     gx = GemmArgs{};
     gx.m = n; gx.n = D; gx.n_terms = 3;
     gx.t[0] = {dQ, p->n_pad, 0, Wq, D, 1, p->dq};
@@ -567,8 +569,6 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
     gx.c = dXn; gx.c_rpad = p->n_pad; gx.seq = p->d.seq; gx.t_pad = p->t_pad;
     tc = tc && gemm_tc_supported(p, gx);
     if (tc) {
-      // the four weight gradients (longest reduction loops: first in the work list) and dXn in one launch; sliced
-      // reductions leave fp32 sums, which one rounding launch turns into the four matrices
       ConvertGroup cg = {};
       if (split_qkv) {
         float* acc = (float*)(sc + p->sb_acc_qkv);
@@ -579,22 +579,23 @@ int fbl_layer_bwd(const fbl_plan* p, const void* dY, const void* X, const float*
         }
         cg.count = 3;
       }
-      if (split_o) {
-        gs[3].ksplit = p->ksplit_o; gs[3].acc = (float*)(sc + p->sb_acc_o);
-        cg.src[cg.count] = gs[3].acc; cg.dst[cg.count] = dWo; cg.n[cg.count] = up8(p->dq) * (int64_t)D;
+      if (dwo_round) {
+        cg.src[cg.count] = (const float*)(sc + p->sb_acc_o); cg.dst[cg.count] = dWo; cg.n[cg.count] = up8(p->dq) * (int64_t)D;
         cg.count++;
+        dwo_round = false;
       }
-      FBL_STEP("dW+dXn", 1, launch_gemm_tc_group(p, gs, 5, status, st, FBL_GEMM_DW_DXN));
+      FBL_STEP("dWqkv+dXn", 1, launch_gemm_tc_group(p, gs, 4, status, st, FBL_GEMM_DWQKV_DXN));
       if (cg.count > 0) FBL_STEP("dW round", 1, launch_convert_f32_group(cg, st));     // one rounding launch for all sliced GEMMs
-      dwo_pending = false;
     } else {
       FBL_STEP("dXn", 1, run_gemm(p, gx, status, st));
       for (int i = 0; i < 3; ++i)
         FBL_STEP(i == 0 ? "dWq" : i == 1 ? "dWk" : "dWv", 1, run_gemm(p, gs[i], status, st));
     }
   }
-  if (dwo_pending) {                // paths without the grouped launch: dWo on its own, unsliced
-    FBL_STEP("dWo", 1, run_gemm(p, gw, status, st));
+  if (dwo_round) {
+    ConvertGroup cg = {};
+    cg.src[0] = (const float*)(sc + p->sb_acc_o); cg.dst[0] = dWo; cg.n[0] = up8(p->dq) * (int64_t)D; cg.count = 1;
+    FBL_STEP("dW round", 1, launch_convert_f32_group(cg, st));
   }
   // every bias gradient is a token-axis column sum: the four of them share their launches, and the second stage
   // shares the norm backward's second kernel where that kernel exists

@@ -24,7 +24,7 @@ from .binding import _check, lib
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 DEFAULT_TABLE = os.path.join(HERE, "tuned_b200.json")
-LAUNCHES = ["proj_qkv", "proj_o", "dA", "dW+dXn"]          # FBL_GEMM_* ids in order
+LAUNCHES = ["proj_qkv", "proj_o", "dWo+dA", "dWqkv+dXn"]          # FBL_GEMM_* ids in order
 
 
 class RtileCand(C.Structure):
@@ -62,8 +62,8 @@ def launch_ops(cfg):
     """Per launch: its operators as (M, N, K) products."""
     n, d, dq, dkv = cfg.batch * cfg.seq, cfg.d_model, cfg.d_q, cfg.d_kv
     return {"proj_qkv": [(n, dq, d), (n, dkv, d), (n, dkv, d)], "proj_o": [(n, d, dq)],
-            "dA": [(n, dq, d)],
-            "dW+dXn": [(d, dq, n), (d, dkv, n), (d, dkv, n), (dq, d, n), (n, d, dq + 2 * dkv)]}
+            "dWo+dA": [(dq, d, n), (n, dq, d)],
+            "dWqkv+dXn": [(d, dq, n), (d, dkv, n), (d, dkv, n), (n, d, dq + 2 * dkv)]}
 
 
 L2_RESIDENT_BYTES = 96e6           # of the 126 MB L2: a launch whose operands fit is re-read from L2, not from HBM
