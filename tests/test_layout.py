@@ -178,3 +178,48 @@ def test_partial_sum_area_covers_what_the_backward_kernels_write():
         _, _, sb = plan.workspace_bytes()
         assert nbytes >= need, (cfg, nbytes, need)
         assert off + nbytes <= sb
+
+
+def test_cross_attention_plan_host_maps_follow_the_memory_side():
+    # K, V, Wk, Wv (and the memory itself) of a cross-attention plan take the memory's sequence length and width;
+    # everything else keeps the query side's.  Element map against the layout oracle, sizes, and the rejections.
+    from fbl_inputs import XattnConfig
+    from paper_2607_21624_b200 import WS
+    cfg = XattnConfig("xl", 2, 13, 21, 128, 192, 2, 1, 64, "bf16", "layernorm", True, True, 1e-5, 0, 0.02)
+    plan = Plan(desc_from_config(cfg), cross=(cfg.seq_kv, cfg.d_mem))
+    tw, tq_pad, tk_pad = 64, 16, 24
+    assert plan.tensor_bytes(TENSOR["X"]) == 2 * tq_pad * 128 * 2
+    assert plan.tensor_bytes(TENSOR["MEM"]) == plan.tensor_bytes(TENSOR["DMEM"]) == 2 * tk_pad * 192 * 2
+    assert plan.tensor_bytes(TENSOR["K"]) == 2 * tk_pad * 64 * 2 and plan.tensor_bytes(TENSOR["Q"]) == 2 * tq_pad * 128 * 2
+    assert plan.tensor_bytes(TENSOR["WK"]) == 192 * 64 * 2 and plan.tensor_bytes(TENSOR["WQ"]) == 128 * 128 * 2
+    seen = set()
+    for b in range(cfg.batch):
+        for t in range(cfg.seq_kv):
+            for c in range(0, cfg.d_mem, 5):
+                got = plan.tile_offset(TENSOR["MEM"], [b, t, c])
+                assert got == lo.rtile_offset(b * tk_pad + t, c, 2 * tk_pad, 8, tw)
+                seen.add(got)
+            for d in range(0, 64, 7):
+                assert plan.tile_offset(TENSOR["K_HEADS"], [b, 0, t, d]) == plan.tile_offset(TENSOR["K"], [b, t, d]) == \
+                    lo.rtile_offset(b * tk_pad + t, d, 2 * tk_pad, 8, tw)
+    assert len(seen) == cfg.batch * cfg.seq_kv * len(range(0, cfg.d_mem, 5))
+    assert plan.tile_offset(TENSOR["K_HEADS"], [0, 0, cfg.seq_kv, 0]) < 0          # past the memory's length
+    assert plan.tile_offset(TENSOR["Q_HEADS"], [0, 0, cfg.seq, 0]) < 0              # past the query side's
+    assert plan.tile_offset(TENSOR["Q_HEADS"], [1, 1, cfg.seq - 1, 63]) == lo.rtile_offset(tq_pad + cfg.seq - 1, 127, 2 * tq_pad, 8, tw)
+    for r in range(0, cfg.d_mem, 11):
+        assert plan.tile_offset(TENSOR["WK"], [r, 3]) == lo.rtile_offset(r, 3, cfg.d_mem, 8, tw) == plan.tile_offset(TENSOR["WK_T"], [3, r])
+    # the workspace areas of K, V, dK, dV are sized by the memory's rows and do not overlap their neighbours
+    areas = sorted(plan.workspace_offset(WS[k]) for k in ("STATS", "XN", "Q", "K", "V", "A", "LSE"))
+    for (o0, n0), (o1, _) in zip(areas, areas[1:]):
+        assert o0 + n0 <= o1
+    assert plan.workspace_offset(WS["K"])[1] == plan.workspace_offset(WS["DK"])[1] == 2 * tk_pad * 64 * 2
+    # a self-attention plan has no memory; a cross plan takes no mask, and its memory width must be whole tiles
+    with pytest.raises(FblError):
+        Plan(desc_from_config(small())).tensor_bytes(TENSOR["MEM"])
+    import dataclasses
+    with pytest.raises(FblError):
+        Plan(desc_from_config(dataclasses.replace(cfg, causal=True)), cross=(cfg.seq_kv, cfg.d_mem))
+    with pytest.raises(FblError):
+        Plan(desc_from_config(cfg), cross=(cfg.seq_kv, 100))
+    with pytest.raises(FblError):
+        Plan(desc_from_config(cfg), cross=(0, cfg.d_mem))
